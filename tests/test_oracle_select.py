@@ -1,0 +1,86 @@
+"""Pins for the token-budget selection of the CPU oracle (Sec. 3.1, 3.2): brute force by
+numpy's lexicographic sort, crafted ties, k = 1, k = n, all-equal scores, zeros of both
+signs, NaN.  No GPU needed."""
+import numpy as np
+import pytest
+
+import oracle
+
+
+def _brute(scores, n, k):
+    """k-1 best of blocks [0, n-1) by (score desc, index asc) + block n-1, ascending."""
+    s = scores[: n - 1].astype(np.float64)
+    s = np.where(np.isnan(s), -np.inf, s)
+    nan_last = np.isnan(scores[: n - 1]).astype(np.int64)
+    order = np.lexsort((np.arange(n - 1), -s, nan_last))     # last key is the primary one
+    return sorted(list(order[: max(0, k - 1)]) + [n - 1])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_scores_against_lexsort(seed):
+    r = np.random.default_rng(seed)
+    B, Hkv, b, max_blocks, max_sel = 3, 2, 16, 40, 12
+    lens = np.array([40 * 16, 17 * 16 - 5, 3], np.int32)
+    sc = r.normal(size=(B, Hkv, max_blocks)).astype(np.float32)
+    if seed % 2:
+        sc = np.round(sc * 2) / 2                # many exact ties
+    budget = [16 * 7, 16 * 12, 16 * 100, 5][seed % 4]
+    idx, cnt = oracle.select(sc, lens, b, budget, max_sel)
+    for i in range(B):
+        n = -(-int(lens[i]) // b)
+        k = min(max(1, budget // b), n, max_sel)
+        for h in range(Hkv):
+            want = _brute(sc[i, h], n, k)
+            assert cnt[i, h] == len(want) == k
+            assert list(idx[i, h, :k]) == want
+            assert np.all(idx[i, h, k:] == -1)
+
+
+def test_crafted_ties_prefer_lower_index():
+    sc = np.array([[[1.0, 5.0, 5.0, 5.0, 0.0, 5.0, 9.0, 123.0]]], np.float32)
+    lens = [8 * 4]                                # n = 8, block 7 forced, its score ignored
+    idx, cnt = oracle.select(sc, lens, 4, 4 * 4, 8)
+    assert list(idx[0, 0, :4]) == [1, 2, 6, 7] and cnt[0, 0] == 4
+    idx, cnt = oracle.select(sc, lens, 4, 4 * 1, 8)          # k = 1: only the last block
+    assert list(idx[0, 0]) == [7] + [-1] * 7 and cnt[0, 0] == 1
+    idx, cnt = oracle.select(sc, lens, 4, 4 * 8, 8)          # k = n: everything
+    assert list(idx[0, 0]) == list(range(8))
+    idx, cnt = oracle.select(sc, lens, 4, 4 * 50, 8)         # budget beyond the sequence
+    assert list(idx[0, 0]) == list(range(8))
+    idx, cnt = oracle.select(sc, lens, 4, 0, 8)              # budget below one block -> k = 1
+    assert cnt[0, 0] == 1 and idx[0, 0, 0] == 7
+
+
+def test_all_equal_scores_take_the_first_blocks():
+    sc = np.full((1, 1, 10), 0.25, np.float32)
+    idx, cnt = oracle.select(sc, [10 * 8], 8, 8 * 4, 6)
+    assert list(idx[0, 0]) == [0, 1, 2, 9, -1, -1]
+
+
+def test_signed_zeros_tie_and_nan_ranks_last():
+    sc = np.array([[[-0.0, 0.0, -1.0, np.nan, -0.0, 7.0]]], np.float32)
+    idx, _ = oracle.select(sc, [6], 1, 3, 6)                 # n = 6, k = 3
+    assert list(idx[0, 0, :3]) == [0, 1, 5]                  # -0 at index 0 ties with +0 at 1
+    sc = np.array([[[np.nan, -np.inf, np.nan, -3.0, 0.0]]], np.float32)
+    idx, _ = oracle.select(sc, [5], 1, 4, 5)                 # candidates 0..3, k-1 = 3
+    assert list(idx[0, 0, :4]) == [0, 1, 3, 4]               # -3, -inf, then the first NaN
+    idx, _ = oracle.select(sc, [5], 1, 3, 5)
+    assert list(idx[0, 0, :3]) == [1, 3, 4]
+
+
+def test_partial_tail_and_single_block():
+    sc = np.arange(8, dtype=np.float32).reshape(1, 1, 8)
+    idx, cnt = oracle.select(sc, [33], 8, 16, 4)             # n = 5 (tail of 1 token), k = 2
+    assert list(idx[0, 0, :2]) == [3, 4] and cnt[0, 0] == 2
+    idx, cnt = oracle.select(sc, [5], 8, 64, 4)              # n = 1
+    assert list(idx[0, 0]) == [0, -1, -1, -1] and cnt[0, 0] == 1
+    idx, cnt = oracle.select(sc, [0], 8, 64, 4)              # empty sequence
+    assert cnt[0, 0] == 0 and np.all(idx == -1)
+
+
+def test_positive_scaling_never_changes_the_selection():
+    r = np.random.default_rng(9)
+    sc = r.normal(size=(2, 2, 64)).astype(np.float32)
+    a = oracle.select(sc, [64 * 8, 50 * 8], 8, 8 * 9, 16)
+    b = oracle.select(sc * np.float32(0.125), [64 * 8, 50 * 8], 8, 8 * 9, 16)   # exact scaling
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])

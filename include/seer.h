@@ -1,0 +1,213 @@
+/*
+ * seer.h -- C ABI of the B200 (sm_100a) decode library for SeerAttention-R:
+ * AttnGate scoring over a K compression cache, token-budget block selection,
+ * block-sparse GQA split-KV flash decoding with a log-sum-exp combine, the
+ * compressed-K cache update, and a dense decode kernel of the same design.
+ *
+ * General rules
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller, unless a
+ *    comment says "host".  The structs themselves are read on the host.
+ *  - bf16 tensors are raw 16-bit bfloat16; strides are in ELEMENTS.
+ *  - Every entry point is asynchronous on the CUDA stream passed as
+ *    `stream` (a cudaStream_t cast to void*, NULL = default stream), performs
+ *    no host synchronisation and no device allocation.  The library allocates
+ *    device memory only in seer_create (context workspace).
+ *  - Errors that the host can see (null pointers, unsupported shapes, a too
+ *    small workspace) return a status at once and launch nothing.  Problems
+ *    only the device can see (a block index or page id out of range) never
+ *    trap: the entry is skipped and a sticky flag is raised that
+ *    seer_get_device_status reports.
+ *  - A context serialises its calls through its workspace: calls that share a
+ *    context must be ordered on one stream (or by events).  Use one context
+ *    per concurrent stream.
+ *  - Supported: head_dim 128; block_size 64 or 128; group size
+ *    num_q_heads / num_kv_heads in 1..8; bf16 inputs, fp32 accumulation.
+ *
+ * Notation: B batch, Hq query heads, Hkv KV heads, g = Hq / Hkv, d head_dim,
+ * b block_size, L_i KV length of sequence i INCLUDING the token being decoded,
+ * n_i = ceil(L_i / b) blocks.  Query head hq belongs to KV head hq / g.
+ */
+#ifndef SEER_H_
+#define SEER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct seer_ctx seer_ctx;
+
+typedef enum {
+    SEER_OK = 0,
+    SEER_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, bad stride/alignment */
+    SEER_ERR_UNSUPPORTED = 2,   /* shape outside the supported set listed above */
+    SEER_ERR_WORKSPACE = 3,     /* context workspace too small for this call */
+    SEER_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed (see seer_last_error) */
+    SEER_ERR_BAD_INDEX = 5,     /* device saw a block index / page id out of range (skipped) */
+    SEER_ERR_TIMEOUT = 6        /* a bounded device-side wait gave up (results invalid) */
+} seer_status;
+
+/* Problem shape shared by all calls. */
+typedef struct {
+    int batch;          /* B */
+    int num_q_heads;    /* Hq */
+    int num_kv_heads;   /* Hkv, divides Hq */
+    int head_dim;       /* d = 128 */
+    int block_size;     /* b = 64 or 128 (sparsity block of the gate, Sec. 2.2 / 3.1) */
+    float sm_scale;     /* softmax scale applied to <q,k>, e.g. 1/sqrt(d) */
+} seer_shape;
+
+/*
+ * bf16 K/V cache.  Two layouts:
+ *  contiguous (page_table == NULL): element (i, h, t, c) of K is at
+ *      k[i*stride_batch + h*stride_head + t*stride_token + c], t < max_seq_len.
+ *      Any order of the batch/head/token axes works ([B,Hkv,S,d], [B,S,Hkv,d] ...).
+ *  paged (page_table != NULL): the cache is a pool of num_pages pages of
+ *      page_size tokens; token t of sequence i lives in page
+ *      p = page_table[i*page_table_stride + t/page_size] at
+ *      k[p*stride_batch + h*stride_head + (t % page_size)*stride_token + c].
+ *      page_size must be a multiple of 64.  (The paper leaves paged KV to
+ *      future work, Sec. 6; this layout is the library's own.)
+ * All strides must be multiples of 8 elements and k, v 16-byte aligned.
+ * Rows at positions >= L_i may hold anything (they are masked, never used).
+ */
+typedef struct {
+    const void* k;
+    const void* v;
+    int64_t stride_batch;           /* between sequences, or between pages when paged */
+    int64_t stride_head;
+    int64_t stride_token;
+    const int32_t* page_table;      /* device, or NULL for the contiguous layout */
+    int64_t page_table_stride;      /* entries per sequence row of the page table */
+    int page_size;                  /* tokens per page (paged only) */
+    int num_pages;                  /* pages in the pool (paged only) */
+    const int32_t* seq_lens;        /* device [B]: L_i */
+    int max_seq_len;                /* token capacity per sequence (contiguous) or the
+                                       largest L_i the page table covers (paged) */
+} seer_kv;
+
+/*
+ * AttnGate parameters and the K compression cache (Eq. 1, Sec. 3.2).
+ *  w_q   [Hkv, d_gate, g*d]  bf16: one projection per KV head over the g
+ *        pre-RoPE query heads of its group laid end to end (index u*d + c).
+ *  w_k   [Hkv, d_gate, 3*d]  bf16: input order [max-pool | min-pool | avg-pool].
+ *  kcomp [B, Hkv, max_blocks, d_gate] bf16: entry j is the compressed key of
+ *        block j (after pooling, projection and RoPE at position j*b).
+ * RoPE inside the gate: rotate-half pairing (c, c + d_gate/2), angle
+ * pos * rope_theta^(-2c/d_gate).  d_gate must be a multiple of 16, <= 256.
+ */
+typedef struct {
+    int d_gate;
+    float rope_theta;
+    const void* w_q;
+    const void* w_k;
+    void* kcomp;
+    int max_blocks;
+} seer_gate;
+
+/* ---- context ----------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` and allocates its workspace
+ * (workspace_bytes, 0 = a default of 64 MiB; partial results of split
+ * sequences, gate scratch, status words).  *out is NULL on failure. */
+seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes);
+/* Frees the workspace.  The caller must have synchronised the streams used. */
+void seer_destroy(seer_ctx* ctx);
+const char* seer_status_string(seer_status s);
+/* Human-readable detail of the last failing call on this context (host string,
+ * owned by the context, valid until the next call). */
+const char* seer_last_error(const seer_ctx* ctx);
+/* Synchronises `stream`, returns the sticky device-side status (SEER_OK,
+ * SEER_ERR_BAD_INDEX or SEER_ERR_TIMEOUT) and clears it. */
+seer_status seer_get_device_status(seer_ctx* ctx, void* stream);
+/* Workspace bytes a context needs for calls of this shape (upper bound);
+ * max_blocks = largest number of blocks per sequence. */
+size_t seer_workspace_bytes(const seer_shape* shape, int max_blocks, int d_gate);
+/* Number of kernels launched by this context so far (all entry points). */
+uint64_t seer_launch_count(const seer_ctx* ctx);
+
+/* ---- the four operations ------------------------------------------------ */
+
+/*
+ * Dense decode attention (the baseline of the paper's kernel comparison,
+ * Sec. 4.4, here the library's own kernel): for every sequence i and query
+ * head hq,  out[i,hq,:] = sum_{t < L_i} softmax_t(sm_scale <q[i,hq], k[i,hq/g,t]>) v[i,hq/g,t].
+ *  q   [B,Hq,d] bf16 contiguous;  out [B,Hq,d] bf16 contiguous;
+ *  lse [B,Hq] fp32 or NULL: natural-log sum of exp of the scaled scores.
+ * L_i == 0 gives out = 0, lse = -inf.
+ */
+seer_status seer_dense_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv,
+                              const void* q, void* out, float* lse, void* stream);
+
+/*
+ * Block-sparse split-KV flash decoding (Sec. 3.3): the same sum restricted to
+ * the tokens of the selected blocks, t in [j*b, min((j+1)*b, L_i)) for j in
+ * the list of (i, hq/g); all query heads of a group share the list.
+ *  block_idx [B,Hkv,max_sel] int32: block numbers; negative entries are
+ *            padding and are skipped; entries >= n_i are skipped and raise
+ *            SEER_ERR_BAD_INDEX; repeated entries are a caller error
+ *            (the block would be counted twice).  Any order.
+ *  block_cnt [B,Hkv] int32 or NULL: number of leading entries to read per
+ *            list (NULL = all max_sel entries, relying on negative padding).
+ * The selected blocks of all (sequence, KV head) pairs are cut into 64-token
+ * tiles and dealt out evenly over the CTAs; pieces of one pair meet in a
+ * log-sum-exp combine done by the last CTA to finish (no second launch).
+ * A list with no valid entry gives out = 0, lse = -inf.
+ */
+seer_status seer_sparse_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv,
+                               const void* q, const int32_t* block_idx,
+                               const int32_t* block_cnt, int max_sel,
+                               void* out, float* lse, void* stream);
+
+/*
+ * AttnGate scoring and token-budget selection (Eq. 1a, 1c; Sec. 3.1, 3.2).
+ *  Scores: q_gate = RoPE_{pos = L_i-1}(w_q[h] x), score[j] = <q_gate, kcomp[i,h,j]> / sqrt(d_gate)
+ *  for the blocks j < n_i - 1 (the softmax of Eq. 1c is not needed for a
+ *  top-k decision and is not computed).
+ *  Selection: k = min(max(1, token_budget / b), n_i, max_sel); the last block
+ *  n_i - 1 is always selected and counts against k; the other k-1 are the
+ *  highest-scoring of blocks [0, n_i-1), ties broken towards the lower block
+ *  number (-0 == +0, NaN below every number).  Lists are written in ascending
+ *  block order and padded with -1.
+ *  q_nope    [B,Hq,d] bf16 pre-RoPE queries; may be NULL iff scores_in is given.
+ *  scores_in [B,Hkv,max_blocks] fp32 or NULL: use these scores instead of
+ *            computing them (selection on caller-provided scores).
+ *  scores_out[B,Hkv,max_blocks] fp32 or NULL: receives the computed scores.
+ *  block_idx [B,Hkv,max_sel] int32 out; block_cnt [B,Hkv] int32 out.
+ *  seq_lens  device [B].
+ */
+seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                             const int32_t* seq_lens, const void* q_nope,
+                             const float* scores_in, int token_budget,
+                             int32_t* block_idx, int32_t* block_cnt, int max_sel,
+                             float* scores_out, void* stream);
+
+/*
+ * K compression cache update (Eq. 1b; Sec. 2.2 "Pooling-based Compression of
+ * K", Sec. 3.2): for block j of (i, h): per channel max, min and mean over the
+ * block's b rows of pre-RoPE K, concatenated [max|min|avg], multiplied by
+ * w_k[h], rotated at position j*b, stored as bf16 in kcomp[i,h,j,:].
+ *  k_nope: bf16, row for token t of (i,h) at
+ *          k_nope[i*stride_batch + h*stride_head + r*stride_token + c] with
+ *          r = t (rows_block_local == 0) or r = t - j*b (rows_block_local != 0:
+ *          the buffer holds just the block being appended, e.g. a rolling
+ *          window of the last b tokens).
+ *  first_block >= 0: write blocks first_block .. first_block+num_blocks-1 of
+ *          every sequence, skipping blocks that are not complete
+ *          (j >= floor(L_i / b)) -- the bulk build after prefill.
+ *  first_block == -1: per sequence, write the block that has just filled,
+ *          j = L_i/b - 1, if L_i % b == 0 and L_i > 0; otherwise nothing
+ *          (num_blocks is ignored) -- the once-per-b-tokens update of decoding.
+ */
+seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                              const int32_t* seq_lens, const void* k_nope,
+                              int64_t stride_batch, int64_t stride_head, int64_t stride_token,
+                              int rows_block_local, int first_block, int num_blocks,
+                              void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEER_H_ */

@@ -1,0 +1,425 @@
+// C ABI of the library: context, argument validation, tensor-map construction, launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/seer.h"
+#include "seer_device.cuh"
+#include "seer_internal.h"
+
+using namespace seer;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct MapKey {
+    const void* base;
+    uint64_t dims[4];
+    uint64_t strides[3];
+    bool operator==(const MapKey& o) const { return memcmp(this, &o, sizeof(MapKey)) == 0; }
+};
+
+constexpr int kMapCache = 16;
+
+}  // namespace
+
+struct seer_ctx {
+    int device;
+    int num_sms;
+    unsigned char* ws;          // device workspace
+    size_t ws_bytes;
+    EncodeTiledFn encode;
+    MapKey map_keys[kMapCache];
+    CUtensorMap maps[kMapCache];
+    int map_used;
+    int map_next;
+    uint64_t launches;
+    char err[512];
+};
+
+namespace {
+
+constexpr size_t kStatusBytes = 256;
+
+seer_status fail(seer_ctx* ctx, seer_status s, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof ctx->err, fmt, ap);
+        va_end(ap);
+    }
+    return s;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WsLayout {
+    size_t tickets, part_o, part_ml, q_gate, scores, total;
+};
+
+WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks) {
+    WsLayout w;
+    size_t off = kStatusBytes;
+    w.tickets = off; off = align_up(off + sizeof(int) * (size_t)num_units, 256);
+    w.part_o = off;  off = align_up(off + sizeof(float) * (size_t)slots * kMaxGroup * kHeadDim, 256);
+    w.part_ml = off; off = align_up(off + sizeof(float) * (size_t)slots * 2 * kMaxGroup, 256);
+    w.q_gate = off;  off = align_up(off + sizeof(float) * (size_t)num_units * (size_t)(d_gate > 0 ? d_gate : 0), 256);
+    w.scores = off;  off = align_up(off + sizeof(float) * (size_t)num_units * (size_t)(max_blocks > 0 ? max_blocks : 0), 256);
+    w.total = off;
+    return w;
+}
+
+constexpr int kMaxGridCtas = 148 * 2 * 4;   // generous bound used for workspace sizing only
+
+seer_status check_shape(seer_ctx* ctx, const seer_shape* s) {
+    if (!s) return fail(ctx, SEER_ERR_INVALID_ARG, "shape is NULL");
+    if (s->batch <= 0 || s->num_q_heads <= 0 || s->num_kv_heads <= 0)
+        return fail(ctx, SEER_ERR_INVALID_ARG, "batch/head counts must be positive");
+    if (s->head_dim != kHeadDim) return fail(ctx, SEER_ERR_UNSUPPORTED, "head_dim %d (only 128)", s->head_dim);
+    if (s->block_size != 64 && s->block_size != 128)
+        return fail(ctx, SEER_ERR_UNSUPPORTED, "block_size %d (only 64 or 128)", s->block_size);
+    if (s->num_q_heads % s->num_kv_heads != 0)
+        return fail(ctx, SEER_ERR_INVALID_ARG, "num_q_heads %d not a multiple of num_kv_heads %d",
+                    s->num_q_heads, s->num_kv_heads);
+    const int g = s->num_q_heads / s->num_kv_heads;
+    if (g < 1 || g > kMaxGroup) return fail(ctx, SEER_ERR_UNSUPPORTED, "group size %d (supported 1..8)", g);
+    if ((long long)s->batch * s->num_kv_heads > 65535)
+        return fail(ctx, SEER_ERR_UNSUPPORTED, "batch * num_kv_heads above 65535");
+    return SEER_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+seer_status get_map(seer_ctx* ctx, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
+                    const CUtensorMap** out) {
+    MapKey key;
+    memset(&key, 0, sizeof key);
+    key.base = base;
+    for (int a = 0; a < 4; ++a) key.dims[a] = dims[a];
+    for (int a = 0; a < 3; ++a) key.strides[a] = strides_bytes[a];
+    for (int a = 0; a < ctx->map_used; ++a)
+        if (ctx->map_keys[a] == key) { *out = &ctx->maps[a]; return SEER_OK; }
+    int slot;
+    if (ctx->map_used < kMapCache) slot = ctx->map_used++;
+    else { slot = ctx->map_next; ctx->map_next = (ctx->map_next + 1) % kMapCache; }
+    cuuint64_t gd[4] = {dims[0], dims[1], dims[2], dims[3]};
+    cuuint64_t gs[3] = {strides_bytes[0], strides_bytes[1], strides_bytes[2]};
+    cuuint32_t box[4] = {64, (cuuint32_t)kTileTokens, 1, 1};       // 64 channels (128 B) x 64 tokens
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = ctx->encode(&ctx->maps[slot], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gd, gs,
+                             box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        memset(&ctx->map_keys[slot], 0, sizeof(MapKey));
+        return fail(ctx, SEER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    }
+    ctx->map_keys[slot] = key;
+    *out = &ctx->maps[slot];
+    return SEER_OK;
+}
+
+seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q,
+                          const int32_t* block_idx, const int32_t* block_cnt, int max_sel, bool sparse,
+                          void* out, float* lse, void* stream) {
+    if (!ctx) return SEER_ERR_INVALID_ARG;
+    seer_status st = check_shape(ctx, shape);
+    if (st != SEER_OK) return st;
+    if (!kv || !kv->k || !kv->v || !kv->seq_lens || !q || !out)
+        return fail(ctx, SEER_ERR_INVALID_ARG, "NULL pointer among kv/k/v/seq_lens/q/out");
+    if (!aligned16(kv->k) || !aligned16(kv->v) || !aligned16(q) || !aligned16(out))
+        return fail(ctx, SEER_ERR_INVALID_ARG, "k, v, q and out must be 16-byte aligned");
+    if (kv->stride_batch % 8 || kv->stride_head % 8 || kv->stride_token % 8 || kv->stride_batch <= 0 ||
+        kv->stride_head <= 0 || kv->stride_token < kHeadDim)
+        return fail(ctx, SEER_ERR_INVALID_ARG, "K/V strides must be positive multiples of 8 elements");
+    if (kv->max_seq_len <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_seq_len must be positive");
+    const bool paged = kv->page_table != nullptr;
+    if (paged) {
+        if (kv->page_size <= 0 || kv->page_size % kTileTokens != 0)
+            return fail(ctx, SEER_ERR_UNSUPPORTED, "page_size %d (must be a multiple of 64)", kv->page_size);
+        if (kv->num_pages <= 0 || kv->page_table_stride <= 0)
+            return fail(ctx, SEER_ERR_INVALID_ARG, "num_pages and page_table_stride must be positive");
+        if ((long long)kv->page_table_stride * kv->page_size < kv->max_seq_len)
+            return fail(ctx, SEER_ERR_INVALID_ARG, "page table row shorter than max_seq_len");
+    }
+    if (sparse) {
+        if (!block_idx) return fail(ctx, SEER_ERR_INVALID_ARG, "block_idx is NULL");
+        if (max_sel <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_sel must be positive");
+    }
+    const int U = shape->batch * shape->num_kv_heads;
+    const int tpb = shape->block_size / kTileTokens;
+
+    cudaError_t ce = cudaSetDevice(ctx->device);
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
+    const int per_sm = decode_ctas_per_sm(sparse, paged);
+    if (per_sm <= 0) return fail(ctx, SEER_ERR_CUDA, "decode kernel cannot be resident (shared memory)");
+    long long max_tiles = sparse ? (long long)U * max_sel * tpb
+                                 : (long long)U * ((kv->max_seq_len + kTileTokens - 1) / kTileTokens);
+    int grid = ctx->num_sms * per_sm;
+    if (max_tiles < grid) grid = (int)(max_tiles > 0 ? max_tiles : 1);
+    const int slots = grid + U;
+    const WsLayout w = ws_layout(U, slots, 0, 0);
+    if (w.total > ctx->ws_bytes)
+        return fail(ctx, SEER_ERR_WORKSPACE, "workspace %zu bytes, call needs %zu", ctx->ws_bytes, w.total);
+
+    // tensor maps: (channel, token row, head, sequence-or-page)
+    const uint64_t rows = paged ? (uint64_t)kv->page_size : (uint64_t)kv->max_seq_len;
+    const uint64_t outer = paged ? (uint64_t)kv->num_pages : (uint64_t)shape->batch;
+    const uint64_t dims[4] = {(uint64_t)kHeadDim, rows, (uint64_t)shape->num_kv_heads, outer};
+    const uint64_t strides[3] = {(uint64_t)kv->stride_token * 2, (uint64_t)kv->stride_head * 2,
+                                 (uint64_t)kv->stride_batch * 2};
+    const CUtensorMap *mk, *mv;
+    st = get_map(ctx, kv->k, dims, strides, &mk);
+    if (st != SEER_OK) return st;
+    const CUtensorMap mk_copy = *mk;       // the second lookup may evict the first
+    st = get_map(ctx, kv->v, dims, strides, &mv);
+    if (st != SEER_OK) return st;
+
+    DecodeParams p;
+    memset(&p, 0, sizeof p);
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.lse = lse;
+    p.seq_lens = kv->seq_lens;
+    p.block_idx = block_idx;
+    p.block_cnt = block_cnt;
+    p.page_table = kv->page_table;
+    p.page_table_stride = kv->page_table_stride;
+    p.max_sel = max_sel;
+    p.page_size = kv->page_size;
+    p.num_pages = kv->num_pages;
+    p.batch = shape->batch;
+    p.num_q_heads = shape->num_q_heads;
+    p.num_kv_heads = shape->num_kv_heads;
+    p.group = shape->num_q_heads / shape->num_kv_heads;
+    p.block_size = shape->block_size;
+    p.tiles_per_block = tpb;
+    p.num_units = U;
+    p.max_blocks_cap = (kv->max_seq_len + kTileTokens - 1) / kTileTokens;
+    p.scale_log2 = shape->sm_scale * 1.4426950408889634f;
+    p.status = reinterpret_cast<unsigned int*>(ctx->ws);
+    p.tickets = reinterpret_cast<int*>(ctx->ws + w.tickets);
+    p.part_o = reinterpret_cast<float*>(ctx->ws + w.part_o);
+    p.part_ml = reinterpret_cast<float*>(ctx->ws + w.part_ml);
+
+    ce = launch_decode(sparse, paged, mk_copy, *mv, p, grid, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "decode launch: %s", cudaGetErrorString(ce));
+    ctx->launches += 1;
+    return SEER_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes) {
+    if (!out) return SEER_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return SEER_ERR_CUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return SEER_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SEER_ERR_CUDA;
+    if (prop.major != 10) return SEER_ERR_UNSUPPORTED;    // kernels are built for sm_100a only
+    seer_ctx* ctx = new (std::nothrow) seer_ctx;
+    if (!ctx) return SEER_ERR_CUDA;
+    memset(ctx, 0, sizeof *ctx);
+    ctx->device = device;
+    ctx->num_sms = prop.multiProcessorCount;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) {
+        delete ctx;
+        return SEER_ERR_CUDA;
+    }
+    ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    ctx->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)64 << 20;
+    if (ctx->ws_bytes < 4096) ctx->ws_bytes = 4096;
+    if (cudaMalloc(reinterpret_cast<void**>(&ctx->ws), ctx->ws_bytes) != cudaSuccess) {
+        delete ctx;
+        return SEER_ERR_CUDA;
+    }
+    if (cudaMemset(ctx->ws, 0, ctx->ws_bytes) != cudaSuccess) {
+        cudaFree(ctx->ws);
+        delete ctx;
+        return SEER_ERR_CUDA;
+    }
+    *out = ctx;
+    return SEER_OK;
+}
+
+void seer_destroy(seer_ctx* ctx) {
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->ws);
+    delete ctx;
+}
+
+const char* seer_status_string(seer_status s) {
+    switch (s) {
+        case SEER_OK: return "ok";
+        case SEER_ERR_INVALID_ARG: return "invalid argument";
+        case SEER_ERR_UNSUPPORTED: return "unsupported shape";
+        case SEER_ERR_WORKSPACE: return "workspace too small";
+        case SEER_ERR_CUDA: return "CUDA error";
+        case SEER_ERR_BAD_INDEX: return "block index or page id out of range (skipped)";
+        case SEER_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+const char* seer_last_error(const seer_ctx* ctx) { return ctx ? ctx->err : "context is NULL"; }
+
+uint64_t seer_launch_count(const seer_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
+    if (!ctx) return SEER_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, ctx->ws, sizeof word, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws, 0, sizeof word, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "status read: %s", cudaGetErrorString(e));
+    if (word & DEV_TIMEOUT) {
+        // a piece that gave up may have left tickets behind: clear them for the next call
+        cudaMemsetAsync(ctx->ws + kStatusBytes, 0, ctx->ws_bytes < (1u << 20) ? ctx->ws_bytes - kStatusBytes
+                                                                              : (1u << 20) - kStatusBytes, s);
+        cudaStreamSynchronize(s);
+        return fail(ctx, SEER_ERR_TIMEOUT, "a device-side wait gave up; results of that call are invalid");
+    }
+    if (word & DEV_BAD_INDEX) return fail(ctx, SEER_ERR_BAD_INDEX, "out-of-range block index or page id skipped");
+    return SEER_OK;
+}
+
+size_t seer_workspace_bytes(const seer_shape* shape, int max_blocks, int d_gate) {
+    if (!shape || shape->batch <= 0 || shape->num_kv_heads <= 0) return 0;
+    const int U = shape->batch * shape->num_kv_heads;
+    return ws_layout(U, kMaxGridCtas + U, d_gate, max_blocks).total;
+}
+
+seer_status seer_dense_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q, void* out,
+                              float* lse, void* stream) {
+    return decode_common(ctx, shape, kv, q, nullptr, nullptr, 0, false, out, lse, stream);
+}
+
+seer_status seer_sparse_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q,
+                               const int32_t* block_idx, const int32_t* block_cnt, int max_sel, void* out,
+                               float* lse, void* stream) {
+    return decode_common(ctx, shape, kv, q, block_idx, block_cnt, max_sel, true, out, lse, stream);
+}
+
+seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,
+                             const void* q_nope, const float* scores_in, int token_budget, int32_t* block_idx,
+                             int32_t* block_cnt, int max_sel, float* scores_out, void* stream) {
+    if (!ctx) return SEER_ERR_INVALID_ARG;
+    seer_status st = check_shape(ctx, shape);
+    if (st != SEER_OK) return st;
+    if (!gate || !seq_lens || !block_idx || !block_cnt)
+        return fail(ctx, SEER_ERR_INVALID_ARG, "NULL pointer among gate/seq_lens/block_idx/block_cnt");
+    if (max_sel <= 0 || gate->max_blocks <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_sel and max_blocks must be positive");
+    if (token_budget < 0) return fail(ctx, SEER_ERR_INVALID_ARG, "token_budget is negative");
+    if (!scores_in) {
+        if (!q_nope || !gate->w_q || !gate->kcomp)
+            return fail(ctx, SEER_ERR_INVALID_ARG, "q_nope, w_q and kcomp are needed when scores_in is NULL");
+        if (gate->d_gate <= 0 || gate->d_gate % 16 || gate->d_gate > 256)
+            return fail(ctx, SEER_ERR_UNSUPPORTED, "d_gate %d (multiple of 16, at most 256)", gate->d_gate);
+        if (!aligned16(q_nope) || !aligned16(gate->w_q) || !aligned16(gate->kcomp))
+            return fail(ctx, SEER_ERR_INVALID_ARG, "q_nope, w_q and kcomp must be 16-byte aligned");
+        if (!(gate->rope_theta > 0.f)) return fail(ctx, SEER_ERR_INVALID_ARG, "rope_theta must be positive");
+    }
+    const int U = shape->batch * shape->num_kv_heads;
+    const WsLayout w = ws_layout(U, kMaxGridCtas + U, scores_in ? 0 : gate->d_gate, scores_in ? 0 : gate->max_blocks);
+    if (w.total > ctx->ws_bytes)
+        return fail(ctx, SEER_ERR_WORKSPACE, "workspace %zu bytes, call needs %zu", ctx->ws_bytes, w.total);
+    cudaError_t ce = cudaSetDevice(ctx->device);
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
+
+    GateParams p;
+    memset(&p, 0, sizeof p);
+    p.q_nope = static_cast<const __nv_bfloat16*>(q_nope);
+    p.w_q = static_cast<const __nv_bfloat16*>(gate->w_q);
+    p.kcomp = static_cast<const __nv_bfloat16*>(gate->kcomp);
+    p.seq_lens = seq_lens;
+    p.scores_in = scores_in;
+    p.scores = scores_out ? scores_out : reinterpret_cast<float*>(ctx->ws + w.scores);
+    p.q_gate = reinterpret_cast<float*>(ctx->ws + w.q_gate);
+    p.block_idx = block_idx;
+    p.block_cnt = block_cnt;
+    p.batch = shape->batch;
+    p.num_q_heads = shape->num_q_heads;
+    p.num_kv_heads = shape->num_kv_heads;
+    p.group = shape->num_q_heads / shape->num_kv_heads;
+    p.block_size = shape->block_size;
+    p.d_gate = gate->d_gate;
+    p.max_blocks = gate->max_blocks;
+    p.max_sel = max_sel;
+    p.token_budget = token_budget;
+    p.rope_theta = gate->rope_theta;
+    p.status = reinterpret_cast<unsigned int*>(ctx->ws);
+    int launched = 0;
+    ce = launch_gate_select(p, static_cast<cudaStream_t>(stream), &launched);
+    ctx->launches += launched;
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "gate launch: %s", cudaGetErrorString(ce));
+    return SEER_OK;
+}
+
+seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,
+                              const void* k_nope, int64_t stride_batch, int64_t stride_head, int64_t stride_token,
+                              int rows_block_local, int first_block, int num_blocks, void* stream) {
+    if (!ctx) return SEER_ERR_INVALID_ARG;
+    seer_status st = check_shape(ctx, shape);
+    if (st != SEER_OK) return st;
+    if (!gate || !seq_lens || !k_nope || !gate->w_k || !gate->kcomp)
+        return fail(ctx, SEER_ERR_INVALID_ARG, "NULL pointer among gate/seq_lens/k_nope/w_k/kcomp");
+    if (gate->d_gate <= 0 || gate->d_gate % 16 || gate->d_gate > 256)
+        return fail(ctx, SEER_ERR_UNSUPPORTED, "d_gate %d (multiple of 16, at most 256)", gate->d_gate);
+    if (gate->max_blocks <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_blocks must be positive");
+    if (!(gate->rope_theta > 0.f)) return fail(ctx, SEER_ERR_INVALID_ARG, "rope_theta must be positive");
+    if (!aligned16(k_nope) || !aligned16(gate->w_k) || !aligned16(gate->kcomp))
+        return fail(ctx, SEER_ERR_INVALID_ARG, "k_nope, w_k and kcomp must be 16-byte aligned");
+    if (stride_batch % 8 || stride_head % 8 || stride_token % 8 || stride_token < kHeadDim || stride_batch < 0 ||
+        stride_head < 0)
+        return fail(ctx, SEER_ERR_INVALID_ARG, "k_nope strides must be multiples of 8 elements");
+    if (first_block < -1) return fail(ctx, SEER_ERR_INVALID_ARG, "first_block must be >= -1");
+    if (first_block >= 0 && num_blocks < 0) return fail(ctx, SEER_ERR_INVALID_ARG, "num_blocks is negative");
+    if (first_block >= 0 && rows_block_local && num_blocks > 1)
+        return fail(ctx, SEER_ERR_INVALID_ARG, "a block-local buffer holds one block only");
+    cudaError_t ce = cudaSetDevice(ctx->device);
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
+
+    KcompParams p;
+    memset(&p, 0, sizeof p);
+    p.k_nope = static_cast<const __nv_bfloat16*>(k_nope);
+    p.w_k = static_cast<const __nv_bfloat16*>(gate->w_k);
+    p.kcomp = static_cast<__nv_bfloat16*>(gate->kcomp);
+    p.seq_lens = seq_lens;
+    p.stride_batch = stride_batch;
+    p.stride_head = stride_head;
+    p.stride_token = stride_token;
+    p.rows_block_local = rows_block_local;
+    p.first_block = first_block;
+    p.num_blocks = num_blocks;
+    p.batch = shape->batch;
+    p.num_kv_heads = shape->num_kv_heads;
+    p.block_size = shape->block_size;
+    p.d_gate = gate->d_gate;
+    p.max_blocks = gate->max_blocks;
+    p.rope_theta = gate->rope_theta;
+    int launched = 0;
+    ce = launch_kcomp_append(p, static_cast<cudaStream_t>(stream), &launched);
+    ctx->launches += launched;
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "kcomp launch: %s", cudaGetErrorString(ce));
+    return SEER_OK;
+}
+
+}  // extern "C"

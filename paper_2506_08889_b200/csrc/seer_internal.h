@@ -1,0 +1,80 @@
+// Host-side declarations shared by the translation units of the library.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace seer {
+
+constexpr int kHeadDim = 128;       // d
+constexpr int kTileTokens = 64;     // tokens per staged K (or V) tile
+constexpr int kMaxGroup = 8;        // query heads per KV head handled by one MMA N-tile
+
+// Everything the decode kernels need besides the two tensor maps.
+struct DecodeParams {
+    const __nv_bfloat16* q;
+    __nv_bfloat16* out;
+    float* lse;
+    const int32_t* seq_lens;
+    const int32_t* block_idx;       // sparse only
+    const int32_t* block_cnt;       // sparse only, may be null
+    const int32_t* page_table;      // paged only
+    int64_t page_table_stride;
+    int max_sel;
+    int page_size;
+    int num_pages;
+    int batch, num_q_heads, num_kv_heads, group, block_size, tiles_per_block;
+    int num_units;                  // batch * num_kv_heads
+    int max_blocks_cap;             // tile-count clamp for dense: capacity in tiles
+    float scale_log2;               // sm_scale * log2(e)
+    unsigned int* status;
+    int* tickets;                   // [num_units], zero between launches
+    float* part_o;                  // [slots][8][128]
+    float* part_ml;                 // [slots][2][8]  (max, sum)
+};
+
+struct DecodeLaunch {
+    int grid;
+    cudaStream_t stream;
+};
+
+// Returns resident CTAs per SM for the decode kernel (queried once).
+int decode_ctas_per_sm(bool sparse, bool paged);
+cudaError_t launch_decode(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
+                          const DecodeParams& p, int grid, cudaStream_t stream);
+
+struct GateParams {
+    const __nv_bfloat16* q_nope;    // [B,Hq,d]
+    const __nv_bfloat16* w_q;       // [Hkv,dg,g*d]
+    const __nv_bfloat16* kcomp;     // [B,Hkv,max_blocks,dg]
+    const int32_t* seq_lens;
+    const float* scores_in;         // may be null
+    float* scores;                  // [B,Hkv,max_blocks] (workspace or caller's scores_out)
+    float* q_gate;                  // [B,Hkv,dg] workspace
+    int32_t* block_idx;
+    int32_t* block_cnt;
+    int batch, num_q_heads, num_kv_heads, group, block_size;
+    int d_gate, max_blocks, max_sel, token_budget;
+    float rope_theta;
+    unsigned int* status;
+};
+// Launches the scoring kernels (unless scores_in is given) and the selection kernel.
+// Returns the number of kernels launched through *launched.
+cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* launched);
+
+struct KcompParams {
+    const __nv_bfloat16* k_nope;
+    const __nv_bfloat16* w_k;       // [Hkv,dg,3d]
+    __nv_bfloat16* kcomp;           // [B,Hkv,max_blocks,dg]
+    const int32_t* seq_lens;
+    int64_t stride_batch, stride_head, stride_token;
+    int rows_block_local;
+    int first_block, num_blocks;    // first_block == -1: the block that just filled
+    int batch, num_kv_heads, block_size, d_gate, max_blocks;
+    float rope_theta;
+};
+cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* launched);
+
+}  // namespace seer

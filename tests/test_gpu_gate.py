@@ -1,0 +1,205 @@
+"""GPU parity of seer_kcomp_append and seer_gate_select against the fp64 oracle (C ABI).
+
+Stage isolation: each stage's oracle is fed the GPU's output of the stage before it, so a
+rounding difference in one stage cannot cascade into a different (equally valid) decision
+in the next.  The selection itself is compared bit for bit on identical fp32 scores."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_08889_b200 import binding, synth
+from util import bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+THETA = 1.0e6
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.close()
+
+
+def _bf16_ulp_close(got_bits, want_f64, ulps=1.0):
+    got = synth.bits_to_bf16(got_bits).to(torch.float64).numpy()
+    # one bf16 ulp at |x| (2^-7 |x| bounds it), plus the fp32-vs-fp64 accumulation noise that
+    # dominates for entries that happen to land near zero
+    tol = ulps * np.abs(want_f64) * 2.0 ** -7 + 1e-5 * np.abs(want_f64).max()
+    bad = np.abs(got - want_f64) > tol
+    assert not bad.any(), f"{bad.sum()} entries off by more than {ulps} ulp; worst {np.abs(got - want_f64).max()}"
+
+
+@pytest.mark.parametrize("b,dg,token_major", [(64, 128, False), (128, 128, True), (64, 64, False)])
+def test_kcomp_bulk_build(ctx, b, dg, token_major):
+    B, Hkv, d = 2, 3, 128
+    nb = 11
+    S = nb * b
+    lens = np.array([S, S - b - 5], np.int32)             # second sequence: 9 complete blocks
+    if token_major:
+        kn = synth.normal_bf16((B, S, Hkv, d), 5, "kn", DEV).permute(0, 2, 1, 3)
+    else:
+        kn = synth.normal_bf16((B, Hkv, S, d), 5, "kn", DEV)
+    wk = synth.normal_bf16((Hkv, dg, 3 * d), 5, "wk", DEV, std=0.02)
+    kc = torch.zeros((B, Hkv, nb, dg), dtype=torch.bfloat16, device=DEV)
+    shape = binding.make_shape(B, Hkv * 4, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, None, wk, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    ctx.seer_kcomp_append(shape, gate, lens_t, kn, first_block=0, num_blocks=nb)
+    torch.cuda.synchronize()
+    _, want = oracle.kcomp(bits(kn), bits(wk), b, 0, nb, nb, THETA)
+    got = bits(kc)
+    _bf16_ulp_close(got[0], want[0])
+    _bf16_ulp_close(got[1, :, :9], want[1, :, :9])
+    assert np.all(got[1, :, 9:] == 0)                     # incomplete blocks are not written
+    # a sub-range only touches its own entries
+    kc2 = torch.zeros_like(kc)
+    gate2 = binding.make_gate(dg, THETA, None, wk, kc2, nb)
+    ctx.seer_kcomp_append(shape, gate2, lens_t, kn, first_block=3, num_blocks=5)
+    torch.cuda.synchronize()
+    got2 = bits(kc2)
+    assert np.array_equal(got2[:, :, 3:8], got[:, :, 3:8])
+    assert np.all(got2[:, :, :3] == 0) and np.all(got2[:, :, 8:] == 0)
+
+
+def test_kcomp_append_when_a_block_fills(ctx):
+    B, Hkv, d, dg, b, nb = 3, 2, 128, 128, 64, 8
+    lens = np.array([5 * b, 5 * b + 1, 3 * b], np.int32)  # sequences 0 and 2 just filled a block
+    kn = synth.normal_bf16((B, Hkv, nb * b, d), 6, "kn", DEV)
+    wk = synth.normal_bf16((Hkv, dg, 3 * d), 6, "wk", DEV, std=0.02)
+    kc = torch.zeros((B, Hkv, nb, dg), dtype=torch.bfloat16, device=DEV)
+    shape = binding.make_shape(B, Hkv * 4, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, None, wk, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    ctx.seer_kcomp_append(shape, gate, lens_t, kn)        # first_block = -1
+    torch.cuda.synchronize()
+    _, want = oracle.kcomp(bits(kn), bits(wk), b, 0, nb, nb, THETA)
+    got = bits(kc)
+    _bf16_ulp_close(got[0, :, 4], want[0, :, 4])
+    _bf16_ulp_close(got[2, :, 2], want[2, :, 2])
+    mask = np.ones((B, nb), bool); mask[0, 4] = False; mask[2, 2] = False
+    assert np.all(got.transpose(0, 2, 1, 3)[mask] == 0)
+    # the same update from a rolling window that holds only the block being appended
+    win = torch.stack([kn[0, :, 4 * b:5 * b], kn[1, :, 4 * b:5 * b], kn[2, :, 2 * b:3 * b]]).contiguous()
+    kc3 = torch.zeros_like(kc)
+    gate3 = binding.make_gate(dg, THETA, None, wk, kc3, nb)
+    ctx.seer_kcomp_append(shape, gate3, lens_t, win, rows_block_local=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(kc3), got)
+
+
+@pytest.mark.parametrize("g,b", [(4, 64), (5, 64), (8, 128), (1, 64)])
+def test_gate_scores_and_selection(ctx, g, b):
+    B, Hkv, d, dg = 3, 2, 128, 128
+    Hq = g * Hkv
+    nbmax = 40
+    lens = np.array([nbmax * b, 17 * b + 9, 2 * b - 1], np.int32)
+    qn = synth.normal_bf16((B, Hq, d), 8, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, g * d), 8, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nbmax, dg), 8, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    max_sel = 12
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nbmax), dtype=torch.float32, device=DEV)
+    budget = 7 * b
+    ctx.seer_gate_select(shape, gate, lens_t, qn, None, budget, idx, cnt, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    n = [-(-int(L) // b) for L in lens]
+    want_sc, _ = oracle.scores(bits(qn), bits(wq), bits(kc), [x - 1 for x in n], [int(L) - 1 for L in lens], THETA)
+    got_sc = sc.cpu().numpy()
+    for i in range(B):
+        assert np.abs(got_sc[i, :, :n[i] - 1] - want_sc[i, :, :n[i] - 1]).max() <= 1e-3
+    # selection is exact on the scores the GPU itself produced
+    want_idx, want_cnt = oracle.select(got_sc, lens, b, budget, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx)
+    assert np.array_equal(cnt.cpu().numpy(), want_cnt)
+    # without scores_out the internal scratch gives the same lists
+    idx2 = torch.zeros_like(idx); cnt2 = torch.zeros_like(cnt)
+    ctx.seer_gate_select(shape, gate, lens_t, qn, None, budget, idx2, cnt2, max_sel)
+    torch.cuda.synchronize()
+    assert torch.equal(idx, idx2) and torch.equal(cnt, cnt2)
+
+
+@pytest.mark.parametrize("case", ["normal", "ties", "all_equal", "specials"])
+@pytest.mark.parametrize("b", [64, 128])
+def test_selection_bit_exact_on_given_scores(ctx, case, b):
+    B, Hkv, nbmax = 4, 3, 700
+    r = synth.np_rng(9, case)
+    sc = r.normal(size=(B, Hkv, nbmax)).astype(np.float32)
+    if case == "ties":
+        sc = np.round(sc * 4) / 4
+    elif case == "all_equal":
+        sc[:] = 0.5
+    elif case == "specials":
+        sc[:, :, ::7] = 0.0
+        sc[:, :, 3::11] = -0.0
+        sc[:, :, 5::13] = np.nan
+        sc[:, :, 6::17] = -np.inf
+        sc[:, :, 8::19] = np.inf
+    lens = np.array([nbmax * b, 333 * b + 1, b, 2 * b], np.int32)
+    shape = binding.make_shape(B, Hkv * 4, Hkv, 128, b, 0.1)
+    gate = binding.make_gate(128, THETA, None, None, None, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    sc_t = torch.as_tensor(sc, device=DEV)
+    for budget, max_sel in [(64 * b, 64), (b, 8), (0, 8), (700 * b, 700), (650 * b, 700), (300 * b, 100)]:
+        idx = torch.full((B, Hkv, max_sel), 77, dtype=torch.int32, device=DEV)
+        cnt = torch.full((B, Hkv), 77, dtype=torch.int32, device=DEV)
+        ctx.seer_gate_select(shape, gate, lens_t, None, sc_t, budget, idx, cnt, max_sel)
+        torch.cuda.synchronize()
+        want_idx, want_cnt = oracle.select(sc, lens, b, budget, max_sel)
+        assert np.array_equal(cnt.cpu().numpy(), want_cnt), (case, budget)
+        assert np.array_equal(idx.cpu().numpy(), want_idx), (case, budget)
+
+
+def test_gate_then_decode_end_to_end_14b_shape_small(ctx):
+    # K_nope := K cache, bulk build of the compressed keys, gate, selection, sparse decode
+    B, Hq, Hkv, d, dg, b = 2, 10, 2, 128, 128, 64
+    nb = 48
+    S = nb * b
+    lens = np.array([S, S - 3 * b - 7], np.int32)
+    q = synth.normal_bf16((B, Hq, d), 12, "q", DEV)
+    qn = synth.normal_bf16((B, Hq, d), 12, "qn", DEV)
+    k = synth.normal_bf16((B, Hkv, S, d), 12, "k", DEV)
+    v = synth.normal_bf16((B, Hkv, S, d), 12, "v", DEV)
+    wq = synth.normal_bf16((Hkv, dg, 5 * d), 12, "wq", DEV, std=0.02)
+    wk = synth.normal_bf16((Hkv, dg, 3 * d), 12, "wk", DEV, std=0.02)
+    kc = torch.zeros((B, Hkv, nb, dg), dtype=torch.bfloat16, device=DEV)
+    scale = 1.0 / np.sqrt(d)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, scale)
+    gate = binding.make_gate(dg, THETA, wq, wk, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    max_sel = 8
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nb), dtype=torch.float32, device=DEV)
+    out = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros((B, Hq), dtype=torch.float32, device=DEV)
+    kv = binding.make_kv(k, v, lens_t)
+    ctx.seer_kcomp_append(shape, gate, lens_t, k, first_block=0, num_blocks=nb)
+    ctx.seer_gate_select(shape, gate, lens_t, qn, None, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+    ctx.seer_sparse_decode(shape, kv, q, idx, cnt, max_sel, out, lse)
+    torch.cuda.synchronize()
+    # stage 1: compressed keys
+    _, kc_want = oracle.kcomp(bits(k), bits(wk), b, 0, nb, nb, THETA)
+    got_kc = bits(kc)
+    _bf16_ulp_close(got_kc[0], kc_want[0])
+    _bf16_ulp_close(got_kc[1, :, :44], kc_want[1, :, :44])
+    # stage 2: scores on the GPU's compressed keys
+    n = [-(-int(L) // b) for L in lens]
+    want_sc, _ = oracle.scores(bits(qn), bits(wq), got_kc, [x - 1 for x in n], [int(L) - 1 for L in lens], THETA)
+    got_sc = sc.cpu().numpy()
+    for i in range(B):
+        assert np.abs(got_sc[i, :, :n[i] - 1] - want_sc[i, :, :n[i] - 1]).max() <= 1e-3
+    # stage 3: selection on the GPU's scores, exact
+    want_idx, want_cnt = oracle.select(got_sc, lens, b, max_sel * b, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx) and np.array_equal(cnt.cpu().numpy(), want_cnt)
+    # stage 4: attention over the GPU's lists
+    from util import check_attention
+    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, want_idx, want_cnt, b, scale)
+    check_attention(out, lse, *ref, what="end to end")
+    assert ctx.device_status() == binding.SEER_OK

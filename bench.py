@@ -1,0 +1,459 @@
+#!/usr/bin/env python
+"""Benchmark of the decode hot path on B200: one "step" is one pass of the whole path for one
+attention layer and one new token per sequence --
+
+    seer_kcomp_append (the block that just filled)  ->  seer_gate_select (Q branch, scores,
+    token-budget top-k)  ->  seer_sparse_decode (split-KV attention + LSE combine)
+
+-- on the long-context sweep workload (batch 8, 40 query / 8 KV heads, head_dim 128,
+KV length 131072, block 64, 90 % of the blocks skipped), with seer_dense_decode timed
+beside it as the speed-up denominator.  Inputs are seeded and synthetic.  Prints ONE JSON
+line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--sparsity S] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sparse_decode_selected_kv_GBps"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one sparse-decode launch on this workload,
+# from the ncu capture summarised under profiles/ (None until a capture exists).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._nvml = None
+
+    def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nvml = None
+            return
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def _run(self):
+        nv = self._nvml
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=2)
+        out = {"sm_mhz": int(np.median(self.samples)) if self.samples else None,
+               "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        return out
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# --------------------------------------------------------------------------------------------
+def build_layers(w, n_layers, seed, dev):
+    """Per layer: K/V cache (K doubles as the pre-RoPE keys the gate pools), gate weights,
+    compressed-K cache (built in bulk by the library, untimed), queries."""
+    import torch
+    from paper_2506_08889_b200 import binding, synth
+    B, Hq, Hkv, d, b, L = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size, w.seq_len
+    layers = []
+    for l in range(n_layers):
+        tag = f"{w.name}:L{l}:"
+        lay = {
+            "k": synth.normal_bf16((B, Hkv, L, d), seed, tag + "k", dev),
+            "v": synth.normal_bf16((B, Hkv, L, d), seed, tag + "v", dev),
+            "q": synth.normal_bf16((B, Hq, d), seed, tag + "q", dev),
+            "qn": synth.normal_bf16((B, Hq, d), seed, tag + "qn", dev),
+            "wq": synth.normal_bf16((Hkv, w.d_gate, w.group * d), seed, tag + "wq", dev, std=w.gate_weight_std),
+            "wk": synth.normal_bf16((Hkv, w.d_gate, 3 * d), seed, tag + "wk", dev, std=w.gate_weight_std),
+            "kc": torch.zeros((B, Hkv, L // b, w.d_gate), dtype=torch.bfloat16, device=dev),
+        }
+        layers.append(lay)
+    return layers
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2506_08889_b200 import binding, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+
+    w = synth.workload(4)
+    w.sparsity = args.sparsity
+    if args.batch:
+        w.batch = args.batch                        # smaller cases for profiler captures
+    if args.seq_len:
+        w.seq_len = args.seq_len
+    B, Hq, Hkv, d, b, L = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size, w.seq_len
+    n_blocks = L // b
+    k_sel = w.keep(n_blocks)
+    budget = k_sel * b
+    seed = synth.BASE_SEED + 1000 * rank            # every rank decodes its own batch of sequences
+    n_layers = args.layers
+    layers = build_layers(w, n_layers, seed, dev)
+
+    ctx = binding.Context(local)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, w.sm_scale)
+    lens_t = torch.full((B,), L, dtype=torch.int32, device=dev)
+    idx = torch.zeros((B, Hkv, k_sel), dtype=torch.int32, device=dev)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+    out = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=dev)
+    out_dense = torch.zeros_like(out)
+    for lay in layers:
+        lay["gate"] = binding.make_gate(w.d_gate, w.rope_theta, lay["wq"], lay["wk"], lay["kc"], n_blocks)
+        lay["kv"] = binding.make_kv(lay["k"], lay["v"], lens_t)
+        # compressed keys of all blocks but the one the timed step appends
+        ctx.seer_kcomp_append(shape, lay["gate"], lens_t, lay["k"], first_block=0, num_blocks=n_blocks - 1)
+    torch.cuda.synchronize()
+
+    def step(lay, ev=None):
+        ctx.seer_kcomp_append(shape, lay["gate"], lens_t, lay["k"])                 # L % b == 0: appends
+        ctx.seer_gate_select(shape, lay["gate"], lens_t, lay["qn"], None, budget, idx, cnt, k_sel)
+        if ev is not None:
+            ev[0].record()
+        ctx.seer_sparse_decode(shape, lay["kv"], lay["q"], idx, cnt, k_sel, out)
+        if ev is not None:
+            ev[1].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # algorithmic bytes of one step (what the method itself must move)
+    sel_kv_bytes = B * Hkv * k_sel * b * d * 2 * 2
+    decode_bytes = sel_kv_bytes + 2 * B * Hq * d * 2 + 4 * B * Hkv * k_sel
+    gate_bytes = B * Hkv * (n_blocks - 1) * w.d_gate * 2 + Hkv * w.d_gate * w.group * d * 2 + 2 * 4 * B * Hkv * (n_blocks - 1)
+    kcomp_bytes = B * Hkv * b * d * 2 + Hkv * w.d_gate * 3 * d * 2 + B * Hkv * w.d_gate * 2
+    dense_bytes = B * Hkv * L * d * 2 * 2 + 2 * B * Hq * d * 2
+
+    K, W = args.steps, max(args.warmup, 3)
+    for s in range(W):
+        step(layers[s % n_layers])
+        ctx.seer_dense_decode(shape, layers[s % n_layers]["kv"], layers[s % n_layers]["q"], out_dense)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.SEER_OK
+
+    # ---- timed region: exactly K steps, device timed, max over ranks ------------------------
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launch_count()
+    barrier()
+    t0.record()
+    for s in range(K):
+        step(layers[s % n_layers], evs[s])
+    t1.record()
+    barrier()
+    launches = ctx.launch_count() - launches0
+    step_ms = t0.elapsed_time(t1) / K
+    sparse_ms = float(np.mean([a.elapsed_time(bq) for a, bq in evs]))
+
+    # dense decode on the same tensors (speed-up denominator), same protocol
+    Kd = max(8, min(K, 200))
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    d0.record()
+    for s in range(Kd):
+        ctx.seer_dense_decode(shape, layers[s % n_layers]["kv"], layers[s % n_layers]["q"], out_dense)
+    d1.record()
+    barrier()
+    dense_ms = d0.elapsed_time(d1) / Kd
+    # sparse kernel alone, back to back (no events inside), for the kernel-only speed-up
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    s0.record()
+    for s in range(K):
+        lay = layers[s % n_layers]
+        ctx.seer_sparse_decode(shape, lay["kv"], lay["q"], idx, cnt, k_sel, out)
+    s1.record()
+    barrier()
+    sparse_b2b_ms = s0.elapsed_time(s1) / K
+    clocks = sampler.stop()
+
+    # ---- end to end through the same API with host buffers ----------------------------------
+    # Per-step inputs (queries, pre-RoPE queries, the new token's K and V rows, lengths) start in
+    # pinned host memory; the result is read back to the host.  The KV cache is device state.
+    hq = layers[0]["q"].cpu().pin_memory()
+    hqn = layers[0]["qn"].cpu().pin_memory()
+    hk_new = layers[0]["k"][:, :, L - 1, :].contiguous().cpu().pin_memory()
+    hv_new = layers[0]["v"][:, :, L - 1, :].contiguous().cpu().pin_memory()
+    hlens = lens_t.cpu().pin_memory()
+    hout = torch.empty((B, Hq, d), dtype=torch.bfloat16).pin_memory()
+    dq, dqn = torch.empty_like(layers[0]["q"]), torch.empty_like(layers[0]["qn"])
+    dk_new = torch.empty((B, Hkv, d), dtype=torch.bfloat16, device=dev)
+    dv_new = torch.empty_like(dk_new)
+    dlens = torch.empty_like(lens_t)
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hqn, hk_new, hv_new, hlens))
+    d2h = hout.numel() * hout.element_size()
+
+    def e2e_step(lay):
+        dq.copy_(hq, non_blocking=True)
+        dqn.copy_(hqn, non_blocking=True)
+        dk_new.copy_(hk_new, non_blocking=True)
+        dv_new.copy_(hv_new, non_blocking=True)
+        dlens.copy_(hlens, non_blocking=True)
+        lay["k"][:, :, L - 1, :] = dk_new            # the caller's append of the new token
+        lay["v"][:, :, L - 1, :] = dv_new
+        kv = lay["kv_e2e"]
+        ctx.seer_kcomp_append(shape, lay["gate"], dlens, lay["k"])
+        ctx.seer_gate_select(shape, lay["gate"], dlens, dqn, None, budget, idx, cnt, k_sel)
+        ctx.seer_sparse_decode(shape, kv, dq, idx, cnt, k_sel, out)
+        hout.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for lay in layers:
+        lay["kv_e2e"] = binding.make_kv(lay["k"], lay["v"], dlens)
+    Ke = max(8, min(K, 300))
+    for s in range(3):
+        e2e_step(layers[s % n_layers])
+    barrier()
+    w0 = time.perf_counter()
+    for s in range(Ke):
+        e2e_step(layers[s % n_layers])
+    barrier()
+    e2e_ms = (time.perf_counter() - w0) * 1e3 / Ke
+    assert ctx.device_status() == binding.SEER_OK
+
+    # ---- reduce over ranks -------------------------------------------------------------------
+    vals = torch.tensor([step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms = [float(x) for x in vals.cpu()]
+
+    result = None
+    if rank == 0:
+        peak, peak_kind = measured_hbm_peak()
+        value = world * sel_kv_bytes / (step_ms * 1e-3) / 1e9
+        kern_gbs = decode_bytes / (sparse_ms * 1e-3) / 1e9
+        result = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": round(step_ms, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "batch_per_gpu": B, "num_q_heads": Hq, "num_kv_heads": Hkv,
+                       "head_dim": d, "seq_len": L, "block_size": b, "sparsity": args.sparsity,
+                       "selected_blocks": k_sel, "of_blocks": n_blocks, "parallelism": f"replicated-batches x{world}",
+                       "step": "kcomp_append + gate_select + sparse_decode (one layer, one token per sequence)",
+                       "l2": f"steps rotate over {n_layers} layer caches ({n_layers * dense_bytes / 1e9:.1f} GB), "
+                             f"selected bytes per step {sel_kv_bytes / 1e6:.0f} MB > L2"},
+            "e2e": {"value": round(world * sel_kv_bytes / (e2e_ms * 1e-3) / 1e9, 1), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 5)},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "decode_kernel<sparse>", "achieved": round(kern_gbs, 1),
+                         "peak": peak, "unit": "GB/s", "frac": round(kern_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
+                         "frac_of_nominal_8000": round(kern_gbs / NOMINAL_HBM_GBS, 4),
+                         "algorithmic_bytes_per_launch": decode_bytes, "us_per_launch": round(sparse_ms * 1e3, 2),
+                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
+            "extra": {
+                "tokens_per_s_per_layer": round(world * B / (step_ms * 1e-3), 1),
+                "selected_kv_bytes_per_step": sel_kv_bytes,
+                "step_algorithmic_bytes": decode_bytes + gate_bytes + kcomp_bytes,
+                "sparse_kernel_us": round(sparse_ms * 1e3, 2), "sparse_kernel_back_to_back_us": round(sparse_b2b_ms * 1e3, 2),
+                "dense_kernel_us": round(dense_ms * 1e3, 2),
+                "dense_kernel_GBps": round(dense_bytes / (dense_ms * 1e-3) / 1e9, 1),
+                "dense_frac_of_measured_peak": round(dense_bytes / (dense_ms * 1e-3) / 1e9 / peak, 4),
+                "gate_plus_kcomp_us": round((step_ms - sparse_ms) * 1e3, 2),
+                "speedup_vs_dense_kernel": round(dense_ms / sparse_b2b_ms, 3),
+                "speedup_vs_dense_step": round(dense_ms / step_ms, 3),
+                "ideal_speedup": round(n_blocks / k_sel, 3),
+            },
+        }
+        if not args.no_cpu_baseline and world == 1:
+            result["cpu_baseline"] = cpu_baseline(w, layers[0], k_sel, budget, sel_kv_bytes, seconds=args.cpu_seconds)
+    ctx.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(result))
+
+
+# --------------------------------------------------------------------------------------------
+def oracle_step(w, host, n_seq, n_kv_heads, budget, k_sel):
+    """The whole step on the CPU oracle for the first n_seq sequences and the first
+    n_kv_heads KV heads (with their query-head groups).  Returns the selected-KV bytes."""
+    import oracle
+    b, L, g = w.block_size, w.seq_len, w.group
+    n_blocks = L // b
+    lens = np.full(n_seq, L, np.int32)
+    k, v = host["k"][:n_seq, :n_kv_heads], host["v"][:n_seq, :n_kv_heads]          # views
+    kc = host["kc"][:n_seq, :n_kv_heads]
+    wk, wq = host["wk"][:n_kv_heads], host["wq"][:n_kv_heads]
+    q, qn = host["q"][:n_seq, :n_kv_heads * g], host["qn"][:n_seq, :n_kv_heads * g]
+    kc, _ = oracle.kcomp(k, wk, b, n_blocks - 1, 1, n_blocks, w.rope_theta, kc_bf16=kc)
+    sc, _ = oracle.scores(qn, wq, kc, [n_blocks - 1] * n_seq, [L - 1] * n_seq, w.rope_theta)
+    idx, cnt = oracle.select(sc.astype(np.float32), lens, b, budget, k_sel)
+    oracle.sparse(q, k, v, lens, idx, cnt, b, w.sm_scale)
+    return n_seq * n_kv_heads * k_sel * b * w.head_dim * 2 * 2
+
+
+def host_copy(lay):
+    from paper_2506_08889_b200 import synth
+    return {name: synth.bf16_bits(lay[name]) for name in ("k", "v", "q", "qn", "wq", "wk", "kc")}
+
+
+def cpu_baseline(w, lay, k_sel, budget, sel_kv_bytes, seconds=15.0):
+    import oracle
+    host = host_copy(lay)
+    H = w.num_kv_heads
+    t0 = time.perf_counter()
+    nbytes = oracle_step(w, host, 1, H, budget, k_sel)
+    one = time.perf_counter() - t0
+    n_seq = int(max(1, min(w.batch, seconds / max(one, 1e-3))))
+    reps = int(max(1, min(5, seconds / max(one * n_seq, 1e-3))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        nbytes = oracle_step(w, host, n_seq, H, budget, k_sel)
+    one = (time.perf_counter() - t0) / reps
+    return {"value": round(nbytes / one / 1e9, 4), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"the whole step (kcomp + scores + select + sparse attention) for {n_seq} of {w.batch} "
+                      f"sequences, all heads, {reps} repetition(s), {one:.2f} s each",
+            "host_cores": os.cpu_count()}
+
+
+def run_reference(args):
+    """The reference arm: the fp64 oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    import oracle
+    from paper_2506_08889_b200 import synth
+    w = synth.workload(4)
+    w.sparsity = args.sparsity
+    b, L = w.block_size, w.seq_len
+    n_blocks = L // b
+    k_sel = w.keep(n_blocks)
+    budget = k_sel * b
+    K, W = args.steps, args.warmup
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    w_small = synth.workload(4)
+    w_small.batch = 1
+    lay = build_layers(w_small, 1, synth.BASE_SEED, dev)[0]
+    host = host_copy(lay)
+    del lay
+    # the compressed keys of the earlier blocks come from the oracle itself (untimed set-up)
+    host["kc"], _ = oracle.kcomp(host["k"], host["wk"], b, 0, n_blocks - 1, n_blocks, w.rope_theta)
+    # bounded sample: as many KV heads of one sequence per step as keep the whole run within minutes
+    budget_s = 150.0
+    heads = w.num_kv_heads
+    while True:
+        t0 = time.perf_counter()
+        oracle_step(w, host, 1, heads, budget, k_sel)
+        probe = time.perf_counter() - t0
+        if probe * (K + W) <= budget_s or heads == 1:
+            break
+        heads //= 2
+    K_eff = K if probe * (K + W) <= budget_s else max(1, int(budget_s / probe) - W)
+    for _ in range(W):
+        oracle_step(w, host, 1, heads, budget, k_sel)
+    t0 = time.perf_counter()
+    for _ in range(K_eff):
+        nbytes = oracle_step(w, host, 1, heads, budget, k_sel)
+    ms = (time.perf_counter() - t0) * 1e3 / K_eff
+    value = round(nbytes / (ms * 1e-3) / 1e9, 4)
+    sample = (f"one step = the whole path for 1 of {w.batch} sequences, {heads} of {w.num_kv_heads} KV heads "
+              f"({heads * w.group} query heads), {K_eff} timed steps")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K_eff, "warmup": W, "ms_per_step": round(ms, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sparsity": args.sparsity, "selected_blocks": k_sel, "of_blocks": n_blocks,
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--sparsity", type=float, default=0.9)
+    ap.add_argument("--layers", type=int, default=4, help="distinct layer caches the steps rotate over")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling cases)")
+    ap.add_argument("--seq-len", type=int, default=0, help="override the workload's KV length (multiple of 64)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -339,6 +339,69 @@ def run_ours(args):
 
 
 # --------------------------------------------------------------------------------------------
+def run_sweep(args):
+    """Sparsity sweep of the long-context workload (kernel-only times, one GPU): sparse decode at
+    each sparsity level against the dense kernel on the same tensors.  Writes one JSON document."""
+    import torch
+    from paper_2506_08889_b200 import binding, synth
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = synth.workload(4)
+    if args.batch:
+        w.batch = args.batch
+    if args.seq_len:
+        w.seq_len = args.seq_len
+    B, Hq, Hkv, d, b, L = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size, w.seq_len
+    n_blocks = L // b
+    n_layers = args.layers
+    layers = build_layers(w, n_layers, synth.BASE_SEED, dev)
+    ctx = binding.Context(0)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, w.sm_scale)
+    lens_t = torch.full((B,), L, dtype=torch.int32, device=dev)
+    out = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=dev)
+    for lay in layers:
+        lay["kv"] = binding.make_kv(lay["k"], lay["v"], lens_t)
+    peak, peak_kind = measured_hbm_peak()
+    K = args.steps
+
+    def timed(fn, iters):
+        for s in range(5):
+            fn(s)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for s in range(iters):
+            fn(s)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters * 1e3      # us
+
+    dense_us = timed(lambda s: ctx.seer_dense_decode(shape, layers[s % n_layers]["kv"], layers[s % n_layers]["q"], out),
+                     max(8, K // 10))
+    dense_bytes = B * Hkv * L * d * 4
+    rows = []
+    for sp in (0.0, 0.5, 0.75, 0.9, 0.95):
+        k_sel = synth.keep_count(n_blocks, sp)
+        scores = synth.normal_f32((B, Hkv, n_blocks), synth.BASE_SEED, f"sweep:{sp}", dev)
+        idx = torch.zeros((B, Hkv, k_sel), dtype=torch.int32, device=dev)
+        cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+        gate = binding.make_gate(w.d_gate, w.rope_theta, None, None, None, n_blocks)
+        ctx.seer_gate_select(shape, gate, lens_t, None, scores, k_sel * b, idx, cnt, k_sel)
+        us = timed(lambda s: ctx.seer_sparse_decode(shape, layers[s % n_layers]["kv"], layers[s % n_layers]["q"],
+                                                    idx, cnt, k_sel, out), K)
+        sel_bytes = B * Hkv * k_sel * b * d * 4
+        rows.append({"sparsity": sp, "selected_blocks": k_sel, "of_blocks": n_blocks, "sparse_us": round(us, 2),
+                     "selected_kv_MB": round(sel_bytes / 1e6, 1), "GBps": round(sel_bytes / us / 1e3, 1),
+                     "frac_of_measured_peak": round(sel_bytes / us / 1e3 / peak, 4),
+                     "frac_of_8000": round(sel_bytes / us / 1e3 / NOMINAL_HBM_GBS, 4),
+                     "speedup_vs_dense": round(dense_us / us, 3), "ideal_speedup": round(n_blocks / k_sel, 3)})
+    assert ctx.device_status() == binding.SEER_OK
+    doc = {"workload": w.name, "batch": B, "seq_len": L, "layers_rotated": n_layers, "dense_us": round(dense_us, 2),
+           "dense_GBps": round(dense_bytes / dense_us / 1e3, 1), "peak_GBps": peak, "peak_kind": peak_kind, "rows": rows}
+    print(json.dumps(doc))
+    ctx.close()
+
+
 def oracle_step(w, host, n_seq, n_kv_heads, budget, k_sel):
     """The whole step on the CPU oracle for the first n_seq sequences and the first
     n_kv_heads KV heads (with their query-head groups).  Returns the selected-KV bytes."""
@@ -446,10 +509,13 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling cases)")
     ap.add_argument("--seq-len", type=int, default=0, help="override the workload's KV length (multiple of 64)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep", action="store_true", help="kernel-only sparsity sweep instead of the step benchmark")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

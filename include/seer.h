@@ -96,7 +96,7 @@ typedef struct {
  *  kcomp [B, Hkv, max_blocks, d_gate] bf16: entry j is the compressed key of
  *        block j (after pooling, projection and RoPE at position j*b).
  * RoPE inside the gate: rotate-half pairing (c, c + d_gate/2), angle
- * pos * rope_theta^(-2c/d_gate).  d_gate must be a multiple of 16, <= 256.
+ * pos * rope_theta^(-2c/d_gate).  d_gate is 64, 128 or 256.
  */
 typedef struct {
     int d_gate;

@@ -63,13 +63,14 @@ seer_status fail(seer_ctx* ctx, seer_status s, const char* fmt, ...) {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t tickets, part_o, part_ml, q_gate, scores, total;
+    size_t tickets, gate_tickets, part_o, part_ml, q_gate, scores, total;
 };
 
 WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks) {
     WsLayout w;
     size_t off = kStatusBytes;
     w.tickets = off; off = align_up(off + sizeof(int) * (size_t)num_units, 256);
+    w.gate_tickets = off; off = align_up(off + sizeof(int) * (size_t)num_units, 256);
     w.part_o = off;  off = align_up(off + sizeof(float) * (size_t)slots * kMaxGroup * kHeadDim, 256);
     w.part_ml = off; off = align_up(off + sizeof(float) * (size_t)slots * 2 * kMaxGroup, 256);
     w.q_gate = off;  off = align_up(off + sizeof(float) * (size_t)num_units * (size_t)(d_gate > 0 ? d_gate : 0), 256);
@@ -95,6 +96,11 @@ seer_status check_shape(seer_ctx* ctx, const seer_shape* s) {
     if ((long long)s->batch * s->num_kv_heads > 65535)
         return fail(ctx, SEER_ERR_UNSUPPORTED, "batch * num_kv_heads above 65535");
     return SEER_OK;
+}
+
+// Rotary frequencies theta^(-2c/d_gate) in double (the device only multiplies by the position).
+void fill_inv_freq(double* dst, int d_gate, float theta) {
+    for (int c = 0; c < d_gate / 2; ++c) dst[c] = pow((double)theta, -2.0 * (double)c / (double)d_gate);
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -210,6 +216,9 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.part_o = reinterpret_cast<float*>(ctx->ws + w.part_o);
     p.part_ml = reinterpret_cast<float*>(ctx->ws + w.part_ml);
 
+#ifdef SEER_DECODE_TRACE
+    p.trace = reinterpret_cast<unsigned long long*>(ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)));
+#endif
     ce = launch_decode(sparse, paged, mk_copy, *mv, p, grid, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "decode launch: %s", cudaGetErrorString(ce));
     ctx->launches += 1;
@@ -281,6 +290,11 @@ const char* seer_last_error(const seer_ctx* ctx) { return ctx ? ctx->err : "cont
 
 uint64_t seer_launch_count(const seer_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+#ifdef SEER_DECODE_TRACE
+/* diagnostic builds only: device address of the per-CTA time stamps of the last decode launch */
+void* seer_debug_trace_ptr(seer_ctx* ctx) { return ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)); }
+#endif
+
 seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
     if (!ctx) return SEER_ERR_INVALID_ARG;
     cudaSetDevice(ctx->device);
@@ -331,8 +345,8 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
     if (!scores_in) {
         if (!q_nope || !gate->w_q || !gate->kcomp)
             return fail(ctx, SEER_ERR_INVALID_ARG, "q_nope, w_q and kcomp are needed when scores_in is NULL");
-        if (gate->d_gate <= 0 || gate->d_gate % 16 || gate->d_gate > 256)
-            return fail(ctx, SEER_ERR_UNSUPPORTED, "d_gate %d (multiple of 16, at most 256)", gate->d_gate);
+        if (gate->d_gate != 64 && gate->d_gate != 128 && gate->d_gate != 256)
+            return fail(ctx, SEER_ERR_UNSUPPORTED, "d_gate %d (supported: 64, 128, 256)", gate->d_gate);
         if (!aligned16(q_nope) || !aligned16(gate->w_q) || !aligned16(gate->kcomp))
             return fail(ctx, SEER_ERR_INVALID_ARG, "q_nope, w_q and kcomp must be 16-byte aligned");
         if (!(gate->rope_theta > 0.f)) return fail(ctx, SEER_ERR_INVALID_ARG, "rope_theta must be positive");
@@ -364,8 +378,9 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
     p.max_blocks = gate->max_blocks;
     p.max_sel = max_sel;
     p.token_budget = token_budget;
-    p.rope_theta = gate->rope_theta;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
+    p.tickets = reinterpret_cast<int*>(ctx->ws + w.gate_tickets);
+    if (!scores_in) fill_inv_freq(p.inv_freq, gate->d_gate, gate->rope_theta);
     int launched = 0;
     ce = launch_gate_select(p, static_cast<cudaStream_t>(stream), &launched);
     ctx->launches += launched;
@@ -381,8 +396,8 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
     if (st != SEER_OK) return st;
     if (!gate || !seq_lens || !k_nope || !gate->w_k || !gate->kcomp)
         return fail(ctx, SEER_ERR_INVALID_ARG, "NULL pointer among gate/seq_lens/k_nope/w_k/kcomp");
-    if (gate->d_gate <= 0 || gate->d_gate % 16 || gate->d_gate > 256)
-        return fail(ctx, SEER_ERR_UNSUPPORTED, "d_gate %d (multiple of 16, at most 256)", gate->d_gate);
+    if (gate->d_gate != 64 && gate->d_gate != 128 && gate->d_gate != 256)
+        return fail(ctx, SEER_ERR_UNSUPPORTED, "d_gate %d (supported: 64, 128, 256)", gate->d_gate);
     if (gate->max_blocks <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_blocks must be positive");
     if (!(gate->rope_theta > 0.f)) return fail(ctx, SEER_ERR_INVALID_ARG, "rope_theta must be positive");
     if (!aligned16(k_nope) || !aligned16(gate->w_k) || !aligned16(gate->kcomp))
@@ -414,7 +429,7 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
     p.block_size = shape->block_size;
     p.d_gate = gate->d_gate;
     p.max_blocks = gate->max_blocks;
-    p.rope_theta = gate->rope_theta;
+    fill_inv_freq(p.inv_freq, gate->d_gate, gate->rope_theta);
     int launched = 0;
     ce = launch_kcomp_append(p, static_cast<cudaStream_t>(stream), &launched);
     ctx->launches += launched;

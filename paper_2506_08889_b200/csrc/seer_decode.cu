@@ -55,6 +55,21 @@ struct __align__(1024) Smem {
     int start_off;
 };
 
+// Programmatic dependent launch: the kernel may start while its predecessor in the stream is
+// still running; nothing the predecessor writes is read before pdl_wait().
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+#ifdef SEER_DECODE_TRACE
+__device__ __forceinline__ void trace_stamp(const DecodeParams& p, int slot) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    p.trace[(size_t)blockIdx.x * 8 + slot] = t;
+}
+#define SEER_STAMP(slot) trace_stamp(p, slot)
+#else
+#define SEER_STAMP(slot) ((void)0)
+#endif
+
 template <bool SPARSE>
 __device__ __forceinline__ int tiles_of(const DecodeParams& p, int u) {
     int L = p.seq_lens[u / p.num_kv_heads];
@@ -111,6 +126,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         tma_prefetch_desc(&map_v);
     }
 
+    if (tid == 0) SEER_STAMP(0);
+    pdl_wait();
+    if (tid == 0) SEER_STAMP(1);
+
     // ---- every CTA sums the units' tile counts and finds where its own range starts ----
     const int per = (U + kThreads - 1) / kThreads;
     const int u_lo = min(U, tid * per), u_hi = min(U, u_lo + per);
@@ -158,6 +177,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     }
     __syncthreads();
     const int n_tiles = t_end - t_begin;
+    if (tid == 0) SEER_STAMP(2);
 
     if (warp == kConsumerWarps) {
         // =========================== producer warp ====================================
@@ -251,6 +271,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     } else {
                         mbar_arrive(&sm.full[st]);
                     }
+                    if (it == 0) SEER_STAMP(3);
+                    if (it == n_tiles - 1) SEER_STAMP(4);
                 }
             }
         }
@@ -262,10 +284,23 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     const int qd = lane & 3;            // column pair: heads 2*qd, 2*qd+1
     const int rw = lane >> 2;           // row within an 8-row slab
     uint32_t bq[8][2];                  // Q^T B-fragments for the 8 k-steps over d
+    uint32_t bq_pre[8][2];              // the same for the unit expected next (prefetched)
     float o[8][4];                      // O^T accumulators: 8 m-tiles over d
     float m_run[2], l_run[2];
     int cur_unit = -1;
     int seg = 0;
+    auto load_q = [&](uint32_t (&dst)[8][2], int unit) {
+        const int i = unit / p.num_kv_heads, h = unit % p.num_kv_heads;
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+            p.q + ((size_t)i * p.num_q_heads + (size_t)h * p.group + rw) * kHeadDim);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            dst[ks][0] = (rw < p.group) ? __ldg(qrow + (16 * ks + 2 * qd) / 2) : 0u;
+            dst[ks][1] = (rw < p.group) ? __ldg(qrow + (16 * ks + 8 + 2 * qd) / 2) : 0u;
+        }
+    };
+    int pre_unit = sm.start_unit;       // requested now, long before the first tile lands
+    if (pre_unit < U) load_q(bq_pre, pre_unit);
 
     // lane-constant parts of the ldmatrix addresses (swizzle: 16-B chunk ^= row & 7)
     const int k_row = 16 * w + ((lane >> 3) & 1) * 8 + (lane & 7);
@@ -278,16 +313,17 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         const int st = it % kStages;
         if (!mbar_wait(&sm.full[st], (it / kStages) & 1, p.status)) return;
         const StageMeta mt = sm.meta[st];
+        if (it == 0 && tid == 0) SEER_STAMP(5);
         if (mt.unit != cur_unit) {
             cur_unit = mt.unit;
-            const int i = cur_unit / p.num_kv_heads, h = cur_unit % p.num_kv_heads;
-            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-                p.q + ((size_t)i * p.num_q_heads + (size_t)h * p.group + rw) * kHeadDim);
+            if (cur_unit == pre_unit) {
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                bq[ks][0] = (rw < p.group) ? __ldg(qrow + (16 * ks + 2 * qd) / 2) : 0u;
-                bq[ks][1] = (rw < p.group) ? __ldg(qrow + (16 * ks + 8 + 2 * qd) / 2) : 0u;
+                for (int ks = 0; ks < 8; ++ks) { bq[ks][0] = bq_pre[ks][0]; bq[ks][1] = bq_pre[ks][1]; }
+            } else {
+                load_q(bq, cur_unit);
             }
+            pre_unit = cur_unit + 1;    // units follow one another (empty ones excepted)
+            if (pre_unit < U) load_q(bq_pre, pre_unit);
 #pragma unroll
             for (int a = 0; a < 8; ++a)
 #pragma unroll
@@ -362,6 +398,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.empty[st]);
 
+        if (it == n_tiles - 1 && tid == 0) SEER_STAMP(6);
         if (mt.last) {
             // ---------------- end of this CTA's piece of the unit ----------------------
             float l0 = l_run[0], l1 = l_run[1];
@@ -452,41 +489,53 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     if (lane == 0) ticket = atomicAdd(&p.tickets[u], 1);
                     ticket = __shfl_sync(0xffffffffu, ticket, 0);
                     if (ticket == n_parts - 1) {
-                        // last piece in: log-sum-exp combine of all pieces of the unit
+                        // Last piece in: log-sum-exp combine of all pieces of the unit.  Lane t takes
+                        // head t/4, channels 32*(t%4) .. +31 of every piece; the loads of a pass do
+                        // not depend on one another, so they are all in flight together.
                         __threadfence();
-                        float mm[2] = {-INFINITY, -INFINITY};
+                        const int hh = lane >> 2, d0 = 32 * (lane & 3);
+                        const size_t s_first = (size_t)c_first + u;
+                        float M = -INFINITY;
+#pragma unroll 8
+                        for (int s2 = 0; s2 < n_parts; ++s2)
+                            M = fmaxf(M, __ldcg(p.part_ml + (s_first + s2) * (2 * kMaxGroup) + hh));
+                        float acc[32];
+#pragma unroll
+                        for (int x = 0; x < 32; ++x) acc[x] = 0.f;
+                        float lsum = 0.f;
+#pragma unroll 2
                         for (int s2 = 0; s2 < n_parts; ++s2) {
-                            const float* pm = p.part_ml + ((size_t)c_first + s2 + u) * (2 * kMaxGroup);
-                            mm[0] = fmaxf(mm[0], __ldcg(pm + 2 * qd));
-                            mm[1] = fmaxf(mm[1], __ldcg(pm + 2 * qd + 1));
-                        }
+                            const float* pm = p.part_ml + (s_first + s2) * (2 * kMaxGroup);
+                            const float4* qo = reinterpret_cast<const float4*>(
+                                p.part_o + (s_first + s2) * (kMaxGroup * kHeadDim) + hh * kHeadDim + d0);
+                            const float ms = __ldcg(pm + hh);
+                            const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
+                            lsum += f * __ldcg(pm + kMaxGroup + hh);
 #pragma unroll
-                        for (int a = 0; a < 8; ++a)
-#pragma unroll
-                            for (int b = 0; b < 4; ++b) o[a][b] = 0.f;
-                        float ll[2] = {0.f, 0.f};
-                        for (int s2 = 0; s2 < n_parts; ++s2) {
-                            const size_t sl = (size_t)c_first + s2 + u;
-                            const float* pm = p.part_ml + sl * (2 * kMaxGroup);
-                            const float* qo = p.part_o + sl * (kMaxGroup * kHeadDim);
-                            const float ms0 = __ldcg(pm + 2 * qd), ms1 = __ldcg(pm + 2 * qd + 1);
-                            const float f0 = (ms0 == -INFINITY) ? 0.f : fast_exp2(ms0 - mm[0]);
-                            const float f1 = (ms1 == -INFINITY) ? 0.f : fast_exp2(ms1 - mm[1]);
-                            ll[0] += f0 * __ldcg(pm + kMaxGroup + 2 * qd);
-                            ll[1] += f1 * __ldcg(pm + kMaxGroup + 2 * qd + 1);
-#pragma unroll
-                            for (int a = 0; a < 8; ++a) {
-                                const int d0 = 16 * a + rw;
-                                o[a][0] += f0 * __ldcg(qo + (2 * qd) * kHeadDim + d0);
-                                o[a][1] += f1 * __ldcg(qo + (2 * qd + 1) * kHeadDim + d0);
-                                o[a][2] += f0 * __ldcg(qo + (2 * qd) * kHeadDim + d0 + 8);
-                                o[a][3] += f1 * __ldcg(qo + (2 * qd + 1) * kHeadDim + d0 + 8);
+                            for (int x = 0; x < 8; ++x) {
+                                const float4 v4 = __ldcg(qo + x);
+                                acc[4 * x] += f * v4.x; acc[4 * x + 1] += f * v4.y;
+                                acc[4 * x + 2] += f * v4.z; acc[4 * x + 3] += f * v4.w;
                             }
                         }
-                        m_all[0] = mm[0]; m_all[1] = mm[1];
-                        l_all[0] = ll[0]; l_all[1] = ll[1];
                         if (lane == 0) p.tickets[u] = 0;     // ready for the next launch
-                        write_final = true;
+                        if (hh < p.group) {
+                            const int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
+                            const size_t row = (size_t)i * p.num_q_heads + (size_t)h * p.group + hh;
+                            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                            uint4* dst = reinterpret_cast<uint4*>(p.out + row * kHeadDim + d0);
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) {
+                                uint4 pk;
+                                pk.x = pack_bf16x2(acc[8 * x] * inv, acc[8 * x + 1] * inv);
+                                pk.y = pack_bf16x2(acc[8 * x + 2] * inv, acc[8 * x + 3] * inv);
+                                pk.z = pack_bf16x2(acc[8 * x + 4] * inv, acc[8 * x + 5] * inv);
+                                pk.w = pack_bf16x2(acc[8 * x + 6] * inv, acc[8 * x + 7] * inv);
+                                dst[x] = pk;
+                            }
+                            if (p.lse && (lane & 3) == 0)
+                                p.lse[row] = lsum > 0.f ? (M + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
+                        }
                     }
                 }
                 if (write_final) {
@@ -520,6 +569,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             cur_unit = -1;      // a later piece (another unit) starts from fresh state
         }
     }
+    if (tid == 0) SEER_STAMP(7);
 }
 
 size_t decode_smem_bytes() { return sizeof(Smem) + 1024; }
@@ -548,8 +598,19 @@ template <bool SPARSE, bool PAGED>
 cudaError_t launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& p, int grid,
                    cudaStream_t stream) {
     if (occupancy<SPARSE, PAGED>() <= 0) return cudaErrorInvalidConfiguration;
-    decode_kernel<SPARSE, PAGED><<<grid, kThreads, decode_smem_bytes(), stream>>>(mk, mv, p);
-    return cudaGetLastError();
+    // launched as a programmatic dependent: barrier set-up and tensor-map prefetch may overlap
+    // the tail of the previous kernel in the stream (the kernel waits before its first read)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = decode_smem_bytes();
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_kernel<SPARSE, PAGED>, mk, mv, p);
 }
 
 }  // namespace

@@ -112,4 +112,14 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// sin and cos of pos * inv_freq for the rotary embedding.  The angle reaches 1e5..1e6 rad at
+// long context, so the product and the reduction to one turn are done in double (a handful
+// of operations); the reduced angle is then accurate to about 1e-10 turns and the fp32
+// sincospi of it to about 1e-7.
+__device__ __forceinline__ void rope_sincos(double pos, double inv_freq, float* sn, float* cs) {
+    double turns = pos * inv_freq * 0.15915494309189535;   // 1 / (2 pi)
+    turns -= rint(turns);                                   // in [-0.5, 0.5]
+    sincospif((float)(2.0 * turns), sn, cs);
+}
+
 }  // namespace seer

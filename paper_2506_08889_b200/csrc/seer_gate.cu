@@ -1,11 +1,19 @@
-// AttnGate at decode time (Eq. 1a, 1c; Sec. 3.1): Q-branch projection + RoPE, block scores
-// against the K compression cache, and the token-budget top-k with the forced last block.
+// AttnGate at decode time (Eq. 1a, 1c; Sec. 3.1, 3.2): the Q-branch projection + RoPE in a
+// small first kernel, then block scores against the K compression cache fused with the
+// token-budget top-k (forced last block) in a second one that is launched as a programmatic
+// dependent of the first, so that its key loads are already in flight when the gate query
+// becomes available.
 #include "seer_device.cuh"
 #include "seer_internal.h"
 
 namespace seer {
 
 namespace {
+
+constexpr int kGateThreads = 512;
+constexpr int kGateWarps = kGateThreads / 32;
+constexpr int kCached = 8;                  // candidate keys a thread can keep in registers
+constexpr int kProjThreads = 256;
 
 __device__ __forceinline__ float dot8(const uint4& a, const float* x) {
     const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&a);
@@ -18,76 +26,25 @@ __device__ __forceinline__ float dot8(const uint4& a, const float* x) {
     }
     return acc;
 }
-
-// ---- q_gate = RoPE_{L_i - 1}( W_q[h] . concat_g(Q_nope) ) ----------------------------------
-// grid (B*Hkv, ceil(dg/2 / 4)), 128 threads; each warp computes one rotary pair (c, c + dg/2).
-__global__ void __launch_bounds__(128) gate_qproj_kernel(const GateParams p) {
-    __shared__ float x[kMaxGroup * kHeadDim];
-    const int u = blockIdx.x, i = u / p.num_kv_heads, h = u % p.num_kv_heads;
-    const int n = p.group * kHeadDim;
-    const __nv_bfloat16* src = p.q_nope + ((size_t)i * p.num_q_heads + (size_t)h * p.group) * kHeadDim;
-    for (int c = threadIdx.x; c < n; c += blockDim.x) x[c] = __bfloat162float(src[c]);
-    __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int half = p.d_gate / 2;
-    const int c = blockIdx.y * 4 + warp;
-    if (c >= half) return;
-    const __nv_bfloat16* w0 = p.w_q + ((size_t)h * p.d_gate + c) * n;
-    const __nv_bfloat16* w1 = p.w_q + ((size_t)h * p.d_gate + c + half) * n;
-    float a0 = 0.f, a1 = 0.f;
-    for (int ch = lane; ch < n / 8; ch += 32) {
-        const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(w0) + ch);
-        const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(w1) + ch);
-        a0 += dot8(v0, x + 8 * ch);
-        a1 += dot8(v1, x + 8 * ch);
-    }
+__device__ __forceinline__ float dot8(const uint4& a, const uint4& b) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* g = reinterpret_cast<const __nv_bfloat162*>(&b);
+    float acc = 0.f;
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        a0 += __shfl_xor_sync(0xffffffffu, a0, off);
-        a1 += __shfl_xor_sync(0xffffffffu, a1, off);
+    for (int k = 0; k < 4; ++k) {
+        const float2 f = __bfloat1622float2(h[k]), e = __bfloat1622float2(g[k]);
+        acc = fmaf(f.x, e.x, acc);
+        acc = fmaf(f.y, e.y, acc);
     }
-    if (lane == 0) {
-        const int L = p.seq_lens[i];
-        const double pos = (double)(L > 0 ? L - 1 : 0);
-        const double ang = pos * pow((double)p.rope_theta, -2.0 * (double)c / (double)p.d_gate);
-        double sn, cs;
-        sincos(ang, &sn, &cs);
-        float* dst = p.q_gate + (size_t)u * p.d_gate;
-        dst[c] = (float)((double)a0 * cs - (double)a1 * sn);
-        dst[c + half] = (float)((double)a1 * cs + (double)a0 * sn);
-    }
+    return acc;
 }
 
-// ---- score[j] = <q_gate, Kc[j]> / sqrt(dg) for j < n_i - 1 ----------------------------------
-// grid (ceil(max_blocks / 64), B*Hkv), 128 threads; 16 lanes per block entry.
-__global__ void __launch_bounds__(128) gate_scores_kernel(const GateParams p) {
-    __shared__ float qg[256];
-    const int u = blockIdx.y, i = u / p.num_kv_heads;
-    const int L = p.seq_lens[i];
-    const int n_i = (L + p.block_size - 1) / p.block_size;
-    const int n_cand = min(n_i - 1, p.max_blocks);
-    const int j0 = blockIdx.x * 64;
-    if (j0 >= n_cand) return;
-    for (int c = threadIdx.x; c < p.d_gate; c += blockDim.x) qg[c] = p.q_gate[(size_t)u * p.d_gate + c];
-    __syncthreads();
-    const int sub = threadIdx.x & 15, grp = threadIdx.x >> 4;       // 8 groups of 16 lanes
-    const float inv = rsqrtf((float)p.d_gate);
-    const int chunks = p.d_gate / 8;
-    for (int jj = grp; jj < 64; jj += 8) {
-        const int j = j0 + jj;
-        const bool live = j < n_cand;
-        float acc = 0.f;
-        if (live) {
-            const uint4* row = reinterpret_cast<const uint4*>(p.kcomp + ((size_t)u * p.max_blocks + j) * p.d_gate);
-            for (int ch = sub; ch < chunks; ch += 16) acc += dot8(__ldg(row + ch), qg + 8 * ch);
-        }
-#pragma unroll
-        for (int off = 8; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (live && sub == 0) p.scores[(size_t)u * p.max_blocks + j] = acc * inv;
-    }
-}
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
+// start while its predecessor is still running; it must pass pdl_wait() before it touches
+// anything the predecessor writes.  Without the attribute both calls do nothing.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 
-// ---- token-budget selection ------------------------------------------------------------------
 // Order-preserving key: larger score <-> larger key; -0 == +0; NaN below everything.
 __device__ __forceinline__ uint32_t score_key(float s) {
     if (s != s) return 0u;
@@ -96,109 +53,301 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-constexpr int kSelThreads = 256;
+struct SelectSmem {
+    int hist[4][256];                       // one histogram per radix pass
+    unsigned long long warp_tot[kGateWarps];
+    uint32_t prefix;
+    int rem;
+};
 
-// One CTA per (sequence, KV head).  Radix select (4 passes of 8 bits) finds the key of the
-// (k-1)-th best candidate; a final ordered pass emits, in ascending block order, every
-// candidate above it plus the first few equal to it (lower block number wins a tie), then
-// the forced last block.  Comparisons only: the result is exact.
-__global__ void __launch_bounds__(kSelThreads) gate_topk_kernel(const GateParams p) {
-    __shared__ int hist[256];
-    __shared__ int warp_cnt[2][kSelThreads / 32];
-    __shared__ uint32_t sh_prefix;
-    __shared__ int sh_need;
-    const int u = blockIdx.x, i = u / p.num_kv_heads;
+// Token-budget selection for one unit, run by a whole CTA.  Thread t owns the candidates
+// [t*E, (t+1)*E).  A radix select (4 passes of 8 bits over order-preserving keys) finds the key
+// of the (k-1)-th best candidate; one ordered pass then emits, in ascending block order, every
+// candidate above it and the first few equal to it (the lower block number wins a tie), and
+// the forced last block closes the list.  Comparisons only: the result is exact.
+template <bool CACHED>
+__device__ void select_unit(const GateParams& p, int u, const float* sc, SelectSmem& sm) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int i = u / p.num_kv_heads;
     int32_t* dst = p.block_idx + (size_t)u * p.max_sel;
-    const float* sc = (p.scores_in ? p.scores_in : p.scores) + (size_t)u * p.max_blocks;
     const int L = p.seq_lens[i];
     const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
     if (n_i <= 0) {
-        for (int e = tid; e < p.max_sel; e += kSelThreads) dst[e] = -1;
+        for (int e = tid; e < p.max_sel; e += kGateThreads) dst[e] = -1;
         if (tid == 0) p.block_cnt[u] = 0;
         return;
     }
-    int k = p.token_budget / p.block_size;
-    k = max(k, 1);
+    int k = max(p.token_budget / p.block_size, 1);
     k = min(k, min(n_i, p.max_sel));
     const int n_cand = min(n_i - 1, p.max_blocks);
-    int need = min(k - 1, n_cand);          // candidates to take besides the last block
+    const int need = min(k - 1, n_cand);             // candidates to take besides the last block
+    const int E = (n_cand + kGateThreads - 1) / kGateThreads;
+    const int j_lo = min(n_cand, tid * E), j_hi = min(n_cand, j_lo + E);
 
-    uint32_t thr = 0u;                      // key of the need-th best candidate
-    int take_eq = 0;                        // how many candidates equal to thr to take
+    uint32_t keys[kCached];
+    if (CACHED) {
+#pragma unroll
+        for (int e = 0; e < kCached; ++e) keys[e] = (j_lo + e < j_hi) ? score_key(__ldcg(sc + j_lo + e)) : 0u;
+    }
+    auto key_at = [&](int e) -> uint32_t { return score_key(__ldcg(sc + j_lo + e)); };
+
+    uint32_t thr = 0u;                               // key of the need-th best candidate
+    int take_eq = n_cand;                            // candidates equal to thr that are taken
     if (need > 0 && need < n_cand) {
+        for (int x = tid; x < 4 * 256; x += kGateThreads) (&sm.hist[0][0])[x] = 0;
+        __syncthreads();
         uint32_t prefix = 0u;
         int rem = need;
         for (int pass = 0; pass < 4; ++pass) {
             const int shift = 24 - 8 * pass;
             const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-            for (int b = tid; b < 256; b += kSelThreads) hist[b] = 0;
-            __syncthreads();
-            for (int j = tid; j < n_cand; j += kSelThreads) {
-                const uint32_t key = score_key(sc[j]);
-                if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
-            }
-            __syncthreads();
-            if (tid == 0) {
-                int acc = 0, b = 255;
-                for (; b > 0; --b) {
-                    if (acc + hist[b] >= rem) break;
-                    acc += hist[b];
+            int* hist = sm.hist[pass];
+            if (CACHED) {
+#pragma unroll
+                for (int e = 0; e < kCached; ++e)
+                    if (j_lo + e < j_hi && (keys[e] & himask) == prefix)
+                        atomicAdd(&hist[(keys[e] >> shift) & 255u], 1);
+            } else {
+                for (int e = 0; j_lo + e < j_hi; ++e) {
+                    const uint32_t key = key_at(e);
+                    if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
                 }
-                sh_prefix = prefix | ((uint32_t)b << shift);
-                sh_need = rem - acc;
             }
             __syncthreads();
-            prefix = sh_prefix;
-            rem = sh_need;
+            if (warp == 0) {
+                // lane l owns bins 255-8l .. 248-8l (descending); a warp scan gives the number of
+                // keys in all higher bins, then the lane that straddles `rem` walks its 8 bins
+                int c[8], mine = 0;
+#pragma unroll
+                for (int b = 0; b < 8; ++b) { c[b] = hist[255 - 8 * lane - b]; mine += c[b]; }
+                int incl = mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                int above = incl - mine;
+                if (above < rem && rem <= incl) {
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) {
+                        if (above < rem && rem <= above + c[b]) {
+                            sm.prefix = prefix | ((uint32_t)(255 - 8 * lane - b) << shift);
+                            sm.rem = rem - above;
+                        }
+                        above += c[b];
+                    }
+                }
+            }
+            __syncthreads();
+            prefix = sm.prefix;
+            rem = sm.rem;
         }
         thr = prefix;
         take_eq = rem;
-    } else if (need >= n_cand) {
-        thr = 0u;                           // everything qualifies: key >= 0 always
-        take_eq = n_cand;
-        need = n_cand;
     }
 
-    // ordered emission
-    int out_base = 0, eq_base = 0;
     if (need > 0) {
-        for (int j0 = 0; j0 < n_cand; j0 += kSelThreads) {
-            const int j = j0 + tid;
-            uint32_t key = 0u;
-            const bool live = j < n_cand;
-            if (live) key = score_key(sc[j]);
-            const bool gt = live && key > thr;
-            const bool eq = live && key == thr;
-            const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
-            if (lane == 0) { warp_cnt[0][warp] = __popc(bg); warp_cnt[1][warp] = __popc(be); }
-            __syncthreads();
-            int gt_before = 0, eq_before = 0, gt_total = 0, eq_total = 0;
+        int n_gt = 0, n_eq = 0;
+        if (CACHED) {
 #pragma unroll
-            for (int w2 = 0; w2 < kSelThreads / 32; ++w2) {
-                const int a = warp_cnt[0][w2], b = warp_cnt[1][w2];
-                if (w2 < warp) { gt_before += a; eq_before += b; }
-                gt_total += a; eq_total += b;
+            for (int e = 0; e < kCached; ++e)
+                if (j_lo + e < j_hi) { n_gt += keys[e] > thr; n_eq += keys[e] == thr; }
+        } else {
+            for (int e = 0; j_lo + e < j_hi; ++e) {
+                const uint32_t key = key_at(e);
+                n_gt += key > thr; n_eq += key == thr;
             }
-            const unsigned lt_mask = (1u << lane) - 1u;
-            gt_before += __popc(bg & lt_mask);
-            eq_before += __popc(be & lt_mask);
-            // equal-key candidates are taken in index order until take_eq are in
-            const int eq_rank = eq_base + eq_before;
-            const int eq_taken_before = min(eq_rank, take_eq);
-            const bool sel = gt || (eq && eq_rank < take_eq);
-            if (sel) dst[out_base + gt_before + eq_taken_before - min(eq_base, take_eq)] = j;
-            out_base += gt_total + (min(eq_base + eq_total, take_eq) - min(eq_base, take_eq));
-            eq_base += eq_total;
-            __syncthreads();
+        }
+        // one block-wide exclusive scan of both counts packed into one 64-bit word
+        const unsigned long long packed = ((unsigned long long)n_gt << 32) | (unsigned long long)n_eq;
+        unsigned long long incl = packed;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) sm.warp_tot[warp] = incl;
+        __syncthreads();
+        unsigned long long base = 0;
+#pragma unroll
+        for (int w2 = 0; w2 < kGateWarps; ++w2) base += (w2 < warp) ? sm.warp_tot[w2] : 0ull;
+        const unsigned long long excl = base + incl - packed;
+        const int gt_before = (int)(excl >> 32);
+        int eq_rank = (int)(excl & 0xffffffffull);
+        int pos = gt_before + min(eq_rank, take_eq);
+        if (CACHED) {
+#pragma unroll
+            for (int e = 0; e < kCached; ++e) {
+                if (j_lo + e < j_hi) {
+                    const bool gt = keys[e] > thr, eq = keys[e] == thr;
+                    if (gt || (eq && eq_rank < take_eq)) dst[pos++] = j_lo + e;
+                    eq_rank += eq;
+                }
+            }
+        } else {
+            for (int e = 0; j_lo + e < j_hi; ++e) {
+                const uint32_t key = key_at(e);
+                const bool gt = key > thr, eq = key == thr;
+                if (gt || (eq && eq_rank < take_eq)) dst[pos++] = j_lo + e;
+                eq_rank += eq;
+            }
         }
     }
-    // forced last block, padding, count
     if (tid == 0) {
-        dst[need] = n_i - 1;
+        dst[need] = n_i - 1;                         // the last block is always active
         p.block_cnt[u] = need + 1;
     }
-    for (int e = need + 1 + tid; e < p.max_sel; e += kSelThreads) dst[e] = -1;
+    for (int e = need + 1 + tid; e < p.max_sel; e += kGateThreads) dst[e] = -1;
+}
+
+__device__ __forceinline__ void select_dispatch(const GateParams& p, int u, const float* sc, SelectSmem& sm) {
+    if (p.max_blocks <= kCached * kGateThreads) select_unit<true>(p, u, sc, sm);
+    else select_unit<false>(p, u, sc, sm);
+}
+
+// Selection on caller-provided scores: one CTA per unit.
+__global__ void __launch_bounds__(kGateThreads) gate_select_only_kernel(const GateParams p) {
+    __shared__ SelectSmem sm;
+    const int u = blockIdx.x;
+    select_dispatch(p, u, p.scores_in + (size_t)u * p.max_blocks, sm);
+}
+
+// ---- q_gate = RoPE_{L_i - 1}( W_q[h] . concat_g(Q_nope) )  (Eq. 1a) ---------------------------
+// grid (B*Hkv, d_gate/32): a CTA computes 16 rotary pairs; each of its 8 warps takes two pairs,
+// i.e. rows c, c+1, c+d_gate/2, c+1+d_gate/2, with all of their loads in flight together.
+// NIT = 16-byte pieces of a row per lane (row length g*128 bf16 = g*16 pieces over 32 lanes).
+template <int NIT>
+__global__ void __launch_bounds__(kProjThreads) gate_qproj_kernel(const GateParams p) {
+    pdl_launch_dependents();
+    const int u = blockIdx.x, i = u / p.num_kv_heads, h = u % p.num_kv_heads;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n = p.group * kHeadDim, chunks = n / 8, half = p.d_gate / 2;
+    const int c0 = blockIdx.y * 16 + warp * 2;
+    if (c0 >= half) return;
+    const uint4* xsrc = reinterpret_cast<const uint4*>(
+        p.q_nope + ((size_t)i * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
+    const int L = __ldg(p.seq_lens + i);
+    uint4 xv[NIT], wv[4][NIT];
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) {
+        const int ch = lane + 32 * it;
+        xv[it] = ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int r = c0 + (k & 1) + (k >> 1) * half;
+        const uint4* wrow = reinterpret_cast<const uint4*>(p.w_q + ((size_t)h * p.d_gate + r) * n);
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int ch = lane + 32 * it;
+            wv[k][it] = ch < chunks ? __ldg(wrow + ch) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    float acc[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        acc[k] = 0.f;
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) acc[k] += dot8(wv[k][it], xv[it]);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
+    }
+    if (lane < 2) {
+        const int c = c0 + lane;
+        float sn, cs;
+        rope_sincos((double)(L > 0 ? L - 1 : 0), p.inv_freq[c], &sn, &cs);
+        const float a = lane ? acc[1] : acc[0], b = lane ? acc[3] : acc[2];
+        float* dst = p.q_gate + (size_t)u * p.d_gate;
+        dst[c] = a * cs - b * sn;
+        dst[c + half] = b * cs + a * sn;
+    }
+}
+
+// ---- scores (Eq. 1c without the softmax) and selection ------------------------------------------
+// grid (S, B*Hkv): the compressed keys of one (sequence, KV head) unit are cut into S slices of
+// `per` entries.  A slice is one flat run of 16-byte pieces; thread t takes pieces t, t+512, ...
+// (kBatch in flight at a time; the first batch is requested before the kernel waits for the
+// projection kernel), and the d_gate/8 neighbouring lanes that hold one key's pieces add up by
+// shuffles.  Each CTA publishes its scores and takes a ticket; the CTA that draws the unit's
+// last ticket runs the selection over all of the unit's scores.  No CTA waits for another.
+__global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(const GateParams p, int per) {
+    __shared__ SelectSmem sm;
+    __shared__ int is_last;
+    const int u = blockIdx.y, i = u / p.num_kv_heads;
+    const int S = gridDim.x, slice = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int lpk = p.d_gate / 8;                      // lanes per key: 8, 16 or 32
+    const int csub = tid & (lpk - 1);
+    const int j0 = min(p.max_blocks, slice * per), j1 = min(p.max_blocks, j0 + per);
+    const uint4* kc = reinterpret_cast<const uint4*>(p.kcomp + ((size_t)u * p.max_blocks + j0) * p.d_gate);
+    const int total = (j1 - j0) * lpk;
+    constexpr int kBatch = 8;
+    uint4 kv[kBatch];
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k) {                 // entries past n_i - 1 exist in memory: harmless
+        const int c = k * kGateThreads + tid;
+        kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    pdl_wait();                                        // q_gate is complete from here on
+    pdl_launch_dependents();
+    const int L = __ldg(p.seq_lens + i);
+    const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
+    const int n_cand = max(0, min(n_i - 1, p.max_blocks));
+    float* sc_out = p.scores + (size_t)u * p.max_blocks;
+    float qsub[8];
+    {
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(p.q_gate + (size_t)u * p.d_gate + 8 * csub));
+        const float4 b = __ldcg(reinterpret_cast<const float4*>(p.q_gate + (size_t)u * p.d_gate + 8 * csub + 4));
+        qsub[0] = a.x; qsub[1] = a.y; qsub[2] = a.z; qsub[3] = a.w;
+        qsub[4] = b.x; qsub[5] = b.y; qsub[6] = b.z; qsub[7] = b.w;
+    }
+    const float inv = rsqrtf((float)p.d_gate);
+    for (int cb = 0; cb < total; cb += kGateThreads * kBatch) {
+        float acc[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
+        if (cb + kGateThreads * kBatch < total) {      // next batch on its way while this one reduces
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                const int c = cb + (kBatch + k) * kGateThreads + tid;
+                kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+            for (int off = lpk >> 1; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
+            const int c = cb + k * kGateThreads + tid;
+            const int j = j0 + c / lpk;
+            if (c < total && csub == 0 && j < n_cand) __stcg(sc_out + j, acc[k] * inv);
+        }
+    }
+    // ---- ticket: the last slice of the unit to finish does the selection --------------------
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int t = atomicAdd(&p.tickets[u], 1);
+        is_last = (t == S - 1);
+        if (is_last) p.tickets[u] = 0;               // ready for the next launch
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    select_dispatch(p, u, sc_out, sm);
+}
+
+template <typename... Args>
+cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 }  // namespace
@@ -206,18 +355,29 @@ __global__ void __launch_bounds__(kSelThreads) gate_topk_kernel(const GateParams
 cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* launched) {
     const int U = p.batch * p.num_kv_heads;
     *launched = 0;
-    if (!p.scores_in) {
-        const int half = p.d_gate / 2;
-        gate_qproj_kernel<<<dim3(U, (half + 3) / 4), 128, 0, stream>>>(p);
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-        gate_scores_kernel<<<dim3((p.max_blocks + 63) / 64, U), 128, 0, stream>>>(p);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-        *launched += 2;
+    if (p.scores_in) {
+        gate_select_only_kernel<<<U, kGateThreads, 0, stream>>>(p);
+        *launched = 1;
+        return cudaGetLastError();
     }
-    gate_topk_kernel<<<U, kSelThreads, 0, stream>>>(p);
-    *launched += 1;
+    const dim3 pgrid(U, (p.d_gate / 2 + 15) / 16);
+    const int nit = (p.group * kHeadDim / 8 + 31) / 32;
+    switch (nit) {
+        case 1: gate_qproj_kernel<1><<<pgrid, kProjThreads, 0, stream>>>(p); break;
+        case 2: gate_qproj_kernel<2><<<pgrid, kProjThreads, 0, stream>>>(p); break;
+        case 3: gate_qproj_kernel<3><<<pgrid, kProjThreads, 0, stream>>>(p); break;
+        default: gate_qproj_kernel<4><<<pgrid, kProjThreads, 0, stream>>>(p); break;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    *launched = 1;
+    // slices of about 512 compressed keys, at most 8 per unit
+    int S = (p.max_blocks + 511) / 512;
+    S = S < 1 ? 1 : (S > 8 ? 8 : S);
+    const int per = (p.max_blocks + S - 1) / S;
+    e = launch_pdl(gate_score_select_kernel, dim3(S, U), dim3(kGateThreads), stream, p, per);
+    if (e != cudaSuccess) return e;
+    *launched = 2;
     return cudaGetLastError();
 }
 

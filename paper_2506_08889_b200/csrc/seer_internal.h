@@ -11,6 +11,7 @@ namespace seer {
 constexpr int kHeadDim = 128;       // d
 constexpr int kTileTokens = 64;     // tokens per staged K (or V) tile
 constexpr int kMaxGroup = 8;        // query heads per KV head handled by one MMA N-tile
+constexpr int kMaxDGate = 256;      // gate width: 64, 128 or 256
 
 // Everything the decode kernels need besides the two tensor maps.
 struct DecodeParams {
@@ -33,6 +34,9 @@ struct DecodeParams {
     int* tickets;                   // [num_units], zero between launches
     float* part_o;                  // [slots][8][128]
     float* part_ml;                 // [slots][2][8]  (max, sum)
+#ifdef SEER_DECODE_TRACE
+    unsigned long long* trace;      // [grid][8] %globaltimer stamps (diagnostic builds only)
+#endif
 };
 
 struct DecodeLaunch {
@@ -57,8 +61,9 @@ struct GateParams {
     int32_t* block_cnt;
     int batch, num_q_heads, num_kv_heads, group, block_size;
     int d_gate, max_blocks, max_sel, token_budget;
-    float rope_theta;
     unsigned int* status;
+    int* tickets;                   // [B*Hkv], zero between launches
+    double inv_freq[kMaxDGate / 2]; // rope_theta^(-2c/d_gate), computed on the host in double
 };
 // Launches the scoring kernels (unless scores_in is given) and the selection kernel.
 // Returns the number of kernels launched through *launched.
@@ -73,7 +78,7 @@ struct KcompParams {
     int rows_block_local;
     int first_block, num_blocks;    // first_block == -1: the block that just filled
     int batch, num_kv_heads, block_size, d_gate, max_blocks;
-    float rope_theta;
+    double inv_freq[kMaxDGate / 2];
 };
 cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* launched);
 

@@ -1,6 +1,6 @@
 // K compression cache update (Eq. 1b; Sec. 3.2): per block, max/min/mean pooling of the
 // pre-RoPE keys over the block's rows, projection by W_k, RoPE at the block's first token,
-// bf16 store.  One CTA handles up to kBlocksPerCta consecutive blocks of one (sequence,
+// bf16 store.  In the bulk build one CTA handles four consecutive blocks of one (sequence,
 // KV head) so that every W_k element fetched is used for all of them.
 #include "seer_device.cuh"
 #include "seer_internal.h"
@@ -9,31 +9,51 @@ namespace seer {
 
 namespace {
 
-constexpr int kBlocksPerCta = 4;
 constexpr int kKcThreads = 256;
-constexpr int kMaxDGate = 256;
+constexpr int kKcWarps = kKcThreads / 32;
+constexpr int kInChunks = 3 * kHeadDim / 8;          // 48 pieces of 16 B per W_k row
 
+// grid (block groups, B*Hkv, row splits).  NB = blocks per CTA (4 for the bulk build, 1 for the
+// per-step append, where the output rows are split over gridDim.z CTAs instead so that the
+// one block's latency chain is short).  Every warp owns rotary pairs (c, c + d_gate/2), two at
+// a time: their four W_k rows are requested before the pooling starts.
+template <int NB>
 __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) {
-    __shared__ float red[kKcThreads / 32][3][kHeadDim];                 // per-warp pooled partials
-    __shared__ __align__(16) float feat[kBlocksPerCta][3 * kHeadDim];   // [max | min | avg]
-    __shared__ float y[kBlocksPerCta][kMaxDGate];
-    __shared__ int blk_of[kBlocksPerCta];
+    __shared__ float red[kKcWarps][3][kHeadDim];                   // per-warp pooled partials
+    __shared__ __align__(16) float feat[NB][3 * kHeadDim];         // [max | min | avg]
 
     const int u = blockIdx.y, i = u / p.num_kv_heads, h = u % p.num_kv_heads;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int L = p.seq_lens[i];
     const int b = p.block_size;
-    const int complete = L > 0 ? L / b : 0;           // blocks with all b rows present
+    const int half = p.d_gate / 2;
+    const int pps = half / gridDim.z;                 // rotary pairs per row split
+    const int pair_base = blockIdx.z * pps;
 
+    // first batch of W_k rows (does not depend on anything else)
+    uint4 wv[4][2];
+    auto load_rows = [&](int pb) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int c = min(pair_base + pb + (k & 1), half - 1);
+            const int r = c + (k >> 1) * half;
+            const uint4* wrow = reinterpret_cast<const uint4*>(p.w_k + ((size_t)h * p.d_gate + r) * 3 * kHeadDim);
+            wv[k][0] = __ldg(wrow + lane);
+            wv[k][1] = lane < 16 ? __ldg(wrow + 32 + lane) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+    load_rows(warp * 2);
+
+    const int L = p.seq_lens[i];
+    const int complete = L > 0 ? L / b : 0;           // blocks with all b rows present
     int nb = 0;                                       // blocks this CTA really handles
     int j_first;
     if (p.first_block < 0) {
         j_first = complete - 1;
         nb = (blockIdx.x == 0 && L > 0 && L % b == 0 && j_first < p.max_blocks) ? 1 : 0;
     } else {
-        j_first = p.first_block + blockIdx.x * kBlocksPerCta;
+        j_first = p.first_block + blockIdx.x * NB;
         const int j_end = min(min(p.first_block + p.num_blocks, complete), p.max_blocks);
-        nb = max(0, min(kBlocksPerCta, j_end - j_first));
+        nb = max(0, min(NB, j_end - j_first));
     }
     if (nb == 0) return;
 
@@ -47,6 +67,7 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
         float mx[8], mn[8], sm[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) { mx[c] = -INFINITY; mn[c] = INFINITY; sm[c] = 0.f; }
+#pragma unroll 4
         for (int r = rgrp; r < b; r += 16) {
             const uint4 v = __ldg(reinterpret_cast<const uint4*>(
                 p.k_nope + base + (row0 + r) * p.stride_token + 8 * cchunk));
@@ -77,7 +98,7 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
         if (tid < kHeadDim) {
             float a = -INFINITY, m2 = INFINITY, s = 0.f;
 #pragma unroll
-            for (int w2 = 0; w2 < kKcThreads / 32; ++w2) {
+            for (int w2 = 0; w2 < kKcWarps; ++w2) {
                 a = fmaxf(a, red[w2][0][tid]);
                 m2 = fminf(m2, red[w2][1][tid]);
                 s += red[w2][2][tid];
@@ -86,63 +107,76 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
             feat[q][kHeadDim + tid] = m2;
             feat[q][2 * kHeadDim + tid] = s / (float)b;
         }
-        if (tid == 0) blk_of[q] = j;
         __syncthreads();
     }
-    for (int q = nb; q < kBlocksPerCta; ++q)
+    for (int q = nb; q < NB; ++q)
         for (int c = tid; c < 3 * kHeadDim; c += kKcThreads) feat[q][c] = 0.f;
     __syncthreads();
 
-    // projection: one warp per output row, all blocks of the CTA at once
-    const int in_chunks = 3 * kHeadDim / 8;           // 48 x 16 B per W_k row
-    for (int r = warp; r < p.d_gate; r += kKcThreads / 32) {
-        const uint4* wrow = reinterpret_cast<const uint4*>(p.w_k + ((size_t)h * p.d_gate + r) * 3 * kHeadDim);
-        float acc[kBlocksPerCta];
+    // this lane's pieces of the features, all blocks (reused by every row)
+    float fr[2][NB][8];
 #pragma unroll
-        for (int q = 0; q < kBlocksPerCta; ++q) acc[q] = 0.f;
-        for (int ch = lane; ch < in_chunks; ch += 32) {
-            const uint4 wv = __ldg(wrow + ch);
-            const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&wv);
-            float wf[8];
+    for (int part = 0; part < 2; ++part) {
+        const int ch = lane + 32 * part;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const float2 f = __bfloat1622float2(hh[c]);
-                wf[2 * c] = f.x; wf[2 * c + 1] = f.y;
-            }
+        for (int q = 0; q < NB; ++q)
 #pragma unroll
-            for (int q = 0; q < kBlocksPerCta; ++q) {
-                const float4 f0 = *reinterpret_cast<const float4*>(&feat[q][8 * ch]);
-                const float4 f1 = *reinterpret_cast<const float4*>(&feat[q][8 * ch + 4]);
-                acc[q] = fmaf(wf[0], f0.x, acc[q]); acc[q] = fmaf(wf[1], f0.y, acc[q]);
-                acc[q] = fmaf(wf[2], f0.z, acc[q]); acc[q] = fmaf(wf[3], f0.w, acc[q]);
-                acc[q] = fmaf(wf[4], f1.x, acc[q]); acc[q] = fmaf(wf[5], f1.y, acc[q]);
-                acc[q] = fmaf(wf[6], f1.z, acc[q]); acc[q] = fmaf(wf[7], f1.w, acc[q]);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < kBlocksPerCta; ++q) {
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], off);
-        }
-        if (lane == 0) {
-#pragma unroll
-            for (int q = 0; q < kBlocksPerCta; ++q) y[q][r] = acc[q];
-        }
+            for (int c = 0; c < 8; ++c) fr[part][q][c] = ch < kInChunks ? feat[q][8 * ch + c] : 0.f;
     }
-    __syncthreads();
 
-    // RoPE at the position of the block's first token, then the bf16 store
-    const int half = p.d_gate / 2;
-    for (int x = tid; x < nb * half; x += kKcThreads) {
-        const int q = x / half, c = x % half;
-        const int j = blk_of[q];
-        const double ang = (double)j * (double)b * pow((double)p.rope_theta, -2.0 * (double)c / (double)p.d_gate);
-        double sn, cs;
-        sincos(ang, &sn, &cs);
-        const double a = y[q][c], bb = y[q][c + half];
-        __nv_bfloat16* dst = p.kcomp + ((size_t)u * p.max_blocks + j) * p.d_gate;
-        dst[c] = __double2bfloat16(a * cs - bb * sn);
-        dst[c + half] = __double2bfloat16(bb * cs + a * sn);
+    for (int pb = warp * 2; pb < pps; pb += kKcWarps * 2) {
+        float acc[4][NB];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+#pragma unroll
+            for (int q = 0; q < NB; ++q) acc[k][q] = 0.f;
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&wv[k][part]);
+                float wf[8];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float2 f = __bfloat1622float2(hh[c]);
+                    wf[2 * c] = f.x; wf[2 * c + 1] = f.y;
+                }
+#pragma unroll
+                for (int q = 0; q < NB; ++q) {
+                    float a = acc[k][q];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) a = fmaf(wf[c], fr[part][q][c], a);
+                    acc[k][q] = a;
+                }
+            }
+        }
+        if (pb + kKcWarps * 2 < pps) load_rows(pb + kKcWarps * 2);     // next batch on its way
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int q = 0; q < NB; ++q)
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc[k][q] += __shfl_xor_sync(0xffffffffu, acc[k][q], off);
+        // RoPE at the position of the block's first token, then the bf16 store:
+        // lane (2q + e) finishes pair e of block q
+        if (lane < 2 * NB) {
+            const int q = lane >> 1, e = lane & 1;
+            const int c = pair_base + pb + e;
+            if (q < nb && pb + e < pps) {
+                float a = 0.f, bb = 0.f;
+#pragma unroll
+                for (int qq = 0; qq < NB; ++qq) {
+                    if (qq == q) {
+                        a = e ? acc[1][qq] : acc[0][qq];
+                        bb = e ? acc[3][qq] : acc[2][qq];
+                    }
+                }
+                const int j = j_first + q;
+                float sn, cs;
+                rope_sincos((double)j * (double)b, p.inv_freq[c], &sn, &cs);
+                __nv_bfloat16* dst = p.kcomp + ((size_t)u * p.max_blocks + j) * p.d_gate;
+                dst[c] = __float2bfloat16(a * cs - bb * sn);
+                dst[c + half] = __float2bfloat16(bb * cs + a * sn);
+            }
+        }
     }
 }
 
@@ -150,10 +184,16 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
 
 cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* launched) {
     const int U = p.batch * p.num_kv_heads;
-    const int gx = p.first_block < 0 ? 1 : (p.num_blocks + kBlocksPerCta - 1) / kBlocksPerCta;
     *launched = 0;
-    if (gx <= 0 || U <= 0) return cudaSuccess;
-    kcomp_kernel<<<dim3(gx, U), kKcThreads, 0, stream>>>(p);
+    if (U <= 0) return cudaSuccess;
+    if (p.first_block < 0) {
+        // one block per unit: split the d_gate/2 rotary pairs over 4 CTAs (16, 8 or 32 pairs each)
+        kcomp_kernel<1><<<dim3(1, U, 4), kKcThreads, 0, stream>>>(p);
+    } else {
+        const int gx = (p.num_blocks + 3) / 4;
+        if (gx <= 0) return cudaSuccess;
+        kcomp_kernel<4><<<dim3(gx, U, 1), kKcThreads, 0, stream>>>(p);
+    }
     *launched = 1;
     return cudaGetLastError();
 }

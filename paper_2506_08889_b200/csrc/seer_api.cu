@@ -4,6 +4,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -43,6 +44,8 @@ struct seer_ctx {
     int map_used;
     int map_next;
     uint64_t launches;
+    unsigned int generation;    // stamps the partials of a decode launch
+    int pool_div;               // decode scheduling: share of tiles handed out dynamically
     char err[512];
 };
 
@@ -62,24 +65,37 @@ seer_status fail(seer_ctx* ctx, seer_status s, const char* fmt, ...) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Workspace: [status][scheduler counters][decode tickets][gate tickets] at fixed offsets, then one
+// scratch region that a decode call uses for its partials and a gate call for its gate query and
+// scores (calls on a context are ordered, and neither kind of scratch outlives its call).
+constexpr int kMaxGridCtas = 148 * 2 * 4;   // generous bound on the decode grid, for workspace sizing
+
 struct WsLayout {
-    size_t tickets, gate_tickets, part_o, part_ml, q_gate, scores, total;
+    size_t sched, steal, tickets, gate_tickets, prefix, scratch;
+    size_t part_o, part_ml, q_gate, scores, total;
 };
 
 WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks) {
     WsLayout w;
     size_t off = kStatusBytes;
+    w.sched = off; off += 256;
+    w.steal = off; off = align_up(off + sizeof(int) * (size_t)kMaxGridCtas, 256);
     w.tickets = off; off = align_up(off + sizeof(int) * (size_t)num_units, 256);
     w.gate_tickets = off; off = align_up(off + sizeof(int) * (size_t)num_units, 256);
-    w.part_o = off;  off = align_up(off + sizeof(float) * (size_t)slots * kMaxGroup * kHeadDim, 256);
-    w.part_ml = off; off = align_up(off + sizeof(float) * (size_t)slots * 2 * kMaxGroup, 256);
-    w.q_gate = off;  off = align_up(off + sizeof(float) * (size_t)num_units * (size_t)(d_gate > 0 ? d_gate : 0), 256);
-    w.scores = off;  off = align_up(off + sizeof(float) * (size_t)num_units * (size_t)(max_blocks > 0 ? max_blocks : 0), 256);
-    w.total = off;
+    w.prefix = off; off = align_up(off + sizeof(int) * ((size_t)num_units + 1), 256);
+    w.scratch = off;
+    // decode view of the scratch
+    size_t d = off;
+    w.part_ml = d; d = align_up(d + sizeof(float) * (size_t)slots * 32, 256);
+    w.part_o = d;  d = align_up(d + sizeof(float) * (size_t)slots * kMaxGroup * kHeadDim, 256);
+    // gate view of the scratch
+    size_t g = off;
+    w.q_gate = g;  g = align_up(g + sizeof(float) * (size_t)num_units * (size_t)(d_gate > 0 ? d_gate : 0), 256);
+    w.scores = g;  g = align_up(g + sizeof(float) * (size_t)num_units * (size_t)(max_blocks > 0 ? max_blocks : 0), 256);
+    w.total = d > g ? d : g;
     return w;
 }
 
-constexpr int kMaxGridCtas = 148 * 2 * 4;   // generous bound used for workspace sizing only
 
 seer_status check_shape(seer_ctx* ctx, const seer_shape* s) {
     if (!s) return fail(ctx, SEER_ERR_INVALID_ARG, "shape is NULL");
@@ -170,8 +186,9 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     long long max_tiles = sparse ? (long long)U * max_sel * tpb
                                  : (long long)U * ((kv->max_seq_len + kTileTokens - 1) / kTileTokens);
     int grid = ctx->num_sms * per_sm;
+    if (grid > kMaxGridCtas) grid = kMaxGridCtas;
     if (max_tiles < grid) grid = (int)(max_tiles > 0 ? max_tiles : 1);
-    const int slots = grid + U;
+    const int slots = decode_max_intervals(grid) + U;
     const WsLayout w = ws_layout(U, slots, 0, 0);
     if (w.total > ctx->ws_bytes)
         return fail(ctx, SEER_ERR_WORKSPACE, "workspace %zu bytes, call needs %zu", ctx->ws_bytes, w.total);
@@ -210,9 +227,14 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.tiles_per_block = tpb;
     p.num_units = U;
     p.max_blocks_cap = (kv->max_seq_len + kTileTokens - 1) / kTileTokens;
+    p.pool_div = ctx->pool_div;
     p.scale_log2 = shape->sm_scale * 1.4426950408889634f;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
     p.tickets = reinterpret_cast<int*>(ctx->ws + w.tickets);
+    p.sched = reinterpret_cast<int*>(ctx->ws + w.sched);
+    p.prefix = reinterpret_cast<int*>(ctx->ws + w.prefix);
+    p.steal = reinterpret_cast<int*>(ctx->ws + w.steal);
+    p.generation = ++ctx->generation;
     p.part_o = reinterpret_cast<float*>(ctx->ws + w.part_o);
     p.part_ml = reinterpret_cast<float*>(ctx->ws + w.part_ml);
 
@@ -251,6 +273,8 @@ seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes) {
         return SEER_ERR_CUDA;
     }
     ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    ctx->pool_div = 4;
+    if (const char* e = getenv("SEER_DECODE_POOL_DIV")) ctx->pool_div = atoi(e);
     ctx->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)64 << 20;
     if (ctx->ws_bytes < 4096) ctx->ws_bytes = 4096;
     if (cudaMalloc(reinterpret_cast<void**>(&ctx->ws), ctx->ws_bytes) != cudaSuccess) {
@@ -293,6 +317,7 @@ uint64_t seer_launch_count(const seer_ctx* ctx) { return ctx ? ctx->launches : 0
 #ifdef SEER_DECODE_TRACE
 /* diagnostic builds only: device address of the per-CTA time stamps of the last decode launch */
 void* seer_debug_trace_ptr(seer_ctx* ctx) { return ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)); }
+int seer_debug_ctas_per_sm(int sparse, int paged) { return decode_ctas_per_sm(sparse != 0, paged != 0); }
 #endif
 
 seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
@@ -305,7 +330,7 @@ seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "status read: %s", cudaGetErrorString(e));
     if (word & DEV_TIMEOUT) {
-        // a piece that gave up may have left tickets behind: clear them for the next call
+        // a CTA that gave up may have left tickets or scheduler counters behind: clear them
         cudaMemsetAsync(ctx->ws + kStatusBytes, 0, ctx->ws_bytes < (1u << 20) ? ctx->ws_bytes - kStatusBytes
                                                                               : (1u << 20) - kStatusBytes, s);
         cudaStreamSynchronize(s);
@@ -318,7 +343,7 @@ seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
 size_t seer_workspace_bytes(const seer_shape* shape, int max_blocks, int d_gate) {
     if (!shape || shape->batch <= 0 || shape->num_kv_heads <= 0) return 0;
     const int U = shape->batch * shape->num_kv_heads;
-    return ws_layout(U, kMaxGridCtas + U, d_gate, max_blocks).total;
+    return ws_layout(U, decode_max_intervals(kMaxGridCtas) + U, d_gate, max_blocks).total;
 }
 
 seer_status seer_dense_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q, void* out,
@@ -352,7 +377,7 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
         if (!(gate->rope_theta > 0.f)) return fail(ctx, SEER_ERR_INVALID_ARG, "rope_theta must be positive");
     }
     const int U = shape->batch * shape->num_kv_heads;
-    const WsLayout w = ws_layout(U, kMaxGridCtas + U, scores_in ? 0 : gate->d_gate, scores_in ? 0 : gate->max_blocks);
+    const WsLayout w = ws_layout(U, 0, scores_in ? 0 : gate->d_gate, scores_in ? 0 : gate->max_blocks);
     if (w.total > ctx->ws_bytes)
         return fail(ctx, SEER_ERR_WORKSPACE, "workspace %zu bytes, call needs %zu", ctx->ws_bytes, w.total);
     cudaError_t ce = cudaSetDevice(ctx->device);

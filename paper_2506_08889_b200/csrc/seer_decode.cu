@@ -3,14 +3,24 @@
 //
 // Work decomposition.  A "unit" is one (sequence, KV head) pair; its work is the list of
 // 64-token tiles of its selected blocks (sparse) or of its whole sequence (dense).  All
-// units' tile lists are laid end to end and cut into `gridDim.x` equal contiguous ranges,
-// one per CTA, so every CTA streams the same number of KV bytes whatever the per-unit
-// selection counts are.  A CTA whose range covers a unit completely writes the final
-// output; otherwise it writes an un-normalised partial (o, max, sum) and takes a ticket;
-// the CTA that draws the last ticket of a unit merges the partials (log-sum-exp combine).
-// There is no spin-wait anywhere: the merge is done by whoever finishes last.
+// units' tile lists are laid end to end (T tiles) and cut into one equal contiguous range per
+// CTA.  The first three quarters of a range are its CTA's static share; the last quarter is
+// cut into chunks that double in size towards the end of the range (two tiles ... 1/8 of the
+// range).  The owner of a range claims its chunks from the front, so its work stays one
+// contiguous run; a CTA that has finished its own range steals other ranges' chunks from the
+// back, the big ones first, as in steal-half work stealing.
+// SMs that get less memory bandwidth than others thus shed work to faster ones and all finish
+// together, while a unit is cut into few pieces.  Claims are single atomic adds on a per-range
+// counter; nobody ever waits for another CTA.
 //
-// Inside a CTA: one producer warp walks the range, turns each tile into TMA box loads
+// A piece is a maximal run of one unit's tiles that one CTA processes in one go.  A piece that
+// covers its unit completely writes the final output.  Any other piece writes an un-normalised
+// partial (o, max, sum), stamped with the launch's generation number, into the slot of the
+// interval it starts in.  When a CTA has finished streaming it adds the tile counts of its pieces
+// to their units' counters; whoever completes a unit's count merges that unit's partials
+// (log-sum-exp combine over the valid slots among the unit's intervals), with all of its warps.
+//
+// Inside a CTA: one producer warp walks the intervals, turns each tile into TMA box loads
 // (K and V, 2 x 64x64 bf16 boxes each, 128-byte swizzle) into a ring of shared-memory
 // stages, and passes per-tile metadata beside the data.  Four consumer warps each own 16
 // of a tile's 64 tokens and keep private online-softmax state (running max, sum, and the
@@ -28,32 +38,63 @@ namespace {
 
 constexpr int kStages = 3;
 constexpr int kConsumerWarps = 4;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;
 constexpr int kHalfTileBytes = kTileTokens * 128;          // 64 rows x 128 B (64 bf16 channels)
 constexpr int kTileBytes = 2 * kHalfTileBytes;             // one K or V tile: 16 KiB
 constexpr int kStageBytes = 2 * kTileBytes;                // K + V
 constexpr int kMergeStride = 132;                          // floats per head row (bank spread)
+constexpr int kMaxPieces = 32;                             // partial pieces a CTA can hold back to its end
+constexpr int kListInts = 2 * kStageBytes / 4;              // slot numbers that fit in two stage buffers
+constexpr int kMaxSteals = 14;                             // chunks a CTA may take from other ranges
+constexpr int kMinChunk = 2;                               // smallest dynamic chunk, in tiles
+constexpr int kMinStaticTilesPerCta = 8;                   // below this everything is static
 
 struct StageMeta {
-    int nvalid;        // tokens of this tile that exist (0 = nothing was loaded)
+    int nvalid;        // tokens of this tile that exist (0 = nothing was loaded); -1 = end of stream
     int unit;          // (sequence, KV head) index
-    int last;          // last tile of this CTA's piece of the unit
+    int flags;         // bit 0: first tile of a piece
     int unit_first;    // global index of the unit's first tile
     int unit_tiles;    // tiles of the unit
+    int interval;      // interval this tile belongs to
+};
+
+struct Piece {
+    int unit, tiles, unit_first, unit_tiles;   // a partial this CTA wrote; merged: first_slot, n_slots
+};
+
+// Geometry of the intervals, identical in every CTA (derived from T and gridDim.x).  Range c is
+// [c*T/G, (c+1)*T/G); with len its length, b its end and ts = b - (len>>2) the start of its
+// tail, its intervals are
+//   0: [a, ts)   1: [ts, ts + (len>>(R+1)))   2: [.., ts + (len>>R))  ...  R: [ts + (len>>3), b),
+// i.e. the tail's chunks double in size towards the end of the range.
+struct Schedule {
+    int T, G;                      // tiles, ranges (G <= T)
+    int R;                         // dynamic chunks per range (0: everything is static)
 };
 
 struct __align__(1024) Smem {
     unsigned char stage[kStages][kStageBytes];
-    float merge_o[kConsumerWarps - 1][kMaxGroup][kMergeStride];
-    float merge_ml[2][kConsumerWarps][2][kMaxGroup];   // double-buffered by piece parity
+    float merge_o[kConsumerWarps - 1][kMaxGroup][kMergeStride];   // warps 1..3 -> warp 0
+    float merge_ml[kConsumerWarps - 1][2][kMaxGroup];
     uint64_t full[kStages];
     uint64_t empty[kStages];
-    uint64_t merge_bar[2];
+    uint64_t merge_bar[2];           // [0]: scratch filled (3 arrivals), [1]: scratch free again / end sync
+    uint64_t end_bar;                // all consumer warps: streams over, the list of combines is final
+    uint64_t list_bar;               // all consumer warps: the lists of valid slots are written
+    volatile int issued;             // tiles whose metadata the producer has written so far
     StageMeta meta[kStages];
+    Schedule sched;
+    Piece pieces[kMaxPieces];
+    int pieces_n;
     int scan_warp[kThreads / 32];
     int start_unit;
     int start_off;
 };
+
+// two CTAs per SM: 2 * (sizeof(Smem) + 1 KiB alignment slack + 1 KiB reserved by the system) must
+// fit in the SM's 228 KiB
+static_assert(sizeof(Smem) + 1024 <= 113 * 1024, "decode kernel no longer fits two CTAs per SM");
 
 // Programmatic dependent launch: the kernel may start while its predecessor in the stream is
 // still running; nothing the predecessor writes is read before pdl_wait().
@@ -84,10 +125,45 @@ __device__ __forceinline__ int tiles_of(const DecodeParams& p, int u) {
     }
 }
 
-// CTA that owns global tile t when T tiles are cut into G equal contiguous ranges
+// Range that owns tile t when T tiles are cut into G equal contiguous ranges
 // (range c = [floor(c*T/G), floor((c+1)*T/G)) ).
-__device__ __forceinline__ int cta_of(long long t, long long T, long long G) {
+__device__ __forceinline__ int range_of(long long t, long long T, long long G) {
     return (int)(((t + 1) * G - 1) / T);
+}
+__device__ __forceinline__ int range_begin(const Schedule& s, int c) { return (int)(((long long)c * s.T) / s.G); }
+
+__device__ void build_schedule(Schedule& s, int T, int grid, int pool_div) {
+    s.T = T;
+    s.G = max(1, min(grid, T));
+    s.R = 0;
+    const int len = T / s.G;                        // shortest range
+    if (pool_div > 0 && len >= kMinStaticTilesPerCta) {
+        int R = 1;
+        while (R < kMaxRounds && (len >> (R + 2)) >= kMinChunk) ++R;
+        s.R = R;
+    }
+}
+
+// Interval j (0 = static share, 1..R = chunks, small ones first) of range c.
+__device__ __forceinline__ void interval_range(const Schedule& s, int c, int j, int* begin, int* end) {
+    const int a = range_begin(s, c), b = range_begin(s, c + 1), len = b - a;
+    if (s.R == 0) { *begin = a; *end = b; return; }
+    const int ts = b - (len >> 2);                  // the tail: last quarter of the range
+    if (j == 0) { *begin = a; *end = ts; return; }
+    *begin = j == 1 ? ts : ts + (len >> (s.R + 3 - j));
+    *end = ts + (len >> (s.R + 2 - j));
+}
+
+// Number (c * (R+1) + j, increasing with the tile position) of the interval that holds tile t.
+__device__ __forceinline__ int interval_of(const Schedule& s, int t) {
+    const int c = range_of(t, s.T, s.G);
+    if (s.R == 0) return c;
+    const int a = range_begin(s, c), b = range_begin(s, c + 1), len = b - a;
+    const int off = t - (b - (len >> 2));           // position inside the tail
+    if (off < 0) return c * (s.R + 1);
+    int j = 1;
+    while (j < s.R && off >= (len >> (s.R + 2 - j))) ++j;
+    return c * (s.R + 1) + j;
 }
 
 __device__ __forceinline__ void write_zero_unit(const DecodeParams& p, int u) {
@@ -97,6 +173,85 @@ __device__ __forceinline__ void write_zero_unit(const DecodeParams& p, int u) {
         for (int c = 0; c < kHeadDim; ++c) p.out[row * kHeadDim + c] = __float2bfloat16(0.f);
         if (p.lse) p.lse[row] = -INFINITY;
     }
+}
+
+constexpr int kMlStride = 32;      // floats per slot in part_ml: [0..7] max, [8..15] sum, [16] generation
+
+// Log-sum-exp combine of one unit's partials by the CTA's consumer threads.  Thread t takes head
+// t/16, channels 8*(t%16) .. +7 of every partial.
+struct MergeState {
+    float M, lsum, acc[8];
+};
+__device__ __forceinline__ void merge_init(MergeState& st) {
+    st.M = -INFINITY;
+    st.lsum = 0.f;
+#pragma unroll
+    for (int x = 0; x < 8; ++x) st.acc[x] = 0.f;
+}
+// Adds the partials in the n listed slots.  A batch of partials is loaded in full before any
+// arithmetic, so a batch costs one round trip to L2.
+__device__ void merge_accumulate(const DecodeParams& p, MergeState& st, const int* slots, int n, int t) {
+    const int hh = t >> 4, d0 = 8 * (t & 15);
+    constexpr int kB = 8;
+    for (int s0 = 0; s0 < n; s0 += kB) {
+        float ms[kB], ls[kB];
+        float4 va[kB], vb[kB];
+#pragma unroll
+        for (int k = 0; k < kB; ++k) {
+            const size_t sl = (size_t)slots[min(s0 + k, n - 1)];
+            const float* pm = p.part_ml + sl * kMlStride;
+            const float4* qo = reinterpret_cast<const float4*>(p.part_o + sl * (kMaxGroup * kHeadDim) +
+                                                               hh * kHeadDim + d0);
+            ms[k] = __ldcg(pm + hh);
+            ls[k] = __ldcg(pm + kMaxGroup + hh);
+            va[k] = __ldcg(qo);
+            vb[k] = __ldcg(qo + 1);
+        }
+#pragma unroll
+        for (int k = 0; k < kB; ++k) {
+            if (s0 + k < n && ms[k] != -INFINITY) {
+                const float Mn = fmaxf(st.M, ms[k]);
+                const float fo = (st.M == -INFINITY) ? 0.f : fast_exp2(st.M - Mn);
+                const float fn = fast_exp2(ms[k] - Mn);
+                st.M = Mn;
+                st.lsum = st.lsum * fo + ls[k] * fn;
+                st.acc[0] = st.acc[0] * fo + va[k].x * fn; st.acc[1] = st.acc[1] * fo + va[k].y * fn;
+                st.acc[2] = st.acc[2] * fo + va[k].z * fn; st.acc[3] = st.acc[3] * fo + va[k].w * fn;
+                st.acc[4] = st.acc[4] * fo + vb[k].x * fn; st.acc[5] = st.acc[5] * fo + vb[k].y * fn;
+                st.acc[6] = st.acc[6] * fo + vb[k].z * fn; st.acc[7] = st.acc[7] * fo + vb[k].w * fn;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void merge_finalize(const DecodeParams& p, const MergeState& st, int u, int t) {
+    const int hh = t >> 4, d0 = 8 * (t & 15);
+    if (hh < p.group) {
+        const int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
+        const size_t row = (size_t)i * p.num_q_heads + (size_t)h * p.group + hh;
+        const float inv = st.lsum > 0.f ? 1.f / st.lsum : 0.f;
+        uint4 pk;
+        pk.x = pack_bf16x2(st.acc[0] * inv, st.acc[1] * inv);
+        pk.y = pack_bf16x2(st.acc[2] * inv, st.acc[3] * inv);
+        pk.z = pack_bf16x2(st.acc[4] * inv, st.acc[5] * inv);
+        pk.w = pack_bf16x2(st.acc[6] * inv, st.acc[7] * inv);
+        *reinterpret_cast<uint4*>(p.out + row * kHeadDim + d0) = pk;
+        if (p.lse && (t & 15) == 0)
+            p.lse[row] = st.lsum > 0.f ? (st.M + log2f(st.lsum)) * 0.6931471805599453f : -INFINITY;
+    }
+}
+// One warp: the slots among [first, first + n_slots) that carry this launch's generation stamp,
+// written to `list` in order; returns how many.
+__device__ __forceinline__ int scan_valid_slots(const DecodeParams& p, int first, int n_slots, int* list, int lane) {
+    int n = 0;
+    for (int s0 = 0; s0 < n_slots; s0 += 32) {
+        const int sl = first + s0 + lane;
+        const bool ok = s0 + lane < n_slots &&
+                        __float_as_uint(__ldcg(p.part_ml + (size_t)sl * kMlStride + 16)) == p.generation;
+        const unsigned m = __ballot_sync(0xffffffffu, ok);
+        if (ok) list[n + __popc(m & ((1u << lane) - 1u))] = sl;
+        n += __popc(m);
+    }
+    return n;
 }
 
 template <bool SPARSE, bool PAGED>
@@ -115,22 +270,24 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             mbar_init(&sm.full[s], 1);
             mbar_init(&sm.empty[s], kConsumerWarps);
         }
-        mbar_init(&sm.merge_bar[0], kConsumerWarps);
-        mbar_init(&sm.merge_bar[1], kConsumerWarps);
+        mbar_init(&sm.merge_bar[0], kConsumerWarps - 1);
+        mbar_init(&sm.merge_bar[1], 1);
+        mbar_init(&sm.end_bar, kConsumerWarps);
+        mbar_init(&sm.list_bar, kConsumerWarps);
         mbar_fence_init();
+        sm.issued = 0;
         sm.start_unit = U;
         sm.start_off = 0;
+        sm.pieces_n = 0;
     }
     if (warp == kConsumerWarps && lane == 0) {
         tma_prefetch_desc(&map_k);
         tma_prefetch_desc(&map_v);
     }
 
-    if (tid == 0) SEER_STAMP(0);
     pdl_wait();
-    if (tid == 0) SEER_STAMP(1);
 
-    // ---- every CTA sums the units' tile counts and finds where its own range starts ----
+    // ---- every CTA sums the units' tile counts and finds where its static share starts ----
     const int per = (U + kThreads - 1) / kThreads;
     const int u_lo = min(U, tid * per), u_hi = min(U, u_lo + per);
     int mine = 0;
@@ -147,133 +304,232 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     }
     if (lane == 31) sm.scan_warp[warp] = incl;
     __syncthreads();
-    int warp_base = 0, T_i = 0;
+    int warp_base = 0, T = 0;
 #pragma unroll
     for (int w = 0; w < kThreads / 32; ++w) {
         int v = sm.scan_warp[w];
         if (w < warp) warp_base += v;
-        T_i += v;
+        T += v;
     }
-    const long long T = T_i;
-    if (T == 0) return;
-    // never more ranges than tiles: every range in use is non-empty, so a unit's pieces are
-    // exactly the CTAs between the owners of its first and last tile
-    const long long G = min((long long)gridDim.x, T);
-    if (cta >= G) return;
+    if (tid == 0) build_schedule(sm.sched, T, gridDim.x, p.pool_div);
+    __syncthreads();
+    const Schedule& sc = sm.sched;
+    int t_begin = 0, t_end = 0;                      // this CTA's static share
+    if (T > 0 && cta < sc.G) interval_range(sc, cta, 0, &t_begin, &t_end);
     const int excl = warp_base + incl - mine;
-    const int t_begin = (int)((cta * T) / G), t_end = (int)(((cta + 1) * T) / G);
-    if (t_begin >= t_end) return;
-    if (mine > 0 && excl <= t_begin && t_begin < excl + mine) {
+    {
+        // prefix sums of the tile counts, for locating a tile's unit later.  Every CTA writes
+        // the same values; a CTA only relies on its own writes being visible to itself.
+        const bool want_start = t_begin < t_end;
         int acc = excl;
         for (int u = u_lo; u < u_hi; ++u) {
-            int t = tiles_of<SPARSE>(p, u);
-            if (t_begin < acc + t) {
+            const int t = tiles_of<SPARSE>(p, u);
+            if (sc.R > 0) p.prefix[u] = acc;
+            if (want_start && t > 0 && acc <= t_begin && t_begin < acc + t) {
                 sm.start_unit = u;
                 sm.start_off = t_begin - acc;
-                break;
             }
             acc += t;
         }
+        if (sc.R > 0 && tid == 0) p.prefix[U] = T;
     }
     __syncthreads();
-    const int n_tiles = t_end - t_begin;
-    if (tid == 0) SEER_STAMP(2);
 
     if (warp == kConsumerWarps) {
         // =========================== producer warp ====================================
-        int cu = sm.start_unit, ce = sm.start_off;
-        if (cu >= U) return;
-        int cut = tiles_of<SPARSE>(p, cu);
-        int cpu = t_begin - ce;
+        // position in the units' tile lists: unit cu, whose first tile is global tile cpu and
+        // which has cut tiles
+        int cu = 0, cpu = 0, cut = 0;
+        if (t_begin < t_end) {
+            cu = sm.start_unit;
+            cut = cu < U ? tiles_of<SPARSE>(p, cu) : 0;
+            cpu = t_begin - sm.start_off;
+        }
         int it = 0;
-        for (int t = 0; t < n_tiles; t += 32) {
-            const int n_chunk = min(32, n_tiles - t);
-            // deal the next n_chunk tiles to lanes, walking over unit boundaries
-            int my_u = -1, my_e = 0, my_ut = 0, my_pu = 0;
-            int base = 0;
-            while (base < n_chunk) {
-                int avail = cut - ce;
-                if (avail <= 0) {
-                    cpu += cut;
-                    ++cu;
-                    ce = 0;
-                    if (cu >= U) { cut = 0; break; }
-                    cut = tiles_of<SPARSE>(p, cu);
-                    continue;
+        int iv_begin = t_begin, iv_end = t_end, iv_id = cta * (sc.R + 1);
+        bool have = t_begin < t_end;
+        bool own = cta < sc.G;           // still claiming chunks of the own range
+        bool contiguous = true;          // the next interval continues the previous one
+        int fails = 0, steals = 0;
+        const int R = sc.R, G = sc.G;
+        for (;;) {
+            if (!have) {
+                if (R == 0 || T == 0) break;
+                int c, j;
+                if (own) {
+                    // own range, from the front: low half of the counter counts front claims
+                    int old = 0;
+                    if (lane == 0) old = atomicAdd(&p.steal[cta], 1);
+                    old = __shfl_sync(0xffffffffu, old, 0);
+                    if ((old & 0xffff) + (old >> 16) >= R) { own = false; continue; }
+                    c = cta;
+                    j = (old & 0xffff) + 1;
+                    contiguous = true;
+                } else {
+                    // Somebody else's range, from the back.  Look at every range's claim counter
+                    // and go for the one with the most chunks left (its owner is the furthest
+                    // behind); ties are broken differently by every thief.
+                    if (fails >= 3 || steals >= kMaxSteals) break;
+                    int best = -1;
+                    for (int c0 = 0; c0 < G; c0 += 32) {
+                        const int cc = c0 + lane;
+                        if (cc < G && cc != cta) {
+                            const int st = __ldcg(p.steal + cc);
+                            const int left = R - (st & 0xffff) - (st >> 16);
+                            if (left > 0) {
+                                const int rot = (cc - cta + G) % G;          // this thief's order of preference
+                                best = max(best, (left << 20) | (0xfffff - min(rot, 0xfffff)));
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+                    if (best < 0) break;                                  // nothing left anywhere
+                    c = (cta + (0xfffff - (best & 0xfffff))) % G;
+                    int old = 0;
+                    if (lane == 0) old = atomicAdd(&p.steal[c], 1 << 16);
+                    old = __shfl_sync(0xffffffffu, old, 0);
+                    if ((old & 0xffff) + (old >> 16) >= R) { ++fails; continue; }
+                    fails = 0;
+                    ++steals;
+                    j = R - (old >> 16);
+                    contiguous = false;
                 }
-                int take = min(avail, n_chunk - base);
-                if (lane >= base && lane < base + take) {
-                    my_u = cu; my_e = ce + lane - base; my_ut = cut; my_pu = cpu;
+                interval_range(sc, c, j, &iv_begin, &iv_end);
+                iv_id = c * (R + 1) + j;
+                if (!contiguous) {
+                    // unit that holds tile iv_begin: 32-ary search in the prefix sums
+                    int lo = 0, hi = U;                       // prefix[lo] <= iv_begin < prefix[hi]
+                    while (hi - lo > 1) {
+                        const int step = (hi - lo + 31) / 32;
+                        const int cand = lo + min((lane + 1) * step, hi - lo);
+                        const int pv = cand < hi ? __ldcg(p.prefix + cand) : 0x7fffffff;
+                        const unsigned m = __ballot_sync(0xffffffffu, pv > iv_begin);
+                        const int f = __ffs(m) - 1;             // the last lane always votes yes
+                        const int new_hi = __shfl_sync(0xffffffffu, cand, f);
+                        const int new_lo = f == 0 ? lo : __shfl_sync(0xffffffffu, cand, f - 1);
+                        hi = new_hi;
+                        lo = new_lo;
+                    }
+                    cu = lo;
+                    cpu = __ldcg(p.prefix + lo);
+                    cut = __ldcg(p.prefix + lo + 1) - cpu;
+                    if (iv_begin < cpu || iv_begin >= cpu + cut) break;   // counts changed under us
                 }
-                base += take;
-                ce += take;
             }
-            // per-lane tile descriptor
-            int nvalid = 0, row = 0, outer = 0, head = 0, last = 0;
-            if (my_u >= 0) {
-                const int i = my_u / p.num_kv_heads;
-                head = my_u % p.num_kv_heads;
-                const int L = p.seq_lens[i];
-                int tok0 = 0;
-                if (SPARSE) {
-                    const int blk = p.block_idx[(size_t)my_u * p.max_sel + my_e / p.tiles_per_block];
-                    const int n_i = (L + p.block_size - 1) / p.block_size;
-                    if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
-                    if (blk >= 0 && blk < n_i) {
-                        tok0 = blk * p.block_size + (my_e % p.tiles_per_block) * kTileTokens;
+            const bool fresh = have || !contiguous;  // this interval starts a new piece
+            have = false;
+            int ce = iv_begin - cpu;                  // offset of the next tile inside unit cu
+            const int n_tiles = iv_end - iv_begin;
+            for (int t = 0; t < n_tiles; t += 32) {
+                const int n_chunk = min(32, n_tiles - t);
+                // deal the next n_chunk tiles to lanes, walking over unit boundaries
+                int my_u = -1, my_e = 0, my_ut = 0, my_pu = 0;
+                int base = 0;
+                while (base < n_chunk) {
+                    int avail = cut - ce;
+                    if (avail <= 0) {
+                        cpu += cut;
+                        ++cu;
+                        ce = 0;
+                        if (cu >= U) { cut = 0; break; }
+                        cut = tiles_of<SPARSE>(p, cu);
+                        continue;
+                    }
+                    int take = min(avail, n_chunk - base);
+                    if (lane >= base && lane < base + take) {
+                        my_u = cu; my_e = ce + lane - base; my_ut = cut; my_pu = cpu;
+                    }
+                    base += take;
+                    ce += take;
+                }
+                // per-lane tile descriptor
+                int nvalid = 0, row = 0, outer = 0, head = 0, flags = 0;
+                if (my_u >= 0) {
+                    const int i = my_u / p.num_kv_heads;
+                    head = my_u % p.num_kv_heads;
+                    const int L = p.seq_lens[i];
+                    int tok0 = 0;
+                    if (SPARSE) {
+                        const int blk = p.block_idx[(size_t)my_u * p.max_sel + my_e / p.tiles_per_block];
+                        const int n_i = (L + p.block_size - 1) / p.block_size;
+                        if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
+                        if (blk >= 0 && blk < n_i) {
+                            tok0 = blk * p.block_size + (my_e % p.tiles_per_block) * kTileTokens;
+                            nvalid = max(0, min(kTileTokens, L - tok0));
+                        }
+                    } else {
+                        tok0 = my_e * kTileTokens;
                         nvalid = max(0, min(kTileTokens, L - tok0));
                     }
-                } else {
-                    tok0 = my_e * kTileTokens;
-                    nvalid = max(0, min(kTileTokens, L - tok0));
-                }
-                if (PAGED) {
-                    if (nvalid > 0) {
-                        const int pg = p.page_table[(size_t)i * p.page_table_stride + tok0 / p.page_size];
-                        if (pg < 0 || pg >= p.num_pages) {
-                            raise_status(p.status, DEV_BAD_INDEX);
-                            nvalid = 0;
+                    if (PAGED) {
+                        if (nvalid > 0) {
+                            const int pg = p.page_table[(size_t)i * p.page_table_stride + tok0 / p.page_size];
+                            if (pg < 0 || pg >= p.num_pages) {
+                                raise_status(p.status, DEV_BAD_INDEX);
+                                nvalid = 0;
+                            }
+                            outer = pg;
+                            row = tok0 % p.page_size;
                         }
-                        outer = pg;
-                        row = tok0 % p.page_size;
-                    }
-                } else {
-                    outer = i;
-                    row = tok0;
-                }
-                last = (my_e == my_ut - 1) || (t + lane == n_tiles - 1);
-            } else if (lane < n_chunk) {
-                // the counts changed under us: keep the pipeline protocol, load nothing
-                my_u = 0; my_ut = 1; last = (t + lane == n_tiles - 1);
-                raise_status(p.status, DEV_BAD_INDEX);
-            }
-            for (int s = 0; s < n_chunk; ++s, ++it) {
-                const int s_nvalid = __shfl_sync(0xffffffffu, nvalid, s);
-                const int s_row = __shfl_sync(0xffffffffu, row, s);
-                const int s_outer = __shfl_sync(0xffffffffu, outer, s);
-                const int s_head = __shfl_sync(0xffffffffu, head, s);
-                const int s_last = __shfl_sync(0xffffffffu, last, s);
-                const int s_u = __shfl_sync(0xffffffffu, my_u, s);
-                const int s_pu = __shfl_sync(0xffffffffu, my_pu, s);
-                const int s_ut = __shfl_sync(0xffffffffu, my_ut, s);
-                if (lane == 0) {
-                    const int st = it % kStages;
-                    if (!mbar_wait(&sm.empty[st], ((it / kStages) & 1) ^ 1, p.status)) return;
-                    sm.meta[st] = StageMeta{s_nvalid, s_u, s_last, s_pu, s_ut};
-                    if (s_nvalid > 0) {
-                        unsigned char* dst = sm.stage[st];
-                        mbar_arrive_expect_tx(&sm.full[st], kStageBytes);
-                        tma_load_4d(dst, &map_k, &sm.full[st], 0, s_row, s_head, s_outer);
-                        tma_load_4d(dst + kHalfTileBytes, &map_k, &sm.full[st], 64, s_row, s_head, s_outer);
-                        tma_load_4d(dst + kTileBytes, &map_v, &sm.full[st], 0, s_row, s_head, s_outer);
-                        tma_load_4d(dst + kTileBytes + kHalfTileBytes, &map_v, &sm.full[st], 64, s_row,
-                                    s_head, s_outer);
                     } else {
-                        mbar_arrive(&sm.full[st]);
+                        outer = i;
+                        row = tok0;
                     }
-                    if (it == 0) SEER_STAMP(3);
-                    if (it == n_tiles - 1) SEER_STAMP(4);
+                    // bit 0: first tile of a piece; (the piece's end is found by the consumers)
+                    flags = (my_e == 0 || (fresh && t + lane == 0)) ? 1 : 0;
+                } else if (lane < n_chunk) {
+                    // the counts changed under us: keep the pipeline protocol, load nothing
+                    my_u = 0; my_ut = 1; flags = 1;
+                    raise_status(p.status, DEV_BAD_INDEX);
                 }
+                for (int s = 0; s < n_chunk; ++s, ++it) {
+                    const int s_nvalid = __shfl_sync(0xffffffffu, nvalid, s);
+                    const int s_row = __shfl_sync(0xffffffffu, row, s);
+                    const int s_outer = __shfl_sync(0xffffffffu, outer, s);
+                    const int s_head = __shfl_sync(0xffffffffu, head, s);
+                    const int s_flags = __shfl_sync(0xffffffffu, flags, s);
+                    const int s_u = __shfl_sync(0xffffffffu, my_u, s);
+                    const int s_pu = __shfl_sync(0xffffffffu, my_pu, s);
+                    const int s_ut = __shfl_sync(0xffffffffu, my_ut, s);
+                    if (lane == 0) {
+                        const int st = it % kStages;
+                        if (!mbar_wait(&sm.empty[st], ((it / kStages) & 1) ^ 1, p.status)) return;
+                        sm.meta[st] = StageMeta{s_nvalid, s_u, s_flags, s_pu, s_ut, iv_id};
+                        __threadfence_block();
+                        sm.issued = it + 1;                  // consumers may look ahead at this tile
+                        if (s_nvalid > 0) {
+                            unsigned char* dst = sm.stage[st];
+                            mbar_arrive_expect_tx(&sm.full[st], kStageBytes);
+                            tma_load_4d(dst, &map_k, &sm.full[st], 0, s_row, s_head, s_outer);
+                            tma_load_4d(dst + kHalfTileBytes, &map_k, &sm.full[st], 64, s_row, s_head, s_outer);
+                            tma_load_4d(dst + kTileBytes, &map_v, &sm.full[st], 0, s_row, s_head, s_outer);
+                            tma_load_4d(dst + kTileBytes + kHalfTileBytes, &map_v, &sm.full[st], 64, s_row,
+                                        s_head, s_outer);
+                        } else {
+                            mbar_arrive(&sm.full[st]);
+                        }
+                    }
+                }
+            }
+        }
+#ifdef SEER_DECODE_TRACE
+        if (lane == 0) { p.trace[(size_t)blockIdx.x * 8 + 3] = steals; p.trace[(size_t)blockIdx.x * 8 + 1] = it; SEER_STAMP(2); }
+#endif
+        if (lane == 0) {
+            // end-of-stream marker for the consumers
+            const int st = it % kStages;
+            if (!mbar_wait(&sm.empty[st], ((it / kStages) & 1) ^ 1, p.status)) return;
+            sm.meta[st] = StageMeta{-1, -1, 1, 0, 0, 0};
+            __threadfence_block();
+            sm.issued = it + 1;
+            mbar_arrive(&sm.full[st]);
+            // the last CTA to stop claiming work re-arms the counters for the next launch
+            __threadfence();
+            if (atomicAdd(&p.sched[1], 1) == (int)gridDim.x - 1) {
+                for (int c = 0; c < (int)gridDim.x; ++c) p.steal[c] = 0;
+                p.sched[0] = 0;
+                p.sched[1] = 0;
             }
         }
         return;
@@ -287,8 +543,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     uint32_t bq_pre[8][2];              // the same for the unit expected next (prefetched)
     float o[8][4];                      // O^T accumulators: 8 m-tiles over d
     float m_run[2], l_run[2];
-    int cur_unit = -1;
-    int seg = 0;
+    int seg = 0;                        // pieces finished so far
+    int piece_tiles = 0, piece_iv = 0;  // tiles in the current piece, interval it started in
     auto load_q = [&](uint32_t (&dst)[8][2], int unit) {
         const int i = unit / p.num_kv_heads, h = unit % p.num_kv_heads;
         const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
@@ -300,7 +556,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         }
     };
     int pre_unit = sm.start_unit;       // requested now, long before the first tile lands
-    if (pre_unit < U) load_q(bq_pre, pre_unit);
+    if (pre_unit < U) load_q(bq_pre, pre_unit); else pre_unit = -1;
 
     // lane-constant parts of the ldmatrix addresses (swizzle: 16-B chunk ^= row & 7)
     const int k_row = 16 * w + ((lane >> 3) & 1) * 8 + (lane & 7);
@@ -309,28 +565,47 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     const int v_csel = (lane >> 3) & 1;
     const int sw = lane & 7;
 
-    for (int it = 0; it < n_tiles; ++it) {
+    // the first tile's metadata
+    if (!mbar_wait(&sm.full[0], 0, p.status)) return;
+    StageMeta mt = sm.meta[0];
+    if (tid == 0) SEER_STAMP(5);
+    for (int it = 0; mt.nvalid >= 0; ++it) {
         const int st = it % kStages;
-        if (!mbar_wait(&sm.full[st], (it / kStages) & 1, p.status)) return;
-        const StageMeta mt = sm.meta[st];
-        if (it == 0 && tid == 0) SEER_STAMP(5);
-        if (mt.unit != cur_unit) {
-            cur_unit = mt.unit;
-            if (cur_unit == pre_unit) {
+        {
+            // look ahead: request the queries of the next unit as soon as the producer has issued a
+            // tile of it (its metadata is stable from then until we release that stage)
+            const int iss = sm.issued;
+            __threadfence_block();
+#pragma unroll
+            for (int look = 1; look < kStages; ++look) {
+                if (it + look < iss) {
+                    const int u2 = *reinterpret_cast<volatile int*>(&sm.meta[(it + look) % kStages].unit);
+                    if (u2 >= 0 && u2 != mt.unit && u2 != pre_unit) {
+                        load_q(bq_pre, u2);
+                        pre_unit = u2;
+                        break;
+                    }
+                }
+            }
+        }
+        if (mt.flags & 1) {
+            // first tile of a piece: fresh state, the unit's queries
+            if (mt.unit == pre_unit) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) { bq[ks][0] = bq_pre[ks][0]; bq[ks][1] = bq_pre[ks][1]; }
             } else {
-                load_q(bq, cur_unit);
+                load_q(bq, mt.unit);
             }
-            pre_unit = cur_unit + 1;    // units follow one another (empty ones excepted)
-            if (pre_unit < U) load_q(bq_pre, pre_unit);
 #pragma unroll
             for (int a = 0; a < 8; ++a)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) o[a][b] = 0.f;
             m_run[0] = m_run[1] = -INFINITY;
             l_run[0] = l_run[1] = 0.f;
+            piece_tiles = 0;
+            piece_iv = mt.interval;
         }
+        ++piece_tiles;
         const int nvalid = mt.nvalid;
         if (nvalid > 16 * w) {
             const uint32_t kbase = smem_u32(sm.stage[st]);
@@ -398,75 +673,76 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.empty[st]);
 
-        if (it == n_tiles - 1 && tid == 0) SEER_STAMP(6);
-        if (mt.last) {
-            // ---------------- end of this CTA's piece of the unit ----------------------
+        // the next tile's metadata tells whether the piece goes on
+        const int nst = (it + 1) % kStages;
+        if (!mbar_wait(&sm.full[nst], ((it + 1) / kStages) & 1, p.status)) return;
+        const StageMeta nx = sm.meta[nst];
+        if (nx.flags & 1) {
+            // ---------------- the current piece ends here ------------------------------------
             float l0 = l_run[0], l1 = l_run[1];
 #pragma unroll
             for (int off = 4; off < 32; off <<= 1) {
                 l0 += __shfl_xor_sync(0xffffffffu, l0, off);
                 l1 += __shfl_xor_sync(0xffffffffu, l1, off);
             }
-            if (rw == 0) {
-                sm.merge_ml[seg & 1][w][0][2 * qd] = m_run[0];
-                sm.merge_ml[seg & 1][w][0][2 * qd + 1] = m_run[1];
-                sm.merge_ml[seg & 1][w][1][2 * qd] = l0;
-                sm.merge_ml[seg & 1][w][1][2 * qd + 1] = l1;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.merge_bar[0]);
-            if (!mbar_wait(&sm.merge_bar[0], seg & 1, p.status)) return;
-            float m_all[2], l_all[2], sc[2];
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                const int hh = 2 * qd + x;
-                float mm = -INFINITY;
-#pragma unroll
-                for (int ww = 0; ww < kConsumerWarps; ++ww) mm = fmaxf(mm, sm.merge_ml[seg & 1][ww][0][hh]);
-                float ll = 0.f;
-#pragma unroll
-                for (int ww = 0; ww < kConsumerWarps; ++ww) {
-                    const float mw = sm.merge_ml[seg & 1][ww][0][hh];
-                    ll += (mw == -INFINITY) ? 0.f : sm.merge_ml[seg & 1][ww][1][hh] * fast_exp2(mw - mm);
-                }
-                m_all[x] = mm;
-                l_all[x] = ll;
-                sc[x] = (m_run[x] == -INFINITY) ? 0.f : fast_exp2(m_run[x] - mm);
-            }
             if (w > 0) {
+                // hand (o, max, sum) to warp 0 through shared memory and move on
+                if (seg > 0 && !mbar_wait(&sm.merge_bar[1], (seg - 1) & 1, p.status)) return;   // scratch free?
 #pragma unroll
                 for (int a = 0; a < 8; ++a) {
                     const int d0 = 16 * a + rw;
-                    sm.merge_o[w - 1][2 * qd][d0] = o[a][0] * sc[0];
-                    sm.merge_o[w - 1][2 * qd + 1][d0] = o[a][1] * sc[1];
-                    sm.merge_o[w - 1][2 * qd][d0 + 8] = o[a][2] * sc[0];
-                    sm.merge_o[w - 1][2 * qd + 1][d0 + 8] = o[a][3] * sc[1];
+                    sm.merge_o[w - 1][2 * qd][d0] = o[a][0];
+                    sm.merge_o[w - 1][2 * qd + 1][d0] = o[a][1];
+                    sm.merge_o[w - 1][2 * qd][d0 + 8] = o[a][2];
+                    sm.merge_o[w - 1][2 * qd + 1][d0 + 8] = o[a][3];
                 }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.merge_bar[1]);
-            if (w == 0) {
-                if (!mbar_wait(&sm.merge_bar[1], seg & 1, p.status)) return;
-#pragma unroll
-                for (int a = 0; a < 8; ++a) {
-                    const int d0 = 16 * a + rw;
-                    o[a][0] *= sc[0]; o[a][1] *= sc[1]; o[a][2] *= sc[0]; o[a][3] *= sc[1];
+                if (rw == 0) {
+                    sm.merge_ml[w - 1][0][2 * qd] = m_run[0];
+                    sm.merge_ml[w - 1][0][2 * qd + 1] = m_run[1];
+                    sm.merge_ml[w - 1][1][2 * qd] = l0;
+                    sm.merge_ml[w - 1][1][2 * qd + 1] = l1;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.merge_bar[0]);
+            } else {
+                const int u = mt.unit;
+                if (!mbar_wait(&sm.merge_bar[0], seg & 1, p.status)) return;
+                float m_all[2], l_all[2];
+                {
+                    float mw[kConsumerWarps - 1][2], lw[kConsumerWarps - 1][2];
+                    m_all[0] = m_run[0]; m_all[1] = m_run[1];
 #pragma unroll
                     for (int ww = 0; ww < kConsumerWarps - 1; ++ww) {
-                        o[a][0] += sm.merge_o[ww][2 * qd][d0];
-                        o[a][1] += sm.merge_o[ww][2 * qd + 1][d0];
-                        o[a][2] += sm.merge_o[ww][2 * qd][d0 + 8];
-                        o[a][3] += sm.merge_o[ww][2 * qd + 1][d0 + 8];
+                        mw[ww][0] = sm.merge_ml[ww][0][2 * qd]; mw[ww][1] = sm.merge_ml[ww][0][2 * qd + 1];
+                        lw[ww][0] = sm.merge_ml[ww][1][2 * qd]; lw[ww][1] = sm.merge_ml[ww][1][2 * qd + 1];
+                        m_all[0] = fmaxf(m_all[0], mw[ww][0]); m_all[1] = fmaxf(m_all[1], mw[ww][1]);
+                    }
+                    const float f0 = (m_run[0] == -INFINITY) ? 0.f : fast_exp2(m_run[0] - m_all[0]);
+                    const float f1 = (m_run[1] == -INFINITY) ? 0.f : fast_exp2(m_run[1] - m_all[1]);
+                    l_all[0] = l0 * f0; l_all[1] = l1 * f1;
+#pragma unroll
+                    for (int a = 0; a < 8; ++a) { o[a][0] *= f0; o[a][1] *= f1; o[a][2] *= f0; o[a][3] *= f1; }
+#pragma unroll
+                    for (int ww = 0; ww < kConsumerWarps - 1; ++ww) {
+                        const float g0 = (mw[ww][0] == -INFINITY) ? 0.f : fast_exp2(mw[ww][0] - m_all[0]);
+                        const float g1 = (mw[ww][1] == -INFINITY) ? 0.f : fast_exp2(mw[ww][1] - m_all[1]);
+                        l_all[0] += lw[ww][0] * g0; l_all[1] += lw[ww][1] * g1;
+#pragma unroll
+                        for (int a = 0; a < 8; ++a) {
+                            const int d0 = 16 * a + rw;
+                            o[a][0] += g0 * sm.merge_o[ww][2 * qd][d0];
+                            o[a][1] += g1 * sm.merge_o[ww][2 * qd + 1][d0];
+                            o[a][2] += g0 * sm.merge_o[ww][2 * qd][d0 + 8];
+                            o[a][3] += g1 * sm.merge_o[ww][2 * qd + 1][d0 + 8];
+                        }
                     }
                 }
-                const int u = mt.unit;
-                const long long first = mt.unit_first;
-                const int c_first = cta_of(first, T, G);
-                const int c_last = cta_of(first + mt.unit_tiles - 1, T, G);
-                const int n_parts = c_last - c_first + 1;
-                bool write_final = (n_parts == 1);
-                if (!write_final) {
-                    const size_t slot = (size_t)cta + u;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.merge_bar[1]);    // scratch may be refilled
+                const int n_held = sm.pieces_n;
+                if (piece_tiles < mt.unit_tiles && n_held < kMaxPieces) {
+                    // part of the unit: partial into the slot of the interval the piece began in
+                    const size_t slot = (size_t)piece_iv + u;
                     float* po = p.part_o + slot * (kMaxGroup * kHeadDim);
 #pragma unroll
                     for (int a = 0; a < 8; ++a) {
@@ -476,69 +752,21 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                         po[(2 * qd) * kHeadDim + d0 + 8] = o[a][2];
                         po[(2 * qd + 1) * kHeadDim + d0 + 8] = o[a][3];
                     }
+                    float* pm = p.part_ml + slot * kMlStride;
                     if (rw == 0) {
-                        float* pm = p.part_ml + slot * (2 * kMaxGroup);
                         pm[2 * qd] = m_all[0];
                         pm[2 * qd + 1] = m_all[1];
                         pm[kMaxGroup + 2 * qd] = l_all[0];
                         pm[kMaxGroup + 2 * qd + 1] = l_all[1];
                     }
-                    __threadfence();
-                    __syncwarp();
-                    int ticket = 0;
-                    if (lane == 0) ticket = atomicAdd(&p.tickets[u], 1);
-                    ticket = __shfl_sync(0xffffffffu, ticket, 0);
-                    if (ticket == n_parts - 1) {
-                        // Last piece in: log-sum-exp combine of all pieces of the unit.  Lane t takes
-                        // head t/4, channels 32*(t%4) .. +31 of every piece; the loads of a pass do
-                        // not depend on one another, so they are all in flight together.
-                        __threadfence();
-                        const int hh = lane >> 2, d0 = 32 * (lane & 3);
-                        const size_t s_first = (size_t)c_first + u;
-                        float M = -INFINITY;
-#pragma unroll 8
-                        for (int s2 = 0; s2 < n_parts; ++s2)
-                            M = fmaxf(M, __ldcg(p.part_ml + (s_first + s2) * (2 * kMaxGroup) + hh));
-                        float acc[32];
-#pragma unroll
-                        for (int x = 0; x < 32; ++x) acc[x] = 0.f;
-                        float lsum = 0.f;
-#pragma unroll 2
-                        for (int s2 = 0; s2 < n_parts; ++s2) {
-                            const float* pm = p.part_ml + (s_first + s2) * (2 * kMaxGroup);
-                            const float4* qo = reinterpret_cast<const float4*>(
-                                p.part_o + (s_first + s2) * (kMaxGroup * kHeadDim) + hh * kHeadDim + d0);
-                            const float ms = __ldcg(pm + hh);
-                            const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - M);
-                            lsum += f * __ldcg(pm + kMaxGroup + hh);
-#pragma unroll
-                            for (int x = 0; x < 8; ++x) {
-                                const float4 v4 = __ldcg(qo + x);
-                                acc[4 * x] += f * v4.x; acc[4 * x + 1] += f * v4.y;
-                                acc[4 * x + 2] += f * v4.z; acc[4 * x + 3] += f * v4.w;
-                            }
-                        }
-                        if (lane == 0) p.tickets[u] = 0;     // ready for the next launch
-                        if (hh < p.group) {
-                            const int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
-                            const size_t row = (size_t)i * p.num_q_heads + (size_t)h * p.group + hh;
-                            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-                            uint4* dst = reinterpret_cast<uint4*>(p.out + row * kHeadDim + d0);
-#pragma unroll
-                            for (int x = 0; x < 4; ++x) {
-                                uint4 pk;
-                                pk.x = pack_bf16x2(acc[8 * x] * inv, acc[8 * x + 1] * inv);
-                                pk.y = pack_bf16x2(acc[8 * x + 2] * inv, acc[8 * x + 3] * inv);
-                                pk.z = pack_bf16x2(acc[8 * x + 4] * inv, acc[8 * x + 5] * inv);
-                                pk.w = pack_bf16x2(acc[8 * x + 6] * inv, acc[8 * x + 7] * inv);
-                                dst[x] = pk;
-                            }
-                            if (p.lse && (lane & 3) == 0)
-                                p.lse[row] = lsum > 0.f ? (M + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
-                        }
+                    if (lane == 0) {
+                        pm[16] = __uint_as_float(p.generation);
+                        sm.pieces[n_held] = Piece{u, piece_tiles, mt.unit_first, mt.unit_tiles};
+                        sm.pieces_n = n_held + 1;
                     }
-                }
-                if (write_final) {
+                    __syncwarp();
+                } else if (piece_tiles >= mt.unit_tiles) {
+                    // the whole unit in one piece: final output
                     const int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
                     const float inv0 = l_all[0] > 0.f ? 1.f / l_all[0] : 0.f;
                     const float inv1 = l_all[1] > 0.f ? 1.f / l_all[1] : 0.f;
@@ -563,10 +791,99 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                         if (h0) p.lse[row0] = l_all[0] > 0.f ? (m_all[0] + log2f(l_all[0])) * ln2 : -INFINITY;
                         if (h1) p.lse[row0 + 1] = l_all[1] > 0.f ? (m_all[1] + log2f(l_all[1])) * ln2 : -INFINITY;
                     }
+                } else {
+                    // (cannot happen with the schedule's bound on pieces per CTA) no room to hold
+                    // the piece back: flag it rather than lose it silently
+                    raise_status(p.status, DEV_TIMEOUT);
                 }
             }
             ++seg;
-            cur_unit = -1;      // a later piece (another unit) starts from fresh state
+        }
+        mt = nx;
+    }
+    // ---- the stream is over: make this CTA's partials count, and do the combines it owes ------
+    if (tid == 0) SEER_STAMP(6);
+    if (w == 0) {
+        const int n_held = sm.pieces_n;
+#ifdef SEER_DECODE_TRACE
+        if (lane == 0) p.trace[(size_t)blockIdx.x * 8 + 4] = n_held;
+#endif
+        __threadfence();                               // the partials above are visible from here on
+        __syncwarp();
+        bool owe = false;
+        Piece pc = Piece{0, 0, 0, 0};
+        if (lane < n_held) {
+            pc = sm.pieces[lane];
+            const int before = atomicAdd(&p.tickets[pc.unit], pc.tiles);
+            owe = before + pc.tiles == pc.unit_tiles;  // this piece completed the unit's count
+        }
+        __threadfence();
+        // rewrite the list: the units this CTA has to combine, with their candidate slots
+        const unsigned m = __ballot_sync(0xffffffffu, owe);
+        __syncwarp();
+        if (owe) {
+            p.tickets[pc.unit] = 0;                    // ready for the next launch
+            const int iv_first = interval_of(sm.sched, pc.unit_first);
+            const int iv_last = interval_of(sm.sched, pc.unit_first + pc.unit_tiles - 1);
+            sm.pieces[__popc(m & ((1u << lane) - 1u))] = Piece{pc.unit, 0, iv_first + pc.unit, iv_last - iv_first + 1};
+        }
+        if (lane == 0) sm.pieces_n = __popc(m);
+    }
+    // every warp is done with the stage buffers, and warp 0's list of owed units is written
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.end_bar);
+    if (!mbar_wait(&sm.end_bar, 0, p.status)) return;
+    const int n_owed = sm.pieces_n;
+    // The combines use the stage buffers as scratch (the stream is over, nothing is in flight): the
+    // slots that really hold a partial of a unit are found by looking at the generation stamps of
+    // the unit's candidate slots, then all threads combine them.
+    int* lists = reinterpret_cast<int*>(sm.stage[0]);            // kListInts slot numbers (two stages)
+    int* counts = reinterpret_cast<int*>(sm.stage[2]);
+    int sync_phase = 0;
+    auto sync_consumers = [&]() -> bool {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.list_bar);
+        const bool ok = mbar_wait(&sm.list_bar, sync_phase & 1, p.status);
+        ++sync_phase;
+        return ok;
+    };
+    int total_cand = 0;
+    for (int e = 0; e < n_owed; ++e) total_cand += sm.pieces[e].unit_tiles;
+    if (total_cand <= kListInts) {
+        // usual case: every owed unit's candidates fit at once; warp e%4 scans unit e
+        int base = 0;
+        for (int e = 0; e < n_owed; ++e) {
+            if ((e & (kConsumerWarps - 1)) == w) {
+                const int n = scan_valid_slots(p, sm.pieces[e].unit_first, sm.pieces[e].unit_tiles, lists + base, lane);
+                if (lane == 0) counts[e] = n;
+            }
+            base += sm.pieces[e].unit_tiles;
+        }
+        if (!sync_consumers()) return;
+        base = 0;
+        for (int e = 0; e < n_owed; ++e) {
+            MergeState ms;
+            merge_init(ms);
+            merge_accumulate(p, ms, lists + base, counts[e], tid);
+            merge_finalize(p, ms, sm.pieces[e].unit, tid);
+            base += sm.pieces[e].unit_tiles;
+        }
+    } else {
+        // a unit cut into thousands of pieces: go through its candidates in windows
+        constexpr int kWin = kListInts / kConsumerWarps;
+        for (int e = 0; e < n_owed; ++e) {
+            MergeState ms;
+            merge_init(ms);
+            const int first = sm.pieces[e].unit_first, n_slots = sm.pieces[e].unit_tiles;
+            for (int w0 = 0; w0 < n_slots; w0 += kListInts) {
+                const int lo = w0 + w * kWin, hi = min(n_slots, min(w0 + kListInts, lo + kWin));
+                const int n = lo < hi ? scan_valid_slots(p, first + lo, hi - lo, lists + w * kWin, lane) : 0;
+                if (lane == 0) counts[w] = n;
+                if (!sync_consumers()) return;
+                for (int ww = 0; ww < kConsumerWarps; ++ww) merge_accumulate(p, ms, lists + ww * kWin, counts[ww], tid);
+                if (!sync_consumers()) return;
+            }
+            merge_finalize(p, ms, sm.pieces[e].unit, tid);
         }
     }
     if (tid == 0) SEER_STAMP(7);
@@ -619,6 +936,8 @@ int decode_ctas_per_sm(bool sparse, bool paged) {
     if (sparse) return paged ? occupancy<true, true>() : occupancy<true, false>();
     return paged ? occupancy<false, true>() : occupancy<false, false>();
 }
+
+int decode_max_intervals(int grid) { return grid * (kMaxRounds + 1) + 1; }
 
 cudaError_t launch_decode(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
                           const DecodeParams& p, int grid, cudaStream_t stream) {

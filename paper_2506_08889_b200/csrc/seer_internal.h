@@ -12,6 +12,7 @@ constexpr int kHeadDim = 128;       // d
 constexpr int kTileTokens = 64;     // tokens per staged K (or V) tile
 constexpr int kMaxGroup = 8;        // query heads per KV head handled by one MMA N-tile
 constexpr int kMaxDGate = 256;      // gate width: 64, 128 or 256
+constexpr int kMaxRounds = 12;      // halving rounds of the decode kernels' dynamic tile pool
 
 // Everything the decode kernels need besides the two tensor maps.
 struct DecodeParams {
@@ -29,11 +30,16 @@ struct DecodeParams {
     int batch, num_q_heads, num_kv_heads, group, block_size, tiles_per_block;
     int num_units;                  // batch * num_kv_heads
     int max_blocks_cap;             // tile-count clamp for dense: capacity in tiles
+    int pool_div;                   // 1/pool_div of the tiles are handed out dynamically (0: none)
     float scale_log2;               // sm_scale * log2(e)
     unsigned int* status;
     int* tickets;                   // [num_units], zero between launches
+    int* sched;                     // [2]: theft cursor, exit counter; zero between launches
+    int* steal;                     // [grid]: per-range claim counters (front | back << 16); zero between launches
+    unsigned int generation;        // stamp that marks this launch's partials
+    int* prefix;                    // [num_units + 1] prefix sums of the units' tile counts
     float* part_o;                  // [slots][8][128]
-    float* part_ml;                 // [slots][2][8]  (max, sum)
+    float* part_ml;                 // [slots][32]: max[8], sum[8], generation stamp
 #ifdef SEER_DECODE_TRACE
     unsigned long long* trace;      // [grid][8] %globaltimer stamps (diagnostic builds only)
 #endif
@@ -46,6 +52,8 @@ struct DecodeLaunch {
 
 // Returns resident CTAs per SM for the decode kernel (queried once).
 int decode_ctas_per_sm(bool sparse, bool paged);
+// Upper bound on the number of work intervals (static ranges + dynamic chunks) of a launch.
+int decode_max_intervals(int grid);
 cudaError_t launch_decode(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
                           const DecodeParams& p, int grid, cudaStream_t stream);
 

@@ -391,6 +391,7 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
     p.seq_lens = seq_lens;
     p.scores_in = scores_in;
     p.scores = scores_out ? scores_out : reinterpret_cast<float*>(ctx->ws + w.scores);
+    p.scores_user = scores_out;
     p.q_gate = reinterpret_cast<float*>(ctx->ws + w.q_gate);
     p.block_idx = block_idx;
     p.block_cnt = block_cnt;

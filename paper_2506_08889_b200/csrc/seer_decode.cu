@@ -96,10 +96,6 @@ struct __align__(1024) Smem {
 // fit in the SM's 228 KiB
 static_assert(sizeof(Smem) + 1024 <= 113 * 1024, "decode kernel no longer fits two CTAs per SM");
 
-// Programmatic dependent launch: the kernel may start while its predecessor in the stream is
-// still running; nothing the predecessor writes is read before pdl_wait().
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 #ifdef SEER_DECODE_TRACE
 __device__ __forceinline__ void trace_stamp(const DecodeParams& p, int slot) {
     unsigned long long t;
@@ -113,13 +109,13 @@ __device__ __forceinline__ void trace_stamp(const DecodeParams& p, int slot) {
 
 template <bool SPARSE>
 __device__ __forceinline__ int tiles_of(const DecodeParams& p, int u) {
-    int L = p.seq_lens[u / p.num_kv_heads];
-    if (L <= 0) return 0;
+    const int L = p.seq_lens[u / p.num_kv_heads];
     if (SPARSE) {
-        int c = p.block_cnt ? p.block_cnt[u] : p.max_sel;
+        int c = p.block_cnt ? p.block_cnt[u] : p.max_sel;     // not behind the test on L: both loads in flight
         c = max(0, min(c, p.max_sel));
-        return c * p.tiles_per_block;
+        return L <= 0 ? 0 : c * p.tiles_per_block;
     } else {
+        if (L <= 0) return 0;
         int t = (L + kTileTokens - 1) / kTileTokens;
         return min(t, p.max_blocks_cap);
     }
@@ -802,6 +798,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         mt = nx;
     }
     // ---- the stream is over: make this CTA's partials count, and do the combines it owes ------
+    pdl_launch_dependents();
     if (tid == 0) SEER_STAMP(6);
     if (w == 0) {
         const int n_held = sm.pieces_n;
@@ -817,7 +814,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             const int before = atomicAdd(&p.tickets[pc.unit], pc.tiles);
             owe = before + pc.tiles == pc.unit_tiles;  // this piece completed the unit's count
         }
-        __threadfence();
         // rewrite the list: the units this CTA has to combine, with their candidate slots
         const unsigned m = __ballot_sync(0xffffffffu, owe);
         __syncwarp();
@@ -915,19 +911,7 @@ template <bool SPARSE, bool PAGED>
 cudaError_t launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& p, int grid,
                    cudaStream_t stream) {
     if (occupancy<SPARSE, PAGED>() <= 0) return cudaErrorInvalidConfiguration;
-    // launched as a programmatic dependent: barrier set-up and tensor-map prefetch may overlap
-    // the tail of the previous kernel in the stream (the kernel waits before its first read)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = decode_smem_bytes();
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_kernel<SPARSE, PAGED>, mk, mv, p);
+    return launch_pdl(decode_kernel<SPARSE, PAGED>, dim3(grid), dim3(kThreads), decode_smem_bytes(), stream, mk, mv, p);
 }
 
 }  // namespace

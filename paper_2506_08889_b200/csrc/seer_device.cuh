@@ -112,6 +112,15 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// Programmatic dependent launch.  Every kernel of the library is launched with the stream-
+// serialisation attribute: it may start while its predecessor in the stream is still running,
+// and touches nothing in global memory before pdl_wait(), which returns once every earlier
+// kernel has completed.  pdl_launch_dependents() lets the next kernel start its own set-up; a
+// kernel calls it only after its own pdl_wait(), so a dependent never overlaps a kernel two
+// places back.  Launched without the attribute both calls do nothing.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
 // sin and cos of pos * inv_freq for the rotary embedding.  The angle reaches 1e5..1e6 rad at
 // long context, so the product and the reduction to one turn are done in double (a handful
 // of operations); the reduced angle is then accurate to about 1e-10 turns and the fp32

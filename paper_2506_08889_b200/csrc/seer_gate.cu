@@ -11,8 +11,6 @@ namespace seer {
 namespace {
 
 constexpr int kGateThreads = 512;
-constexpr int kGateWarps = kGateThreads / 32;
-constexpr int kCached = 8;                  // candidate keys a thread can keep in registers
 constexpr int kProjThreads = 256;
 
 __device__ __forceinline__ float dot8(const uint4& a, const float* x) {
@@ -39,12 +37,6 @@ __device__ __forceinline__ float dot8(const uint4& a, const uint4& b) {
     return acc;
 }
 
-// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
-// start while its predecessor is still running; it must pass pdl_wait() before it touches
-// anything the predecessor writes.  Without the attribute both calls do nothing.
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
-
 // Order-preserving key: larger score <-> larger key; -0 == +0; NaN below everything.
 __device__ __forceinline__ uint32_t score_key(float s) {
     if (s != s) return 0u;
@@ -53,9 +45,12 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+constexpr int kUnitThreads = 1024;          // one-CTA-per-unit gate kernel
+constexpr int kUnitMaxBlocks = 4096;        // ... and the compressed keys it can score
+
 struct SelectSmem {
     int hist[4][256];                       // one histogram per radix pass
-    unsigned long long warp_tot[kGateWarps];
+    unsigned long long warp_tot[kUnitThreads / 32];
     uint32_t prefix;
     int rem;
 };
@@ -65,15 +60,17 @@ struct SelectSmem {
 // of the (k-1)-th best candidate; one ordered pass then emits, in ascending block order, every
 // candidate above it and the first few equal to it (the lower block number wins a tie), and
 // the forced last block closes the list.  Comparisons only: the result is exact.
-template <bool CACHED>
+// NT = threads of the CTA; SMEM = the scores are in shared memory (else read from L2).
+template <int NT, bool CACHED, bool SMEM>
 __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectSmem& sm) {
+    constexpr int kCachedT = CACHED ? (NT >= 1024 ? 4 : 8) : 1;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int i = u / p.num_kv_heads;
     int32_t* dst = p.block_idx + (size_t)u * p.max_sel;
     const int L = p.seq_lens[i];
     const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
     if (n_i <= 0) {
-        for (int e = tid; e < p.max_sel; e += kGateThreads) dst[e] = -1;
+        for (int e = tid; e < p.max_sel; e += NT) dst[e] = -1;
         if (tid == 0) p.block_cnt[u] = 0;
         return;
     }
@@ -81,20 +78,21 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
     k = min(k, min(n_i, p.max_sel));
     const int n_cand = min(n_i - 1, p.max_blocks);
     const int need = min(k - 1, n_cand);             // candidates to take besides the last block
-    const int E = (n_cand + kGateThreads - 1) / kGateThreads;
+    const int E = (n_cand + NT - 1) / NT;
     const int j_lo = min(n_cand, tid * E), j_hi = min(n_cand, j_lo + E);
 
-    uint32_t keys[kCached];
+    auto score_at = [&](int j) -> float { return SMEM ? sc[j] : __ldcg(sc + j); };
+    uint32_t keys[kCachedT];
     if (CACHED) {
 #pragma unroll
-        for (int e = 0; e < kCached; ++e) keys[e] = (j_lo + e < j_hi) ? score_key(__ldcg(sc + j_lo + e)) : 0u;
+        for (int e = 0; e < kCachedT; ++e) keys[e] = (j_lo + e < j_hi) ? score_key(score_at(j_lo + e)) : 0u;
     }
-    auto key_at = [&](int e) -> uint32_t { return score_key(__ldcg(sc + j_lo + e)); };
+    auto key_at = [&](int e) -> uint32_t { return score_key(score_at(j_lo + e)); };
 
     uint32_t thr = 0u;                               // key of the need-th best candidate
     int take_eq = n_cand;                            // candidates equal to thr that are taken
     if (need > 0 && need < n_cand) {
-        for (int x = tid; x < 4 * 256; x += kGateThreads) (&sm.hist[0][0])[x] = 0;
+        for (int x = tid; x < 4 * 256; x += NT) (&sm.hist[0][0])[x] = 0;
         __syncthreads();
         uint32_t prefix = 0u;
         int rem = need;
@@ -104,7 +102,7 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
             int* hist = sm.hist[pass];
             if (CACHED) {
 #pragma unroll
-                for (int e = 0; e < kCached; ++e)
+                for (int e = 0; e < kCachedT; ++e)
                     if (j_lo + e < j_hi && (keys[e] & himask) == prefix)
                         atomicAdd(&hist[(keys[e] >> shift) & 255u], 1);
             } else {
@@ -150,7 +148,7 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
         int n_gt = 0, n_eq = 0;
         if (CACHED) {
 #pragma unroll
-            for (int e = 0; e < kCached; ++e)
+            for (int e = 0; e < kCachedT; ++e)
                 if (j_lo + e < j_hi) { n_gt += keys[e] > thr; n_eq += keys[e] == thr; }
         } else {
             for (int e = 0; j_lo + e < j_hi; ++e) {
@@ -170,14 +168,14 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
         __syncthreads();
         unsigned long long base = 0;
 #pragma unroll
-        for (int w2 = 0; w2 < kGateWarps; ++w2) base += (w2 < warp) ? sm.warp_tot[w2] : 0ull;
+        for (int w2 = 0; w2 < NT / 32; ++w2) base += (w2 < warp) ? sm.warp_tot[w2] : 0ull;
         const unsigned long long excl = base + incl - packed;
         const int gt_before = (int)(excl >> 32);
         int eq_rank = (int)(excl & 0xffffffffull);
         int pos = gt_before + min(eq_rank, take_eq);
         if (CACHED) {
 #pragma unroll
-            for (int e = 0; e < kCached; ++e) {
+            for (int e = 0; e < kCachedT; ++e) {
                 if (j_lo + e < j_hi) {
                     const bool gt = keys[e] > thr, eq = keys[e] == thr;
                     if (gt || (eq && eq_rank < take_eq)) dst[pos++] = j_lo + e;
@@ -197,19 +195,22 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
         dst[need] = n_i - 1;                         // the last block is always active
         p.block_cnt[u] = need + 1;
     }
-    for (int e = need + 1 + tid; e < p.max_sel; e += kGateThreads) dst[e] = -1;
+    for (int e = need + 1 + tid; e < p.max_sel; e += NT) dst[e] = -1;
 }
 
+template <int NT, bool SMEM>
 __device__ __forceinline__ void select_dispatch(const GateParams& p, int u, const float* sc, SelectSmem& sm) {
-    if (p.max_blocks <= kCached * kGateThreads) select_unit<true>(p, u, sc, sm);
-    else select_unit<false>(p, u, sc, sm);
+    if (p.max_blocks <= (NT >= 1024 ? 4 : 8) * NT) select_unit<NT, true, SMEM>(p, u, sc, sm);
+    else select_unit<NT, false, SMEM>(p, u, sc, sm);
 }
 
 // Selection on caller-provided scores: one CTA per unit.
 __global__ void __launch_bounds__(kGateThreads) gate_select_only_kernel(const GateParams p) {
     __shared__ SelectSmem sm;
     const int u = blockIdx.x;
-    select_dispatch(p, u, p.scores_in + (size_t)u * p.max_blocks, sm);
+    pdl_wait();
+    pdl_launch_dependents();
+    select_dispatch<kGateThreads, false>(p, u, p.scores_in + (size_t)u * p.max_blocks, sm);
 }
 
 // ---- q_gate = RoPE_{L_i - 1}( W_q[h] . concat_g(Q_nope) )  (Eq. 1a) ---------------------------
@@ -218,7 +219,8 @@ __global__ void __launch_bounds__(kGateThreads) gate_select_only_kernel(const Ga
 // NIT = 16-byte pieces of a row per lane (row length g*128 bf16 = g*16 pieces over 32 lanes).
 template <int NIT>
 __global__ void __launch_bounds__(kProjThreads) gate_qproj_kernel(const GateParams p) {
-    pdl_launch_dependents();
+    pdl_wait();
+    pdl_launch_dependents();      // the score kernel may start requesting its keys
     const int u = blockIdx.x, i = u / p.num_kv_heads, h = u % p.num_kv_heads;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n = p.group * kHeadDim, chunks = n / 8, half = p.d_gate / 2;
@@ -331,23 +333,106 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
     }
     __syncthreads();
     if (!is_last) return;
-    __threadfence();
-    select_dispatch(p, u, sc_out, sm);
+    select_dispatch<kGateThreads, false>(p, u, sc_out, sm);   // reads the scores with ld.cg, after the ticket
 }
 
-template <typename... Args>
-cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, args...);
+// ---- the whole gate of one (sequence, KV head) unit in one CTA --------------------------------
+// Used when a unit's compressed keys are few enough that one SM streams them as fast as the
+// split version would (which has to publish scores, fence, take tickets and read the scores
+// back): projection + RoPE, scores into shared memory, selection, all in one launch.
+template <int NIT>
+__global__ void __launch_bounds__(kUnitThreads, 1) gate_unit_kernel(const GateParams p) {
+    __shared__ float qg[kMaxDGate];
+    __shared__ float sc[kUnitMaxBlocks];
+    __shared__ SelectSmem sm;
+    pdl_wait();
+    pdl_launch_dependents();
+    const int u = blockIdx.x, i = u / p.num_kv_heads, h = u % p.num_kv_heads;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int L = __ldg(p.seq_lens + i);
+    const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
+    const int n_cand = max(0, min(n_i - 1, p.max_blocks));
+    const int lpk = p.d_gate / 8;                      // lanes per key: 8, 16 or 32
+    const int csub = tid & (lpk - 1);
+    const uint4* kc = reinterpret_cast<const uint4*>(p.kcomp + (size_t)u * p.max_blocks * p.d_gate);
+    const int total = n_cand * lpk;
+    constexpr int kBatch = 8;
+    // first batch of keys: independent of the gate query, so it travels while W_q is applied
+    uint4 kv[kBatch];
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k) {
+        const int c = k * kUnitThreads + tid;
+        kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    // ---- q_gate: every warp takes rotary pairs two at a time (rows c, c+1, c+half, c+1+half) ----
+    {
+        const int n = p.group * kHeadDim, chunks = n / 8, half = p.d_gate / 2;
+        const uint4* xsrc = reinterpret_cast<const uint4*>(
+            p.q_nope + ((size_t)i * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
+        uint4 xv[NIT];
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int ch = lane + 32 * it;
+            xv[it] = ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        for (int c0 = warp * 2; c0 < half; c0 += (kUnitThreads / 32) * 2) {
+            float acc[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int r = c0 + (k & 1) + (k >> 1) * half;
+                const uint4* wrow = reinterpret_cast<const uint4*>(p.w_q + ((size_t)h * p.d_gate + r) * n);
+                acc[k] = 0.f;
+#pragma unroll
+                for (int it = 0; it < NIT; ++it) {
+                    const int ch = lane + 32 * it;
+                    if (ch < chunks) acc[k] += dot8(__ldg(wrow + ch), xv[it]);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
+            if (lane < 2) {
+                const int c = c0 + lane;
+                float sn, cs;
+                rope_sincos((double)(L > 0 ? L - 1 : 0), p.inv_freq[c], &sn, &cs);
+                const float a = lane ? acc[1] : acc[0], b = lane ? acc[3] : acc[2];
+                qg[c] = a * cs - b * sn;
+                qg[c + half] = b * cs + a * sn;
+            }
+        }
+    }
+    __syncthreads();
+    // ---- scores into shared memory (and to scores_out if the caller wants them) ----------------
+    float qsub[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) qsub[c] = qg[8 * csub + c];
+    const float inv = rsqrtf((float)p.d_gate);
+    float* sc_out = p.scores_user ? p.scores_user + (size_t)u * p.max_blocks : nullptr;
+    for (int cb = 0; cb < total; cb += kUnitThreads * kBatch) {
+        float acc[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
+        if (cb + kUnitThreads * kBatch < total) {      // next batch on its way while this one reduces
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                const int c = cb + (kBatch + k) * kUnitThreads + tid;
+                kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+            for (int off = lpk >> 1; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
+            const int c = cb + k * kUnitThreads + tid;
+            if (c < total && csub == 0) {
+                const float v = acc[k] * inv;
+                sc[c / lpk] = v;
+                if (sc_out) sc_out[c / lpk] = v;
+            }
+        }
+    }
+    __syncthreads();
+    select_dispatch<kUnitThreads, true>(p, u, sc, sm);
 }
 
 }  // namespace
@@ -356,26 +441,41 @@ cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* la
     const int U = p.batch * p.num_kv_heads;
     *launched = 0;
     if (p.scores_in) {
-        gate_select_only_kernel<<<U, kGateThreads, 0, stream>>>(p);
         *launched = 1;
-        return cudaGetLastError();
+        return launch_pdl(gate_select_only_kernel, dim3(U), dim3(kGateThreads), 0, stream, p);
+    }
+    const int nit = (p.group * kHeadDim / 8 + 31) / 32;
+    // One CTA per unit when a unit's keys are few enough: one SM streams them at roughly 25 GB/s
+    // (measured), the split version gets the whole chip but pays about 4 us for publishing scores
+    // and taking tickets.
+    const double one_cta_us = p.max_blocks * p.d_gate * 2.0 / 0.025e6;
+    const double split_us = (double)U * p.max_blocks * p.d_gate * 2.0 / 6.0e6 + 4.0;
+    if (p.max_blocks <= kUnitMaxBlocks && one_cta_us <= split_us) {
+        cudaError_t e;
+        switch (nit) {
+            case 1: e = launch_pdl(gate_unit_kernel<1>, dim3(U), dim3(kUnitThreads), 0, stream, p); break;
+            case 2: e = launch_pdl(gate_unit_kernel<2>, dim3(U), dim3(kUnitThreads), 0, stream, p); break;
+            case 3: e = launch_pdl(gate_unit_kernel<3>, dim3(U), dim3(kUnitThreads), 0, stream, p); break;
+            default: e = launch_pdl(gate_unit_kernel<4>, dim3(U), dim3(kUnitThreads), 0, stream, p); break;
+        }
+        *launched = 1;
+        return e;
     }
     const dim3 pgrid(U, (p.d_gate / 2 + 15) / 16);
-    const int nit = (p.group * kHeadDim / 8 + 31) / 32;
+    cudaError_t e;
     switch (nit) {
-        case 1: gate_qproj_kernel<1><<<pgrid, kProjThreads, 0, stream>>>(p); break;
-        case 2: gate_qproj_kernel<2><<<pgrid, kProjThreads, 0, stream>>>(p); break;
-        case 3: gate_qproj_kernel<3><<<pgrid, kProjThreads, 0, stream>>>(p); break;
-        default: gate_qproj_kernel<4><<<pgrid, kProjThreads, 0, stream>>>(p); break;
+        case 1: e = launch_pdl(gate_qproj_kernel<1>, pgrid, dim3(kProjThreads), 0, stream, p); break;
+        case 2: e = launch_pdl(gate_qproj_kernel<2>, pgrid, dim3(kProjThreads), 0, stream, p); break;
+        case 3: e = launch_pdl(gate_qproj_kernel<3>, pgrid, dim3(kProjThreads), 0, stream, p); break;
+        default: e = launch_pdl(gate_qproj_kernel<4>, pgrid, dim3(kProjThreads), 0, stream, p); break;
     }
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     *launched = 1;
     // slices of about 512 compressed keys, at most 8 per unit
     int S = (p.max_blocks + 511) / 512;
     S = S < 1 ? 1 : (S > 8 ? 8 : S);
     const int per = (p.max_blocks + S - 1) / S;
-    e = launch_pdl(gate_score_select_kernel, dim3(S, U), dim3(kGateThreads), stream, p, per);
+    e = launch_pdl(gate_score_select_kernel, dim3(S, U), dim3(kGateThreads), 0, stream, p, per);
     if (e != cudaSuccess) return e;
     *launched = 2;
     return cudaGetLastError();

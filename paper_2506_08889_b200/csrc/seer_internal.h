@@ -14,6 +14,23 @@ constexpr int kMaxGroup = 8;        // query heads per KV head handled by one MM
 constexpr int kMaxDGate = 256;      // gate width: 64, 128 or 256
 constexpr int kMaxRounds = 12;      // halving rounds of the decode kernels' dynamic tile pool
 
+// Launch with the programmatic-stream-serialisation attribute (see pdl_wait in seer_device.cuh).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Everything the decode kernels need besides the two tensor maps.
 struct DecodeParams {
     const __nv_bfloat16* q;
@@ -64,6 +81,7 @@ struct GateParams {
     const int32_t* seq_lens;
     const float* scores_in;         // may be null
     float* scores;                  // [B,Hkv,max_blocks] (workspace or caller's scores_out)
+    float* scores_user;             // caller's scores_out or null
     float* q_gate;                  // [B,Hkv,dg] workspace
     int32_t* block_idx;
     int32_t* block_cnt;

@@ -29,7 +29,9 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
     const int pps = half / gridDim.z;                 // rotary pairs per row split
     const int pair_base = blockIdx.z * pps;
 
-    // first batch of W_k rows (does not depend on anything else)
+    pdl_wait();
+    pdl_launch_dependents();
+    // first batch of W_k rows, requested before the pooling starts
     uint4 wv[4][2];
     auto load_rows = [&](int pb) {
 #pragma unroll
@@ -188,11 +190,15 @@ cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* 
     if (U <= 0) return cudaSuccess;
     if (p.first_block < 0) {
         // one block per unit: split the d_gate/2 rotary pairs over 4 CTAs (16, 8 or 32 pairs each)
-        kcomp_kernel<1><<<dim3(1, U, 4), kKcThreads, 0, stream>>>(p);
+        cudaError_t e = launch_pdl(kcomp_kernel<1>, dim3(1, U, 4), dim3(kKcThreads), 0, stream, p);
+        *launched = 1;
+        return e;
     } else {
         const int gx = (p.num_blocks + 3) / 4;
         if (gx <= 0) return cudaSuccess;
-        kcomp_kernel<4><<<dim3(gx, U, 1), kKcThreads, 0, stream>>>(p);
+        cudaError_t e = launch_pdl(kcomp_kernel<4>, dim3(gx, U, 1), dim3(kKcThreads), 0, stream, p);
+        *launched = 1;
+        return e;
     }
     *launched = 1;
     return cudaGetLastError();

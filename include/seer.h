@@ -207,6 +207,41 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
                               int rows_block_local, int first_block, int num_blocks,
                               void* stream);
 
+/*
+ * seer_gate_select without a context and without any allocation.  (The paper has no counterpart:
+ * this entry point exists for hosts of the library, not for the method.)
+ *
+ * Some callers may not allocate device memory at all: an inference server that hands every byte
+ * of HBM to its own pool at start-up and forbids cudaMalloc afterwards (a late allocation can
+ * fail, or stall the GPU, under its memory plan), or code that runs inside a region where the
+ * CUDA allocator must not be entered.  seer_create allocates a workspace, so those callers
+ * cannot have a context.  This call computes exactly what seer_gate_select computes from
+ * q_nope (same kernels, same results) but keeps the scratch it needs -- per-unit tickets, the gate
+ * query, and the block scores unless scores_out is given -- in an array of
+ * SEER_STATIC_SCRATCH_BYTES that is part of the library image.  Every GPU on which the library
+ * is used holds one copy of that array from first use until the process exits.
+ *
+ *  - It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *  - A call whose scratch need, 4*B*Hkv + 4*B*Hkv*d_gate (+ 4*B*Hkv*max_blocks without scores_out),
+ *    each part rounded up to 256 bytes, exceeds the array returns SEER_ERR_WORKSPACE and launches
+ *    nothing; `err` says how much was needed.  (Example that fits: B*Hkv = 64, d_gate 128,
+ *    max_blocks 2048.)
+ *  - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device made current).  Make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents.  The
+ *    call clears the part that must start at zero (the tickets) on `stream`; two calls that
+ *    overlap on the GPU (different streams without ordering, or concurrent host threads) race on
+ *    it and give wrong results.  Order them.
+ *  - err / err_len: optional caller buffer that receives a one-line message on failure.
+ * Arguments otherwise as for seer_gate_select (scores_in is not offered: selection on given
+ * scores needs no scratch and no context-free variant).
+ */
+#define SEER_STATIC_SCRATCH_BYTES (1 << 20)
+seer_status seer_gate_select_static(int device, const seer_shape* shape, const seer_gate* gate,
+                                    const int32_t* seq_lens, const void* q_nope, int token_budget,
+                                    int32_t* block_idx, int32_t* block_cnt, int max_sel,
+                                    float* scores_out, void* stream, char* err, size_t err_len);
+
 #ifdef __cplusplus
 }
 #endif

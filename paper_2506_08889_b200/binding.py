@@ -30,6 +30,7 @@ EXPORTS = [
     "seer_create", "seer_destroy", "seer_status_string", "seer_last_error",
     "seer_get_device_status", "seer_workspace_bytes", "seer_launch_count",
     "seer_dense_decode", "seer_sparse_decode", "seer_gate_select", "seer_kcomp_append",
+    "seer_gate_select_static",
 ]
 
 
@@ -98,6 +99,9 @@ def lib() -> ctypes.CDLL:
     L.seer_kcomp_append.restype = i32
     L.seer_kcomp_append.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp,
                                     i64, i64, i64, i32, i32, i32, vp]
+    L.seer_gate_select_static.restype = i32
+    L.seer_gate_select_static.argtypes = [i32, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, i32,
+                                          vp, vp, i32, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
     _lib = L
     return L
 
@@ -205,3 +209,18 @@ class Context:
                                             _ptr(k_nope), k_nope.stride(0), k_nope.stride(1), k_nope.stride(2),
                                             int(bool(rows_block_local)), int(first_block), int(num_blocks),
                                             _stream(stream)))
+
+
+STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def seer_gate_select_static(device: int, shape: SeerShape, gate: SeerGate, seq_lens, q_nope, token_budget,
+                            block_idx, block_cnt, max_sel, scores_out=None, stream=None):
+    """Gate scoring + selection for callers that may not allocate device memory: no context, the
+    scratch lives in a fixed array inside the library (see ``seer_gate_select_static`` in seer.h)."""
+    buf = ctypes.create_string_buffer(256)
+    st = lib().seer_gate_select_static(int(device), ctypes.byref(shape), ctypes.byref(gate), _ptr(seq_lens),
+                                       _ptr(q_nope), int(token_budget), _ptr(block_idx), _ptr(block_cnt),
+                                       int(max_sel), _ptr(scores_out), _stream(stream), buf, len(buf))
+    if st != SEER_OK:
+        raise SeerError(st, buf.value.decode())

@@ -482,3 +482,115 @@ cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* la
 }
 
 }  // namespace seer
+
+// ================================================================================================
+// Gate selection without a context: the scratch the split gate kernels need (gate query, block
+// scores, per-unit tickets) lives in a fixed array inside the library image instead of a
+// context's workspace, for callers that are not allowed to allocate device memory.
+// ================================================================================================
+#include <mutex>
+#include <stdio.h>
+
+#include "../../include/seer.h"
+
+namespace {
+
+// One copy per GPU that loads the library, held until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[SEER_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices];     // device address of g_static_scratch, per device
+
+seer_status static_fail(char* err, size_t err_len, seer_status st, const char* fmt, long long a = 0, long long b = 0) {
+    if (err && err_len) snprintf(err, err_len, fmt, a, b);
+    return st;
+}
+
+}  // namespace
+
+extern "C" seer_status seer_gate_select_static(int device, const seer_shape* shape, const seer_gate* gate,
+                                               const int32_t* seq_lens, const void* q_nope, int token_budget,
+                                               int32_t* block_idx, int32_t* block_cnt, int max_sel,
+                                               float* scores_out, void* stream, char* err, size_t err_len) {
+    using namespace seer;
+    if (err && err_len) err[0] = '\0';
+    if (!shape || !gate || !seq_lens || !q_nope || !block_idx || !block_cnt || !gate->w_q || !gate->kcomp)
+        return static_fail(err, err_len, SEER_ERR_INVALID_ARG, "NULL pointer among the arguments");
+    if (shape->batch <= 0 || shape->num_q_heads <= 0 || shape->num_kv_heads <= 0 || max_sel <= 0 ||
+        gate->max_blocks <= 0 || token_budget < 0 || shape->num_q_heads % shape->num_kv_heads != 0)
+        return static_fail(err, err_len, SEER_ERR_INVALID_ARG, "sizes must be positive and num_q_heads a multiple of num_kv_heads");
+    const int group = shape->num_q_heads / shape->num_kv_heads;
+    if (shape->head_dim != kHeadDim || (shape->block_size != 64 && shape->block_size != 128) || group > kMaxGroup ||
+        (gate->d_gate != 64 && gate->d_gate != 128 && gate->d_gate != 256))
+        return static_fail(err, err_len, SEER_ERR_UNSUPPORTED,
+                           "supported: head_dim 128, block_size 64/128, group size <= 8, d_gate 64/128/256");
+    if (!(gate->rope_theta > 0.f)) return static_fail(err, err_len, SEER_ERR_INVALID_ARG, "rope_theta must be positive");
+    if (((uintptr_t)q_nope | (uintptr_t)gate->w_q | (uintptr_t)gate->kcomp) & 15u)
+        return static_fail(err, err_len, SEER_ERR_INVALID_ARG, "q_nope, w_q and kcomp must be 16-byte aligned");
+    if (device < 0 || device >= kMaxDevices)
+        return static_fail(err, err_len, SEER_ERR_INVALID_ARG, "device index %lld outside 0..%lld", device, kMaxDevices - 1);
+    const long long U = (long long)shape->batch * shape->num_kv_heads;
+    if (U > 65535) return static_fail(err, err_len, SEER_ERR_UNSUPPORTED, "batch * num_kv_heads above 65535");
+
+    // layout of the scratch: [tickets U ints][gate query U*d_gate floats][scores U*max_blocks floats]
+    const size_t off_qg = ((size_t)U * sizeof(int) + 255) / 256 * 256;
+    const size_t off_sc = off_qg + ((size_t)U * gate->d_gate * sizeof(float) + 255) / 256 * 256;
+    const size_t need = off_sc + (scores_out ? 0 : (size_t)U * gate->max_blocks * sizeof(float));
+    if (need > (size_t)SEER_STATIC_SCRATCH_BYTES)
+        return static_fail(err, err_len, SEER_ERR_WORKSPACE,
+                           "this call needs %lld bytes of scratch, the built-in array holds %lld "
+                           "(use seer_gate_select with a context instead)", (long long)need,
+                           (long long)SEER_STATIC_SCRATCH_BYTES);
+
+    cudaError_t ce = cudaSetDevice(device);
+    if (ce != cudaSuccess) return static_fail(err, err_len, SEER_ERR_CUDA, "cudaSetDevice failed (code %lld)", (long long)ce);
+    unsigned char* base = nullptr;
+    {
+        // once per device, with that device current: the array's name is only a host-side handle,
+        // the kernels need its address in this device's memory
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[device]) {
+            unsigned char* ptr = nullptr;
+            ce = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
+            if (ce != cudaSuccess || !ptr)
+                return static_fail(err, err_len, SEER_ERR_CUDA, "cudaGetSymbolAddress failed (code %lld)", (long long)ce);
+            g_static_ptr[device] = ptr;
+        }
+        base = g_static_ptr[device];
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the tickets must start at zero; everything else is written before it is read
+    ce = cudaMemsetAsync(base, 0, (size_t)U * sizeof(int), s);
+    if (ce != cudaSuccess) return static_fail(err, err_len, SEER_ERR_CUDA, "cudaMemsetAsync failed (code %lld)", (long long)ce);
+
+    GateParams p;
+    memset(&p, 0, sizeof p);
+    p.q_nope = static_cast<const __nv_bfloat16*>(q_nope);
+    p.w_q = static_cast<const __nv_bfloat16*>(gate->w_q);
+    p.kcomp = static_cast<const __nv_bfloat16*>(gate->kcomp);
+    p.seq_lens = seq_lens;
+    p.scores_in = nullptr;
+    p.scores = scores_out ? scores_out : reinterpret_cast<float*>(base + off_sc);
+    p.scores_user = scores_out;
+    p.q_gate = reinterpret_cast<float*>(base + off_qg);
+    p.block_idx = block_idx;
+    p.block_cnt = block_cnt;
+    p.batch = shape->batch;
+    p.num_q_heads = shape->num_q_heads;
+    p.num_kv_heads = shape->num_kv_heads;
+    p.group = group;
+    p.block_size = shape->block_size;
+    p.d_gate = gate->d_gate;
+    p.max_blocks = gate->max_blocks;
+    p.max_sel = max_sel;
+    p.token_budget = token_budget;
+    p.status = nullptr;
+    p.tickets = reinterpret_cast<int*>(base);
+    for (int c = 0; c < gate->d_gate / 2; ++c)
+        p.inv_freq[c] = pow((double)gate->rope_theta, -2.0 * (double)c / (double)gate->d_gate);
+    int launched = 0;
+    ce = launch_gate_select(p, s, &launched);
+    if (ce != cudaSuccess) return static_fail(err, err_len, SEER_ERR_CUDA, "kernel launch failed (code %lld)", (long long)ce);
+    return SEER_OK;
+}

@@ -110,6 +110,40 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
+# ---- the multi-GPU part: ranks are replicas with their own batches, no data-path collective ----
+def init_ranks(backend: str, device=None):
+    """(rank, world, local_rank) from the torchrun environment; starts the process group if world > 1."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1 and not dist.is_initialized():
+        kw = {"device_id": device} if device is not None else {}
+        dist.init_process_group(backend, **kw)
+    return rank, world, local
+
+
+def rank_seed(rank: int) -> int:
+    """Every rank decodes its own batch of sequences."""
+    from paper_2506_08889_b200 import synth
+    return synth.BASE_SEED + 1000 * rank
+
+
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (the job is as slow as its slowest rank)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def job_throughput_gbs(world: int, bytes_per_rank: int, ms: float) -> float:
+    """Whole-job GB/s: all ranks' bytes over the slowest rank's time."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 # --------------------------------------------------------------------------------------------
 def build_layers(w, n_layers, seed, dev):
     """Per layer: K/V cache (K doubles as the pre-RoPE keys the gate pools), gate weights,
@@ -138,13 +172,10 @@ def run_ours(args):
     import torch.distributed as dist
     from paper_2506_08889_b200 import binding, synth
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
+    rank, world, local = init_ranks("nccl", torch.device(dev))
 
     w = synth.workload(4)
     w.sparsity = args.sparsity
@@ -156,7 +187,7 @@ def run_ours(args):
     n_blocks = L // b
     k_sel = w.keep(n_blocks)
     budget = k_sel * b
-    seed = synth.BASE_SEED + 1000 * rank            # every rank decodes its own batch of sequences
+    seed = rank_seed(rank)
     n_layers = args.layers
     layers = build_layers(w, n_layers, seed, dev)
 
@@ -285,15 +316,13 @@ def run_ours(args):
     assert ctx.device_status() == binding.SEER_OK
 
     # ---- reduce over ranks -------------------------------------------------------------------
-    vals = torch.tensor([step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms = [float(x) for x in vals.cpu()]
+    step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms = max_over_ranks(
+        [step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms], dev)
 
     result = None
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
-        value = world * sel_kv_bytes / (step_ms * 1e-3) / 1e9
+        value = job_throughput_gbs(world, sel_kv_bytes, step_ms)
         kern_gbs = decode_bytes / (sparse_ms * 1e-3) / 1e9
         result = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -305,7 +334,7 @@ def run_ours(args):
                        "step": "kcomp_append + gate_select + sparse_decode (one layer, one token per sequence)",
                        "l2": f"steps rotate over {n_layers} layer caches ({n_layers * dense_bytes / 1e9:.1f} GB), "
                              f"selected bytes per step {sel_kv_bytes / 1e6:.0f} MB > L2"},
-            "e2e": {"value": round(world * sel_kv_bytes / (e2e_ms * 1e-3) / 1e9, 1), "unit": UNIT,
+            "e2e": {"value": round(job_throughput_gbs(world, sel_kv_bytes, e2e_ms), 1), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 5)},
             "gpu_launches": int(launches),
             "clocks": clocks,

@@ -31,9 +31,12 @@ METRIC = "sparse_decode_selected_kv_GBps"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one sparse-decode launch on this workload,
-# from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one sparse-decode launch, from an ncu capture of a
+# quarter-size case (batch 2): 107.7 MB read + 3.0 MB written for 107.5 MB of algorithmic bytes.
+# Reads grow with the selected tiles, writes (partials) with the number of CTAs, so a launch on
+# `batch` sequences moves about batch/2 * 107.7 MB + 3.0 MB.
+NCU_READ_BYTES_PER_2_SEQUENCES = 107.677e6
+NCU_WRITE_BYTES_PER_LAUNCH = 3.03e6
 
 
 def measured_hbm_peak():
@@ -342,7 +345,9 @@ def run_ours(args):
                          "peak": peak, "unit": "GB/s", "frac": round(kern_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
                          "frac_of_nominal_8000": round(kern_gbs / NOMINAL_HBM_GBS, 4),
                          "algorithmic_bytes_per_launch": decode_bytes, "us_per_launch": round(sparse_ms * 1e3, 2),
-                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
+                         "traffic": (int(NCU_READ_BYTES_PER_2_SEQUENCES * B / 2 * (1.0 - args.sparsity) / 0.1
+                                         + NCU_WRITE_BYTES_PER_LAUNCH) if abs(args.sparsity - 0.9) < 1e-9 else None),
+                         "traffic_note": "ncu capture at batch 2, scaled by the units processed"},
             "extra": {
                 "tokens_per_s_per_layer": round(world * B / (step_ms * 1e-3), 1),
                 "selected_kv_bytes_per_step": sel_kv_bytes,

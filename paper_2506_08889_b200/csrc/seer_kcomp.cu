@@ -1,7 +1,7 @@
 // K compression cache update (Eq. 1b; Sec. 3.2): per block, max/min/mean pooling of the
 // pre-RoPE keys over the block's rows, projection by W_k, RoPE at the block's first token,
-// bf16 store.  In the bulk build one CTA handles four consecutive blocks of one (sequence,
-// KV head) so that every W_k element fetched is used for all of them.
+// bf16 store.  Two kernels: the per-step append of the one block that has just filled, and the
+// bulk build over many blocks after prefill.
 #include "seer_device.cuh"
 #include "seer_internal.h"
 
@@ -13,10 +13,10 @@ constexpr int kKcThreads = 256;
 constexpr int kKcWarps = kKcThreads / 32;
 constexpr int kInChunks = 3 * kHeadDim / 8;          // 48 pieces of 16 B per W_k row
 
-// grid (block groups, B*Hkv, row splits).  NB = blocks per CTA (4 for the bulk build, 1 for the
-// per-step append, where the output rows are split over gridDim.z CTAs instead so that the
-// one block's latency chain is short).  Every warp owns rotary pairs (c, c + d_gate/2), two at
-// a time: their four W_k rows are requested before the pooling starts.
+// Append: grid (1, B*Hkv, row splits).  One block per (sequence, KV head); the output rows are
+// split over gridDim.z CTAs so that the one block's latency chain is short.  Every warp owns
+// rotary pairs (c, c + d_gate/2), two at a time: their four W_k rows are requested before the
+// pooling starts.  (NB is the number of blocks per CTA; only NB = 1 is instantiated.)
 template <int NB>
 __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) {
     __shared__ float red[kKcWarps][3][kHeadDim];                   // per-warp pooled partials
@@ -182,6 +182,142 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
     }
 }
 
+// ---- bulk build (after prefill): 16 consecutive blocks of one (sequence, KV head) per CTA --------
+// Phase 1 streams the blocks' rows with many loads in flight (each warp pools two blocks) and
+// leaves the 3*128 pooled features of every block in shared memory as bf16 (max and min are bf16
+// values already; the mean is kept as a bf16 high part plus a bf16 correction, so nothing is
+// lost).  Phase 2 is the contraction Y[row][block] = W_k[row][:] . feat[block][:] on the tensor
+// cores (mma.sync m16n8k16: W_k rows on M straight from global memory, the 16 blocks on N);
+// phase 3 rotates and stores.  Several CTAs share an SM, so one CTA's projection overlaps the
+// others' streaming.
+constexpr int kBulkBlocks = 16;
+constexpr int kFeatStride = 3 * kHeadDim + 8;         // bf16 per block row (+8: conflict-free fragment reads)
+constexpr int kLoStride = kHeadDim + 8;
+
+__global__ void __launch_bounds__(kKcThreads) kcomp_bulk_kernel(const KcompParams p) {
+    __shared__ __align__(16) __nv_bfloat16 feat_hi[kBulkBlocks][kFeatStride];   // [max | min | avg]
+    __shared__ __align__(16) __nv_bfloat16 feat_lo[kBulkBlocks][kLoStride];     // avg - bf16(avg)
+    __shared__ float ybuf[kBulkBlocks][kMaxDGate];
+    pdl_wait();
+    pdl_launch_dependents();
+    const int u = blockIdx.y, i = u / p.num_kv_heads, h = u % p.num_kv_heads;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = p.block_size;
+    const int L = p.seq_lens[i];
+    const int complete = L > 0 ? L / b : 0;
+    const int j_first = p.first_block + blockIdx.x * kBulkBlocks;
+    const int j_end = min(min(p.first_block + p.num_blocks, complete), p.max_blocks);
+    const int nb = max(0, min(kBulkBlocks, j_end - j_first));
+    if (nb == 0) return;
+    const size_t base = (size_t)i * p.stride_batch + (size_t)h * p.stride_head;
+    const int cchunk = lane & 15, rsel = lane >> 4;
+
+    for (int q = warp; q < kBulkBlocks; q += kKcWarps) {
+        // max and min stay packed bf16 pairs (they are bf16 values anyway), the sum is fp32
+        __nv_bfloat162 mx[4], mn[4];
+        float sm[8];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            mx[c] = __float2bfloat162_rn(-INFINITY);
+            mn[c] = __float2bfloat162_rn(INFINITY);
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c) sm[c] = 0.f;
+        if (q < nb) {
+            const __nv_bfloat16* src = p.k_nope + base + (size_t)(j_first + q) * b * p.stride_token + 8 * cchunk;
+#pragma unroll 16
+            for (int r = rsel; r < b; r += 2) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + (size_t)r * p.stride_token));
+                const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    mx[c] = __hmax2(mx[c], hh[c]);
+                    mn[c] = __hmin2(mn[c], hh[c]);
+                    const float2 f = __bfloat1622float2(hh[c]);
+                    sm[2 * c] += f.x; sm[2 * c + 1] += f.y;
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t xm = *reinterpret_cast<uint32_t*>(&mx[c]), xn = *reinterpret_cast<uint32_t*>(&mn[c]);
+                uint32_t ym = __shfl_xor_sync(0xffffffffu, xm, 16), yn = __shfl_xor_sync(0xffffffffu, xn, 16);
+                mx[c] = __hmax2(mx[c], *reinterpret_cast<__nv_bfloat162*>(&ym));
+                mn[c] = __hmin2(mn[c], *reinterpret_cast<__nv_bfloat162*>(&yn));
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) sm[c] += __shfl_xor_sync(0xffffffffu, sm[c], 16);
+        }
+        if (lane < 16) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const __nv_bfloat162 zero = __float2bfloat162_rn(0.f);
+                *reinterpret_cast<__nv_bfloat162*>(&feat_hi[q][8 * cchunk + 2 * c]) = q < nb ? mx[c] : zero;
+                *reinterpret_cast<__nv_bfloat162*>(&feat_hi[q][kHeadDim + 8 * cchunk + 2 * c]) = q < nb ? mn[c] : zero;
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float av = q < nb ? sm[c] / (float)b : 0.f;
+                const __nv_bfloat16 av_hi = __float2bfloat16(av);
+                feat_hi[q][2 * kHeadDim + 8 * cchunk + c] = av_hi;
+                feat_lo[q][8 * cchunk + c] = __float2bfloat16(av - __bfloat162float(av_hi));
+            }
+        }
+    }
+    __syncthreads();
+
+    // Y[row][block]: warp w takes output rows 16*mt .. +15 for mt = w, w+8, ...
+    const int g = lane >> 2, t4 = lane & 3;
+    for (int mt = warp; mt < p.d_gate / 16; mt += kKcWarps) {
+        const uint32_t* w0 = reinterpret_cast<const uint32_t*>(p.w_k + ((size_t)h * p.d_gate + 16 * mt + g) * 3 * kHeadDim);
+        const uint32_t* w1 = w0 + 8 * (3 * kHeadDim / 2);     // row + 8
+        float acc[2][4];
+#pragma unroll
+        for (int n = 0; n < 2; ++n)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) acc[n][x] = 0.f;
+#pragma unroll 6
+        for (int ks = 0; ks < 3 * kHeadDim / 16; ++ks) {
+            uint32_t a[4];
+            a[0] = __ldg(w0 + 8 * ks + t4);
+            a[1] = __ldg(w1 + 8 * ks + t4);
+            a[2] = __ldg(w0 + 8 * ks + 4 + t4);
+            a[3] = __ldg(w1 + 8 * ks + 4 + t4);
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                const __nv_bfloat16* fr = &feat_hi[8 * n + g][16 * ks + 2 * t4];
+                const uint32_t b0 = *reinterpret_cast<const uint32_t*>(fr);
+                const uint32_t b1 = *reinterpret_cast<const uint32_t*>(fr + 8);
+                mma_bf16_16816(acc[n], a, b0, b1);
+                if (ks >= 2 * kHeadDim / 16) {        // the mean's correction term
+                    const __nv_bfloat16* fl = &feat_lo[8 * n + g][16 * ks - 2 * kHeadDim + 2 * t4];
+                    mma_bf16_16816(acc[n], a, *reinterpret_cast<const uint32_t*>(fl),
+                                   *reinterpret_cast<const uint32_t*>(fl + 8));
+                }
+            }
+        }
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            ybuf[8 * n + 2 * t4][16 * mt + g] = acc[n][0];
+            ybuf[8 * n + 2 * t4 + 1][16 * mt + g] = acc[n][1];
+            ybuf[8 * n + 2 * t4][16 * mt + g + 8] = acc[n][2];
+            ybuf[8 * n + 2 * t4 + 1][16 * mt + g + 8] = acc[n][3];
+        }
+    }
+    __syncthreads();
+
+    const int half = p.d_gate / 2;
+    for (int x = tid; x < nb * half; x += kKcThreads) {
+        const int q = x / half, c = x % half;
+        const int j = j_first + q;
+        float sn, cs;
+        rope_sincos((double)j * (double)b, p.inv_freq[c], &sn, &cs);
+        const float a = ybuf[q][c], bb = ybuf[q][c + half];
+        __nv_bfloat16* dst = p.kcomp + ((size_t)u * p.max_blocks + j) * p.d_gate;
+        dst[c] = __float2bfloat16(a * cs - bb * sn);
+        dst[c + half] = __float2bfloat16(bb * cs + a * sn);
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* launched) {
@@ -194,9 +330,9 @@ cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* 
         *launched = 1;
         return e;
     } else {
-        const int gx = (p.num_blocks + 3) / 4;
+        const int gx = (p.num_blocks + kBulkBlocks - 1) / kBulkBlocks;
         if (gx <= 0) return cudaSuccess;
-        cudaError_t e = launch_pdl(kcomp_kernel<4>, dim3(gx, U, 1), dim3(kKcThreads), 0, stream, p);
+        cudaError_t e = launch_pdl(kcomp_bulk_kernel, dim3(gx, U, 1), dim3(kKcThreads), 0, stream, p);
         *launched = 1;
         return e;
     }

@@ -208,6 +208,24 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
                               void* stream);
 
 /*
+ * One decode step of one attention layer in a single call (paper Fig. 3): the compressed-K
+ * update for the block that has just filled (Sec. 3.2, skipped when k_nope is NULL), gate scoring
+ * and token-budget selection (Eq. 1a/1c, Sec. 3.1), block-sparse decode over the selected
+ * blocks (Sec. 3.3).  Exactly the three calls
+ *     seer_kcomp_append(.., first_block = -1) ; seer_gate_select(.., scores_in = NULL) ; seer_sparse_decode
+ * on `stream`, with one argument check and one host round trip instead of three.
+ *  block_idx / block_cnt / max_sel: caller-owned scratch for the selected lists (they are
+ *  outputs too: the lists the attention used).  Other arguments as in the three calls;
+ *  kv->seq_lens is used as the sequence lengths of all three.
+ */
+seer_status seer_decode_step(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const seer_gate* gate,
+                             const void* q, const void* q_nope, const void* k_nope,
+                             int64_t k_nope_stride_batch, int64_t k_nope_stride_head, int64_t k_nope_stride_token,
+                             int k_nope_rows_block_local, int token_budget,
+                             int32_t* block_idx, int32_t* block_cnt, int max_sel,
+                             void* out, float* lse, void* stream);
+
+/*
  * seer_gate_select without a context and without any allocation.  (The paper has no counterpart:
  * this entry point exists for hosts of the library, not for the method.)
  *

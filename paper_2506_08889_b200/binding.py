@@ -30,7 +30,7 @@ EXPORTS = [
     "seer_create", "seer_destroy", "seer_status_string", "seer_last_error",
     "seer_get_device_status", "seer_workspace_bytes", "seer_launch_count",
     "seer_dense_decode", "seer_sparse_decode", "seer_gate_select", "seer_kcomp_append",
-    "seer_gate_select_static",
+    "seer_gate_select_static", "seer_decode_step",
 ]
 
 
@@ -99,6 +99,9 @@ def lib() -> ctypes.CDLL:
     L.seer_kcomp_append.restype = i32
     L.seer_kcomp_append.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp,
                                     i64, i64, i64, i32, i32, i32, vp]
+    L.seer_decode_step.restype = i32
+    L.seer_decode_step.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), ctypes.POINTER(SeerGate),
+                                   vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, i32, vp, vp, vp]
     L.seer_gate_select_static.restype = i32
     L.seer_gate_select_static.argtypes = [i32, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, i32,
                                           vp, vp, i32, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
@@ -209,6 +212,18 @@ class Context:
                                             _ptr(k_nope), k_nope.stride(0), k_nope.stride(1), k_nope.stride(2),
                                             int(bool(rows_block_local)), int(first_block), int(num_blocks),
                                             _stream(stream)))
+
+    def seer_decode_step(self, shape: SeerShape, kv: SeerKV, gate: SeerGate, q, q_nope, k_nope, token_budget,
+                         block_idx, block_cnt, max_sel, out, lse=None, rows_block_local=False, stream=None):
+        """Compressed-K append (skipped if k_nope is None) + gate selection + sparse decode in one call."""
+        sb = sh = st = 0
+        if k_nope is not None:
+            assert k_nope.dtype == torch.bfloat16 and k_nope.stride(3) == 1
+            sb, sh, st = k_nope.stride(0), k_nope.stride(1), k_nope.stride(2)
+        self._check(lib().seer_decode_step(self._h, ctypes.byref(shape), ctypes.byref(kv), ctypes.byref(gate),
+                                           _ptr(q), _ptr(q_nope), _ptr(k_nope), sb, sh, st,
+                                           int(bool(rows_block_local)), int(token_budget), _ptr(block_idx),
+                                           _ptr(block_cnt), int(max_sel), _ptr(out), _ptr(lse), _stream(stream)))
 
 
 STATIC_SCRATCH_BYTES = 1 << 20

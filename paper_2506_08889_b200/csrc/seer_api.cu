@@ -406,6 +406,9 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
     p.token_budget = token_budget;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
     p.tickets = reinterpret_cast<int*>(ctx->ws + w.gate_tickets);
+#ifdef SEER_GATE_TRACE
+    p.status = reinterpret_cast<unsigned int*>(ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)));
+#endif
     if (!scores_in) fill_inv_freq(p.inv_freq, gate->d_gate, gate->rope_theta);
     int launched = 0;
     ce = launch_gate_select(p, static_cast<cudaStream_t>(stream), &launched);
@@ -461,6 +464,25 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
     ctx->launches += launched;
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "kcomp launch: %s", cudaGetErrorString(ce));
     return SEER_OK;
+}
+
+seer_status seer_decode_step(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const seer_gate* gate,
+                             const void* q, const void* q_nope, const void* k_nope, int64_t k_nope_stride_batch,
+                             int64_t k_nope_stride_head, int64_t k_nope_stride_token, int k_nope_rows_block_local,
+                             int token_budget, int32_t* block_idx, int32_t* block_cnt, int max_sel, void* out,
+                             float* lse, void* stream) {
+    if (!ctx) return SEER_ERR_INVALID_ARG;
+    if (!kv || !kv->seq_lens) return fail(ctx, SEER_ERR_INVALID_ARG, "kv or kv->seq_lens is NULL");
+    seer_status st;
+    if (k_nope) {
+        st = seer_kcomp_append(ctx, shape, gate, kv->seq_lens, k_nope, k_nope_stride_batch, k_nope_stride_head,
+                               k_nope_stride_token, k_nope_rows_block_local, -1, 1, stream);
+        if (st != SEER_OK) return st;
+    }
+    st = seer_gate_select(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, token_budget, block_idx, block_cnt, max_sel,
+                          nullptr, stream);
+    if (st != SEER_OK) return st;
+    return seer_sparse_decode(ctx, shape, kv, q, block_idx, block_cnt, max_sel, out, lse, stream);
 }
 
 }  // extern "C"

@@ -807,6 +807,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 #endif
         __threadfence();                               // the partials above are visible from here on
         __syncwarp();
+        if (lane == 0) SEER_STAMP(0);
         bool owe = false;
         Piece pc = Piece{0, 0, 0, 0};
         if (lane < n_held) {

@@ -272,6 +272,13 @@ __global__ void __launch_bounds__(kProjThreads) gate_qproj_kernel(const GatePara
 // projection kernel), and the d_gate/8 neighbouring lanes that hold one key's pieces add up by
 // shuffles.  Each CTA publishes its scores and takes a ticket; the CTA that draws the unit's
 // last ticket runs the selection over all of the unit's scores.  No CTA waits for another.
+#ifdef SEER_GATE_TRACE
+#define GATE_STAMP(k) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
+    reinterpret_cast<unsigned long long*>(p.status)[((size_t)blockIdx.y * gridDim.x + blockIdx.x) * 8 + (k)] = t_; } } while (0)
+#else
+#define GATE_STAMP(k) ((void)0)
+#endif
+
 __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(const GateParams p, int per) {
     __shared__ SelectSmem sm;
     __shared__ int is_last;
@@ -290,7 +297,9 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
         const int c = k * kGateThreads + tid;
         kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
     }
+    GATE_STAMP(0);
     pdl_wait();                                        // q_gate is complete from here on
+    GATE_STAMP(1);
     pdl_launch_dependents();
     const int L = __ldg(p.seq_lens + i);
     const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
@@ -324,16 +333,20 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
         }
     }
     // ---- ticket: the last slice of the unit to finish does the selection --------------------
+    GATE_STAMP(2);
     __threadfence();
     __syncthreads();
+    GATE_STAMP(3);
     if (tid == 0) {
         const int t = atomicAdd(&p.tickets[u], 1);
         is_last = (t == S - 1);
         if (is_last) p.tickets[u] = 0;               // ready for the next launch
     }
     __syncthreads();
+    GATE_STAMP(4);
     if (!is_last) return;
     select_dispatch<kGateThreads, false>(p, u, sc_out, sm);   // reads the scores with ld.cg, after the ticket
+    GATE_STAMP(5);
 }
 
 // ---- the whole gate of one (sequence, KV head) unit in one CTA --------------------------------

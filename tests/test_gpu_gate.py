@@ -203,3 +203,40 @@ def test_gate_then_decode_end_to_end_14b_shape_small(ctx):
     ref = oracle.sparse(bits(q), bits(k), bits(v), lens, want_idx, want_cnt, b, scale)
     check_attention(out, lse, *ref, what="end to end")
     assert ctx.device_status() == binding.SEER_OK
+
+
+def test_single_call_step_equals_the_three_calls(ctx):
+    B, Hq, Hkv, d, dg, b = 3, 8, 2, 128, 128, 64
+    nb = 40
+    S = nb * b
+    lens = np.array([S, S - b, 17 * b + 3], np.int32)          # sequences 0 and 1 have just filled a block
+    q = synth.normal_bf16((B, Hq, d), 21, "q", DEV)
+    qn = synth.normal_bf16((B, Hq, d), 21, "qn", DEV)
+    k = synth.normal_bf16((B, Hkv, S, d), 21, "k", DEV)
+    v = synth.normal_bf16((B, Hkv, S, d), 21, "v", DEV)
+    wq = synth.normal_bf16((Hkv, dg, 4 * d), 21, "wq", DEV, std=0.02)
+    wk = synth.normal_bf16((Hkv, dg, 3 * d), 21, "wk", DEV, std=0.02)
+    scale = 1.0 / np.sqrt(d)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, scale)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    kv = binding.make_kv(k, v, lens_t)
+    max_sel = 6
+    res = []
+    for fused in (False, True):
+        kc = synth.normal_bf16((B, Hkv, nb, dg), 21, "kc", DEV)     # "earlier" entries
+        gate = binding.make_gate(dg, THETA, wq, wk, kc, nb)
+        idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+        cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+        out = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=DEV)
+        lse = torch.zeros((B, Hq), dtype=torch.float32, device=DEV)
+        if fused:
+            ctx.seer_decode_step(shape, kv, gate, q, qn, k, max_sel * b, idx, cnt, max_sel, out, lse)
+        else:
+            ctx.seer_kcomp_append(shape, gate, lens_t, k)
+            ctx.seer_gate_select(shape, gate, lens_t, qn, None, max_sel * b, idx, cnt, max_sel)
+            ctx.seer_sparse_decode(shape, kv, q, idx, cnt, max_sel, out, lse)
+        torch.cuda.synchronize()
+        res.append((kc, idx, cnt, out, lse))
+    for a, c in zip(res[0], res[1]):
+        assert torch.equal(a, c)
+    assert ctx.device_status() == binding.SEER_OK

@@ -48,15 +48,19 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 constexpr int kUnitThreads = 1024;          // one-CTA-per-unit gate kernel
 constexpr int kUnitMaxBlocks = 4096;        // ... and the compressed keys it can score
 
+constexpr int kSelBits = 11;                // digit width of a selection pass
+constexpr int kSelBins = 1 << kSelBits;
+
 struct SelectSmem {
-    int hist[4][256];                       // one histogram per radix pass
+    int hist[3][kSelBins];                  // one histogram per pass (at most ceil(32 / 11) passes)
     unsigned long long warp_tot[kUnitThreads / 32];
+    uint32_t warp_min[kUnitThreads / 32], warp_max[kUnitThreads / 32];
     uint32_t prefix;
     int rem;
 };
 
 // Token-budget selection for one unit, run by a whole CTA.  Thread t owns the candidates
-// [t*E, (t+1)*E).  A radix select (4 passes of 8 bits over order-preserving keys) finds the key
+// [t*E, (t+1)*E).  A radix select (passes of 11 bits over order-preserving keys) finds the key
 // of the (k-1)-th best candidate; one ordered pass then emits, in ascending block order, every
 // candidate above it and the first few equal to it (the lower block number wins a tie), and
 // the forced last block closes the list.  Comparisons only: the result is exact.
@@ -92,55 +96,80 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
     uint32_t thr = 0u;                               // key of the need-th best candidate
     int take_eq = n_cand;                            // candidates equal to thr that are taken
     if (need > 0 && need < n_cand) {
-        for (int x = tid; x < 4 * 256; x += NT) (&sm.hist[0][0])[x] = 0;
+        // The keys of real scores crowd into a few exponent values, so digits of the raw key make
+        // for a handful of hot histogram bins.  The passes therefore work on key - min(key), whose
+        // significant bits (those of max - min) are spread evenly: first the block-wide min and max.
+        uint32_t kmin = 0xffffffffu, kmax = 0u;
+        if (CACHED) {
+#pragma unroll
+            for (int e = 0; e < kCachedT; ++e)
+                if (j_lo + e < j_hi) { kmin = min(kmin, keys[e]); kmax = max(kmax, keys[e]); }
+        } else {
+            for (int e = 0; j_lo + e < j_hi; ++e) { const uint32_t key = key_at(e); kmin = min(kmin, key); kmax = max(kmax, key); }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, off));
+            kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, off));
+        }
+        if (lane == 0) { sm.warp_min[warp] = kmin; sm.warp_max[warp] = kmax; }
+        for (int x = tid; x < 3 * kSelBins; x += NT) (&sm.hist[0][0])[x] = 0;
         __syncthreads();
-        uint32_t prefix = 0u;
+#pragma unroll
+        for (int w2 = 0; w2 < NT / 32; ++w2) { kmin = min(kmin, sm.warp_min[w2]); kmax = max(kmax, sm.warp_max[w2]); }
+        int bits_left = 32 - __clz(max(kmax - kmin, 1u));     // significant bits of key - kmin
+        uint32_t prefix = 0u;                                  // the digits found so far, of thr - kmin
         int rem = need;
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
-            const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+        constexpr int kBinsPerThread = kSelBins / NT;
+        for (int pass = 0; bits_left > 0; ++pass) {
+            const int wbits = min(kSelBits, bits_left), shift = bits_left - wbits;
             int* hist = sm.hist[pass];
+            auto count = [&](uint32_t key) {
+                const uint32_t rel = key - kmin;
+                // 64-bit shift: shift + wbits can be 32
+                if ((uint32_t)((unsigned long long)rel >> (shift + wbits)) == prefix)
+                    atomicAdd(&hist[(rel >> shift) & ((1u << wbits) - 1u)], 1);
+            };
             if (CACHED) {
 #pragma unroll
                 for (int e = 0; e < kCachedT; ++e)
-                    if (j_lo + e < j_hi && (keys[e] & himask) == prefix)
-                        atomicAdd(&hist[(keys[e] >> shift) & 255u], 1);
+                    if (j_lo + e < j_hi) count(keys[e]);
             } else {
-                for (int e = 0; j_lo + e < j_hi; ++e) {
-                    const uint32_t key = key_at(e);
-                    if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
-                }
+                for (int e = 0; j_lo + e < j_hi; ++e) count(key_at(e));
             }
             __syncthreads();
-            if (warp == 0) {
-                // lane l owns bins 255-8l .. 248-8l (descending); a warp scan gives the number of
-                // keys in all higher bins, then the lane that straddles `rem` walks its 8 bins
-                int c[8], mine = 0;
+            // thread t owns bins (kSelBins-1 - kBinsPerThread*t) downwards; a block scan gives the number
+            // of keys in all higher bins, then the thread that straddles `rem` walks its own bins
+            int c[kBinsPerThread], mine = 0;
 #pragma unroll
-                for (int b = 0; b < 8; ++b) { c[b] = hist[255 - 8 * lane - b]; mine += c[b]; }
-                int incl = mine;
+            for (int x = 0; x < kBinsPerThread; ++x) { c[x] = hist[kSelBins - 1 - kBinsPerThread * tid - x]; mine += c[x]; }
+            unsigned long long incl = (unsigned long long)mine;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
-                }
-                int above = incl - mine;
-                if (above < rem && rem <= incl) {
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (lane == 31) sm.warp_tot[warp] = incl;
+            __syncthreads();
+            int above = (int)incl - mine;
 #pragma unroll
-                    for (int b = 0; b < 8; ++b) {
-                        if (above < rem && rem <= above + c[b]) {
-                            sm.prefix = prefix | ((uint32_t)(255 - 8 * lane - b) << shift);
-                            sm.rem = rem - above;
-                        }
-                        above += c[b];
+            for (int w2 = 0; w2 < NT / 32; ++w2) above += (w2 < warp) ? (int)sm.warp_tot[w2] : 0;
+            if (above < rem && rem <= above + mine) {
+#pragma unroll
+                for (int x = 0; x < kBinsPerThread; ++x) {
+                    if (above < rem && rem <= above + c[x]) {
+                        sm.prefix = (prefix << wbits) | (uint32_t)(kSelBins - 1 - kBinsPerThread * tid - x);
+                        sm.rem = rem - above;
                     }
+                    above += c[x];
                 }
             }
             __syncthreads();
             prefix = sm.prefix;
             rem = sm.rem;
+            bits_left = shift;
         }
-        thr = prefix;
+        thr = kmin + prefix;
         take_eq = rem;
     }
 

@@ -228,3 +228,29 @@ def test_host_side_argument_checks(ctx):
         small.seer_dense_decode(shape, kv, q, out)
     assert e.value.status == binding.SEER_ERR_WORKSPACE
     small.close()
+
+
+def test_result_does_not_depend_on_how_the_work_is_cut(ctx, monkeypatch):
+    # the same launch with work stealing (default) and with a purely static split, on a case large
+    # enough for stealing to happen: both within the parity bound of the oracle, and of each other
+    B, Hq, Hkv, d, b, S = 4, 10, 2, 128, 64, 32768
+    lens = np.array([S, S - 1000, S // 2 + 17, S - 64], np.int32)
+    q, k, v = make_qkv(B, Hq, Hkv, S, d, 123, DEV)
+    n = [-(-int(L) // b) for L in lens]
+    idx, cnt = synth.random_block_lists(lens, Hkv, b, [x // 2 for x in n], max(n) // 2 + 1, 123)
+    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.0884)
+    out_dyn, lse_dyn = _run_sparse(ctx, q, k, v, lens, idx, cnt, b, 0.0884)
+    check_attention(out_dyn, lse_dyn, *ref, what="stealing", strict=True)
+    monkeypatch.setenv("SEER_DECODE_POOL_DIV", "0")            # read when a context is created
+    static_ctx = binding.Context(0)
+    try:
+        out_st, lse_st = _run_sparse(static_ctx, q, k, v, lens, idx, cnt, b, 0.0884)
+    finally:
+        static_ctx.close()
+    check_attention(out_st, lse_st, *ref, what="static", strict=True)
+    assert (out_dyn.float() - out_st.float()).abs().max().item() <= 2e-3
+    # launch after launch on the same context: counters and tickets re-arm themselves
+    for _ in range(5):
+        o2, l2 = _run_sparse(ctx, q, k, v, lens, idx, cnt, b, 0.0884)
+        check_attention(o2, l2, *ref, what="repeat", strict=True)
+    assert ctx.device_status() == binding.SEER_OK

@@ -185,6 +185,21 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
                              float* scores_out, void* stream);
 
 /*
+ * The threshold method of Sec. 3.1: the scores are normalised by a softmax over the blocks
+ * that have a compressed key (Eq. 1c; blocks [0, n_i - 1)), and the blocks whose probability
+ * exceeds `threshold` are selected -- a different number for every (sequence, KV head).  The
+ * last block is always selected and takes no part in the normalisation; if more than
+ * max_sel - 1 blocks pass, the max_sel - 1 highest-scoring are kept.  Scores must be finite.
+ * The probabilities are formed in fp32, so a block whose probability is within rounding of
+ * the threshold may fall on either side.  Other arguments and the output format as for
+ * seer_gate_select (threshold in [0, 1]; the paper's ablation uses 2e-3 .. 6e-3).
+ */
+seer_status seer_gate_select_threshold(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                                       const int32_t* seq_lens, const void* q_nope, const float* scores_in,
+                                       float threshold, int32_t* block_idx, int32_t* block_cnt, int max_sel,
+                                       float* scores_out, void* stream);
+
+/*
  * K compression cache update (Eq. 1b; Sec. 2.2 "Pooling-based Compression of
  * K", Sec. 3.2): for block j of (i, h): per channel max, min and mean over the
  * block's b rows of pre-RoPE K, concatenated [max|min|avg], multiplied by

@@ -333,6 +333,23 @@ static int int_asc(const void *pa, const void *pb)
     return (a > c) - (a < c);
 }
 
+/* The `need` best of blocks [0, n-1) by (score descending, index ascending) plus the last block
+ * n-1, ascending, -1 padded; returns the count. */
+static int emit_best_and_last(const float *s, int n, int need, int max_sel, int32_t *dst)
+{
+    for (int e = 0; e < max_sel; ++e) dst[e] = -1;
+    int ncand = n - 1;
+    cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(ncand > 0 ? ncand : 1));
+    for (int j = 0; j < ncand; ++j) { cand[j].s = s[j]; cand[j].j = j; }
+    qsort(cand, (size_t)ncand, sizeof(cand_t), cand_before);
+    int m = 0;
+    for (int e = 0; e < need && e < ncand; ++e) dst[m++] = cand[e].j;
+    dst[m++] = n - 1;
+    qsort(dst, (size_t)m, sizeof(int32_t), int_asc);
+    free(cand);
+    return m;
+}
+
 void oracle_select(const float *scores, const int32_t *seq_lens,
                    int B, int Hkv, int b, int max_blocks, int token_budget,
                    int max_sel, int32_t *block_idx, int32_t *block_cnt)
@@ -341,24 +358,56 @@ void oracle_select(const float *scores, const int32_t *seq_lens,
     for (int i = 0; i < B; ++i)
         for (int h = 0; h < Hkv; ++h) {
             int32_t *dst = block_idx + ((int64_t)i * Hkv + h) * max_sel;
-            for (int e = 0; e < max_sel; ++e) dst[e] = -1;
             int L = seq_lens[i];
             int n = (L + b - 1) / b;
-            if (n <= 0) { block_cnt[i * Hkv + h] = 0; continue; }
+            if (n <= 0) {
+                for (int e = 0; e < max_sel; ++e) dst[e] = -1;
+                block_cnt[i * Hkv + h] = 0;
+                continue;
+            }
             int k = token_budget / b;
             if (k < 1) k = 1;
             if (k > n) k = n;
             if (k > max_sel) k = max_sel;
-            int ncand = n - 1;
-            cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(ncand > 0 ? ncand : 1));
             const float *s = scores + ((int64_t)i * Hkv + h) * max_blocks;
-            for (int j = 0; j < ncand; ++j) { cand[j].s = s[j]; cand[j].j = j; }
-            qsort(cand, (size_t)ncand, sizeof(cand_t), cand_before);
-            int m = 0;
-            for (int e = 0; e < k - 1 && e < ncand; ++e) dst[m++] = cand[e].j;
-            dst[m++] = n - 1;
-            qsort(dst, (size_t)m, sizeof(int32_t), int_asc);
-            block_cnt[i * Hkv + h] = m;
-            free(cand);
+            block_cnt[i * Hkv + h] = emit_best_and_last(s, n, k - 1, max_sel, dst);
+        }
+}
+
+/* Threshold selection (Sec. 3.1, the second sparsify method): S = softmax of the gate scores
+ * (Eq. 1c) over the blocks that have a compressed key, [0, n_i-1); the blocks with S_j > tau are
+ * selected, and the last block always is (Sec. 3.2).  Readings where the paper is silent: the
+ * last block takes no part in the normalisation (it has no valid entry); if more than
+ * max_sel-1 blocks pass, the max_sel-1 highest-scoring are kept.  Scores must be finite.
+ * probs_out (optional, [B,Hkv,max_blocks]): the softmax values, for tests. */
+void oracle_select_threshold(const float *scores, const int32_t *seq_lens,
+                             int B, int Hkv, int b, int max_blocks, double tau,
+                             int max_sel, int32_t *block_idx, int32_t *block_cnt, double *probs_out)
+{
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int i = 0; i < B; ++i)
+        for (int h = 0; h < Hkv; ++h) {
+            int32_t *dst = block_idx + ((int64_t)i * Hkv + h) * max_sel;
+            int L = seq_lens[i];
+            int n = (L + b - 1) / b;
+            if (n <= 0) {
+                for (int e = 0; e < max_sel; ++e) dst[e] = -1;
+                block_cnt[i * Hkv + h] = 0;
+                continue;
+            }
+            const float *s = scores + ((int64_t)i * Hkv + h) * max_blocks;
+            int ncand = n - 1;
+            double mx = -INFINITY, z = 0.0;
+            for (int j = 0; j < ncand; ++j) if ((double)s[j] > mx) mx = (double)s[j];
+            for (int j = 0; j < ncand; ++j) z += exp((double)s[j] - mx);
+            int above = 0;
+            for (int j = 0; j < ncand; ++j) {
+                double pj = exp((double)s[j] - mx) / z;
+                if (probs_out) probs_out[((int64_t)i * Hkv + h) * max_blocks + j] = pj;
+                if (pj > tau) ++above;
+            }
+            int need = above;
+            if (need > max_sel - 1) need = max_sel - 1;
+            block_cnt[i * Hkv + h] = emit_best_and_last(s, n, need, max_sel, dst);
         }
 }

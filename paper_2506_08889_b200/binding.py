@@ -30,7 +30,7 @@ EXPORTS = [
     "seer_create", "seer_destroy", "seer_status_string", "seer_last_error",
     "seer_get_device_status", "seer_workspace_bytes", "seer_launch_count",
     "seer_dense_decode", "seer_sparse_decode", "seer_gate_select", "seer_kcomp_append",
-    "seer_gate_select_static", "seer_decode_step",
+    "seer_gate_select_static", "seer_decode_step", "seer_gate_select_threshold",
 ]
 
 
@@ -99,6 +99,9 @@ def lib() -> ctypes.CDLL:
     L.seer_kcomp_append.restype = i32
     L.seer_kcomp_append.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp,
                                     i64, i64, i64, i32, i32, i32, vp]
+    L.seer_gate_select_threshold.restype = i32
+    L.seer_gate_select_threshold.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, vp,
+                                             ctypes.c_float, vp, vp, i32, vp, vp]
     L.seer_decode_step.restype = i32
     L.seer_decode_step.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), ctypes.POINTER(SeerGate),
                                    vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, i32, vp, vp, vp]
@@ -203,6 +206,13 @@ class Context:
         self._check(lib().seer_gate_select(self._h, ctypes.byref(shape), ctypes.byref(gate), _ptr(seq_lens),
                                            _ptr(q_nope), _ptr(scores_in), int(token_budget), _ptr(block_idx),
                                            _ptr(block_cnt), int(max_sel), _ptr(scores_out), _stream(stream)))
+
+    def seer_gate_select_threshold(self, shape: SeerShape, gate: SeerGate, seq_lens, q_nope, scores_in, threshold,
+                                   block_idx, block_cnt, max_sel, scores_out=None, stream=None):
+        self._check(lib().seer_gate_select_threshold(self._h, ctypes.byref(shape), ctypes.byref(gate),
+                                                     _ptr(seq_lens), _ptr(q_nope), _ptr(scores_in),
+                                                     ctypes.c_float(threshold), _ptr(block_idx), _ptr(block_cnt),
+                                                     int(max_sel), _ptr(scores_out), _stream(stream)))
 
     def seer_kcomp_append(self, shape: SeerShape, gate: SeerGate, seq_lens, k_nope, rows_block_local=False,
                           first_block=-1, num_blocks=1, stream=None):

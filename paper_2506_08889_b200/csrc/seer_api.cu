@@ -357,9 +357,10 @@ seer_status seer_sparse_decode(seer_ctx* ctx, const seer_shape* shape, const see
     return decode_common(ctx, shape, kv, q, block_idx, block_cnt, max_sel, true, out, lse, stream);
 }
 
-seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,
-                             const void* q_nope, const float* scores_in, int token_budget, int32_t* block_idx,
-                             int32_t* block_cnt, int max_sel, float* scores_out, void* stream) {
+static seer_status gate_select_common(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                                      const int32_t* seq_lens, const void* q_nope, const float* scores_in,
+                                      int token_budget, int threshold_mode, float threshold, int32_t* block_idx,
+                                      int32_t* block_cnt, int max_sel, float* scores_out, void* stream) {
     if (!ctx) return SEER_ERR_INVALID_ARG;
     seer_status st = check_shape(ctx, shape);
     if (st != SEER_OK) return st;
@@ -404,6 +405,8 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
     p.max_blocks = gate->max_blocks;
     p.max_sel = max_sel;
     p.token_budget = token_budget;
+    p.threshold_mode = threshold_mode;
+    p.threshold = threshold;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
     p.tickets = reinterpret_cast<int*>(ctx->ws + w.gate_tickets);
 #ifdef SEER_GATE_TRACE
@@ -415,6 +418,23 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
     ctx->launches += launched;
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "gate launch: %s", cudaGetErrorString(ce));
     return SEER_OK;
+}
+
+seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,
+                             const void* q_nope, const float* scores_in, int token_budget, int32_t* block_idx,
+                             int32_t* block_cnt, int max_sel, float* scores_out, void* stream) {
+    return gate_select_common(ctx, shape, gate, seq_lens, q_nope, scores_in, token_budget, 0, 0.f, block_idx, block_cnt,
+                              max_sel, scores_out, stream);
+}
+
+seer_status seer_gate_select_threshold(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                                       const int32_t* seq_lens, const void* q_nope, const float* scores_in,
+                                       float threshold, int32_t* block_idx, int32_t* block_cnt, int max_sel,
+                                       float* scores_out, void* stream) {
+    if (ctx && !(threshold >= 0.f && threshold <= 1.f))
+        return fail(ctx, SEER_ERR_INVALID_ARG, "threshold must lie in [0, 1] (it is compared with a softmax probability)");
+    return gate_select_common(ctx, shape, gate, seq_lens, q_nope, scores_in, 0, 1, threshold, block_idx, block_cnt, max_sel,
+                              scores_out, stream);
 }
 
 seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,

@@ -48,6 +48,12 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 constexpr int kUnitThreads = 1024;          // one-CTA-per-unit gate kernel
 constexpr int kUnitMaxBlocks = 4096;        // ... and the compressed keys it can score
 
+// Inverse of score_key (NaN came out as key 0 and goes back as -inf).
+__device__ __forceinline__ float key_score(uint32_t key) {
+    if (key == 0u) return -INFINITY;
+    return __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
+}
+
 constexpr int kSelBits = 11;                // digit width of a selection pass
 constexpr int kSelBins = 1 << kSelBits;
 
@@ -81,7 +87,7 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
     int k = max(p.token_budget / p.block_size, 1);
     k = min(k, min(n_i, p.max_sel));
     const int n_cand = min(n_i - 1, p.max_blocks);
-    const int need = min(k - 1, n_cand);             // candidates to take besides the last block
+    int need = min(k - 1, n_cand);                   // candidates to take besides the last block
     const int E = (n_cand + NT - 1) / NT;
     const int j_lo = min(n_cand, tid * E), j_hi = min(n_cand, j_lo + E);
 
@@ -92,6 +98,48 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
         for (int e = 0; e < kCachedT; ++e) keys[e] = (j_lo + e < j_hi) ? score_key(score_at(j_lo + e)) : 0u;
     }
     auto key_at = [&](int e) -> uint32_t { return score_key(score_at(j_lo + e)); };
+
+    if (p.threshold_mode) {
+        // Threshold method (Sec. 3.1): softmax of the scores over the candidate blocks; the blocks
+        // with probability above tau are taken.  They are the `above` highest-scoring candidates
+        // (equal scores have equal probabilities), so only the count differs from the budget method.
+        auto block_reduce = [&](float v, bool is_max) -> float {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float o = __shfl_xor_sync(0xffffffffu, v, off);
+                v = is_max ? fmaxf(v, o) : v + o;
+            }
+            __syncthreads();                                   // the scratch may still be in use
+            if (lane == 0) sm.warp_min[warp] = __float_as_uint(v);
+            __syncthreads();
+            float r = is_max ? -INFINITY : 0.f;
+#pragma unroll
+            for (int w2 = 0; w2 < NT / 32; ++w2) {
+                const float o = __uint_as_float(sm.warp_min[w2]);
+                r = is_max ? fmaxf(r, o) : r + o;
+            }
+            return r;
+        };
+        auto for_each_score = [&](auto&& fn) {
+            if (CACHED) {
+#pragma unroll
+                for (int e = 0; e < kCachedT; ++e)
+                    if (j_lo + e < j_hi) fn(key_score(keys[e]));
+            } else {
+                for (int e = 0; j_lo + e < j_hi; ++e) fn(key_score(key_at(e)));
+            }
+        };
+        float mx = -INFINITY;
+        for_each_score([&](float v) { mx = fmaxf(mx, v); });
+        mx = block_reduce(mx, true);
+        float z = 0.f;
+        for_each_score([&](float v) { z += __expf(v - mx); });
+        z = block_reduce(z, false);
+        float cnt_above = 0.f;
+        for_each_score([&](float v) { cnt_above += (__expf(v - mx) > p.threshold * z) ? 1.f : 0.f; });
+        const int above = (int)(block_reduce(cnt_above, false) + 0.5f);
+        need = min(min(above, p.max_sel - 1), n_cand);
+    }
 
     uint32_t thr = 0u;                               // key of the need-th best candidate
     int take_eq = n_cand;                            // candidates equal to thr that are taken

@@ -87,6 +87,8 @@ struct GateParams {
     int32_t* block_cnt;
     int batch, num_q_heads, num_kv_heads, group, block_size;
     int d_gate, max_blocks, max_sel, token_budget;
+    int threshold_mode;             // 0: token budget, 1: softmax probability above `threshold`
+    float threshold;
     unsigned int* status;
     int* tickets;                   // [B*Hkv], zero between launches
     double inv_freq[kMaxDGate / 2]; // rope_theta^(-2c/d_gate), computed on the host in double

@@ -240,3 +240,44 @@ def test_single_call_step_equals_the_three_calls(ctx):
     for a, c in zip(res[0], res[1]):
         assert torch.equal(a, c)
     assert ctx.device_status() == binding.SEER_OK
+
+
+@pytest.mark.parametrize("tau", [0.002, 0.006, 0.05])
+def test_threshold_selection(ctx, tau):
+    # the decision is a floating-point comparison (fp32 on the GPU, fp64 in the oracle): blocks
+    # whose probability is not within rounding of tau must agree exactly, the few others may differ
+    B, Hkv, b, nbmax, max_sel = 4, 3, 64, 700, 700
+    r = synth.np_rng(31, "thr")
+    sc = (r.normal(size=(B, Hkv, nbmax)) * 1.5).astype(np.float32)
+    lens = np.array([nbmax * b, 333 * b + 1, b, 2 * b], np.int32)
+    shape = binding.make_shape(B, Hkv * 4, Hkv, 128, b, 0.1)
+    gate = binding.make_gate(128, THETA, None, None, None, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    idx = torch.full((B, Hkv, max_sel), 77, dtype=torch.int32, device=DEV)
+    cnt = torch.full((B, Hkv), 77, dtype=torch.int32, device=DEV)
+    ctx.seer_gate_select_threshold(shape, gate, lens_t, None, torch.as_tensor(sc, device=DEV), tau, idx, cnt, max_sel)
+    torch.cuda.synchronize()
+    want_idx, want_cnt, probs = oracle.select_threshold(sc, lens, b, tau, max_sel)
+    idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+    total = 0
+    for i in range(B):
+        n = -(-int(lens[i]) // b)
+        for h in range(Hkv):
+            got = set(idx[i, h, :cnt[i, h]].tolist())
+            want = set(want_idx[i, h, :want_cnt[i, h]].tolist())
+            assert n - 1 in got and list(idx[i, h, :cnt[i, h]]) == sorted(got)
+            assert np.all(idx[i, h, cnt[i, h]:] == -1)
+            for j in got ^ want:
+                assert abs(probs[i, h, j] - tau) <= 1e-5 * tau + 1e-9, (i, h, j, probs[i, h, j])
+            total += len(got)
+    assert total > B * Hkv                                   # the threshold did select something
+    # too small a list: the highest-scoring max_sel-1 are kept, exactly as the budget method would
+    small = 9
+    idx2 = torch.zeros((B, Hkv, small), dtype=torch.int32, device=DEV)
+    cnt2 = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    ctx.seer_gate_select_threshold(shape, gate, lens_t, None, torch.as_tensor(sc, device=DEV), 1e-7, idx2, cnt2, small)
+    torch.cuda.synchronize()
+    w2, c2, _ = oracle.select_threshold(sc, lens, b, 1e-7, small)
+    assert np.array_equal(idx2.cpu().numpy(), w2) and np.array_equal(cnt2.cpu().numpy(), c2)
+    with pytest.raises(binding.SeerError):
+        ctx.seer_gate_select_threshold(shape, gate, lens_t, None, torch.as_tensor(sc, device=DEV), 1.5, idx2, cnt2, small)

@@ -84,3 +84,53 @@ def test_positive_scaling_never_changes_the_selection():
     a = oracle.select(sc, [64 * 8, 50 * 8], 8, 8 * 9, 16)
     b = oracle.select(sc * np.float32(0.125), [64 * 8, 50 * 8], 8, 8 * 9, 16)   # exact scaling
     assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+# ---- threshold method (Sec. 3.1): blocks whose softmax score exceeds tau, plus the last block ----
+def _softmax64(x):
+    x = x.astype(np.float64)
+    e = np.exp(x - x.max())
+    return e / e.sum()
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_threshold_selection_against_numpy_softmax(seed):
+    r = np.random.default_rng(100 + seed)
+    B, Hkv, b, max_blocks, max_sel = 2, 2, 16, 60, 60
+    lens = np.array([60 * 16, 23 * 16 + 5], np.int32)
+    sc = (r.normal(size=(B, Hkv, max_blocks)) * 2.0).astype(np.float32)
+    tau = [0.002, 0.006, 0.02, 0.5][seed]
+    idx, cnt, probs = oracle.select_threshold(sc, lens, b, tau, max_sel)
+    for i in range(B):
+        n = -(-int(lens[i]) // b)
+        for h in range(Hkv):
+            p = _softmax64(sc[i, h, : n - 1])
+            assert np.allclose(probs[i, h, : n - 1], p, rtol=1e-12) and abs(p.sum() - 1.0) < 1e-12
+            want = sorted([j for j in range(n - 1) if p[j] > tau] + [n - 1])
+            assert list(idx[i, h, : cnt[i, h]]) == want
+            assert np.all(idx[i, h, cnt[i, h]:] == -1)
+
+
+def test_threshold_closed_forms_and_truncation():
+    # equal scores: every block has probability 1/(n-1)
+    sc = np.zeros((1, 1, 9), np.float32)
+    idx, cnt, _ = oracle.select_threshold(sc, [9 * 4], 4, 0.124, 9)       # 1/8 > 0.124: all
+    assert list(idx[0, 0]) == list(range(9))
+    idx, cnt, _ = oracle.select_threshold(sc, [9 * 4], 4, 0.125, 9)       # 1/8 > 1/8 is false: last only
+    assert list(idx[0, 0, :1]) == [8] and cnt[0, 0] == 1
+    # one dominant block
+    sc[0, 0, 3] = 30.0
+    idx, cnt, _ = oracle.select_threshold(sc, [9 * 4], 4, 0.5, 9)
+    assert list(idx[0, 0, :2]) == [3, 8] and cnt[0, 0] == 2
+    # the last block's own score plays no role, and a shift of all scores changes nothing
+    sc2 = sc + np.float32(5.0)
+    sc2[0, 0, 8] = 1e9
+    a = oracle.select_threshold(sc2, [9 * 4], 4, 0.5, 9)
+    assert np.array_equal(a[0], idx)
+    # more blocks pass than fit: the highest-scoring max_sel-1 are kept (ties: lower index)
+    sc3 = np.array([[[1, 3, 2, 3, 0, 1, 9]]], np.float32)
+    idx, cnt, _ = oracle.select_threshold(sc3, [7 * 4], 4, 1e-6, 4)       # all six pass, room for three
+    assert list(idx[0, 0]) == [1, 2, 3, 6] and cnt[0, 0] == 4
+    # a single block: nothing to normalise over
+    idx, cnt, _ = oracle.select_threshold(sc3, [3], 4, 0.1, 4)
+    assert list(idx[0, 0]) == [0, -1, -1, -1] and cnt[0, 0] == 1

@@ -451,6 +451,69 @@ def run_sweep(args):
     ctx.close()
 
 
+def run_grid(args):
+    """The paper's own kernel-benchmark shape (Sec. 4.4): 64 query / 8 KV heads, head_dim 128, over
+    sequence length x batch x sparsity, sparse kernel against the dense kernel on the same tensors.
+    Kernel-only, one GPU, one JSON document; L2 is kept cold by rotating over distinct caches."""
+    import torch
+    from paper_2506_08889_b200 import binding, synth
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    ctx = binding.Context(0)
+    peak, peak_kind = measured_hbm_peak()
+    Hq, Hkv, d, b = 64, 8, 128, args.block_size
+    rows = []
+
+    def timed(fn, iters):
+        for s in range(3):
+            fn(s)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for s in range(iters):
+            fn(s)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters * 1e3
+
+    for L in (8192, 32768, 131072):
+        for B in (1, 4, 16):
+            kv_bytes = B * Hkv * L * d * 4
+            n_copies = max(2, min(8, int(2 * 256e6 // kv_bytes) + 1))     # rotate over > 2x L2
+            caches = []
+            for c in range(n_copies):
+                tag = f"grid:{L}:{B}:{c}:"
+                k = synth.normal_bf16((B, Hkv, L, d), synth.BASE_SEED, tag + "k", dev)
+                v = synth.normal_bf16((B, Hkv, L, d), synth.BASE_SEED, tag + "v", dev)
+                caches.append((k, v))
+            q = synth.normal_bf16((B, Hq, d), synth.BASE_SEED, f"grid:{L}:{B}:q", dev)
+            out = torch.zeros_like(q)
+            lens_t = torch.full((B,), L, dtype=torch.int32, device=dev)
+            shape = binding.make_shape(B, Hq, Hkv, d, b, 1.0 / float(np.sqrt(d)))
+            kvs = [binding.make_kv(k, v, lens_t) for k, v in caches]
+            iters = max(20, min(args.steps, int(3e5 / max(1.0, kv_bytes / 6e6))))
+            dense_us = timed(lambda s: ctx.seer_dense_decode(shape, kvs[s % n_copies], q, out), max(5, iters // 4))
+            nb = L // b
+            for sp in (0.5, 0.7, 0.9):
+                k_sel = synth.keep_count(nb, sp)
+                scores = synth.normal_f32((B, Hkv, nb), synth.BASE_SEED, f"grid:{L}:{B}:{sp}", dev)
+                idx = torch.zeros((B, Hkv, k_sel), dtype=torch.int32, device=dev)
+                cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+                gate = binding.make_gate(128, 1.0e6, None, None, None, nb)
+                ctx.seer_gate_select(shape, gate, lens_t, None, scores, k_sel * b, idx, cnt, k_sel)
+                us = timed(lambda s: ctx.seer_sparse_decode(shape, kvs[s % n_copies], q, idx, cnt, k_sel, out), iters)
+                sel = B * Hkv * k_sel * b * d * 4
+                rows.append({"seq_len": L, "batch": B, "sparsity": sp, "sparse_us": round(us, 2),
+                             "dense_us": round(dense_us, 2), "speedup": round(dense_us / us, 2),
+                             "ideal": round(nb / k_sel, 2), "GBps": round(sel / us / 1e3, 1)})
+            del caches, kvs
+            torch.cuda.empty_cache()
+    assert ctx.device_status() == binding.SEER_OK
+    print(json.dumps({"shape": "64 query / 8 KV heads, head_dim 128", "block_size": b, "peak_GBps": peak,
+                      "peak_kind": peak_kind, "rows": rows}))
+    ctx.close()
+
+
 def oracle_step(w, host, n_seq, n_kv_heads, budget, k_sel):
     """The whole step on the CPU oracle for the first n_seq sequences and the first
     n_kv_heads KV heads (with their query-head groups).  Returns the selected-KV bytes."""
@@ -559,10 +622,14 @@ def main():
     ap.add_argument("--seq-len", type=int, default=0, help="override the workload's KV length (multiple of 64)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true", help="kernel-only sparsity sweep instead of the step benchmark")
+    ap.add_argument("--grid", action="store_true", help="the paper's 64/8-head kernel grid (seq len x batch x sparsity)")
+    ap.add_argument("--block-size", type=int, default=64, help="block size for --grid (64 or 128)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()
-    if args.sweep:
+    if args.grid:
+        run_grid(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -87,9 +87,6 @@ struct __align__(1024) Smem {
     Schedule sched;
     Piece pieces[kMaxPieces];
     int pieces_n;
-    int scan_warp[kThreads / 32];
-    int start_unit;
-    int start_off;
 };
 
 // two CTAs per SM: 2 * (sizeof(Smem) + 1 KiB alignment slack + 1 KiB reserved by the system) must
@@ -272,8 +269,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         mbar_init(&sm.list_bar, kConsumerWarps);
         mbar_fence_init();
         sm.issued = 0;
-        sm.start_unit = U;
-        sm.start_off = 0;
         sm.pieces_n = 0;
     }
     if (warp == kConsumerWarps && lane == 0) {
@@ -281,65 +276,63 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         tma_prefetch_desc(&map_v);
     }
 
+    __syncthreads();                                 // barriers initialised
     pdl_wait();
-
-    // ---- every CTA sums the units' tile counts and finds where its static share starts ----
-    const int per = (U + kThreads - 1) / kThreads;
-    const int u_lo = min(U, tid * per), u_hi = min(U, u_lo + per);
-    int mine = 0;
-    for (int u = u_lo; u < u_hi; ++u) {
-        int t = tiles_of<SPARSE>(p, u);
-        if (t == 0 && cta == 0) write_zero_unit(p, u);   // units without work: zeros, -inf
-        mine += t;
-    }
-    int incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) sm.scan_warp[warp] = incl;
-    __syncthreads();
-    int warp_base = 0, T = 0;
-#pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) {
-        int v = sm.scan_warp[w];
-        if (w < warp) warp_base += v;
-        T += v;
-    }
-    if (tid == 0) build_schedule(sm.sched, T, gridDim.x, p.pool_div);
-    __syncthreads();
-    const Schedule& sc = sm.sched;
-    int t_begin = 0, t_end = 0;                      // this CTA's static share
-    if (T > 0 && cta < sc.G) interval_range(sc, cta, 0, &t_begin, &t_end);
-    const int excl = warp_base + incl - mine;
-    {
-        // prefix sums of the tile counts, for locating a tile's unit later.  Every CTA writes
-        // the same values; a CTA only relies on its own writes being visible to itself.
-        const bool want_start = t_begin < t_end;
-        int acc = excl;
-        for (int u = u_lo; u < u_hi; ++u) {
-            const int t = tiles_of<SPARSE>(p, u);
-            if (sc.R > 0) p.prefix[u] = acc;
-            if (want_start && t > 0 && acc <= t_begin && t_begin < acc + t) {
-                sm.start_unit = u;
-                sm.start_off = t_begin - acc;
-            }
-            acc += t;
-        }
-        if (sc.R > 0 && tid == 0) p.prefix[U] = T;
-    }
-    __syncthreads();
 
     if (warp == kConsumerWarps) {
         // =========================== producer warp ====================================
+        // The warp first sums the units' tile counts by itself (the consumer warps do not need the
+        // result to start waiting), derives the schedule and finds where its static share starts.
+        const int per = (U + 31) / 32;
+        const int u_lo = min(U, lane * per), u_hi = min(U, u_lo + per);
+        int mine = 0;
+        for (int u = u_lo; u < u_hi; ++u) {
+            const int t = tiles_of<SPARSE>(p, u);
+            if (t == 0 && cta == 0) write_zero_unit(p, u);   // units without work: zeros, -inf
+            mine += t;
+        }
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int T = __shfl_sync(0xffffffffu, incl, 31);
+        Schedule sc;
+        build_schedule(sc, T, gridDim.x, p.pool_div);
+        if (lane == 0) sm.sched = sc;                    // the consumers use it when a piece ends
+        int t_begin = 0, t_end = 0;                      // this CTA's static share
+        if (T > 0 && cta < sc.G) interval_range(sc, cta, 0, &t_begin, &t_end);
+        // prefix sums of the tile counts, for locating a tile's unit later (every CTA writes the
+        // same values; a CTA only relies on its own writes), and the unit holding tile t_begin
+        int my_start_u = -1, my_start_off = 0;
+        {
+            int acc = incl - mine;
+            for (int u = u_lo; u < u_hi; ++u) {
+                const int t = tiles_of<SPARSE>(p, u);
+                if (sc.R > 0) p.prefix[u] = acc;
+                if (t_begin < t_end && t > 0 && acc <= t_begin && t_begin < acc + t) {
+                    my_start_u = u;
+                    my_start_off = t_begin - acc;
+                }
+                acc += t;
+            }
+            if (sc.R > 0 && lane == 0) p.prefix[U] = T;
+        }
+        __syncwarp();
         // position in the units' tile lists: unit cu, whose first tile is global tile cpu and
         // which has cut tiles
         int cu = 0, cpu = 0, cut = 0;
-        if (t_begin < t_end) {
-            cu = sm.start_unit;
-            cut = cu < U ? tiles_of<SPARSE>(p, cu) : 0;
-            cpu = t_begin - sm.start_off;
+        {
+            const unsigned m = __ballot_sync(0xffffffffu, my_start_u >= 0);
+            if (m) {
+                const int src = __ffs(m) - 1;
+                cu = __shfl_sync(0xffffffffu, my_start_u, src);
+                cpu = t_begin - __shfl_sync(0xffffffffu, my_start_off, src);
+                cut = tiles_of<SPARSE>(p, cu);
+            } else {
+                t_end = t_begin;                         // (no static share)
+            }
         }
         int it = 0;
         int iv_begin = t_begin, iv_end = t_end, iv_id = cta * (sc.R + 1);
@@ -551,8 +544,17 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             dst[ks][1] = (rw < p.group) ? __ldg(qrow + (16 * ks + 8 + 2 * qd) / 2) : 0u;
         }
     };
-    int pre_unit = sm.start_unit;       // requested now, long before the first tile lands
-    if (pre_unit < U) load_q(bq_pre, pre_unit); else pre_unit = -1;
+    int pre_unit = -1;
+    {
+        // the first tile's unit is known as soon as the producer has issued it, well before its data
+        // lands: request that unit's queries in the meantime
+        for (int spin = 0; spin < (1 << 22) && sm.issued < 1; ++spin) __nanosleep(32);
+        __threadfence_block();
+        if (sm.issued >= 1) {
+            const int u0 = *reinterpret_cast<volatile int*>(&sm.meta[0].unit);
+            if (u0 >= 0) { load_q(bq_pre, u0); pre_unit = u0; }
+        }
+    }
 
     // lane-constant parts of the ldmatrix addresses (swizzle: 16-B chunk ^= row & 7)
     const int k_row = 16 * w + ((lane >> 3) & 1) * 8 + (lane & 7);

@@ -75,14 +75,19 @@ struct WsLayout {
     size_t part_o, part_ml, q_gate, scores, total;
 };
 
+constexpr int kMaxUnits = 65535;            // batch * num_kv_heads (check_shape enforces it)
+
 WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks) {
     WsLayout w;
+    // The regions that must stay zero between launches sit at offsets that do not depend on the
+    // call's shape (they are sized for the largest unit count), so that calls of different shapes on
+    // one context never see one another's scratch in them.
     size_t off = kStatusBytes;
     w.sched = off; off += 256;
     w.steal = off; off = align_up(off + sizeof(int) * (size_t)kMaxGridCtas, 256);
-    w.tickets = off; off = align_up(off + sizeof(int) * (size_t)num_units, 256);
-    w.gate_tickets = off; off = align_up(off + sizeof(int) * (size_t)num_units, 256);
-    w.prefix = off; off = align_up(off + sizeof(int) * ((size_t)num_units + 1), 256);
+    w.tickets = off; off = align_up(off + sizeof(unsigned long long) * (size_t)kMaxUnits, 256);
+    w.gate_tickets = off; off = align_up(off + sizeof(int) * (size_t)kMaxUnits, 256);
+    w.prefix = off; off = align_up(off + sizeof(int) * ((size_t)kMaxUnits + 1), 256);
     w.scratch = off;
     // decode view of the scratch
     size_t d = off;
@@ -230,7 +235,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.pool_div = ctx->pool_div;
     p.scale_log2 = shape->sm_scale * 1.4426950408889634f;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
-    p.tickets = reinterpret_cast<int*>(ctx->ws + w.tickets);
+    p.tickets = reinterpret_cast<unsigned long long*>(ctx->ws + w.tickets);
     p.sched = reinterpret_cast<int*>(ctx->ws + w.sched);
     p.prefix = reinterpret_cast<int*>(ctx->ws + w.prefix);
     p.steal = reinterpret_cast<int*>(ctx->ws + w.steal);
@@ -276,7 +281,7 @@ seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes) {
     ctx->pool_div = 4;
     if (const char* e = getenv("SEER_DECODE_POOL_DIV")) ctx->pool_div = atoi(e);
     ctx->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)64 << 20;
-    if (ctx->ws_bytes < 4096) ctx->ws_bytes = 4096;
+    if (ctx->ws_bytes < 4096) ctx->ws_bytes = 4096;     // (far too small for any call: every call checks)
     if (cudaMalloc(reinterpret_cast<void**>(&ctx->ws), ctx->ws_bytes) != cudaSuccess) {
         delete ctx;
         return SEER_ERR_CUDA;
@@ -331,8 +336,8 @@ seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
     if (e != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "status read: %s", cudaGetErrorString(e));
     if (word & DEV_TIMEOUT) {
         // a CTA that gave up may have left tickets or scheduler counters behind: clear them
-        cudaMemsetAsync(ctx->ws + kStatusBytes, 0, ctx->ws_bytes < (1u << 20) ? ctx->ws_bytes - kStatusBytes
-                                                                              : (1u << 20) - kStatusBytes, s);
+        const size_t fixed = ws_layout(1, 0, 0, 0).scratch;
+        cudaMemsetAsync(ctx->ws + kStatusBytes, 0, (ctx->ws_bytes < fixed ? ctx->ws_bytes : fixed) - kStatusBytes, s);
         cudaStreamSynchronize(s);
         return fail(ctx, SEER_ERR_TIMEOUT, "a device-side wait gave up; results of that call are invalid");
     }

@@ -45,7 +45,8 @@ constexpr int kTileBytes = 2 * kHalfTileBytes;             // one K or V tile: 1
 constexpr int kStageBytes = 2 * kTileBytes;                // K + V
 constexpr int kMergeStride = 132;                          // floats per head row (bank spread)
 constexpr int kMaxPieces = 32;                             // partial pieces a CTA can hold back to its end
-constexpr int kListInts = 2 * kStageBytes / 4;              // slot numbers that fit in two stage buffers
+constexpr int kListInts = kStageBytes / 4 - 64;              // slot numbers that fit in one stage buffer (less 64 counts)
+constexpr int kLandBytes = 2 * kStageBytes;                 // landing area for staged partials: two stage buffers
 constexpr int kMaxSteals = 14;                             // chunks a CTA may take from other ranges
 constexpr int kMinChunk = 2;                               // smallest dynamic chunk, in tiles
 constexpr int kMinStaticTilesPerCta = 8;                   // below this everything is static
@@ -59,8 +60,11 @@ struct StageMeta {
     int interval;      // interval this tile belongs to
 };
 
+// A partial this CTA wrote (unit, tiles, unit_first, unit_tiles, interval it went to); after the
+// counts are taken the same records list the units this CTA has to combine
+// (unit, -, first_slot, n_slots, mask of valid slots or 0 if unknown).
 struct Piece {
-    int unit, tiles, unit_first, unit_tiles;   // a partial this CTA wrote; merged: first_slot, n_slots
+    int unit, tiles, unit_first, unit_tiles, extra;
 };
 
 // Geometry of the intervals, identical in every CTA (derived from T and gridDim.x).  Range c is
@@ -82,6 +86,7 @@ struct __align__(1024) Smem {
     uint64_t merge_bar[2];           // [0]: scratch filled (3 arrivals), [1]: scratch free again / end sync
     uint64_t end_bar;                // all consumer warps: streams over, the list of combines is final
     uint64_t list_bar;               // all consumer warps: the lists of valid slots are written
+    uint64_t land_bar;               // bulk copies of partials into the landing area have arrived
     volatile int issued;             // tiles whose metadata the producer has written so far
     StageMeta meta[kStages];
     Schedule sched;
@@ -181,39 +186,32 @@ __device__ __forceinline__ void merge_init(MergeState& st) {
 #pragma unroll
     for (int x = 0; x < 8; ++x) st.acc[x] = 0.f;
 }
-// Adds the partials in the n listed slots.  A batch of partials is loaded in full before any
-// arithmetic, so a batch costs one round trip to L2.
-__device__ void merge_accumulate(const DecodeParams& p, MergeState& st, const int* slots, int n, int t) {
+// Adds the partials that have been staged in shared memory: land_o + k * o_stride holds the
+// group x 128 floats of partial k, land_ml[k] its 32-float (max, sum, stamp) record.
+__device__ __forceinline__ void merge_accumulate_staged(MergeState& st, const float* land_o, int o_stride,
+                                                        const float* land_ml, int m, int group, int t) {
     const int hh = t >> 4, d0 = 8 * (t & 15);
-    constexpr int kB = 8;
-    for (int s0 = 0; s0 < n; s0 += kB) {
-        float ms[kB], ls[kB];
-        float4 va[kB], vb[kB];
+    if (hh >= group) return;
+    // the round's maximum first, so that the sum below is a chain of independent multiply-adds
+    float Mr = st.M;
+    for (int k = 0; k < m; ++k) Mr = fmaxf(Mr, land_ml[k * kMlStride + hh]);
+    if (Mr == -INFINITY) return;
+    const float fo = (st.M == -INFINITY) ? 0.f : fast_exp2(st.M - Mr);
+    st.M = Mr;
+    st.lsum *= fo;
 #pragma unroll
-        for (int k = 0; k < kB; ++k) {
-            const size_t sl = (size_t)slots[min(s0 + k, n - 1)];
-            const float* pm = p.part_ml + sl * kMlStride;
-            const float4* qo = reinterpret_cast<const float4*>(p.part_o + sl * (kMaxGroup * kHeadDim) +
-                                                               hh * kHeadDim + d0);
-            ms[k] = __ldcg(pm + hh);
-            ls[k] = __ldcg(pm + kMaxGroup + hh);
-            va[k] = __ldcg(qo);
-            vb[k] = __ldcg(qo + 1);
-        }
-#pragma unroll
-        for (int k = 0; k < kB; ++k) {
-            if (s0 + k < n && ms[k] != -INFINITY) {
-                const float Mn = fmaxf(st.M, ms[k]);
-                const float fo = (st.M == -INFINITY) ? 0.f : fast_exp2(st.M - Mn);
-                const float fn = fast_exp2(ms[k] - Mn);
-                st.M = Mn;
-                st.lsum = st.lsum * fo + ls[k] * fn;
-                st.acc[0] = st.acc[0] * fo + va[k].x * fn; st.acc[1] = st.acc[1] * fo + va[k].y * fn;
-                st.acc[2] = st.acc[2] * fo + va[k].z * fn; st.acc[3] = st.acc[3] * fo + va[k].w * fn;
-                st.acc[4] = st.acc[4] * fo + vb[k].x * fn; st.acc[5] = st.acc[5] * fo + vb[k].y * fn;
-                st.acc[6] = st.acc[6] * fo + vb[k].z * fn; st.acc[7] = st.acc[7] * fo + vb[k].w * fn;
-            }
-        }
+    for (int x = 0; x < 8; ++x) st.acc[x] *= fo;
+#pragma unroll 4
+    for (int k = 0; k < m; ++k) {
+        const float ms = land_ml[k * kMlStride + hh];
+        const float fn = (ms == -INFINITY) ? 0.f : fast_exp2(ms - Mr);
+        const float4 va = *reinterpret_cast<const float4*>(land_o + k * o_stride + hh * kHeadDim + d0);
+        const float4 vb = *reinterpret_cast<const float4*>(land_o + k * o_stride + hh * kHeadDim + d0 + 4);
+        st.lsum = fmaf(land_ml[k * kMlStride + kMaxGroup + hh], fn, st.lsum);
+        st.acc[0] = fmaf(va.x, fn, st.acc[0]); st.acc[1] = fmaf(va.y, fn, st.acc[1]);
+        st.acc[2] = fmaf(va.z, fn, st.acc[2]); st.acc[3] = fmaf(va.w, fn, st.acc[3]);
+        st.acc[4] = fmaf(vb.x, fn, st.acc[4]); st.acc[5] = fmaf(vb.y, fn, st.acc[5]);
+        st.acc[6] = fmaf(vb.z, fn, st.acc[6]); st.acc[7] = fmaf(vb.w, fn, st.acc[7]);
     }
 }
 __device__ __forceinline__ void merge_finalize(const DecodeParams& p, const MergeState& st, int u, int t) {
@@ -267,6 +265,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         mbar_init(&sm.merge_bar[1], 1);
         mbar_init(&sm.end_bar, kConsumerWarps);
         mbar_init(&sm.list_bar, kConsumerWarps);
+        mbar_init(&sm.land_bar, 1);
         mbar_fence_init();
         sm.issued = 0;
         sm.pieces_n = 0;
@@ -503,7 +502,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             }
         }
 #ifdef SEER_DECODE_TRACE
-        if (lane == 0) { p.trace[(size_t)blockIdx.x * 8 + 3] = steals; p.trace[(size_t)blockIdx.x * 8 + 1] = it; SEER_STAMP(2); }
 #endif
         if (lane == 0) {
             // end-of-stream marker for the consumers
@@ -566,7 +564,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     // the first tile's metadata
     if (!mbar_wait(&sm.full[0], 0, p.status)) return;
     StageMeta mt = sm.meta[0];
-    if (tid == 0) SEER_STAMP(5);
     for (int it = 0; mt.nvalid >= 0; ++it) {
         const int st = it % kStages;
         {
@@ -759,7 +756,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     }
                     if (lane == 0) {
                         pm[16] = __uint_as_float(p.generation);
-                        sm.pieces[n_held] = Piece{u, piece_tiles, mt.unit_first, mt.unit_tiles};
+                        sm.pieces[n_held] = Piece{u, piece_tiles, mt.unit_first, mt.unit_tiles, piece_iv};
                         sm.pieces_n = n_held + 1;
                     }
                     __syncwarp();
@@ -805,26 +802,36 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (w == 0) {
         const int n_held = sm.pieces_n;
 #ifdef SEER_DECODE_TRACE
-        if (lane == 0) p.trace[(size_t)blockIdx.x * 8 + 4] = n_held;
 #endif
         __threadfence();                               // the partials above are visible from here on
         __syncwarp();
         if (lane == 0) SEER_STAMP(0);
+        // One 64-bit add per piece on its unit's counter: the high half counts tiles, the low half
+        // collects one bit per piece (its slot's place among the unit's candidate slots, when there
+        // are at most 32 of those).  Whoever completes the tile count learns from the same word
+        // which slots hold the unit's partials.
         bool owe = false;
-        Piece pc = Piece{0, 0, 0, 0};
+        Piece pc = Piece{0, 0, 0, 0, 0};
+        int first_slot = 0, n_slots = 0;
+        unsigned int mask = 0u;
         if (lane < n_held) {
             pc = sm.pieces[lane];
-            const int before = atomicAdd(&p.tickets[pc.unit], pc.tiles);
-            owe = before + pc.tiles == pc.unit_tiles;  // this piece completed the unit's count
+            const int iv_first = interval_of(sm.sched, pc.unit_first);
+            const int iv_last = interval_of(sm.sched, pc.unit_first + pc.unit_tiles - 1);
+            first_slot = iv_first + pc.unit;
+            n_slots = iv_last - iv_first + 1;
+            const unsigned int bit = n_slots <= 32 ? 1u << (pc.extra - iv_first) : 0u;
+            const unsigned long long before =
+                atomicAdd(&p.tickets[pc.unit], ((unsigned long long)pc.tiles << 32) | bit);
+            owe = (int)(before >> 32) + pc.tiles == pc.unit_tiles;     // this piece completed the unit's count
+            mask = (unsigned int)before | bit;
         }
         // rewrite the list: the units this CTA has to combine, with their candidate slots
         const unsigned m = __ballot_sync(0xffffffffu, owe);
         __syncwarp();
         if (owe) {
-            p.tickets[pc.unit] = 0;                    // ready for the next launch
-            const int iv_first = interval_of(sm.sched, pc.unit_first);
-            const int iv_last = interval_of(sm.sched, pc.unit_first + pc.unit_tiles - 1);
-            sm.pieces[__popc(m & ((1u << lane) - 1u))] = Piece{pc.unit, 0, iv_first + pc.unit, iv_last - iv_first + 1};
+            p.tickets[pc.unit] = 0ull;                 // ready for the next launch
+            sm.pieces[__popc(m & ((1u << lane) - 1u))] = Piece{pc.unit, 0, first_slot, n_slots, (int)mask};
         }
         if (lane == 0) sm.pieces_n = __popc(m);
     }
@@ -833,12 +840,21 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (lane == 0) mbar_arrive(&sm.end_bar);
     if (!mbar_wait(&sm.end_bar, 0, p.status)) return;
     const int n_owed = sm.pieces_n;
-    // The combines use the stage buffers as scratch (the stream is over, nothing is in flight): the
+#ifdef SEER_DECODE_TRACE
+    if (tid == 0 && n_owed > 0) { SEER_STAMP(2); p.trace[(size_t)blockIdx.x * 8 + 4] = n_owed; }
+#endif
+    // The combines use the stage buffers as scratch (the stream is over, nothing is in flight).  The
     // slots that really hold a partial of a unit are found by looking at the generation stamps of
-    // the unit's candidate slots, then all threads combine them.
-    int* lists = reinterpret_cast<int*>(sm.stage[0]);            // kListInts slot numbers (two stages)
-    int* counts = reinterpret_cast<int*>(sm.stage[2]);
-    int sync_phase = 0;
+    // the unit's candidate slots (lists, in the third stage buffer); the partials themselves are
+    // brought in by bulk copies, kLand at a time, into the first two stage buffers, and added up.
+    int* lists = reinterpret_cast<int*>(sm.stage[2]);            // kListInts slot numbers
+    int* counts = lists + kListInts;                             // per owed unit (or per warp)
+    // only the group's real heads are brought in: group x 512 B + 128 B per partial, one per lane
+    const int o_stride = p.group * kHeadDim;                     // floats per staged partial
+    const int n_land = min(32, kLandBytes / (o_stride * 4 + kMlStride * 4));
+    float* land_o = reinterpret_cast<float*>(sm.stage[0]);       // [n_land][group][128]
+    float* land_ml = land_o + n_land * o_stride;                 // [n_land][32]
+    int sync_phase = 0, land_phase = 0;
     auto sync_consumers = [&]() -> bool {
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.list_bar);
@@ -846,24 +862,70 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         ++sync_phase;
         return ok;
     };
+    // stage the n listed partials, kLand per round, and add them to ms (all consumer threads call)
+    auto accumulate_list = [&](MergeState& ms, const int* slots, int n) -> bool {
+        for (int s0 = 0; s0 < n; s0 += n_land) {
+            const int m = min(n_land, n - s0);
+            if (w == 0) {
+                // warp 0 issues the copies, one partial per lane
+                if (lane == 0) {
+                    fence_proxy_async_smem();        // earlier plain accesses to the landing area are done
+                    mbar_arrive_expect_tx(&sm.land_bar, (uint32_t)m * (o_stride * 4 + kMlStride * 4));
+                }
+                __syncwarp();
+                if (lane < m) {
+                    const size_t sl = (size_t)slots[s0 + lane];
+                    bulk_load(land_o + lane * o_stride, p.part_o + sl * (kMaxGroup * kHeadDim), o_stride * 4, &sm.land_bar);
+                    bulk_load(land_ml + lane * kMlStride, p.part_ml + sl * kMlStride, kMlStride * 4, &sm.land_bar);
+                }
+            }
+            if (!mbar_wait(&sm.land_bar, land_phase & 1, p.status)) return false;
+#ifdef SEER_DECODE_TRACE
+            if (tid == 0 && land_phase == 0) SEER_STAMP(5);
+#endif
+            ++land_phase;
+            merge_accumulate_staged(ms, land_o, o_stride, land_ml, m, p.group, tid);
+            if (!sync_consumers()) return false;     // everybody has read the landing area
+#ifdef SEER_DECODE_TRACE
+            if (tid == 0 && land_phase == 1) SEER_STAMP(1);
+#endif
+        }
+        return true;
+    };
     int total_cand = 0;
     for (int e = 0; e < n_owed; ++e) total_cand += sm.pieces[e].unit_tiles;
     if (total_cand <= kListInts) {
-        // usual case: every owed unit's candidates fit at once; warp e%4 scans unit e
+        // usual case: every owed unit's candidates fit at once; warp e%4 lists unit e's valid slots.
+        // With a static split every candidate slot holds a partial; with at most 32 candidates the
+        // ticket word said which ones do; otherwise the generation stamps are looked at.
         int base = 0;
         for (int e = 0; e < n_owed; ++e) {
             if ((e & (kConsumerWarps - 1)) == w) {
-                const int n = scan_valid_slots(p, sm.pieces[e].unit_first, sm.pieces[e].unit_tiles, lists + base, lane);
+                const int first = sm.pieces[e].unit_first, n_slots = sm.pieces[e].unit_tiles;
+                int n;
+                if (sm.sched.R == 0) {
+                    for (int x = lane; x < n_slots; x += 32) lists[base + x] = first + x;
+                    n = n_slots;
+                } else if (n_slots <= 32) {
+                    const unsigned int mk = (unsigned int)sm.pieces[e].extra;
+                    if ((mk >> lane) & 1u) lists[base + __popc(mk & ((1u << lane) - 1u))] = first + lane;
+                    n = __popc(mk);
+                } else {
+                    n = scan_valid_slots(p, first, n_slots, lists + base, lane);
+                }
                 if (lane == 0) counts[e] = n;
             }
             base += sm.pieces[e].unit_tiles;
         }
         if (!sync_consumers()) return;
+#ifdef SEER_DECODE_TRACE
+        if (tid == 0 && n_owed > 0) { SEER_STAMP(3); p.trace[(size_t)blockIdx.x * 8 + 4] = n_owed * 1000 + counts[0]; }
+#endif
         base = 0;
         for (int e = 0; e < n_owed; ++e) {
             MergeState ms;
             merge_init(ms);
-            merge_accumulate(p, ms, lists + base, counts[e], tid);
+            if (!accumulate_list(ms, lists + base, counts[e])) return;
             merge_finalize(p, ms, sm.pieces[e].unit, tid);
             base += sm.pieces[e].unit_tiles;
         }
@@ -879,7 +941,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 const int n = lo < hi ? scan_valid_slots(p, first + lo, hi - lo, lists + w * kWin, lane) : 0;
                 if (lane == 0) counts[w] = n;
                 if (!sync_consumers()) return;
-                for (int ww = 0; ww < kConsumerWarps; ++ww) merge_accumulate(p, ms, lists + ww * kWin, counts[ww], tid);
+                for (int ww = 0; ww < kConsumerWarps; ++ww)
+                    if (!accumulate_list(ms, lists + ww * kWin, counts[ww])) return;
                 if (!sync_consumers()) return;
             }
             merge_finalize(p, ms, sm.pieces[e].unit, tid);

@@ -50,7 +50,7 @@ struct DecodeParams {
     int pool_div;                   // 1/pool_div of the tiles are handed out dynamically (0: none)
     float scale_log2;               // sm_scale * log2(e)
     unsigned int* status;
-    int* tickets;                   // [num_units], zero between launches
+    unsigned long long* tickets;    // [num_units]: tiles done << 32 | valid-slot bits; zero between launches
     int* sched;                     // [2]: theft cursor, exit counter; zero between launches
     int* steal;                     // [grid]: per-range claim counters (front | back << 16); zero between launches
     unsigned int generation;        // stamp that marks this launch's partials

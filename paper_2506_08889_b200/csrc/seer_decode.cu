@@ -186,6 +186,44 @@ __device__ __forceinline__ void merge_init(MergeState& st) {
 #pragma unroll
     for (int x = 0; x < 8; ++x) st.acc[x] = 0.f;
 }
+// Adds up to kDirect partials straight from global memory: every load is issued before any
+// arithmetic, so the whole batch costs one round trip to L2 (the cheapest way for a few partials).
+constexpr int kDirect = 8;
+__device__ __forceinline__ void merge_accumulate_direct(const DecodeParams& p, MergeState& st, const int* slots,
+                                                        int n, int t) {
+    const int hh = t >> 4, d0 = 8 * (t & 15);
+    float ms[kDirect], ls[kDirect];
+    float4 va[kDirect], vb[kDirect];
+#pragma unroll
+    for (int k = 0; k < kDirect; ++k) {
+        const size_t sl = (size_t)slots[min(k, n - 1)];
+        const float* pm = p.part_ml + sl * kMlStride;
+        const float4* qo = reinterpret_cast<const float4*>(p.part_o + sl * (kMaxGroup * kHeadDim) + hh * kHeadDim + d0);
+        ms[k] = __ldcg(pm + hh);
+        ls[k] = __ldcg(pm + kMaxGroup + hh);
+        va[k] = __ldcg(qo);
+        vb[k] = __ldcg(qo + 1);
+    }
+    float Mr = st.M;
+#pragma unroll
+    for (int k = 0; k < kDirect; ++k) Mr = fmaxf(Mr, k < n ? ms[k] : -INFINITY);
+    if (Mr == -INFINITY) return;
+    const float fo = (st.M == -INFINITY) ? 0.f : fast_exp2(st.M - Mr);
+    st.M = Mr;
+    st.lsum *= fo;
+#pragma unroll
+    for (int x = 0; x < 8; ++x) st.acc[x] *= fo;
+#pragma unroll
+    for (int k = 0; k < kDirect; ++k) {
+        const float fn = (k < n && ms[k] != -INFINITY) ? fast_exp2(ms[k] - Mr) : 0.f;
+        st.lsum = fmaf(ls[k], fn, st.lsum);
+        st.acc[0] = fmaf(va[k].x, fn, st.acc[0]); st.acc[1] = fmaf(va[k].y, fn, st.acc[1]);
+        st.acc[2] = fmaf(va[k].z, fn, st.acc[2]); st.acc[3] = fmaf(va[k].w, fn, st.acc[3]);
+        st.acc[4] = fmaf(vb[k].x, fn, st.acc[4]); st.acc[5] = fmaf(vb[k].y, fn, st.acc[5]);
+        st.acc[6] = fmaf(vb[k].z, fn, st.acc[6]); st.acc[7] = fmaf(vb[k].w, fn, st.acc[7]);
+    }
+}
+
 // Adds the partials that have been staged in shared memory: land_o + k * o_stride holds the
 // group x 128 floats of partial k, land_ml[k] its 32-float (max, sum, stamp) record.
 __device__ __forceinline__ void merge_accumulate_staged(MergeState& st, const float* land_o, int o_stride,
@@ -864,6 +902,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     };
     // stage the n listed partials, kLand per round, and add them to ms (all consumer threads call)
     auto accumulate_list = [&](MergeState& ms, const int* slots, int n) -> bool {
+        if (n > 0 && n <= kDirect) {
+            merge_accumulate_direct(p, ms, slots, n, tid);
+            return true;
+        }
         for (int s0 = 0; s0 < n; s0 += n_land) {
             const int m = min(n_land, n - s0);
             if (w == 0) {

@@ -35,8 +35,8 @@ FALLBACK_HBM_GBS = 6650.0
 # quarter-size case (batch 2): 107.7 MB read + 3.0 MB written for 107.5 MB of algorithmic bytes.
 # Reads grow with the selected tiles, writes (partials) with the number of CTAs, so a launch on
 # `batch` sequences moves about batch/2 * 107.7 MB + 3.0 MB.
-NCU_READ_BYTES_PER_2_SEQUENCES = 107.677e6
-NCU_WRITE_BYTES_PER_LAUNCH = 3.03e6
+NCU_READ_BYTES_PER_2_SEQUENCES = 107.693e6
+NCU_WRITE_BYTES_PER_LAUNCH = 3.32e6
 
 
 def measured_hbm_peak():

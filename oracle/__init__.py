@@ -115,6 +115,28 @@ def sparse(q, k, v, seq_lens, block_idx, block_cnt, block_size, scale):
     return out, lse
 
 
+def sparse_multi(q, k, v, seq_lens, block_idx, block_cnt, block_size, scale):
+    """Block-sparse attention for T query tokens per sequence (the last T cached tokens), causal
+    among them, one block list per (sequence, KV head).  q: [B,T,Hq,d] bf16 bits.
+    Returns (out [B,T,Hq,d] f64, lse [B,T,Hq] f64)."""
+    q = np.ascontiguousarray(_u16(q, "q")); k = _u16(k, "k"); v = _u16(v, "v")
+    B, T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    sb, sh, st = _kv_strides(k, v)
+    seq_lens = _i32(seq_lens)
+    block_idx = _i32(block_idx)
+    assert block_idx.shape[:2] == (B, Hkv)
+    max_sel = block_idx.shape[2]
+    cnt = None if block_cnt is None else _i32(block_cnt)
+    out = np.zeros((B, T, Hq, d), np.float64)
+    lse = np.zeros((B, T, Hq), np.float64)
+    lib().oracle_sparse_multi(_p(q), _p(k), _p(v), sb, sh, st, _p(seq_lens), _p(block_idx), _p(cnt),
+                              ctypes.c_int(max_sel), ctypes.c_int(B), ctypes.c_int(T), ctypes.c_int(Hq),
+                              ctypes.c_int(Hkv), ctypes.c_int(d), ctypes.c_int(block_size),
+                              ctypes.c_double(scale), _p(out), _p(lse))
+    return out, lse
+
+
 def kcomp(k_nope, w_k, block_size, first_block, num_blocks, max_blocks, theta,
           kc_bf16=None):
     """K-branch entries for blocks first_block..first_block+num_blocks-1.

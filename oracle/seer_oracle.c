@@ -189,6 +189,52 @@ void oracle_sparse(const bf16_t *q, const bf16_t *k, const bf16_t *v,
         }
 }
 
+/* Block-sparse attention for T query tokens per sequence (the query-level
+ * parallelism of multi-token prediction / speculative decoding that Sec. 6
+ * "Unify Sparse Prefill and Decoding" points to; the paper gives no formula, so
+ * this is the causal definition written out).  The cache already holds all L_i
+ * tokens, the last T of which are the queries' own: query t (0 <= t < T) sits at
+ * position L_i - T + t and sees the cached tokens at positions <= its own, of
+ * the blocks listed for its (sequence, KV head) -- one list for all T tokens,
+ * as one list serves all heads of a group.  T = 1 is oracle_sparse.
+ * q, out: [B,T,Hq,d]; lse: [B,T,Hq].  A query that sees no token gets a zero
+ * row and lse = -inf.  Sequences with L_i < T: queries at negative positions
+ * see nothing. */
+void oracle_sparse_multi(const bf16_t *q, const bf16_t *k, const bf16_t *v,
+                         int64_t sb, int64_t sh, int64_t st,
+                         const int32_t *seq_lens, const int32_t *block_idx,
+                         const int32_t *block_cnt, int max_sel,
+                         int B, int T, int Hq, int Hkv, int d, int b,
+                         double scale, double *out, double *lse)
+{
+    int g = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int i = 0; i < B; ++i)
+        for (int hq = 0; hq < Hq; ++hq) {
+            int h = hq / g;
+            int L = seq_lens[i];
+            int n = (L + b - 1) / b;
+            unsigned char *listed = (unsigned char *)calloc((size_t)(L > 0 ? L : 1), 1);
+            unsigned char *use = (unsigned char *)calloc((size_t)(L > 0 ? L : 1), 1);
+            int cnt = block_cnt ? block_cnt[i * Hkv + h] : max_sel;
+            if (cnt > max_sel) cnt = max_sel;
+            for (int e = 0; e < cnt; ++e) {
+                int j = block_idx[((int64_t)i * Hkv + h) * max_sel + e];
+                if (j < 0 || j >= n) continue;
+                for (int t = j * b; t < (j + 1) * b && t < L; ++t) listed[t] = 1;
+            }
+            for (int t = 0; t < T; ++t) {
+                int pos = L - T + t;                      /* this query's own position */
+                for (int x = 0; x < L; ++x) use[x] = (unsigned char)(listed[x] && x <= pos);
+                int64_t row = ((int64_t)i * T + t) * Hq + hq;
+                attend_one(q + row * d, k + i * sb + h * sh, v + i * sb + h * sh, st,
+                           L, d, scale, use, out + row * d, lse + row);
+            }
+            free(use);
+            free(listed);
+        }
+}
+
 /* ------------------------------------------------------------------------- */
 /* Rotary embedding inside the gate (Sec. 2.2 "Positional Embedding").  Reading
  * taken where the paper is silent: rotate-half pairing (c, c + dg/2), angle

@@ -230,3 +230,79 @@ def test_transposed_operand_or_wrong_group_mapping_would_be_caught():
         s = 0.4 * (_f64(k[0, h]) @ _f64(q[0, hq]))
         p = np.exp(s - s.max()); p /= p.sum()
         assert np.allclose(out[0, hq], p @ _f64(v[0, h]), atol=1e-13)
+
+
+# ---- T query tokens per sequence (the query-level parallelism Sec. 6 points to) ------------------
+
+def _mk_multi(B, T, Hq, Hkv, S, d, seed, name="m"):
+    q = synth.normal_bf16((B, T, Hq, d), seed, name + "q")
+    k = synth.normal_bf16((B, Hkv, S, d), seed, name + "k")
+    v = synth.normal_bf16((B, Hkv, S, d), seed, name + "v")
+    return q, k, v
+
+
+def test_multi_token_with_one_token_is_the_single_token_routine():
+    q, k, v = _mk_multi(2, 1, 4, 2, 50, 16, 31)
+    lens = [50, 37]
+    idx = np.array([[[0, 3, 6], [1, 2, 6]], [[4, 0, -1], [2, 4, 1]]], np.int32)
+    cnt = np.array([[3, 3], [2, 3]], np.int32)
+    out, lse = oracle.sparse_multi(_bits(q), _bits(k), _bits(v), lens, idx, cnt, 8, 0.25)
+    want, want_lse = oracle.sparse(_bits(q[:, 0]), _bits(k), _bits(v), lens, idx, cnt, 8, 0.25)
+    assert np.array_equal(out[:, 0], want) and np.array_equal(lse[:, 0], want_lse)
+
+
+@pytest.mark.parametrize("T", [2, 3, 8])
+def test_multi_token_query_t_is_single_token_decode_on_the_cache_cut_after_its_position(T):
+    # query t at position L-T+t sees exactly what a one-token decode sees when the cache ends there
+    B, Hq, Hkv, S, d, b = 2, 6, 2, 70, 16, 8
+    q, k, v = _mk_multi(B, T, Hq, Hkv, S, d, 32 + T)
+    lens = np.array([70, 41], np.int32)          # 41: the T tokens straddle a block boundary for T >= 2
+    rng = synth.np_rng(5, "multi-lists")
+    idx = np.stack([np.stack([rng.permutation(9)[:6] for _ in range(Hkv)]) for _ in range(B)]).astype(np.int32)
+    idx[:, :, 0] = (lens[:, None] - 1) // b      # the last block is always there
+    idx[0, 0, 1] = (70 - T) // b                 # and, for one unit, the block the first new token is in
+    out, lse = oracle.sparse_multi(_bits(q), _bits(k), _bits(v), lens, idx, None, b, 0.3)
+    for t in range(T):
+        cut = lens - T + t + 1
+        want, want_lse = oracle.sparse(_bits(q[:, t]), _bits(k), _bits(v), cut, idx, None, b, 0.3)
+        assert np.allclose(out[:, t], want, rtol=0, atol=1e-14)
+        assert np.allclose(lse[:, t], want_lse, rtol=0, atol=1e-13)
+
+
+def test_multi_token_matches_masked_softmax_written_with_matrices():
+    # brute force: one [T, L] mask (listed blocks AND causal) and a plain softmax in numpy
+    B, T, Hq, Hkv, S, d, b = 1, 4, 4, 2, 30, 8, 4
+    q, k, v = _mk_multi(B, T, Hq, Hkv, S, d, 40)
+    L = 27
+    idx = np.array([[[6, 1, 4, 5], [6, 0, 2, 3]]], np.int32)
+    out, lse = oracle.sparse_multi(_bits(q), _bits(k), _bits(v), [L], idx, None, b, 0.5)
+    pos = np.arange(L)
+    for hq in range(Hq):
+        h = hq // 2
+        in_list = np.isin(pos // b, idx[0, h])
+        qpos = L - T + np.arange(T)
+        mask = in_list[None, :] & (pos[None, :] <= qpos[:, None])
+        s = 0.5 * _f64(q[0, :, hq]) @ _f64(k[0, h, :L]).T
+        s = np.where(mask, s, -np.inf)
+        w = np.exp(s - s.max(axis=1, keepdims=True))
+        z = w.sum(axis=1, keepdims=True)
+        assert np.allclose(out[0, :, hq], (w / z) @ _f64(v[0, h, :L]), rtol=0, atol=1e-14)
+        assert np.allclose(lse[0, :, hq], s.max(axis=1) + np.log(z[:, 0]), rtol=0, atol=1e-13)
+
+
+def test_multi_token_earlier_queries_do_not_see_later_tokens_and_unseen_rows_are_zero():
+    B, T, Hq, Hkv, S, d, b = 1, 3, 2, 1, 24, 8, 8
+    q, k, v = _mk_multi(B, T, Hq, Hkv, S, d, 41)
+    L = 17                                        # block 2 holds position 16 only
+    idx = np.array([[[2, 0]]], np.int32)
+    out, lse = oracle.sparse_multi(_bits(q), _bits(k), _bits(v), [L], idx, None, b, 0.4)
+    k2, v2 = k.clone(), v.clone()
+    k2[0, 0, 16] += 1.0                           # the last token: visible to query 2 only
+    v2[0, 0, 16] -= 2.0
+    out2, lse2 = oracle.sparse_multi(_bits(q), _bits(k2), _bits(v2), [L], idx, None, b, 0.4)
+    assert np.array_equal(out[0, :2], out2[0, :2]) and np.array_equal(lse[0, :2], lse2[0, :2])
+    assert not np.allclose(out[0, 2], out2[0, 2])
+    # only the last block listed: queries 0 and 1 (positions 14, 15) see nothing at all
+    out3, lse3 = oracle.sparse_multi(_bits(q), _bits(k), _bits(v), [L], np.array([[[2]]], np.int32), None, b, 0.4)
+    assert np.all(out3[0, :2] == 0.0) and np.all(np.isneginf(lse3[0, :2]))
+    assert np.allclose(out3[0, 2], _f64(v[0, 0, 16])[None, :], rtol=0, atol=1e-15)

@@ -162,6 +162,29 @@ seer_status seer_sparse_decode(seer_ctx* ctx, const seer_shape* shape, const see
                                void* out, float* lse, void* stream);
 
 /*
+ * The same two kernels for q_len query tokens per sequence (1 <= q_len <= 8): the query-level
+ * parallelism of multi-token prediction or speculative decoding that Sec. 6 ("Unify Sparse
+ * Prefill and Decoding") names as a way to more parallelism in sparse decoding.  The paper gives
+ * no formula; this library takes the causal definition.  The cache already holds all L_i tokens
+ * of sequence i, the newest q_len of them being the queries' own; query t (0 <= t < q_len) sits
+ * at position L_i - q_len + t and sees cached tokens at positions <= its own -- for the sparse
+ * call, of the blocks in the list of its (sequence, KV head), one list serving all q_len tokens
+ * as it serves all heads of the group.  q_len = 1 is seer_sparse_decode / seer_dense_decode.
+ *  q   [B,q_len,Hq,d] bf16 contiguous;  out [B,q_len,Hq,d] bf16;  lse [B,q_len,Hq] fp32 or NULL.
+ * A query that sees no listed token (also every query at a negative position, when
+ * L_i < q_len) gets out = 0, lse = -inf.  Tokens share a launch -- and the selected K/V are read
+ * once for all of them -- while q_len * (Hq/Hkv) <= 16; beyond that the call issues
+ * ceil(q_len / floor(16 / (Hq/Hkv))) launches on the stream.  Other arguments, errors and the
+ * treatment of the lists as in the single-token calls.
+ */
+seer_status seer_sparse_decode_multi(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv,
+                                     const void* q, int q_len, const int32_t* block_idx,
+                                     const int32_t* block_cnt, int max_sel, void* out, float* lse,
+                                     void* stream);
+seer_status seer_dense_decode_multi(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv,
+                                    const void* q, int q_len, void* out, float* lse, void* stream);
+
+/*
  * AttnGate scoring and token-budget selection (Eq. 1a, 1c; Sec. 3.1, 3.2).
  *  Scores: q_gate = RoPE_{pos = L_i-1}(w_q[h] x), score[j] = <q_gate, kcomp[i,h,j]> / sqrt(d_gate)
  *  for the blocks j < n_i - 1 (the softmax of Eq. 1c is not needed for a

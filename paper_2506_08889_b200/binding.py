@@ -31,6 +31,7 @@ EXPORTS = [
     "seer_get_device_status", "seer_workspace_bytes", "seer_launch_count",
     "seer_dense_decode", "seer_sparse_decode", "seer_gate_select", "seer_kcomp_append",
     "seer_gate_select_static", "seer_decode_step", "seer_gate_select_threshold",
+    "seer_sparse_decode_multi", "seer_dense_decode_multi",
 ]
 
 
@@ -93,6 +94,11 @@ def lib() -> ctypes.CDLL:
     L.seer_sparse_decode.restype = i32
     L.seer_sparse_decode.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), vp, vp, vp, i32,
                                      vp, vp, vp]
+    L.seer_sparse_decode_multi.restype = i32
+    L.seer_sparse_decode_multi.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), vp, i32, vp, vp,
+                                           i32, vp, vp, vp]
+    L.seer_dense_decode_multi.restype = i32
+    L.seer_dense_decode_multi.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), vp, i32, vp, vp, vp]
     L.seer_gate_select.restype = i32
     L.seer_gate_select.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, vp, i32,
                                    vp, vp, i32, vp, vp]
@@ -200,6 +206,16 @@ class Context:
         self._check(lib().seer_sparse_decode(self._h, ctypes.byref(shape), ctypes.byref(kv), _ptr(q),
                                              _ptr(block_idx), _ptr(block_cnt), int(max_sel), _ptr(out),
                                              _ptr(lse), _stream(stream)))
+
+    def seer_sparse_decode_multi(self, shape: SeerShape, kv: SeerKV, q, q_len, block_idx, block_cnt, max_sel, out,
+                                 lse=None, stream=None):
+        self._check(lib().seer_sparse_decode_multi(self._h, ctypes.byref(shape), ctypes.byref(kv), _ptr(q),
+                                                   int(q_len), _ptr(block_idx), _ptr(block_cnt), int(max_sel),
+                                                   _ptr(out), _ptr(lse), _stream(stream)))
+
+    def seer_dense_decode_multi(self, shape: SeerShape, kv: SeerKV, q, q_len, out, lse=None, stream=None):
+        self._check(lib().seer_dense_decode_multi(self._h, ctypes.byref(shape), ctypes.byref(kv), _ptr(q),
+                                                  int(q_len), _ptr(out), _ptr(lse), _stream(stream)))
 
     def seer_gate_select(self, shape: SeerShape, gate: SeerGate, seq_lens, q_nope, scores_in, token_budget,
                          block_idx, block_cnt, max_sel, scores_out=None, stream=None):

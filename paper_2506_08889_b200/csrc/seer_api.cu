@@ -77,7 +77,7 @@ struct WsLayout {
 
 constexpr int kMaxUnits = 65535;            // batch * num_kv_heads (check_shape enforces it)
 
-WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks) {
+WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks, int n_tiles = 1) {
     WsLayout w;
     // The regions that must stay zero between launches sit at offsets that do not depend on the
     // call's shape (they are sized for the largest unit count), so that calls of different shapes on
@@ -91,8 +91,8 @@ WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks) {
     w.scratch = off;
     // decode view of the scratch
     size_t d = off;
-    w.part_ml = d; d = align_up(d + sizeof(float) * (size_t)slots * 32, 256);
-    w.part_o = d;  d = align_up(d + sizeof(float) * (size_t)slots * kMaxGroup * kHeadDim, 256);
+    w.part_ml = d; d = align_up(d + sizeof(float) * (size_t)slots * 32 * n_tiles, 256);
+    w.part_o = d;  d = align_up(d + sizeof(float) * (size_t)slots * 8 * n_tiles * kHeadDim, 256);
     // gate view of the scratch
     size_t g = off;
     w.q_gate = g;  g = align_up(g + sizeof(float) * (size_t)num_units * (size_t)(d_gate > 0 ? d_gate : 0), 256);
@@ -154,7 +154,7 @@ seer_status get_map(seer_ctx* ctx, const void* base, const uint64_t dims[4], con
     return SEER_OK;
 }
 
-seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q,
+seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q, int q_len,
                           const int32_t* block_idx, const int32_t* block_cnt, int max_sel, bool sparse,
                           void* out, float* lse, void* stream) {
     if (!ctx) return SEER_ERR_INVALID_ARG;
@@ -168,6 +168,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
         kv->stride_head <= 0 || kv->stride_token < kHeadDim)
         return fail(ctx, SEER_ERR_INVALID_ARG, "K/V strides must be positive multiples of 8 elements");
     if (kv->max_seq_len <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_seq_len must be positive");
+    if (q_len < 1 || q_len > 8) return fail(ctx, SEER_ERR_UNSUPPORTED, "q_len %d (supported 1..8)", q_len);
     const bool paged = kv->page_table != nullptr;
     if (paged) {
         if (kv->page_size <= 0 || kv->page_size % kTileTokens != 0)
@@ -186,7 +187,12 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
 
     cudaError_t ce = cudaSetDevice(ctx->device);
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
-    const int per_sm = decode_ctas_per_sm(sparse, paged);
+    // Query tokens share a launch while (tokens x group) fits the kernel's 16 rows; more tokens
+    // take further launches over the same lists (each reads the selected K/V once).
+    const int group = shape->num_q_heads / shape->num_kv_heads;
+    const int tok_per_launch = q_len < 16 / group ? q_len : 16 / group;
+    const int n_tiles = tok_per_launch * group > 8 ? 2 : 1;
+    const int per_sm = decode_ctas_per_sm(sparse, paged, n_tiles);
     if (per_sm <= 0) return fail(ctx, SEER_ERR_CUDA, "decode kernel cannot be resident (shared memory)");
     long long max_tiles = sparse ? (long long)U * max_sel * tpb
                                  : (long long)U * ((kv->max_seq_len + kTileTokens - 1) / kTileTokens);
@@ -194,7 +200,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     if (grid > kMaxGridCtas) grid = kMaxGridCtas;
     if (max_tiles < grid) grid = (int)(max_tiles > 0 ? max_tiles : 1);
     const int slots = decode_max_intervals(grid) + U;
-    const WsLayout w = ws_layout(U, slots, 0, 0);
+    const WsLayout w = ws_layout(U, slots, 0, 0, n_tiles);
     if (w.total > ctx->ws_bytes)
         return fail(ctx, SEER_ERR_WORKSPACE, "workspace %zu bytes, call needs %zu", ctx->ws_bytes, w.total);
 
@@ -227,7 +233,8 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.batch = shape->batch;
     p.num_q_heads = shape->num_q_heads;
     p.num_kv_heads = shape->num_kv_heads;
-    p.group = shape->num_q_heads / shape->num_kv_heads;
+    p.group = group;
+    p.q_len = q_len;
     p.block_size = shape->block_size;
     p.tiles_per_block = tpb;
     p.num_units = U;
@@ -239,16 +246,21 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.sched = reinterpret_cast<int*>(ctx->ws + w.sched);
     p.prefix = reinterpret_cast<int*>(ctx->ws + w.prefix);
     p.steal = reinterpret_cast<int*>(ctx->ws + w.steal);
-    p.generation = ++ctx->generation;
     p.part_o = reinterpret_cast<float*>(ctx->ws + w.part_o);
     p.part_ml = reinterpret_cast<float*>(ctx->ws + w.part_ml);
 
 #ifdef SEER_DECODE_TRACE
     p.trace = reinterpret_cast<unsigned long long*>(ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)));
 #endif
-    ce = launch_decode(sparse, paged, mk_copy, *mv, p, grid, static_cast<cudaStream_t>(stream));
-    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "decode launch: %s", cudaGetErrorString(ce));
-    ctx->launches += 1;
+    for (int t0 = 0; t0 < q_len; t0 += tok_per_launch) {
+        p.t_base = t0;
+        p.t_cnt = q_len - t0 < tok_per_launch ? q_len - t0 : tok_per_launch;
+        p.rows = p.t_cnt * group;
+        p.generation = ++ctx->generation;
+        ce = launch_decode(sparse, paged, n_tiles, mk_copy, *mv, p, grid, static_cast<cudaStream_t>(stream));
+        if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "decode launch: %s", cudaGetErrorString(ce));
+        ctx->launches += 1;
+    }
     return SEER_OK;
 }
 
@@ -322,7 +334,7 @@ uint64_t seer_launch_count(const seer_ctx* ctx) { return ctx ? ctx->launches : 0
 #ifdef SEER_DECODE_TRACE
 /* diagnostic builds only: device address of the per-CTA time stamps of the last decode launch */
 void* seer_debug_trace_ptr(seer_ctx* ctx) { return ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)); }
-int seer_debug_ctas_per_sm(int sparse, int paged) { return decode_ctas_per_sm(sparse != 0, paged != 0); }
+int seer_debug_ctas_per_sm(int sparse, int paged) { return decode_ctas_per_sm(sparse != 0, paged != 0, 1); }
 #endif
 
 seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
@@ -348,18 +360,29 @@ seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
 size_t seer_workspace_bytes(const seer_shape* shape, int max_blocks, int d_gate) {
     if (!shape || shape->batch <= 0 || shape->num_kv_heads <= 0) return 0;
     const int U = shape->batch * shape->num_kv_heads;
-    return ws_layout(U, decode_max_intervals(kMaxGridCtas) + U, d_gate, max_blocks).total;
+    return ws_layout(U, decode_max_intervals(kMaxGridCtas) + U, d_gate, max_blocks, 2).total;
 }
 
 seer_status seer_dense_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q, void* out,
                               float* lse, void* stream) {
-    return decode_common(ctx, shape, kv, q, nullptr, nullptr, 0, false, out, lse, stream);
+    return decode_common(ctx, shape, kv, q, 1, nullptr, nullptr, 0, false, out, lse, stream);
 }
 
 seer_status seer_sparse_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q,
                                const int32_t* block_idx, const int32_t* block_cnt, int max_sel, void* out,
                                float* lse, void* stream) {
-    return decode_common(ctx, shape, kv, q, block_idx, block_cnt, max_sel, true, out, lse, stream);
+    return decode_common(ctx, shape, kv, q, 1, block_idx, block_cnt, max_sel, true, out, lse, stream);
+}
+
+seer_status seer_sparse_decode_multi(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q,
+                                     int q_len, const int32_t* block_idx, const int32_t* block_cnt, int max_sel,
+                                     void* out, float* lse, void* stream) {
+    return decode_common(ctx, shape, kv, q, q_len, block_idx, block_cnt, max_sel, true, out, lse, stream);
+}
+
+seer_status seer_dense_decode_multi(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q,
+                                    int q_len, void* out, float* lse, void* stream) {
+    return decode_common(ctx, shape, kv, q, q_len, nullptr, nullptr, 0, false, out, lse, stream);
 }
 
 static seer_status gate_select_common(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,

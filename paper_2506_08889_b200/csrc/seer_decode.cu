@@ -52,7 +52,7 @@ constexpr int kMinChunk = 2;                               // smallest dynamic c
 constexpr int kMinStaticTilesPerCta = 8;                   // below this everything is static
 
 struct StageMeta {
-    int nvalid;        // tokens of this tile that exist (0 = nothing was loaded); -1 = end of stream
+    int nvalid;        // cached tokens from the tile's first row on, capped at 64 + 7 (0 = nothing was loaded); -1 = end of stream
     int unit;          // (sequence, KV head) index
     int flags;         // bit 0: first tile of a piece
     int unit_first;    // global index of the unit's first tile
@@ -164,118 +164,147 @@ __device__ __forceinline__ int interval_of(const Schedule& s, int t) {
     return c * (s.R + 1) + j;
 }
 
+// Output row of row r on a unit's MMA N side: query token t_base + r / group, head r % group of
+// the KV head's group; rows of q, out and lse are laid out [sequence][token][query head].
+__device__ __forceinline__ size_t unit_row(const DecodeParams& p, int u, int r) {
+    const int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
+    const int tl = r / p.group, gi = r - tl * p.group;
+    return ((size_t)i * p.q_len + p.t_base + tl) * p.num_q_heads + (size_t)h * p.group + gi;
+}
+
 __device__ __forceinline__ void write_zero_unit(const DecodeParams& p, int u) {
-    int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
-    for (int hh = 0; hh < p.group; ++hh) {
-        size_t row = (size_t)i * p.num_q_heads + (size_t)h * p.group + hh;
+    for (int r = 0; r < p.rows; ++r) {
+        const size_t row = unit_row(p, u, r);
         for (int c = 0; c < kHeadDim; ++c) p.out[row * kHeadDim + c] = __float2bfloat16(0.f);
         if (p.lse) p.lse[row] = -INFINITY;
     }
 }
 
-constexpr int kMlStride = 32;      // floats per slot in part_ml: [0..7] max, [8..15] sum, [16] generation
+// floats per slot in part_ml for a kernel with one N-tile: [0..7] max, [8..15] sum, [16] generation;
+// with NT N-tiles: [0..8NT) max, [8NT..16NT) sum, [16NT] generation, 32*NT floats in all
+constexpr int kMlStride = 32;
 
-// Log-sum-exp combine of one unit's partials by the CTA's consumer threads.  Thread t takes head
-// t/16, channels 8*(t%16) .. +7 of every partial.
+// Log-sum-exp combine of one unit's partials by the CTA's consumer threads.  Thread t takes rows
+// t/16 + 8*nt, channels 8*(t%16) .. +7 of every partial.
+template <int NT>
 struct MergeState {
-    float M, lsum, acc[8];
+    float M[NT], lsum[NT], acc[NT][8];
 };
-__device__ __forceinline__ void merge_init(MergeState& st) {
-    st.M = -INFINITY;
-    st.lsum = 0.f;
+template <int NT>
+__device__ __forceinline__ void merge_init(MergeState<NT>& st) {
 #pragma unroll
-    for (int x = 0; x < 8; ++x) st.acc[x] = 0.f;
-}
-// Adds up to kDirect partials straight from global memory: every load is issued before any
-// arithmetic, so the whole batch costs one round trip to L2 (the cheapest way for a few partials).
-constexpr int kDirect = 8;
-__device__ __forceinline__ void merge_accumulate_direct(const DecodeParams& p, MergeState& st, const int* slots,
-                                                        int n, int t) {
-    const int hh = t >> 4, d0 = 8 * (t & 15);
-    float ms[kDirect], ls[kDirect];
-    float4 va[kDirect], vb[kDirect];
+    for (int nt = 0; nt < NT; ++nt) {
+        st.M[nt] = -INFINITY;
+        st.lsum[nt] = 0.f;
 #pragma unroll
-    for (int k = 0; k < kDirect; ++k) {
-        const size_t sl = (size_t)slots[min(k, n - 1)];
-        const float* pm = p.part_ml + sl * kMlStride;
-        const float4* qo = reinterpret_cast<const float4*>(p.part_o + sl * (kMaxGroup * kHeadDim) + hh * kHeadDim + d0);
-        ms[k] = __ldcg(pm + hh);
-        ls[k] = __ldcg(pm + kMaxGroup + hh);
-        va[k] = __ldcg(qo);
-        vb[k] = __ldcg(qo + 1);
+        for (int x = 0; x < 8; ++x) st.acc[nt][x] = 0.f;
     }
-    float Mr = st.M;
+}
+// Adds up to kDirect partials straight from global memory: every load (of one N-tile's rows) is
+// issued before any arithmetic, so the whole batch costs one round trip to L2 per N-tile (the
+// cheapest way for a few partials).
+constexpr int kDirect = 8;
+template <int NT>
+__device__ __forceinline__ void merge_accumulate_direct(const DecodeParams& p, MergeState<NT>& st, const int* slots,
+                                                        int n, int t) {
+    const int d0 = 8 * (t & 15);
 #pragma unroll
-    for (int k = 0; k < kDirect; ++k) Mr = fmaxf(Mr, k < n ? ms[k] : -INFINITY);
-    if (Mr == -INFINITY) return;
-    const float fo = (st.M == -INFINITY) ? 0.f : fast_exp2(st.M - Mr);
-    st.M = Mr;
-    st.lsum *= fo;
+    for (int nt = 0; nt < NT; ++nt) {
+        const int hh = (t >> 4) + 8 * nt;
+        float ms[kDirect], ls[kDirect];
+        float4 va[kDirect], vb[kDirect];
 #pragma unroll
-    for (int x = 0; x < 8; ++x) st.acc[x] *= fo;
+        for (int k = 0; k < kDirect; ++k) {
+            const size_t sl = (size_t)slots[min(k, n - 1)];
+            const float* pm = p.part_ml + sl * (kMlStride * NT);
+            const float4* qo = reinterpret_cast<const float4*>(p.part_o + sl * (8 * NT * kHeadDim) + hh * kHeadDim + d0);
+            ms[k] = __ldcg(pm + hh);
+            ls[k] = __ldcg(pm + 8 * NT + hh);
+            va[k] = __ldcg(qo);
+            vb[k] = __ldcg(qo + 1);
+        }
+        float Mr = st.M[nt];
 #pragma unroll
-    for (int k = 0; k < kDirect; ++k) {
-        const float fn = (k < n && ms[k] != -INFINITY) ? fast_exp2(ms[k] - Mr) : 0.f;
-        st.lsum = fmaf(ls[k], fn, st.lsum);
-        st.acc[0] = fmaf(va[k].x, fn, st.acc[0]); st.acc[1] = fmaf(va[k].y, fn, st.acc[1]);
-        st.acc[2] = fmaf(va[k].z, fn, st.acc[2]); st.acc[3] = fmaf(va[k].w, fn, st.acc[3]);
-        st.acc[4] = fmaf(vb[k].x, fn, st.acc[4]); st.acc[5] = fmaf(vb[k].y, fn, st.acc[5]);
-        st.acc[6] = fmaf(vb[k].z, fn, st.acc[6]); st.acc[7] = fmaf(vb[k].w, fn, st.acc[7]);
+        for (int k = 0; k < kDirect; ++k) Mr = fmaxf(Mr, k < n ? ms[k] : -INFINITY);
+        if (Mr == -INFINITY) continue;
+        const float fo = (st.M[nt] == -INFINITY) ? 0.f : fast_exp2(st.M[nt] - Mr);
+        st.M[nt] = Mr;
+        st.lsum[nt] *= fo;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) st.acc[nt][x] *= fo;
+#pragma unroll
+        for (int k = 0; k < kDirect; ++k) {
+            const float fn = (k < n && ms[k] != -INFINITY) ? fast_exp2(ms[k] - Mr) : 0.f;
+            st.lsum[nt] = fmaf(ls[k], fn, st.lsum[nt]);
+            st.acc[nt][0] = fmaf(va[k].x, fn, st.acc[nt][0]); st.acc[nt][1] = fmaf(va[k].y, fn, st.acc[nt][1]);
+            st.acc[nt][2] = fmaf(va[k].z, fn, st.acc[nt][2]); st.acc[nt][3] = fmaf(va[k].w, fn, st.acc[nt][3]);
+            st.acc[nt][4] = fmaf(vb[k].x, fn, st.acc[nt][4]); st.acc[nt][5] = fmaf(vb[k].y, fn, st.acc[nt][5]);
+            st.acc[nt][6] = fmaf(vb[k].z, fn, st.acc[nt][6]); st.acc[nt][7] = fmaf(vb[k].w, fn, st.acc[nt][7]);
+        }
     }
 }
 
 // Adds the partials that have been staged in shared memory: land_o + k * o_stride holds the
-// group x 128 floats of partial k, land_ml[k] its 32-float (max, sum, stamp) record.
-__device__ __forceinline__ void merge_accumulate_staged(MergeState& st, const float* land_o, int o_stride,
-                                                        const float* land_ml, int m, int group, int t) {
-    const int hh = t >> 4, d0 = 8 * (t & 15);
-    if (hh >= group) return;
-    // the round's maximum first, so that the sum below is a chain of independent multiply-adds
-    float Mr = st.M;
-    for (int k = 0; k < m; ++k) Mr = fmaxf(Mr, land_ml[k * kMlStride + hh]);
-    if (Mr == -INFINITY) return;
-    const float fo = (st.M == -INFINITY) ? 0.f : fast_exp2(st.M - Mr);
-    st.M = Mr;
-    st.lsum *= fo;
+// rows x 128 floats of partial k, land_ml + k * 32 * NT its (max, sum, stamp) record.
+template <int NT>
+__device__ __forceinline__ void merge_accumulate_staged(MergeState<NT>& st, const float* land_o, int o_stride,
+                                                        const float* land_ml, int m, int rows, int t) {
+    const int d0 = 8 * (t & 15);
 #pragma unroll
-    for (int x = 0; x < 8; ++x) st.acc[x] *= fo;
+    for (int nt = 0; nt < NT; ++nt) {
+        const int hh = (t >> 4) + 8 * nt;
+        if (hh >= rows) continue;
+        // the round's maximum first, so that the sum below is a chain of independent multiply-adds
+        float Mr = st.M[nt];
+        for (int k = 0; k < m; ++k) Mr = fmaxf(Mr, land_ml[k * (kMlStride * NT) + hh]);
+        if (Mr == -INFINITY) continue;
+        const float fo = (st.M[nt] == -INFINITY) ? 0.f : fast_exp2(st.M[nt] - Mr);
+        st.M[nt] = Mr;
+        st.lsum[nt] *= fo;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) st.acc[nt][x] *= fo;
 #pragma unroll 4
-    for (int k = 0; k < m; ++k) {
-        const float ms = land_ml[k * kMlStride + hh];
-        const float fn = (ms == -INFINITY) ? 0.f : fast_exp2(ms - Mr);
-        const float4 va = *reinterpret_cast<const float4*>(land_o + k * o_stride + hh * kHeadDim + d0);
-        const float4 vb = *reinterpret_cast<const float4*>(land_o + k * o_stride + hh * kHeadDim + d0 + 4);
-        st.lsum = fmaf(land_ml[k * kMlStride + kMaxGroup + hh], fn, st.lsum);
-        st.acc[0] = fmaf(va.x, fn, st.acc[0]); st.acc[1] = fmaf(va.y, fn, st.acc[1]);
-        st.acc[2] = fmaf(va.z, fn, st.acc[2]); st.acc[3] = fmaf(va.w, fn, st.acc[3]);
-        st.acc[4] = fmaf(vb.x, fn, st.acc[4]); st.acc[5] = fmaf(vb.y, fn, st.acc[5]);
-        st.acc[6] = fmaf(vb.z, fn, st.acc[6]); st.acc[7] = fmaf(vb.w, fn, st.acc[7]);
+        for (int k = 0; k < m; ++k) {
+            const float ms = land_ml[k * (kMlStride * NT) + hh];
+            const float fn = (ms == -INFINITY) ? 0.f : fast_exp2(ms - Mr);
+            const float4 va = *reinterpret_cast<const float4*>(land_o + k * o_stride + hh * kHeadDim + d0);
+            const float4 vb = *reinterpret_cast<const float4*>(land_o + k * o_stride + hh * kHeadDim + d0 + 4);
+            st.lsum[nt] = fmaf(land_ml[k * (kMlStride * NT) + 8 * NT + hh], fn, st.lsum[nt]);
+            st.acc[nt][0] = fmaf(va.x, fn, st.acc[nt][0]); st.acc[nt][1] = fmaf(va.y, fn, st.acc[nt][1]);
+            st.acc[nt][2] = fmaf(va.z, fn, st.acc[nt][2]); st.acc[nt][3] = fmaf(va.w, fn, st.acc[nt][3]);
+            st.acc[nt][4] = fmaf(vb.x, fn, st.acc[nt][4]); st.acc[nt][5] = fmaf(vb.y, fn, st.acc[nt][5]);
+            st.acc[nt][6] = fmaf(vb.z, fn, st.acc[nt][6]); st.acc[nt][7] = fmaf(vb.w, fn, st.acc[nt][7]);
+        }
     }
 }
-__device__ __forceinline__ void merge_finalize(const DecodeParams& p, const MergeState& st, int u, int t) {
-    const int hh = t >> 4, d0 = 8 * (t & 15);
-    if (hh < p.group) {
-        const int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
-        const size_t row = (size_t)i * p.num_q_heads + (size_t)h * p.group + hh;
-        const float inv = st.lsum > 0.f ? 1.f / st.lsum : 0.f;
+template <int NT>
+__device__ __forceinline__ void merge_finalize(const DecodeParams& p, const MergeState<NT>& st, int u, int t) {
+    const int d0 = 8 * (t & 15);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int hh = (t >> 4) + 8 * nt;
+        if (hh >= p.rows) continue;
+        const size_t row = unit_row(p, u, hh);
+        const float inv = st.lsum[nt] > 0.f ? 1.f / st.lsum[nt] : 0.f;
         uint4 pk;
-        pk.x = pack_bf16x2(st.acc[0] * inv, st.acc[1] * inv);
-        pk.y = pack_bf16x2(st.acc[2] * inv, st.acc[3] * inv);
-        pk.z = pack_bf16x2(st.acc[4] * inv, st.acc[5] * inv);
-        pk.w = pack_bf16x2(st.acc[6] * inv, st.acc[7] * inv);
+        pk.x = pack_bf16x2(st.acc[nt][0] * inv, st.acc[nt][1] * inv);
+        pk.y = pack_bf16x2(st.acc[nt][2] * inv, st.acc[nt][3] * inv);
+        pk.z = pack_bf16x2(st.acc[nt][4] * inv, st.acc[nt][5] * inv);
+        pk.w = pack_bf16x2(st.acc[nt][6] * inv, st.acc[nt][7] * inv);
         *reinterpret_cast<uint4*>(p.out + row * kHeadDim + d0) = pk;
         if (p.lse && (t & 15) == 0)
-            p.lse[row] = st.lsum > 0.f ? (st.M + log2f(st.lsum)) * 0.6931471805599453f : -INFINITY;
+            p.lse[row] = st.lsum[nt] > 0.f ? (st.M[nt] + log2f(st.lsum[nt])) * 0.6931471805599453f : -INFINITY;
     }
 }
 // One warp: the slots among [first, first + n_slots) that carry this launch's generation stamp,
 // written to `list` in order; returns how many.
+template <int NT>
 __device__ __forceinline__ int scan_valid_slots(const DecodeParams& p, int first, int n_slots, int* list, int lane) {
     int n = 0;
     for (int s0 = 0; s0 < n_slots; s0 += 32) {
         const int sl = first + s0 + lane;
         const bool ok = s0 + lane < n_slots &&
-                        __float_as_uint(__ldcg(p.part_ml + (size_t)sl * kMlStride + 16)) == p.generation;
+                        __float_as_uint(__ldcg(p.part_ml + (size_t)sl * (kMlStride * NT) + 16 * NT)) == p.generation;
         const unsigned m = __ballot_sync(0xffffffffu, ok);
         if (ok) list[n + __popc(m & ((1u << lane) - 1u))] = sl;
         n += __popc(m);
@@ -283,7 +312,7 @@ __device__ __forceinline__ int scan_valid_slots(const DecodeParams& p, int first
     return n;
 }
 
-template <bool SPARSE, bool PAGED>
+template <bool SPARSE, bool PAGED, int NT>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const DecodeParams p) {
@@ -482,11 +511,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                         if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
                         if (blk >= 0 && blk < n_i) {
                             tok0 = blk * p.block_size + (my_e % p.tiles_per_block) * kTileTokens;
-                            nvalid = max(0, min(kTileTokens, L - tok0));
+                            nvalid = max(0, min(kTileTokens + 7, L - tok0));
                         }
                     } else {
                         tok0 = my_e * kTileTokens;
-                        nvalid = max(0, min(kTileTokens, L - tok0));
+                        nvalid = max(0, min(kTileTokens + 7, L - tok0));
                     }
                     if (PAGED) {
                         if (nvalid > 0) {
@@ -562,33 +591,45 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 
     // =============================== consumer warps =====================================
     const int w = warp;
-    const int qd = lane & 3;            // column pair: heads 2*qd, 2*qd+1
+    const int qd = lane & 3;            // column pair: rows 2*qd, 2*qd+1 of every N-tile
     const int rw = lane >> 2;           // row within an 8-row slab
-    uint32_t bq[8][2];                  // Q^T B-fragments for the 8 k-steps over d
-    uint32_t bq_pre[8][2];              // the same for the unit expected next (prefetched)
-    float o[8][4];                      // O^T accumulators: 8 m-tiles over d
-    float m_run[2], l_run[2];
-    int seg = 0;                        // pieces finished so far
+    uint32_t bq[NT][8][2];              // Q^T B-fragments: NT N-tiles x 8 k-steps over d
+    uint32_t bq_pre[8][2];              // NT == 1: the same for the unit expected next (prefetched)
+    float o[NT][8][4];                  // O^T accumulators: 8 m-tiles over d per N-tile
+    float m_run[NT][2], l_run[NT][2];
+    int seg = 0;                        // merge rounds finished so far (NT per piece)
     int piece_tiles = 0, piece_iv = 0;  // tiles in the current piece, interval it started in
-    auto load_q = [&](uint32_t (&dst)[8][2], int unit) {
-        const int i = unit / p.num_kv_heads, h = unit % p.num_kv_heads;
-        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-            p.q + ((size_t)i * p.num_q_heads + (size_t)h * p.group + rw) * kHeadDim);
+    // Query token of this thread's two columns in every N-tile, as the number of newest cached
+    // tokens it may not see (q_len - 1 - token): column c of N-tile nt is row 8*nt + c of the unit,
+    // i.e. token t_base + row / group.  Rows past p.rows are padding (their result is never stored).
+    int back[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            const int r = 8 * nt + 2 * qd + c;
+            back[nt][c] = r < p.rows ? p.q_len - 1 - (p.t_base + r / p.group) : 0;
+        }
+    // B fragment of N-tile nt: this thread supplies row 8*nt + rw of the unit's queries
+    auto load_q = [&](uint32_t (&dst)[8][2], int unit, int nt) {
+        const int r = 8 * nt + rw;
+        const bool real = r < p.rows;
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + unit_row(p, unit, real ? r : 0) * kHeadDim);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-            dst[ks][0] = (rw < p.group) ? __ldg(qrow + (16 * ks + 2 * qd) / 2) : 0u;
-            dst[ks][1] = (rw < p.group) ? __ldg(qrow + (16 * ks + 8 + 2 * qd) / 2) : 0u;
+            dst[ks][0] = real ? __ldg(qrow + (16 * ks + 2 * qd) / 2) : 0u;
+            dst[ks][1] = real ? __ldg(qrow + (16 * ks + 8 + 2 * qd) / 2) : 0u;
         }
     };
     int pre_unit = -1;
-    {
+    if (NT == 1) {
         // the first tile's unit is known as soon as the producer has issued it, well before its data
         // lands: request that unit's queries in the meantime
         for (int spin = 0; spin < (1 << 22) && sm.issued < 1; ++spin) __nanosleep(32);
         __threadfence_block();
         if (sm.issued >= 1) {
             const int u0 = *reinterpret_cast<volatile int*>(&sm.meta[0].unit);
-            if (u0 >= 0) { load_q(bq_pre, u0); pre_unit = u0; }
+            if (u0 >= 0) { load_q(bq_pre, u0, 0); pre_unit = u0; }
         }
     }
 
@@ -604,7 +645,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     StageMeta mt = sm.meta[0];
     for (int it = 0; mt.nvalid >= 0; ++it) {
         const int st = it % kStages;
-        {
+        if (NT == 1) {
             // look ahead: request the queries of the next unit as soon as the producer has issued a
             // tile of it (its metadata is stable from then until we release that stage)
             const int iss = sm.issued;
@@ -614,7 +655,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 if (it + look < iss) {
                     const int u2 = *reinterpret_cast<volatile int*>(&sm.meta[(it + look) % kStages].unit);
                     if (u2 >= 0 && u2 != mt.unit && u2 != pre_unit) {
-                        load_q(bq_pre, u2);
+                        load_q(bq_pre, u2, 0);
                         pre_unit = u2;
                         break;
                     }
@@ -623,23 +664,29 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         }
         if (mt.flags & 1) {
             // first tile of a piece: fresh state, the unit's queries
-            if (mt.unit == pre_unit) {
+            if (NT == 1 && mt.unit == pre_unit) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) { bq[ks][0] = bq_pre[ks][0]; bq[ks][1] = bq_pre[ks][1]; }
+                for (int ks = 0; ks < 8; ++ks) { bq[0][ks][0] = bq_pre[ks][0]; bq[0][ks][1] = bq_pre[ks][1]; }
             } else {
-                load_q(bq, mt.unit);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) load_q(bq[nt], mt.unit, nt);
             }
 #pragma unroll
-            for (int a = 0; a < 8; ++a)
+            for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
-                for (int b = 0; b < 4; ++b) o[a][b] = 0.f;
-            m_run[0] = m_run[1] = -INFINITY;
-            l_run[0] = l_run[1] = 0.f;
+                for (int a = 0; a < 8; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) o[nt][a][b] = 0.f;
+                m_run[nt][0] = m_run[nt][1] = -INFINITY;
+                l_run[nt][0] = l_run[nt][1] = 0.f;
+            }
             piece_tiles = 0;
             piece_iv = mt.interval;
         }
         ++piece_tiles;
-        const int nvalid = mt.nvalid;
+        // mt.nvalid counts the cached tokens from the tile's first row on (up to 7 beyond the tile, so
+        // that earlier query tokens can be cut off); nvalid is the part of the tile that exists
+        const int nvalid = min(mt.nvalid, kTileTokens);
         if (nvalid > 16 * w) {
             const uint32_t kbase = smem_u32(sm.stage[st]);
             const uint32_t vbase = kbase + kTileBytes;
@@ -658,49 +705,67 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 fence_proxy_async_smem();
                 __syncwarp();
             }
-            // ---- S^T = K . Q^T (two independent accumulator chains) ----
-            float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+            // ---- S^T = K . Q^T (two independent accumulator chains per N-tile) ----
+            float sa[NT][4], sb[NT][4];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) sa[nt][x] = sb[nt][x] = 0.f;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 uint32_t a[4];
                 const int c8 = ((2 * ks) & 7) + k_csel;
                 ldmatrix_x4(a, kbase + (ks >> 2) * kHalfTileBytes + k_row * 128 + ((c8 ^ sw) << 4));
-                if (ks & 1) mma_bf16_16816(sb, a, bq[ks][0], bq[ks][1]);
-                else        mma_bf16_16816(sa, a, bq[ks][0], bq[ks][1]);
-            }
-            float s[4];
 #pragma unroll
-            for (int x = 0; x < 4; ++x) s[x] = (sa[x] + sb[x]) * p.scale_log2;
+                for (int nt = 0; nt < NT; ++nt) {
+                    if (ks & 1) mma_bf16_16816(sb[nt], a, bq[nt][ks][0], bq[nt][ks][1]);
+                    else        mma_bf16_16816(sa[nt], a, bq[nt][ks][0], bq[nt][ks][1]);
+                }
+            }
             const int r0 = 16 * w + rw;
-            if (r0 >= nvalid) s[0] = s[1] = -INFINITY;
-            if (r0 + 8 >= nvalid) s[2] = s[3] = -INFINITY;
-            // ---- online softmax over this warp's 16 tokens, per head column ----
-            float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
+            uint32_t pb[NT][2];
 #pragma unroll
-            for (int off = 4; off < 32; off <<= 1) {
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
-            }
-            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);   // finite: >= 1 valid row
-            const float al0 = fast_exp2(m_run[0] - mn0), al1 = fast_exp2(m_run[1] - mn1);
-            m_run[0] = mn0; m_run[1] = mn1;
-            const float p0 = fast_exp2(s[0] - mn0), p1 = fast_exp2(s[1] - mn1);
-            const float p2 = fast_exp2(s[2] - mn0), p3 = fast_exp2(s[3] - mn1);
-            l_run[0] = l_run[0] * al0 + (p0 + p2);
-            l_run[1] = l_run[1] * al1 + (p1 + p3);
+            for (int nt = 0; nt < NT; ++nt) {
+                float s[4];
 #pragma unroll
-            for (int a = 0; a < 8; ++a) {
-                o[a][0] *= al0; o[a][1] *= al1; o[a][2] *= al0; o[a][3] *= al1;
+                for (int x = 0; x < 4; ++x) s[x] = (sa[nt][x] + sb[nt][x]) * p.scale_log2;
+                // a row's token sees the first mt.nvalid - back cached tokens counted from this tile's start
+                const int lim0 = mt.nvalid - back[nt][0], lim1 = mt.nvalid - back[nt][1];
+                if (r0 >= lim0) s[0] = -INFINITY;
+                if (r0 >= lim1) s[1] = -INFINITY;
+                if (r0 + 8 >= lim0) s[2] = -INFINITY;
+                if (r0 + 8 >= lim1) s[3] = -INFINITY;
+                // ---- online softmax over this warp's 16 tokens, per row (column of S^T) ----
+                float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+                }
+                const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);
+                // a row that has seen nothing so far keeps max = -inf; exponents are then taken against 0
+                const float mb0 = mn0 == -INFINITY ? 0.f : mn0, mb1 = mn1 == -INFINITY ? 0.f : mn1;
+                const float al0 = fast_exp2(m_run[nt][0] - mb0), al1 = fast_exp2(m_run[nt][1] - mb1);
+                m_run[nt][0] = mn0; m_run[nt][1] = mn1;
+                const float p0 = fast_exp2(s[0] - mb0), p1 = fast_exp2(s[1] - mb1);
+                const float p2 = fast_exp2(s[2] - mb0), p3 = fast_exp2(s[3] - mb1);
+                l_run[nt][0] = l_run[nt][0] * al0 + (p0 + p2);
+                l_run[nt][1] = l_run[nt][1] * al1 + (p1 + p3);
+#pragma unroll
+                for (int a = 0; a < 8; ++a) {
+                    o[nt][a][0] *= al0; o[nt][a][1] *= al1; o[nt][a][2] *= al0; o[nt][a][3] *= al1;
+                }
+                pb[nt][0] = movmatrix_trans(pack_bf16x2(p0, p1));   // tokens 0-7 of the slice
+                pb[nt][1] = movmatrix_trans(pack_bf16x2(p2, p3));   // tokens 8-15
             }
-            const uint32_t pb0 = movmatrix_trans(pack_bf16x2(p0, p1));   // tokens 0-7 of the slice
-            const uint32_t pb1 = movmatrix_trans(pack_bf16x2(p2, p3));   // tokens 8-15
             // ---- O^T += V^T . P^T ----
 #pragma unroll
             for (int a = 0; a < 8; ++a) {
                 uint32_t f[4];
                 const int c8 = ((2 * a) & 7) + v_csel;
                 ldmatrix_x4_trans(f, vbase + (a >> 2) * kHalfTileBytes + v_row * 128 + ((c8 ^ sw) << 4));
-                mma_bf16_16816(o[a], f, pb0, pb1);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(o[nt][a], f, pb[nt][0], pb[nt][1]);
             }
         }
         __syncwarp();
@@ -712,117 +777,131 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         const StageMeta nx = sm.meta[nst];
         if (nx.flags & 1) {
             // ---------------- the current piece ends here ------------------------------------
-            float l0 = l_run[0], l1 = l_run[1];
+            // One merge round per N-tile through the same scratch: warps 1..3 hand (o, max, sum) of the
+            // N-tile to warp 0, which folds them into its own.
+            float m_all[NT][2], l_all[NT][2];
 #pragma unroll
-            for (int off = 4; off < 32; off <<= 1) {
-                l0 += __shfl_xor_sync(0xffffffffu, l0, off);
-                l1 += __shfl_xor_sync(0xffffffffu, l1, off);
-            }
-            if (w > 0) {
-                // hand (o, max, sum) to warp 0 through shared memory and move on
-                if (seg > 0 && !mbar_wait(&sm.merge_bar[1], (seg - 1) & 1, p.status)) return;   // scratch free?
+            for (int nt = 0; nt < NT; ++nt) {
+                float l0 = l_run[nt][0], l1 = l_run[nt][1];
 #pragma unroll
-                for (int a = 0; a < 8; ++a) {
-                    const int d0 = 16 * a + rw;
-                    sm.merge_o[w - 1][2 * qd][d0] = o[a][0];
-                    sm.merge_o[w - 1][2 * qd + 1][d0] = o[a][1];
-                    sm.merge_o[w - 1][2 * qd][d0 + 8] = o[a][2];
-                    sm.merge_o[w - 1][2 * qd + 1][d0 + 8] = o[a][3];
+                for (int off = 4; off < 32; off <<= 1) {
+                    l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+                    l1 += __shfl_xor_sync(0xffffffffu, l1, off);
                 }
-                if (rw == 0) {
-                    sm.merge_ml[w - 1][0][2 * qd] = m_run[0];
-                    sm.merge_ml[w - 1][0][2 * qd + 1] = m_run[1];
-                    sm.merge_ml[w - 1][1][2 * qd] = l0;
-                    sm.merge_ml[w - 1][1][2 * qd + 1] = l1;
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.merge_bar[0]);
-            } else {
-                const int u = mt.unit;
-                if (!mbar_wait(&sm.merge_bar[0], seg & 1, p.status)) return;
-                float m_all[2], l_all[2];
-                {
+                if (w > 0) {
+                    if (seg > 0 && !mbar_wait(&sm.merge_bar[1], (seg - 1) & 1, p.status)) return;   // scratch free?
+#pragma unroll
+                    for (int a = 0; a < 8; ++a) {
+                        const int d0 = 16 * a + rw;
+                        sm.merge_o[w - 1][2 * qd][d0] = o[nt][a][0];
+                        sm.merge_o[w - 1][2 * qd + 1][d0] = o[nt][a][1];
+                        sm.merge_o[w - 1][2 * qd][d0 + 8] = o[nt][a][2];
+                        sm.merge_o[w - 1][2 * qd + 1][d0 + 8] = o[nt][a][3];
+                    }
+                    if (rw == 0) {
+                        sm.merge_ml[w - 1][0][2 * qd] = m_run[nt][0];
+                        sm.merge_ml[w - 1][0][2 * qd + 1] = m_run[nt][1];
+                        sm.merge_ml[w - 1][1][2 * qd] = l0;
+                        sm.merge_ml[w - 1][1][2 * qd + 1] = l1;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.merge_bar[0]);
+                } else {
+                    if (!mbar_wait(&sm.merge_bar[0], seg & 1, p.status)) return;
                     float mw[kConsumerWarps - 1][2], lw[kConsumerWarps - 1][2];
-                    m_all[0] = m_run[0]; m_all[1] = m_run[1];
+                    m_all[nt][0] = m_run[nt][0]; m_all[nt][1] = m_run[nt][1];
 #pragma unroll
                     for (int ww = 0; ww < kConsumerWarps - 1; ++ww) {
                         mw[ww][0] = sm.merge_ml[ww][0][2 * qd]; mw[ww][1] = sm.merge_ml[ww][0][2 * qd + 1];
                         lw[ww][0] = sm.merge_ml[ww][1][2 * qd]; lw[ww][1] = sm.merge_ml[ww][1][2 * qd + 1];
-                        m_all[0] = fmaxf(m_all[0], mw[ww][0]); m_all[1] = fmaxf(m_all[1], mw[ww][1]);
+                        m_all[nt][0] = fmaxf(m_all[nt][0], mw[ww][0]); m_all[nt][1] = fmaxf(m_all[nt][1], mw[ww][1]);
                     }
-                    const float f0 = (m_run[0] == -INFINITY) ? 0.f : fast_exp2(m_run[0] - m_all[0]);
-                    const float f1 = (m_run[1] == -INFINITY) ? 0.f : fast_exp2(m_run[1] - m_all[1]);
-                    l_all[0] = l0 * f0; l_all[1] = l1 * f1;
+                    const float f0 = (m_run[nt][0] == -INFINITY) ? 0.f : fast_exp2(m_run[nt][0] - m_all[nt][0]);
+                    const float f1 = (m_run[nt][1] == -INFINITY) ? 0.f : fast_exp2(m_run[nt][1] - m_all[nt][1]);
+                    l_all[nt][0] = l0 * f0; l_all[nt][1] = l1 * f1;
 #pragma unroll
-                    for (int a = 0; a < 8; ++a) { o[a][0] *= f0; o[a][1] *= f1; o[a][2] *= f0; o[a][3] *= f1; }
+                    for (int a = 0; a < 8; ++a) {
+                        o[nt][a][0] *= f0; o[nt][a][1] *= f1; o[nt][a][2] *= f0; o[nt][a][3] *= f1;
+                    }
 #pragma unroll
                     for (int ww = 0; ww < kConsumerWarps - 1; ++ww) {
-                        const float g0 = (mw[ww][0] == -INFINITY) ? 0.f : fast_exp2(mw[ww][0] - m_all[0]);
-                        const float g1 = (mw[ww][1] == -INFINITY) ? 0.f : fast_exp2(mw[ww][1] - m_all[1]);
-                        l_all[0] += lw[ww][0] * g0; l_all[1] += lw[ww][1] * g1;
+                        const float g0 = (mw[ww][0] == -INFINITY) ? 0.f : fast_exp2(mw[ww][0] - m_all[nt][0]);
+                        const float g1 = (mw[ww][1] == -INFINITY) ? 0.f : fast_exp2(mw[ww][1] - m_all[nt][1]);
+                        l_all[nt][0] += lw[ww][0] * g0; l_all[nt][1] += lw[ww][1] * g1;
 #pragma unroll
                         for (int a = 0; a < 8; ++a) {
                             const int d0 = 16 * a + rw;
-                            o[a][0] += g0 * sm.merge_o[ww][2 * qd][d0];
-                            o[a][1] += g1 * sm.merge_o[ww][2 * qd + 1][d0];
-                            o[a][2] += g0 * sm.merge_o[ww][2 * qd][d0 + 8];
-                            o[a][3] += g1 * sm.merge_o[ww][2 * qd + 1][d0 + 8];
+                            o[nt][a][0] += g0 * sm.merge_o[ww][2 * qd][d0];
+                            o[nt][a][1] += g1 * sm.merge_o[ww][2 * qd + 1][d0];
+                            o[nt][a][2] += g0 * sm.merge_o[ww][2 * qd][d0 + 8];
+                            o[nt][a][3] += g1 * sm.merge_o[ww][2 * qd + 1][d0 + 8];
                         }
                     }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.merge_bar[1]);    // scratch may be refilled
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.merge_bar[1]);    // scratch may be refilled
+                ++seg;
+            }
+            if (w == 0) {
+                const int u = mt.unit;
                 const int n_held = sm.pieces_n;
                 if (piece_tiles < mt.unit_tiles && n_held < kMaxPieces) {
                     // part of the unit: partial into the slot of the interval the piece began in
                     const size_t slot = (size_t)piece_iv + u;
-                    float* po = p.part_o + slot * (kMaxGroup * kHeadDim);
+                    float* po = p.part_o + slot * (8 * NT * kHeadDim);
+                    float* pm = p.part_ml + slot * (kMlStride * NT);
 #pragma unroll
-                    for (int a = 0; a < 8; ++a) {
-                        const int d0 = 16 * a + rw;
-                        po[(2 * qd) * kHeadDim + d0] = o[a][0];
-                        po[(2 * qd + 1) * kHeadDim + d0] = o[a][1];
-                        po[(2 * qd) * kHeadDim + d0 + 8] = o[a][2];
-                        po[(2 * qd + 1) * kHeadDim + d0 + 8] = o[a][3];
-                    }
-                    float* pm = p.part_ml + slot * kMlStride;
-                    if (rw == 0) {
-                        pm[2 * qd] = m_all[0];
-                        pm[2 * qd + 1] = m_all[1];
-                        pm[kMaxGroup + 2 * qd] = l_all[0];
-                        pm[kMaxGroup + 2 * qd + 1] = l_all[1];
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const int c0 = 8 * nt + 2 * qd;
+#pragma unroll
+                        for (int a = 0; a < 8; ++a) {
+                            const int d0 = 16 * a + rw;
+                            po[c0 * kHeadDim + d0] = o[nt][a][0];
+                            po[(c0 + 1) * kHeadDim + d0] = o[nt][a][1];
+                            po[c0 * kHeadDim + d0 + 8] = o[nt][a][2];
+                            po[(c0 + 1) * kHeadDim + d0 + 8] = o[nt][a][3];
+                        }
+                        if (rw == 0) {
+                            pm[c0] = m_all[nt][0];
+                            pm[c0 + 1] = m_all[nt][1];
+                            pm[8 * NT + c0] = l_all[nt][0];
+                            pm[8 * NT + c0 + 1] = l_all[nt][1];
+                        }
                     }
                     if (lane == 0) {
-                        pm[16] = __uint_as_float(p.generation);
+                        pm[16 * NT] = __uint_as_float(p.generation);
                         sm.pieces[n_held] = Piece{u, piece_tiles, mt.unit_first, mt.unit_tiles, piece_iv};
                         sm.pieces_n = n_held + 1;
                     }
                     __syncwarp();
                 } else if (piece_tiles >= mt.unit_tiles) {
                     // the whole unit in one piece: final output
-                    const int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
-                    const float inv0 = l_all[0] > 0.f ? 1.f / l_all[0] : 0.f;
-                    const float inv1 = l_all[1] > 0.f ? 1.f / l_all[1] : 0.f;
-                    const size_t row0 = (size_t)i * p.num_q_heads + (size_t)h * p.group + 2 * qd;
-                    __nv_bfloat16* o0 = p.out + row0 * kHeadDim;
-                    __nv_bfloat16* o1 = o0 + kHeadDim;
-                    const bool h0 = 2 * qd < p.group, h1 = 2 * qd + 1 < p.group;
 #pragma unroll
-                    for (int a = 0; a < 8; ++a) {
-                        const int d0 = 16 * a + rw;
-                        if (h0) {
-                            o0[d0] = __float2bfloat16(o[a][0] * inv0);
-                            o0[d0 + 8] = __float2bfloat16(o[a][2] * inv0);
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const int c0 = 8 * nt + 2 * qd;
+                        const float inv0 = l_all[nt][0] > 0.f ? 1.f / l_all[nt][0] : 0.f;
+                        const float inv1 = l_all[nt][1] > 0.f ? 1.f / l_all[nt][1] : 0.f;
+                        const bool h0 = c0 < p.rows, h1 = c0 + 1 < p.rows;
+                        const size_t row0 = unit_row(p, u, h0 ? c0 : 0), row1 = unit_row(p, u, h1 ? c0 + 1 : 0);
+                        __nv_bfloat16* o0 = p.out + row0 * kHeadDim;
+                        __nv_bfloat16* o1 = p.out + row1 * kHeadDim;
+#pragma unroll
+                        for (int a = 0; a < 8; ++a) {
+                            const int d0 = 16 * a + rw;
+                            if (h0) {
+                                o0[d0] = __float2bfloat16(o[nt][a][0] * inv0);
+                                o0[d0 + 8] = __float2bfloat16(o[nt][a][2] * inv0);
+                            }
+                            if (h1) {
+                                o1[d0] = __float2bfloat16(o[nt][a][1] * inv1);
+                                o1[d0 + 8] = __float2bfloat16(o[nt][a][3] * inv1);
+                            }
                         }
-                        if (h1) {
-                            o1[d0] = __float2bfloat16(o[a][1] * inv1);
-                            o1[d0 + 8] = __float2bfloat16(o[a][3] * inv1);
+                        if (p.lse && rw == 0) {
+                            const float ln2 = 0.6931471805599453f;
+                            if (h0) p.lse[row0] = l_all[nt][0] > 0.f ? (m_all[nt][0] + log2f(l_all[nt][0])) * ln2 : -INFINITY;
+                            if (h1) p.lse[row1] = l_all[nt][1] > 0.f ? (m_all[nt][1] + log2f(l_all[nt][1])) * ln2 : -INFINITY;
                         }
-                    }
-                    if (p.lse && rw == 0) {
-                        const float ln2 = 0.6931471805599453f;
-                        if (h0) p.lse[row0] = l_all[0] > 0.f ? (m_all[0] + log2f(l_all[0])) * ln2 : -INFINITY;
-                        if (h1) p.lse[row0 + 1] = l_all[1] > 0.f ? (m_all[1] + log2f(l_all[1])) * ln2 : -INFINITY;
                     }
                 } else {
                     // (cannot happen with the schedule's bound on pieces per CTA) no room to hold
@@ -830,7 +909,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     raise_status(p.status, DEV_TIMEOUT);
                 }
             }
-            ++seg;
         }
         mt = nx;
     }
@@ -887,11 +965,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     // brought in by bulk copies, kLand at a time, into the first two stage buffers, and added up.
     int* lists = reinterpret_cast<int*>(sm.stage[2]);            // kListInts slot numbers
     int* counts = lists + kListInts;                             // per owed unit (or per warp)
-    // only the group's real heads are brought in: group x 512 B + 128 B per partial, one per lane
-    const int o_stride = p.group * kHeadDim;                     // floats per staged partial
-    const int n_land = min(32, kLandBytes / (o_stride * 4 + kMlStride * 4));
-    float* land_o = reinterpret_cast<float*>(sm.stage[0]);       // [n_land][group][128]
-    float* land_ml = land_o + n_land * o_stride;                 // [n_land][32]
+    // only the unit's real rows are brought in: rows x 512 B + 128 B * NT per partial, one per lane
+    constexpr int kMl = kMlStride * NT;                          // floats per (max, sum, stamp) record
+    const int o_stride = p.rows * kHeadDim;                      // floats per staged partial
+    const int n_land = min(32, kLandBytes / (o_stride * 4 + kMl * 4));
+    float* land_o = reinterpret_cast<float*>(sm.stage[0]);       // [n_land][rows][128]
+    float* land_ml = land_o + n_land * o_stride;                 // [n_land][32 * NT]
     int sync_phase = 0, land_phase = 0;
     auto sync_consumers = [&]() -> bool {
         __syncwarp();
@@ -901,9 +980,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         return ok;
     };
     // stage the n listed partials, kLand per round, and add them to ms (all consumer threads call)
-    auto accumulate_list = [&](MergeState& ms, const int* slots, int n) -> bool {
+    auto accumulate_list = [&](MergeState<NT>& ms, const int* slots, int n) -> bool {
         if (n > 0 && n <= kDirect) {
-            merge_accumulate_direct(p, ms, slots, n, tid);
+            merge_accumulate_direct<NT>(p, ms, slots, n, tid);
             return true;
         }
         for (int s0 = 0; s0 < n; s0 += n_land) {
@@ -912,13 +991,13 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 // warp 0 issues the copies, one partial per lane
                 if (lane == 0) {
                     fence_proxy_async_smem();        // earlier plain accesses to the landing area are done
-                    mbar_arrive_expect_tx(&sm.land_bar, (uint32_t)m * (o_stride * 4 + kMlStride * 4));
+                    mbar_arrive_expect_tx(&sm.land_bar, (uint32_t)m * (o_stride * 4 + kMl * 4));
                 }
                 __syncwarp();
                 if (lane < m) {
                     const size_t sl = (size_t)slots[s0 + lane];
-                    bulk_load(land_o + lane * o_stride, p.part_o + sl * (kMaxGroup * kHeadDim), o_stride * 4, &sm.land_bar);
-                    bulk_load(land_ml + lane * kMlStride, p.part_ml + sl * kMlStride, kMlStride * 4, &sm.land_bar);
+                    bulk_load(land_o + lane * o_stride, p.part_o + sl * (8 * NT * kHeadDim), o_stride * 4, &sm.land_bar);
+                    bulk_load(land_ml + lane * kMl, p.part_ml + sl * kMl, kMl * 4, &sm.land_bar);
                 }
             }
             if (!mbar_wait(&sm.land_bar, land_phase & 1, p.status)) return false;
@@ -926,7 +1005,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             if (tid == 0 && land_phase == 0) SEER_STAMP(5);
 #endif
             ++land_phase;
-            merge_accumulate_staged(ms, land_o, o_stride, land_ml, m, p.group, tid);
+            merge_accumulate_staged<NT>(ms, land_o, o_stride, land_ml, m, p.rows, tid);
             if (!sync_consumers()) return false;     // everybody has read the landing area
 #ifdef SEER_DECODE_TRACE
             if (tid == 0 && land_phase == 1) SEER_STAMP(1);
@@ -953,7 +1032,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     if ((mk >> lane) & 1u) lists[base + __popc(mk & ((1u << lane) - 1u))] = first + lane;
                     n = __popc(mk);
                 } else {
-                    n = scan_valid_slots(p, first, n_slots, lists + base, lane);
+                    n = scan_valid_slots<NT>(p, first, n_slots, lists + base, lane);
                 }
                 if (lane == 0) counts[e] = n;
             }
@@ -965,7 +1044,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 #endif
         base = 0;
         for (int e = 0; e < n_owed; ++e) {
-            MergeState ms;
+            MergeState<NT> ms;
             merge_init(ms);
             if (!accumulate_list(ms, lists + base, counts[e])) return;
             merge_finalize(p, ms, sm.pieces[e].unit, tid);
@@ -975,12 +1054,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         // a unit cut into thousands of pieces: go through its candidates in windows
         constexpr int kWin = kListInts / kConsumerWarps;
         for (int e = 0; e < n_owed; ++e) {
-            MergeState ms;
+            MergeState<NT> ms;
             merge_init(ms);
             const int first = sm.pieces[e].unit_first, n_slots = sm.pieces[e].unit_tiles;
             for (int w0 = 0; w0 < n_slots; w0 += kListInts) {
                 const int lo = w0 + w * kWin, hi = min(n_slots, min(w0 + kListInts, lo + kWin));
-                const int n = lo < hi ? scan_valid_slots(p, first + lo, hi - lo, lists + w * kWin, lane) : 0;
+                const int n = lo < hi ? scan_valid_slots<NT>(p, first + lo, hi - lo, lists + w * kWin, lane) : 0;
                 if (lane == 0) counts[w] = n;
                 if (!sync_consumers()) return;
                 for (int ww = 0; ww < kConsumerWarps; ++ww)
@@ -995,19 +1074,19 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 
 size_t decode_smem_bytes() { return sizeof(Smem) + 1024; }
 
-template <bool SPARSE, bool PAGED>
+template <bool SPARSE, bool PAGED, int NT>
 cudaError_t configure() {
-    return cudaFuncSetAttribute(decode_kernel<SPARSE, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(decode_kernel<SPARSE, PAGED, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)decode_smem_bytes());
 }
 
-template <bool SPARSE, bool PAGED>
+template <bool SPARSE, bool PAGED, int NT>
 int occupancy() {
     static int cached = -1;
     if (cached < 0) {
-        if (configure<SPARSE, PAGED>() != cudaSuccess) return 0;
+        if (configure<SPARSE, PAGED, NT>() != cudaSuccess) return 0;
         int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<SPARSE, PAGED>, kThreads,
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<SPARSE, PAGED, NT>, kThreads,
                                                           decode_smem_bytes()) != cudaSuccess)
             return 0;
         cached = n;
@@ -1015,28 +1094,42 @@ int occupancy() {
     return cached;
 }
 
-template <bool SPARSE, bool PAGED>
+template <bool SPARSE, bool PAGED, int NT>
 cudaError_t launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& p, int grid,
                    cudaStream_t stream) {
-    if (occupancy<SPARSE, PAGED>() <= 0) return cudaErrorInvalidConfiguration;
-    return launch_pdl(decode_kernel<SPARSE, PAGED>, dim3(grid), dim3(kThreads), decode_smem_bytes(), stream, mk, mv, p);
+    if (occupancy<SPARSE, PAGED, NT>() <= 0) return cudaErrorInvalidConfiguration;
+    return launch_pdl(decode_kernel<SPARSE, PAGED, NT>, dim3(grid), dim3(kThreads), decode_smem_bytes(), stream, mk, mv,
+                      p);
+}
+
+template <int NT>
+int occupancy_of(bool sparse, bool paged) {
+    if (sparse) return paged ? occupancy<true, true, NT>() : occupancy<true, false, NT>();
+    return paged ? occupancy<false, true, NT>() : occupancy<false, false, NT>();
+}
+
+template <int NT>
+cudaError_t launch_of(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
+                      const DecodeParams& p, int grid, cudaStream_t stream) {
+    if (sparse) return paged ? launch<true, true, NT>(map_k, map_v, p, grid, stream)
+                             : launch<true, false, NT>(map_k, map_v, p, grid, stream);
+    return paged ? launch<false, true, NT>(map_k, map_v, p, grid, stream)
+                 : launch<false, false, NT>(map_k, map_v, p, grid, stream);
 }
 
 }  // namespace
 
-int decode_ctas_per_sm(bool sparse, bool paged) {
-    if (sparse) return paged ? occupancy<true, true>() : occupancy<true, false>();
-    return paged ? occupancy<false, true>() : occupancy<false, false>();
+int decode_ctas_per_sm(bool sparse, bool paged, int n_tiles) {
+    return n_tiles == 1 ? occupancy_of<1>(sparse, paged) : occupancy_of<2>(sparse, paged);
 }
 
 int decode_max_intervals(int grid) { return grid * (kMaxRounds + 1) + 1; }
 
-cudaError_t launch_decode(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
+cudaError_t launch_decode(bool sparse, bool paged, int n_tiles, const CUtensorMap& map_k, const CUtensorMap& map_v,
                           const DecodeParams& p, int grid, cudaStream_t stream) {
-    if (sparse) return paged ? launch<true, true>(map_k, map_v, p, grid, stream)
-                             : launch<true, false>(map_k, map_v, p, grid, stream);
-    return paged ? launch<false, true>(map_k, map_v, p, grid, stream)
-                 : launch<false, false>(map_k, map_v, p, grid, stream);
+    if (n_tiles < 1 || n_tiles > 2 || p.rows > 8 * n_tiles) return cudaErrorInvalidValue;
+    return n_tiles == 1 ? launch_of<1>(sparse, paged, map_k, map_v, p, grid, stream)
+                        : launch_of<2>(sparse, paged, map_k, map_v, p, grid, stream);
 }
 
 }  // namespace seer

@@ -45,6 +45,9 @@ struct DecodeParams {
     int page_size;
     int num_pages;
     int batch, num_q_heads, num_kv_heads, group, block_size, tiles_per_block;
+    int q_len;                      // query tokens per sequence (the last q_len cached tokens), 1 for plain decoding
+    int t_base, t_cnt;              // this launch handles query tokens t_base .. t_base + t_cnt - 1
+    int rows;                       // t_cnt * group: rows on the MMA N side, <= 8 * (N-tiles of the kernel)
     int num_units;                  // batch * num_kv_heads
     int max_blocks_cap;             // tile-count clamp for dense: capacity in tiles
     int pool_div;                   // 1/pool_div of the tiles are handed out dynamically (0: none)
@@ -55,8 +58,8 @@ struct DecodeParams {
     int* steal;                     // [grid]: per-range claim counters (front | back << 16); zero between launches
     unsigned int generation;        // stamp that marks this launch's partials
     int* prefix;                    // [num_units + 1] prefix sums of the units' tile counts
-    float* part_o;                  // [slots][8][128]
-    float* part_ml;                 // [slots][32]: max[8], sum[8], generation stamp
+    float* part_o;                  // [slots][8*NT][128]   (NT: N-tiles of the kernel, 1 or 2)
+    float* part_ml;                 // [slots][32*NT]: max[8*NT], sum[8*NT], generation stamp
 #ifdef SEER_DECODE_TRACE
     unsigned long long* trace;      // [grid][8] %globaltimer stamps (diagnostic builds only)
 #endif
@@ -68,10 +71,11 @@ struct DecodeLaunch {
 };
 
 // Returns resident CTAs per SM for the decode kernel (queried once).
-int decode_ctas_per_sm(bool sparse, bool paged);
+int decode_ctas_per_sm(bool sparse, bool paged, int n_tiles);
 // Upper bound on the number of work intervals (static ranges + dynamic chunks) of a launch.
 int decode_max_intervals(int grid);
-cudaError_t launch_decode(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
+// n_tiles: MMA N-tiles of 8 rows (1 or 2); p.rows <= 8 * n_tiles.
+cudaError_t launch_decode(bool sparse, bool paged, int n_tiles, const CUtensorMap& map_k, const CUtensorMap& map_v,
                           const DecodeParams& p, int grid, cudaStream_t stream);
 
 struct GateParams {

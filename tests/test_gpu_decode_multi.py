@@ -1,0 +1,146 @@
+"""GPU parity of seer_sparse_decode_multi / seer_dense_decode_multi (q_len query tokens per
+sequence, causal among them) against the fp64 oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_08889_b200 import binding, synth
+from util import bits, check_attention, to_paged
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.close()
+
+
+def _make(B, T, Hq, Hkv, S, seed, name=""):
+    q = synth.normal_bf16((B, T, Hq, 128), seed, name + "q", DEV)
+    k = synth.normal_bf16((B, Hkv, S, 128), seed, name + "k", DEV)
+    v = synth.normal_bf16((B, Hkv, S, 128), seed, name + "v", DEV)
+    return q, k, v
+
+
+def _run(ctx, q, k, v, lens, idx, cnt, b, scale, dense=False, page_table=None, page_size=0, max_seq_len=None):
+    B, T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    shape = binding.make_shape(B, Hq, Hkv, d, b, scale)
+    lens_t = torch.as_tensor(np.asarray(lens, np.int32), device=DEV)
+    kv = binding.make_kv(k, v, lens_t, max_seq_len=max_seq_len, page_table=page_table, page_size=page_size)
+    out = torch.full((B, T, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, T, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    if dense:
+        ctx.seer_dense_decode_multi(shape, kv, q, T, out, lse)
+    else:
+        idx_t = torch.as_tensor(idx, device=DEV).contiguous()
+        cnt_t = None if cnt is None else torch.as_tensor(cnt, device=DEV).contiguous()
+        ctx.seer_sparse_decode_multi(shape, kv, q, T, idx_t, cnt_t, idx.shape[2], out, lse)
+    torch.cuda.synchronize()
+    return out, lse
+
+
+def _all_blocks(lens, Hkv, b):
+    n = [-(-int(L) // b) for L in lens]
+    idx = np.full((len(lens), Hkv, max(max(n), 1)), -1, np.int32)
+    cnt = np.zeros((len(lens), Hkv), np.int32)
+    for i, x in enumerate(n):
+        idx[i, :, :x] = np.arange(x)
+        cnt[i] = x
+    return idx, cnt
+
+
+# (Hq, Hkv, q_len): rows on the MMA N side and launches per call
+#   (32,8,2): 8 rows, one N-tile      (40,8,3): 15 rows, two N-tiles     (64,8,2): 16 rows
+#   (40,8,8): 3 + 3 + 2 tokens in three launches   (8,8,8): 8 rows   (16,8,8): 16 rows   (40,8,1): plain decode
+@pytest.mark.parametrize("Hq,Hkv,T", [(32, 8, 2), (40, 8, 3), (64, 8, 2), (40, 8, 8), (8, 8, 8), (16, 8, 8),
+                                      (40, 8, 1), (6, 2, 5)])
+def test_sparse_multi_ragged_lengths_and_boundaries(ctx, Hq, Hkv, T):
+    B, S, b = 6, 1536, 64
+    # 1536: full blocks; 1025: the last block holds one token, the others' own tokens sit in the block before;
+    # 1027 / 517: tokens straddle a block (and tile) boundary for larger T; 70; 3: shorter than q_len for T > 3
+    lens = np.array([1536, 1025, 1027, 517, 70, 3], np.int32)
+    q, k, v = _make(B, T, Hq, Hkv, S, 700 + Hq + T)
+    n = [-(-int(L) // b) for L in lens]
+    keep = [max(1, x // 2) for x in n]
+    idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max(keep) + 2, 700 + T, shuffle=True)
+    ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
+    out, lse = _run(ctx, q, k, v, lens, idx, cnt, b, 0.09)
+    check_attention(out, lse, *ref, what=f"multi Hq={Hq} T={T}")
+    assert ctx.device_status() == binding.SEER_OK
+
+
+@pytest.mark.parametrize("Hq,Hkv,T,b", [(40, 8, 3, 64), (32, 8, 4, 128), (64, 8, 4, 64)])
+def test_dense_multi_equals_oracle_with_every_block_listed(ctx, Hq, Hkv, T, b):
+    B, S = 4, 2048
+    lens = np.array([2048, 1000, 65, 2], np.int32)
+    q, k, v = _make(B, T, Hq, Hkv, S, 800 + T)
+    idx, cnt = _all_blocks(lens, Hkv, b)
+    ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
+    out, lse = _run(ctx, q, k, v, lens, None, None, b, 0.09, dense=True)
+    check_attention(out, lse, *ref, what="dense multi")
+    outs, lses = _run(ctx, q, k, v, lens, idx, cnt, b, 0.09)
+    check_attention(outs, lses, *ref, what="sparse multi, all blocks")
+    assert ctx.device_status() == binding.SEER_OK
+
+
+def test_multi_rows_that_see_nothing_are_zero(ctx):
+    # only the last block is listed and it holds one token: the earlier query tokens see nothing
+    B, T, Hq, Hkv, S, b = 2, 3, 40, 8, 256, 64
+    lens = np.array([129, 193], np.int32)
+    q, k, v = _make(B, T, Hq, Hkv, S, 810)
+    idx = np.array([[[2]] * Hkv, [[3]] * Hkv], np.int32)
+    ref_o, ref_l = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, None, b, 0.09)
+    assert np.isneginf(ref_l[:, :2]).all() and np.isfinite(ref_l[:, 2]).all()
+    out, lse = _run(ctx, q, k, v, lens, idx, None, b, 0.09)
+    check_attention(out, lse, ref_o, ref_l, what="unseen rows")
+    assert (out[:, :2] == 0).all()
+
+
+def test_multi_long_lists_split_over_ctas_and_paged(ctx):
+    # enough tiles per unit that every unit is cut into pieces and merged by the combine
+    B, T, Hq, Hkv, S, b = 2, 3, 40, 8, 16384, 64
+    lens = np.array([16384, 12345], np.int32)
+    q, k, v = _make(B, T, Hq, Hkv, S, 820)
+    n = [-(-int(L) // b) for L in lens]
+    keep = [x // 2 for x in n]
+    idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max(keep), 820)
+    ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.0884)
+    out, lse = _run(ctx, q, k, v, lens, idx, cnt, b, 0.0884)
+    check_attention(out, lse, *ref, what="multi long", strict=True)
+    kp, vp, table = to_paged(k, v, b, 820)
+    outp, lsep = _run(ctx, q, kp, vp, lens, idx, cnt, b, 0.0884, page_table=table, page_size=b, max_seq_len=S)
+    check_attention(outp, lsep, *ref, what="multi long paged", strict=True)
+    assert ctx.device_status() == binding.SEER_OK
+
+
+def test_multi_one_token_is_bitwise_the_single_token_call(ctx):
+    B, Hq, Hkv, S, b = 3, 40, 8, 4096, 64
+    lens = np.array([4096, 3000, 100], np.int32)
+    q, k, v = _make(B, 1, Hq, Hkv, S, 830)
+    idx, cnt = synth.random_block_lists(lens, Hkv, b, [20, 15, 2], 20, 830)
+    out, lse = _run(ctx, q, k, v, lens, idx, cnt, b, 0.0884)
+    shape = binding.make_shape(B, Hq, Hkv, 128, b, 0.0884)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    kv = binding.make_kv(k, v, lens_t)
+    out1 = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device=DEV)
+    lse1 = torch.empty((B, Hq), dtype=torch.float32, device=DEV)
+    ctx.seer_sparse_decode(shape, kv, q[:, 0].contiguous(), torch.as_tensor(idx, device=DEV),
+                           torch.as_tensor(cnt, device=DEV), 20, out1, lse1)
+    torch.cuda.synchronize()
+    assert torch.equal(out[:, 0], out1) and torch.equal(lse[:, 0], lse1)
+
+
+def test_multi_rejects_unsupported_q_len(ctx):
+    B, Hq, Hkv, S, b = 1, 8, 8, 64, 64
+    q, k, v = _make(B, 1, Hq, Hkv, S, 840)
+    shape = binding.make_shape(B, Hq, Hkv, 128, b, 0.1)
+    kv = binding.make_kv(k, v, torch.tensor([64], dtype=torch.int32, device=DEV))
+    out = torch.empty_like(q)
+    for bad in (0, 9):
+        with pytest.raises(binding.SeerError):
+            ctx.seer_dense_decode_multi(shape, kv, q, bad, out)

@@ -129,6 +129,12 @@ __device__ __forceinline__ float fast_exp2(float x) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 
+// Hint: bring [ptr, ptr + bytes) into L2 (ptr 16-byte aligned, bytes a multiple of 16).  Purely a
+// prefetch: no data reaches the SM, later loads read whatever L2 then holds.
+__device__ __forceinline__ void prefetch_l2(const void* ptr, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr), "r"(bytes) : "memory");
+}
+
 // sin and cos of pos * inv_freq for the rotary embedding.  The angle reaches 1e5..1e6 rad at
 // long context, so the product and the reduction to one turn are done in double (a handful
 // of operations); the reduced angle is then accurate to about 1e-10 turns and the fp32

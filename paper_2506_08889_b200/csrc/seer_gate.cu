@@ -1,10 +1,16 @@
-// AttnGate at decode time (Eq. 1a, 1c; Sec. 3.1, 3.2): the Q-branch projection + RoPE in a
-// small first kernel, then block scores against the K compression cache fused with the
-// token-budget top-k (forced last block) in a second one that is launched as a programmatic
-// dependent of the first, so that its key loads are already in flight when the gate query
-// becomes available.
+// AttnGate at decode time (Eq. 1a, 1c; Sec. 3.1, 3.2).  Up to 8192 compressed keys per
+// (sequence, KV head) unit the whole gate is one kernel, one thread-block cluster per unit: Q-branch
+// projection + RoPE spread over the cluster's warps, block scores of each CTA's slice of the K
+// compression cache, and the token-budget top-k (forced last block) by the cluster's first CTA, with
+// distributed shared memory carrying the gate query and the scores between the steps.  Beyond that
+// size the same steps run as a projection kernel and a score + selection kernel (the second a
+// programmatic dependent of the first) that go through global memory and per-unit tickets.
+#include <cooperative_groups.h>
+
 #include "seer_device.cuh"
 #include "seer_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace seer {
 
@@ -45,8 +51,7 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-constexpr int kUnitThreads = 1024;          // one-CTA-per-unit gate kernel
-constexpr int kUnitMaxBlocks = 4096;        // ... and the compressed keys it can score
+constexpr int kUnitThreads = 1024;          // most threads a CTA that runs the selection may have
 
 // Inverse of score_key (NaN came out as key 0 and goes back as -inf).
 __device__ __forceinline__ float key_score(uint32_t key) {
@@ -63,6 +68,9 @@ struct SelectSmem {
     uint32_t warp_min[kUnitThreads / 32], warp_max[kUnitThreads / 32];
     uint32_t prefix;
     int rem;
+    int bin_cnt;                            // one-pass path: candidates in the boundary bin ...
+    int list_n;                             // ... how many of them have been listed ...
+    uint32_t list[32];                      // ... and their keys
 };
 
 // Token-budget selection for one unit, run by a whole CTA.  Thread t owns the candidates
@@ -169,6 +177,85 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
         uint32_t prefix = 0u;                                  // the digits found so far, of thr - kmin
         int rem = need;
         constexpr int kBinsPerThread = kSelBins / NT;
+        // One-pass path.  Scores spread over [smin, smax] like a bell curve put at most a few
+        // candidates into any of 2048 equal-width bins, so one histogram over the monotone map
+        //     bin(s) = floor((s - smin) * 2047 / (smax - smin))
+        // leaves a boundary bin with a handful of candidates, which one warp ranks directly.  The map
+        // only has to be monotone for the result to be exact (equal scores share a bin, a larger score
+        // never lands in a lower one); when it is unusable (non-finite range) or the boundary bin
+        // holds more than 32 candidates, the radix passes below do the job.
+        if (CACHED) {
+            const float smin = key_score(kmin), smax = key_score(kmax);
+            const float range = smax - smin, scale = 2047.f / range;
+            if (smin > -INFINITY && range > 0.f && range < INFINITY && scale < INFINITY) {
+                int* hist = sm.hist[2];
+                auto bin_of = [&](uint32_t key) -> int {
+                    return min(kSelBins - 1, (int)((key_score(key) - smin) * scale));
+                };
+                int my_bin[kCachedT];
+#pragma unroll
+                for (int e = 0; e < kCachedT; ++e) {
+                    my_bin[e] = -1;
+                    if (j_lo + e < j_hi) { my_bin[e] = bin_of(keys[e]); atomicAdd(&hist[my_bin[e]], 1); }
+                }
+                if (tid == 0) sm.list_n = 0;
+                __syncthreads();
+                int c[kBinsPerThread], mine = 0;
+#pragma unroll
+                for (int x = 0; x < kBinsPerThread; ++x) { c[x] = hist[kSelBins - 1 - kBinsPerThread * tid - x]; mine += c[x]; }
+                int incl = mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                if (lane == 31) sm.warp_tot[warp] = (unsigned long long)incl;
+                __syncthreads();
+                int above = incl - mine;
+#pragma unroll
+                for (int w2 = 0; w2 < NT / 32; ++w2) above += (w2 < warp) ? (int)sm.warp_tot[w2] : 0;
+                if (above < rem && rem <= above + mine) {
+#pragma unroll
+                    for (int x = 0; x < kBinsPerThread; ++x) {
+                        if (above < rem && rem <= above + c[x]) {
+                            sm.prefix = (uint32_t)(kSelBins - 1 - kBinsPerThread * tid - x);
+                            sm.rem = rem - above;
+                            sm.bin_cnt = c[x];
+                        }
+                        above += c[x];
+                    }
+                }
+                __syncthreads();
+                const int bbin = (int)sm.prefix, brem = sm.rem, bcnt = sm.bin_cnt;
+                if (bcnt <= 32) {
+                    // list the boundary bin's keys; warp 0 finds the brem-th largest among them
+#pragma unroll
+                    for (int e = 0; e < kCachedT; ++e)
+                        if (my_bin[e] == bbin) sm.list[atomicAdd(&sm.list_n, 1)] = keys[e];
+                    __syncthreads();
+                    if (warp == 0) {
+                        const uint32_t mykey = lane < bcnt ? sm.list[lane] : 0u;
+                        int gt = 0, ge = 0;
+                        for (int m2 = 0; m2 < bcnt; ++m2) {
+                            const uint32_t km = __shfl_sync(0xffffffffu, mykey, m2);
+                            gt += km > mykey;
+                            ge += km >= mykey;
+                        }
+                        if (lane < bcnt && gt < brem && brem <= ge) {     // all such lanes hold the same key
+                            sm.prefix = mykey;
+                            sm.rem = brem - gt;
+                        }
+                    }
+                    __syncthreads();
+                    thr = sm.prefix;
+                    take_eq = sm.rem;
+                    bits_left = 0;                         // the radix passes are not needed
+                } else {
+                    for (int x = tid; x < kSelBins; x += NT) hist[x] = 0;   // used again by the third pass
+                }
+            }
+        }
+        const bool radix = bits_left > 0;
         for (int pass = 0; bits_left > 0; ++pass) {
             const int wbits = min(kSelBits, bits_left), shift = bits_left - wbits;
             int* hist = sm.hist[pass];
@@ -217,8 +304,10 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
             rem = sm.rem;
             bits_left = shift;
         }
-        thr = kmin + prefix;
-        take_eq = rem;
+        if (radix) {
+            thr = kmin + prefix;
+            take_eq = rem;
+        }
     }
 
     if (need > 0) {
@@ -426,103 +515,175 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
     GATE_STAMP(5);
 }
 
-// ---- the whole gate of one (sequence, KV head) unit in one CTA --------------------------------
-// Used when a unit's compressed keys are few enough that one SM streams them as fast as the
-// split version would (which has to publish scores, fence, take tickets and read the scores
-// back): projection + RoPE, scores into shared memory, selection, all in one launch.
+// ---- the whole gate of one unit in one thread-block cluster -------------------------------------
+// grid (S, B*Hkv) with cluster (S, 1, 1): the S CTAs of a cluster share one (sequence, KV head) unit.
+//   1. Every warp of the cluster takes rotary pairs of the Q branch (rows c and c + d_gate/2 of
+//      W_q[h]; the rows of its first pair are requested before the kernel waits for its
+//      predecessor, W_q being a constant), applies RoPE and stores the two results into the
+//      shared memory of all S CTAs (distributed shared memory).
+//   2. Each CTA scores its slice of the compressed keys (requested right after the wait, so they
+//      travel during step 1) and stores the scores into the shared memory of the cluster's first CTA.
+//   3. The first CTA runs the selection on the scores in its shared memory.
+// Between the steps the cluster meets at its hardware barrier; nothing goes through global memory
+// and nobody takes tickets.  NIT = 16-byte pieces of a W_q row per lane.
 template <int NIT>
-__global__ void __launch_bounds__(kUnitThreads, 1) gate_unit_kernel(const GateParams p) {
+__global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const GateParams p, int per) {
+    extern __shared__ float sc_all[];                  // first CTA: the unit's scores [max_blocks]
     __shared__ float qg[kMaxDGate];
-    __shared__ float sc[kUnitMaxBlocks];
     __shared__ SelectSmem sm;
-    pdl_wait();
-    pdl_launch_dependents();
-    const int u = blockIdx.x, i = u / p.num_kv_heads, h = u % p.num_kv_heads;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = (int)cluster.num_blocks(), slice = (int)cluster.block_rank();
+    const int u = blockIdx.y, i = u / p.num_kv_heads, h = u % p.num_kv_heads;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int L = __ldg(p.seq_lens + i);
-    const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
-    const int n_cand = max(0, min(n_i - 1, p.max_blocks));
-    const int lpk = p.d_gate / 8;                      // lanes per key: 8, 16 or 32
-    const int csub = tid & (lpk - 1);
-    const uint4* kc = reinterpret_cast<const uint4*>(p.kcomp + (size_t)u * p.max_blocks * p.d_gate);
-    const int total = n_cand * lpk;
-    constexpr int kBatch = 8;
-    // first batch of keys: independent of the gate query, so it travels while W_q is applied
-    uint4 kv[kBatch];
+    const int n = p.group * kHeadDim, chunks = n / 8, half = p.d_gate / 2;
+    const int gw = slice * (kGateThreads / 32) + warp, n_gw = S * (kGateThreads / 32);
+    // W_q rows of this warp's first rotary pair: constants, requested before the wait
+    uint4 wv[2][NIT];
 #pragma unroll
-    for (int k = 0; k < kBatch; ++k) {
-        const int c = k * kUnitThreads + tid;
-        kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
-    }
-    // ---- q_gate: every warp takes rotary pairs two at a time (rows c, c+1, c+half, c+1+half) ----
-    {
-        const int n = p.group * kHeadDim, chunks = n / 8, half = p.d_gate / 2;
-        const uint4* xsrc = reinterpret_cast<const uint4*>(
-            p.q_nope + ((size_t)i * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
-        uint4 xv[NIT];
+    for (int k = 0; k < 2; ++k) {
+        const uint4* wrow = reinterpret_cast<const uint4*>(p.w_q + ((size_t)h * p.d_gate + min(gw, half - 1) + k * half) * n);
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
             const int ch = lane + 32 * it;
-            xv[it] = ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u);
+            wv[k][it] = (gw < half && ch < chunks) ? __ldg(wrow + ch) : make_uint4(0u, 0u, 0u, 0u);
         }
-        for (int c0 = warp * 2; c0 < half; c0 += (kUnitThreads / 32) * 2) {
-            float acc[4];
+    }
+    // The slice's compressed keys are asked into L2 meanwhile (a hint only; they are read after the
+    // wait): entries of complete earlier blocks do not change any more, so in a decode step the
+    // key stream overlaps the predecessor kernel.
+    {
+        const int pj0 = min(p.max_blocks, slice * per), pj1 = min(p.max_blocks, pj0 + per);
+        const char* base = reinterpret_cast<const char*>(p.kcomp + ((size_t)u * p.max_blocks + pj0) * p.d_gate);
+        const int bytes = (pj1 - pj0) * p.d_gate * 2;
+        for (int off = tid * 512; off < bytes; off += kGateThreads * 512) prefetch_l2(base + off, min(512, bytes - off));
+    }
+    GATE_STAMP(0);
+    pdl_wait();                                        // queries, lengths and compressed keys are final
+    GATE_STAMP(1);
+    pdl_launch_dependents();
+    const uint4* xsrc = reinterpret_cast<const uint4*>(
+        p.q_nope + ((size_t)i * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
+    uint4 xv[NIT];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int r = c0 + (k & 1) + (k >> 1) * half;
-                const uint4* wrow = reinterpret_cast<const uint4*>(p.w_q + ((size_t)h * p.d_gate + r) * n);
-                acc[k] = 0.f;
+    for (int it = 0; it < NIT; ++it) {
+        const int ch = lane + 32 * it;
+        xv[it] = ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    const int L = __ldg(p.seq_lens + i);
+    // ---- 1. gate query ------------------------------------------------------------------------
+    for (int c = gw; c < half; c += n_gw) {
+        if (c != gw) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const uint4* wrow = reinterpret_cast<const uint4*>(p.w_q + ((size_t)h * p.d_gate + c + k * half) * n);
 #pragma unroll
                 for (int it = 0; it < NIT; ++it) {
                     const int ch = lane + 32 * it;
-                    if (ch < chunks) acc[k] += dot8(__ldg(wrow + ch), xv[it]);
+                    wv[k][it] = ch < chunks ? __ldg(wrow + ch) : make_uint4(0u, 0u, 0u, 0u);
                 }
             }
+        }
+        float a = 0.f, b = 0.f;
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
+        for (int it = 0; it < NIT; ++it) { a += dot8(wv[0][it], xv[it]); b += dot8(wv[1][it], xv[it]); }
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
-            if (lane < 2) {
-                const int c = c0 + lane;
-                float sn, cs;
-                rope_sincos((double)(L > 0 ? L - 1 : 0), p.inv_freq[c], &sn, &cs);
-                const float a = lane ? acc[1] : acc[0], b = lane ? acc[3] : acc[2];
-                qg[c] = a * cs - b * sn;
-                qg[c + half] = b * cs + a * sn;
-            }
+        for (int off = 16; off > 0; off >>= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, off);
+            b += __shfl_xor_sync(0xffffffffu, b, off);
+        }
+        float sn, cs;
+        rope_sincos((double)(L > 0 ? L - 1 : 0), p.inv_freq[c], &sn, &cs);
+        const float ra = a * cs - b * sn, rb = b * cs + a * sn;
+        if (lane < S) {                                // lane r stores into CTA r of the cluster
+            float* dst = cluster.map_shared_rank(qg, lane);
+            dst[c] = ra;
+            dst[c + half] = rb;
         }
     }
-    __syncthreads();
-    // ---- scores into shared memory (and to scores_out if the caller wants them) ----------------
+    // The slice's first batch of keys is requested only now, when the registers that held W_q and
+    // the queries are free; it travels during the cluster barrier.
+    const int lpk = p.d_gate / 8;                      // lanes per key: 8, 16 or 32
+    const int csub = tid & (lpk - 1);
+    const int j0 = min(p.max_blocks, slice * per), j1 = min(p.max_blocks, j0 + per);
+    const uint4* kc = reinterpret_cast<const uint4*>(p.kcomp + ((size_t)u * p.max_blocks + j0) * p.d_gate);
+    const int total = (j1 - j0) * lpk;
+    constexpr int kBatch = 8;
+    uint4 kv[kBatch];
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k) {                 // entries past n_i - 1 exist in memory: harmless
+        const int pc = k * kGateThreads + tid;
+        kv[k] = pc < total ? __ldg(kc + pc) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    GATE_STAMP(2);
+    cluster.sync();
+    GATE_STAMP(3);
+    // ---- 2. scores of this slice, into the first CTA's shared memory ---------------------------
+    const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
+    const int n_cand = max(0, min(n_i - 1, p.max_blocks));
+    float* sc0 = cluster.map_shared_rank(sc_all, 0);
+    float* sc_user = p.scores_user ? p.scores_user + (size_t)u * p.max_blocks : nullptr;
     float qsub[8];
 #pragma unroll
     for (int c = 0; c < 8; ++c) qsub[c] = qg[8 * csub + c];
     const float inv = rsqrtf((float)p.d_gate);
-    float* sc_out = p.scores_user ? p.scores_user + (size_t)u * p.max_blocks : nullptr;
-    for (int cb = 0; cb < total; cb += kUnitThreads * kBatch) {
+    for (int cb = 0; cb < total; cb += kGateThreads * kBatch) {
         float acc[kBatch];
 #pragma unroll
         for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
-        if (cb + kUnitThreads * kBatch < total) {      // next batch on its way while this one reduces
+        if (cb + kGateThreads * kBatch < total) {      // next batch on its way while this one reduces
 #pragma unroll
             for (int k = 0; k < kBatch; ++k) {
-                const int c = cb + (kBatch + k) * kUnitThreads + tid;
+                const int c = cb + (kBatch + k) * kGateThreads + tid;
                 kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
             }
         }
 #pragma unroll
         for (int k = 0; k < kBatch; ++k) {
             for (int off = lpk >> 1; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
-            const int c = cb + k * kUnitThreads + tid;
-            if (c < total && csub == 0) {
+            const int c = cb + k * kGateThreads + tid;
+            const int j = j0 + c / lpk;
+            if (c < total && csub == 0 && j < n_cand) {
                 const float v = acc[k] * inv;
-                sc[c / lpk] = v;
-                if (sc_out) sc_out[c / lpk] = v;
+                sc0[j] = v;
+                if (sc_user) sc_user[j] = v;
             }
         }
     }
-    __syncthreads();
-    select_dispatch<kUnitThreads, true>(p, u, sc, sm);
+    GATE_STAMP(4);
+    cluster.sync();
+    GATE_STAMP(5);
+    // ---- 3. selection by the first CTA ----------------------------------------------------------
+    if (slice != 0) return;
+    select_dispatch<kGateThreads, true>(p, u, sc_all, sm);
+    GATE_STAMP(6);
+}
+
+constexpr int kClusterMaxBlocks = 8192;     // compressed keys per unit the cluster kernel holds in shared memory
+
+template <int NIT>
+cudaError_t launch_gate_cluster(const GateParams& p, int S, int per, cudaStream_t stream) {
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(gate_cluster_kernel<NIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   kClusterMaxBlocks * (int)sizeof(float));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S, p.batch * p.num_kv_heads);
+    cfg.blockDim = dim3(kGateThreads);
+    cfg.dynamicSmemBytes = (size_t)p.max_blocks * sizeof(float);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = S;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, gate_cluster_kernel<NIT>, p, per);
 }
 
 }  // namespace
@@ -535,24 +696,22 @@ cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* la
         return launch_pdl(gate_select_only_kernel, dim3(U), dim3(kGateThreads), 0, stream, p);
     }
     const int nit = (p.group * kHeadDim / 8 + 31) / 32;
-    // One CTA per unit when a unit's keys are few enough: one SM streams them at roughly 25 GB/s
-    // (measured), the split version gets the whole chip but pays about 4 us for publishing scores
-    // and taking tickets.
-    const double one_cta_us = p.max_blocks * p.d_gate * 2.0 / 0.025e6;
-    const double split_us = (double)U * p.max_blocks * p.d_gate * 2.0 / 6.0e6 + 4.0;
-    if (p.max_blocks <= kUnitMaxBlocks && one_cta_us <= split_us) {
-        cudaError_t e;
+    cudaError_t e;
+    if (p.max_blocks <= kClusterMaxBlocks) {
+        // one cluster per unit: slices of about 512 compressed keys, at most 8 CTAs
+        int S = (p.max_blocks + 511) / 512;
+        S = S < 1 ? 1 : (S > 8 ? 8 : S);
+        const int per = (p.max_blocks + S - 1) / S;
         switch (nit) {
-            case 1: e = launch_pdl(gate_unit_kernel<1>, dim3(U), dim3(kUnitThreads), 0, stream, p); break;
-            case 2: e = launch_pdl(gate_unit_kernel<2>, dim3(U), dim3(kUnitThreads), 0, stream, p); break;
-            case 3: e = launch_pdl(gate_unit_kernel<3>, dim3(U), dim3(kUnitThreads), 0, stream, p); break;
-            default: e = launch_pdl(gate_unit_kernel<4>, dim3(U), dim3(kUnitThreads), 0, stream, p); break;
+            case 1: e = launch_gate_cluster<1>(p, S, per, stream); break;
+            case 2: e = launch_gate_cluster<2>(p, S, per, stream); break;
+            case 3: e = launch_gate_cluster<3>(p, S, per, stream); break;
+            default: e = launch_gate_cluster<4>(p, S, per, stream); break;
         }
         *launched = 1;
         return e;
     }
     const dim3 pgrid(U, (p.d_gate / 2 + 15) / 16);
-    cudaError_t e;
     switch (nit) {
         case 1: e = launch_pdl(gate_qproj_kernel<1>, pgrid, dim3(kProjThreads), 0, stream, p); break;
         case 2: e = launch_pdl(gate_qproj_kernel<2>, pgrid, dim3(kProjThreads), 0, stream, p); break;

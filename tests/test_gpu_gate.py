@@ -125,6 +125,33 @@ def test_gate_scores_and_selection(ctx, g, b):
     assert torch.equal(idx, idx2) and torch.equal(cnt, cnt2)
 
 
+def test_gate_more_keys_than_one_cluster_holds(ctx):
+    # above 8192 compressed keys per unit the gate runs as projection + score/selection kernels
+    B, Hkv, g, d, dg, b = 1, 2, 2, 128, 64, 64
+    Hq = g * Hkv
+    nbmax = 9000
+    lens = np.array([nbmax * b - 5], np.int32)
+    qn = synth.normal_bf16((B, Hq, d), 18, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, g * d), 18, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nbmax, dg), 18, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    max_sel = 900
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nbmax), dtype=torch.float32, device=DEV)
+    before = ctx.launch_count()
+    ctx.seer_gate_select(shape, gate, lens_t, qn, None, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    assert ctx.launch_count() - before == 2
+    want_sc, _ = oracle.scores(bits(qn), bits(wq), bits(kc), [nbmax - 1], [int(lens[0]) - 1], THETA)
+    got_sc = sc.cpu().numpy()
+    assert np.abs(got_sc[0, :, :nbmax - 1] - want_sc[0, :, :nbmax - 1]).max() <= 1e-3
+    want_idx, want_cnt = oracle.select(got_sc, lens, b, max_sel * b, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx) and np.array_equal(cnt.cpu().numpy(), want_cnt)
+
+
 @pytest.mark.parametrize("case", ["normal", "ties", "all_equal", "specials"])
 @pytest.mark.parametrize("b", [64, 128])
 def test_selection_bit_exact_on_given_scores(ctx, case, b):

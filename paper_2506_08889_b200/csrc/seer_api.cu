@@ -438,7 +438,7 @@ static seer_status gate_select_common(seer_ctx* ctx, const seer_shape* shape, co
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
     p.tickets = reinterpret_cast<int*>(ctx->ws + w.gate_tickets);
 #ifdef SEER_GATE_TRACE
-    p.status = reinterpret_cast<unsigned int*>(ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)));
+    p.status = reinterpret_cast<unsigned int*>(ctx->ws + (ctx->ws_bytes - (size_t)(1 << 19)));
 #endif
     if (!scores_in) fill_inv_freq(p.inv_freq, gate->d_gate, gate->rope_theta);
     int launched = 0;

@@ -102,7 +102,7 @@ static_assert(sizeof(Smem) + 1024 <= 113 * 1024, "decode kernel no longer fits t
 __device__ __forceinline__ void trace_stamp(const DecodeParams& p, int slot) {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    p.trace[(size_t)blockIdx.x * 8 + slot] = t;
+    p.trace[(size_t)blockIdx.x * 16 + slot] = t;
 }
 #define SEER_STAMP(slot) trace_stamp(p, slot)
 #else
@@ -342,8 +342,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         tma_prefetch_desc(&map_v);
     }
 
+    if (tid == 0) SEER_STAMP(8);
     __syncthreads();                                 // barriers initialised
     pdl_wait();
+    if (tid == 0) SEER_STAMP(9);
 
     if (warp == kConsumerWarps) {
         // =========================== producer warp ====================================
@@ -642,6 +644,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 
     // the first tile's metadata
     if (!mbar_wait(&sm.full[0], 0, p.status)) return;
+    if (tid == 0) SEER_STAMP(10);
     StageMeta mt = sm.meta[0];
     for (int it = 0; mt.nvalid >= 0; ++it) {
         const int st = it % kStages;
@@ -957,7 +960,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (!mbar_wait(&sm.end_bar, 0, p.status)) return;
     const int n_owed = sm.pieces_n;
 #ifdef SEER_DECODE_TRACE
-    if (tid == 0 && n_owed > 0) { SEER_STAMP(2); p.trace[(size_t)blockIdx.x * 8 + 4] = n_owed; }
+    if (tid == 0 && n_owed > 0) { SEER_STAMP(2); p.trace[(size_t)blockIdx.x * 16 + 4] = n_owed; }
 #endif
     // The combines use the stage buffers as scratch (the stream is over, nothing is in flight).  The
     // slots that really hold a partial of a unit are found by looking at the generation stamps of
@@ -1040,7 +1043,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         }
         if (!sync_consumers()) return;
 #ifdef SEER_DECODE_TRACE
-        if (tid == 0 && n_owed > 0) { SEER_STAMP(3); p.trace[(size_t)blockIdx.x * 8 + 4] = n_owed * 1000 + counts[0]; }
+        if (tid == 0 && n_owed > 0) { SEER_STAMP(3); p.trace[(size_t)blockIdx.x * 16 + 4] = n_owed * 1000 + counts[0]; }
 #endif
         base = 0;
         for (int e = 0; e < n_owed; ++e) {

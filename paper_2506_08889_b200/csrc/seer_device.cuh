@@ -129,6 +129,15 @@ __device__ __forceinline__ float fast_exp2(float x) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 
+// 16-byte asynchronous copy global -> shared (both 16-byte aligned), not through registers; the
+// issuing thread waits for its own copies with cp_async_wait_all.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+}
+
 // Hint: bring [ptr, ptr + bytes) into L2 (ptr 16-byte aligned, bytes a multiple of 16).  Purely a
 // prefetch: no data reaches the SM, later loads read whatever L2 then holds.
 __device__ __forceinline__ void prefetch_l2(const void* ptr, uint32_t bytes) {

@@ -528,7 +528,7 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
 // and nobody takes tickets.  NIT = 16-byte pieces of a W_q row per lane.
 template <int NIT>
 __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const GateParams p, int per) {
-    extern __shared__ float sc_all[];                  // first CTA: the unit's scores [max_blocks]
+    extern __shared__ __align__(16) float sc_all[];    // scores [max_blocks] (used in the first CTA), staged keys
     __shared__ float qg[kMaxDGate];
     __shared__ SelectSmem sm;
     cg::cluster_group cluster = cg::this_cluster();
@@ -561,6 +561,22 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     pdl_wait();                                        // queries, lengths and compressed keys are final
     GATE_STAMP(1);
     pdl_launch_dependents();
+    // This slice's keys: one flat run of 16-byte pieces, thread t taking pieces t, t + 512, ...
+    // The first kBatch pieces per thread go straight into shared memory by asynchronous copies, issued
+    // now, so that they travel during the projection; the next kBatch are requested into registers
+    // once the projection has freed them; any further ones follow in register batches.
+    const int lpk = p.d_gate / 8;                      // lanes per key: 8, 16 or 32
+    const int csub = tid & (lpk - 1);
+    const int j0 = min(p.max_blocks, slice * per), j1 = min(p.max_blocks, j0 + per);
+    const uint4* kc = reinterpret_cast<const uint4*>(p.kcomp + ((size_t)u * p.max_blocks + j0) * p.d_gate);
+    const int total = (j1 - j0) * lpk;
+    constexpr int kBatch = 8;
+    uint4* staged = reinterpret_cast<uint4*>(sc_all + ((p.max_blocks + 3) & ~3));     // [kBatch * 512] pieces
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k) {                 // entries past n_i - 1 exist in memory: harmless
+        const int pc = k * kGateThreads + tid;
+        if (pc < total) cp_async16(staged + pc, kc + pc);
+    }
     const uint4* xsrc = reinterpret_cast<const uint4*>(
         p.q_nope + ((size_t)i * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
     uint4 xv[NIT];
@@ -600,18 +616,11 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
             dst[c + half] = rb;
         }
     }
-    // The slice's first batch of keys is requested only now, when the registers that held W_q and
-    // the queries are free; it travels during the cluster barrier.
-    const int lpk = p.d_gate / 8;                      // lanes per key: 8, 16 or 32
-    const int csub = tid & (lpk - 1);
-    const int j0 = min(p.max_blocks, slice * per), j1 = min(p.max_blocks, j0 + per);
-    const uint4* kc = reinterpret_cast<const uint4*>(p.kcomp + ((size_t)u * p.max_blocks + j0) * p.d_gate);
-    const int total = (j1 - j0) * lpk;
-    constexpr int kBatch = 8;
+    // second batch of keys, into the registers that held W_q and the queries
     uint4 kv[kBatch];
 #pragma unroll
-    for (int k = 0; k < kBatch; ++k) {                 // entries past n_i - 1 exist in memory: harmless
-        const int pc = k * kGateThreads + tid;
+    for (int k = 0; k < kBatch; ++k) {
+        const int pc = (kBatch + k) * kGateThreads + tid;
         kv[k] = pc < total ? __ldg(kc + pc) : make_uint4(0u, 0u, 0u, 0u);
     }
     GATE_STAMP(2);
@@ -626,17 +635,8 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
 #pragma unroll
     for (int c = 0; c < 8; ++c) qsub[c] = qg[8 * csub + c];
     const float inv = rsqrtf((float)p.d_gate);
-    for (int cb = 0; cb < total; cb += kGateThreads * kBatch) {
-        float acc[kBatch];
-#pragma unroll
-        for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
-        if (cb + kGateThreads * kBatch < total) {      // next batch on its way while this one reduces
-#pragma unroll
-            for (int k = 0; k < kBatch; ++k) {
-                const int c = cb + (kBatch + k) * kGateThreads + tid;
-                kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
-            }
-        }
+    // adds up the lanes of a key and stores its score; acc[k] belongs to piece cb + k * 512 + tid
+    auto finish_batch = [&](float (&acc)[kBatch], int cb) {
 #pragma unroll
         for (int k = 0; k < kBatch; ++k) {
             for (int off = lpk >> 1; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
@@ -648,6 +648,30 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
                 if (sc_user) sc_user[j] = v;
             }
         }
+    };
+    {
+        // the staged batch (each thread reads back the pieces it copied itself)
+        cp_async_wait_all();
+        float acc[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+            const int pc = k * kGateThreads + tid;
+            acc[k] = pc < total ? dot8(staged[pc], qsub) : 0.f;
+        }
+        finish_batch(acc, 0);
+    }
+    for (int cb = kGateThreads * kBatch; cb < total; cb += kGateThreads * kBatch) {
+        float acc[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
+        if (cb + kGateThreads * kBatch < total) {      // next batch on its way while this one reduces
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                const int c = cb + (kBatch + k) * kGateThreads + tid;
+                kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        finish_batch(acc, cb);
     }
     GATE_STAMP(4);
     cluster.sync();
@@ -658,6 +682,7 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     GATE_STAMP(6);
 }
 
+constexpr int kClusterStageBytes = 8 * kGateThreads * 16;   // the staged first batch of a slice's keys
 constexpr int kClusterMaxBlocks = 8192;     // compressed keys per unit the cluster kernel holds in shared memory
 
 template <int NIT>
@@ -665,14 +690,14 @@ cudaError_t launch_gate_cluster(const GateParams& p, int S, int per, cudaStream_
     static bool configured = false;
     if (!configured) {
         const cudaError_t e = cudaFuncSetAttribute(gate_cluster_kernel<NIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   kClusterMaxBlocks * (int)sizeof(float));
+                                                   kClusterMaxBlocks * (int)sizeof(float) + kClusterStageBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S, p.batch * p.num_kv_heads);
     cfg.blockDim = dim3(kGateThreads);
-    cfg.dynamicSmemBytes = (size_t)p.max_blocks * sizeof(float);
+    cfg.dynamicSmemBytes = (size_t)((p.max_blocks + 3) & ~3) * sizeof(float) + kClusterStageBytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -451,6 +451,64 @@ def run_sweep(args):
     ctx.close()
 
 
+def run_multi(args):
+    """Multi-query-token decode (q_len tokens per sequence over one block list) on the long-context
+    workload's cache at the given sparsity, kernel-only, one GPU: time per call and per token for
+    q_len = 1..8 and three group sizes.  Writes one JSON document."""
+    import torch
+    from paper_2506_08889_b200 import binding, synth
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = synth.workload(4)
+    w.sparsity = args.sparsity
+    if args.batch:
+        w.batch = args.batch
+    if args.seq_len:
+        w.seq_len = args.seq_len
+    B, Hkv, d, b, L = w.batch, w.num_kv_heads, w.head_dim, w.block_size, w.seq_len
+    n_blocks = L // b
+    k_sel = w.keep(n_blocks)
+    n_layers = args.layers
+    layers = build_layers(w, n_layers, synth.BASE_SEED, dev)
+    ctx = binding.Context(0)
+    lens_t = torch.full((B,), L, dtype=torch.int32, device=dev)
+    lens = np.full(B, L, np.int32)
+    for l, lay in enumerate(layers):
+        lay["kv"] = binding.make_kv(lay["k"], lay["v"], lens_t)
+        idx, cnt = synth.random_block_lists(lens, Hkv, b, k_sel, k_sel, synth.BASE_SEED, f"multi:{l}")
+        lay["idx"], lay["cnt"] = torch.as_tensor(idx, device=dev), torch.as_tensor(cnt, device=dev)
+    sel_bytes = B * Hkv * k_sel * b * d * 4
+    rows = []
+    for Hq in (32, 40, 64):
+        shape = binding.make_shape(B, Hq, Hkv, d, b, w.sm_scale)
+        for T in (1, 2, 3, 4, 8):
+            q = synth.normal_bf16((B, T, Hq, d), synth.BASE_SEED, f"multi:q:{Hq}:{T}", dev)
+            out = torch.zeros_like(q)
+
+            def step(s):
+                lay = layers[s % n_layers]
+                ctx.seer_sparse_decode_multi(shape, lay["kv"], q, T, lay["idx"], lay["cnt"], k_sel, out)
+            for s in range(5):
+                step(s)
+            torch.cuda.synchronize()
+            n0 = ctx.launch_count()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for s in range(args.steps):
+                step(s)
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) / args.steps * 1e3
+            launches = (ctx.launch_count() - n0) // args.steps
+            rows.append({"num_q_heads": Hq, "q_len": T, "rows_per_unit": T * Hq // Hkv, "launches": launches,
+                         "us_per_call": round(us, 2), "us_per_token": round(us / T, 2),
+                         "GBps_read": round(launches * sel_bytes / us / 1e3, 1)})
+    assert ctx.device_status() == binding.SEER_OK
+    print(json.dumps({"workload": w.name, "batch": B, "seq_len": L, "sparsity": args.sparsity, "selected_blocks": k_sel,
+                      "selected_kv_MB_per_launch": round(sel_bytes / 1e6, 1), "rows": rows}))
+    ctx.close()
+
+
 def run_grid(args):
     """The paper's own kernel-benchmark shape (Sec. 4.4): 64 query / 8 KV heads, head_dim 128, over
     sequence length x batch x sparsity, sparse kernel against the dense kernel on the same tensors.
@@ -623,12 +681,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true", help="kernel-only sparsity sweep instead of the step benchmark")
     ap.add_argument("--grid", action="store_true", help="the paper's 64/8-head kernel grid (seq len x batch x sparsity)")
+    ap.add_argument("--multi", action="store_true", help="multi-query-token decode: q_len 1..8, kernel-only")
     ap.add_argument("--block-size", type=int, default=64, help="block size for --grid (64 or 128)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()
     if args.grid:
         run_grid(args)
+    elif args.multi:
+        run_multi(args)
     elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":

@@ -195,6 +195,40 @@ def select(scores_f32, seq_lens, block_size, token_budget, max_sel):
     return idx, cnt
 
 
+def scores_multi(q_nope, w_q, kc, seq_lens, block_size, theta):
+    """Gate scores for T query tokens per sequence: per block the largest of the tokens' scores, over
+    the blocks wholly before the first query token.  q_nope: [B,T,Hq,d].  Returns [B,Hkv,max_blocks] f64."""
+    q_nope = np.ascontiguousarray(_u16(q_nope, "q_nope"))
+    w_q = np.ascontiguousarray(_u16(w_q, "w_q"))
+    kc = np.ascontiguousarray(_u16(kc, "kc"))
+    B, T, Hq, d = q_nope.shape
+    _, Hkv, max_blocks, dg = kc.shape
+    assert w_q.shape == (Hkv, dg, (Hq // Hkv) * d)
+    seq_lens = _i32(seq_lens)
+    sc = np.zeros((B, Hkv, max_blocks), np.float64)
+    lib().oracle_scores_multi(_p(q_nope), _p(w_q), _p(kc), _p(seq_lens), ctypes.c_int(T),
+                              ctypes.c_int(B), ctypes.c_int(Hq), ctypes.c_int(Hkv), ctypes.c_int(d),
+                              ctypes.c_int(dg), ctypes.c_int(max_blocks), ctypes.c_int(block_size),
+                              ctypes.c_double(theta), _p(sc))
+    return sc
+
+
+def select_multi(scores_f32, seq_lens, block_size, token_budget, q_len, max_sel):
+    """Token-budget top-k for q_len query tokens: the blocks holding the query tokens are forced."""
+    s = np.ascontiguousarray(np.asarray(scores_f32))
+    if s.dtype != np.float32:
+        raise TypeError("selection is defined on fp32 scores")
+    B, Hkv, max_blocks = s.shape
+    seq_lens = _i32(seq_lens)
+    idx = np.zeros((B, Hkv, max_sel), np.int32)
+    cnt = np.zeros((B, Hkv), np.int32)
+    lib().oracle_select_multi(_p(s), _p(seq_lens), ctypes.c_int(B), ctypes.c_int(Hkv),
+                              ctypes.c_int(block_size), ctypes.c_int(max_blocks),
+                              ctypes.c_int(token_budget), ctypes.c_int(q_len), ctypes.c_int(max_sel),
+                              _p(idx), _p(cnt))
+    return idx, cnt
+
+
 def select_threshold(scores_f32, seq_lens, block_size, tau, max_sel):
     """Threshold selection on softmax(scores) with the forced last block.
     Returns (idx, cnt, probs f64 [B,Hkv,max_blocks])."""

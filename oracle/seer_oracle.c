@@ -457,3 +457,94 @@ void oracle_select_threshold(const float *scores, const int32_t *seq_lens,
             block_cnt[i * Hkv + h] = emit_best_and_last(s, n, need, max_sel, dst);
         }
 }
+
+/* ------------------------------------------------------------------------- */
+/* The gate for T query tokens per sequence (the newest T cached tokens; see
+ * oracle_sparse_multi).  The paper has no gate for several decode-time
+ * queries; reading taken: every query token gets its own gate query, rotated
+ * at its own position L_i - T + t; a block's score is the largest of the T
+ * tokens' scores (a block that any token wants is wanted), over the blocks
+ * that lie wholly before the first query token, j < j_f = floor((L_i - T)/b)
+ * (all of them complete).  T = 1 is oracle_scores with n_entries = n_i - 1,
+ * qpos = L_i - 1.  q_nope: [B,T,Hq,d]; scores: [B,Hkv,max_blocks], entries
+ * j >= j_f untouched. */
+void oracle_scores_multi(const bf16_t *q_nope, const bf16_t *w_q, const bf16_t *kc,
+                         const int32_t *seq_lens, int T,
+                         int B, int Hq, int Hkv, int d, int dg, int max_blocks, int b,
+                         double theta, double *scores)
+{
+    int g = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int i = 0; i < B; ++i)
+        for (int h = 0; h < Hkv; ++h) {
+            int L = seq_lens[i];
+            int jf = L - T > 0 ? (L - T) / b : 0;
+            if (jf > max_blocks) jf = max_blocks;
+            double *qg = (double *)malloc(sizeof(double) * (size_t)dg);
+            double *best = scores + ((int64_t)i * Hkv + h) * max_blocks;
+            const bf16_t *w = w_q + (int64_t)h * dg * g * d;
+            const bf16_t *kcb = kc + ((int64_t)i * Hkv + h) * max_blocks * dg;
+            for (int t = 0; t < T; ++t) {
+                const bf16_t *x = q_nope + (((int64_t)i * T + t) * Hq + (int64_t)h * g) * d;
+                for (int r = 0; r < dg; ++r) {
+                    double acc = 0.0;
+                    for (int c = 0; c < g * d; ++c)
+                        acc += bf16_to_f64(w[(int64_t)r * g * d + c]) * bf16_to_f64(x[c]);
+                    qg[r] = acc;
+                }
+                rope_f64(qg, dg, (double)(L - T + t), theta);
+                for (int j = 0; j < jf; ++j) {
+                    double acc = 0.0;
+                    for (int r = 0; r < dg; ++r)
+                        acc += qg[r] * bf16_to_f64(kcb[(int64_t)j * dg + r]);
+                    acc /= sqrt((double)dg);
+                    if (t == 0 || acc > best[j]) best[j] = acc;
+                }
+            }
+            free(qg);
+        }
+}
+
+/* Token-budget selection for T query tokens: the blocks that hold a query
+ * token's own position, j_f .. n_i - 1 (one or two blocks for T <= b), are
+ * always in the list and count against k = min(max(1, budget/b), n_i, max_sel);
+ * the other k - (n_i - j_f) come from blocks [0, j_f) by (score descending,
+ * index ascending).  If the forced blocks alone exceed max_sel the last max_sel
+ * of them are kept.  T = 1 is oracle_select. */
+void oracle_select_multi(const float *scores, const int32_t *seq_lens,
+                         int B, int Hkv, int b, int max_blocks, int token_budget, int T,
+                         int max_sel, int32_t *block_idx, int32_t *block_cnt)
+{
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int i = 0; i < B; ++i)
+        for (int h = 0; h < Hkv; ++h) {
+            int32_t *dst = block_idx + ((int64_t)i * Hkv + h) * max_sel;
+            for (int e = 0; e < max_sel; ++e) dst[e] = -1;
+            int L = seq_lens[i];
+            int n = (L + b - 1) / b;
+            if (n <= 0) { block_cnt[i * Hkv + h] = 0; continue; }
+            int jf = L - T > 0 ? (L - T) / b : 0;
+            int k = token_budget / b;
+            if (k < 1) k = 1;
+            if (k > n) k = n;
+            if (k > max_sel) k = max_sel;
+            int forced = n - jf;
+            if (forced > max_sel) forced = max_sel;
+            int need = k - forced;
+            if (need < 0) need = 0;
+            if (need > jf) need = jf;
+            if (need > max_blocks) need = max_blocks;
+            const float *s = scores + ((int64_t)i * Hkv + h) * max_blocks;
+            int ncand = jf < max_blocks ? jf : max_blocks;
+            cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(ncand > 0 ? ncand : 1));
+            for (int j = 0; j < ncand; ++j) { cand[j].s = s[j]; cand[j].j = j; }
+            qsort(cand, (size_t)ncand, sizeof(cand_t), cand_before);
+            int m = 0;
+            for (int e = 0; e < need && e < ncand; ++e) dst[m++] = cand[e].j;
+            for (int j = n - forced; j < n; ++j) dst[m++] = j;
+            qsort(dst, (size_t)m, sizeof(int32_t), int_asc);
+            free(cand);
+            block_cnt[i * Hkv + h] = m;
+        }
+}
+

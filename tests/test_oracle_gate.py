@@ -174,3 +174,29 @@ def test_score_depends_on_relative_position_only():
     s1 = oracle.rope(x, 2 * b + 3, THETA) @ kc64[0, 0, 1]
     s2 = oracle.rope(x, 5 * b + 3, THETA) @ kc64[0, 0, 4]
     assert abs(s1 - s2) < 1e-10
+
+
+# ---- gate scores for several query tokens ---------------------------------------------------------
+
+def test_multi_token_scores_are_the_maximum_of_single_token_scores_at_each_tokens_position():
+    B, T, Hq, Hkv, d, dg, nb, b = 2, 3, 4, 2, 8, 8, 9, 16
+    qn = synth.normal_bf16((B, T, Hq, d), 6, "qn")
+    w = synth.normal_bf16((Hkv, dg, 2 * d), 6, "w", std=0.2)
+    kc = synth.normal_bf16((B, Hkv, nb, dg), 6, "kc")
+    lens = np.array([9 * 16, 5 * 16 + 2], np.int32)     # 82: the three tokens straddle blocks 4 and 5
+    got = oracle.scores_multi(_bits(qn), _bits(w), _bits(kc), lens, b, THETA)
+    jf = [(int(L) - T) // b for L in lens]
+    assert jf == [8, 4]
+    per_token = []
+    for t in range(T):
+        sc, _ = oracle.scores(_bits(qn[:, t]), _bits(w), _bits(kc), jf, [int(L) - T + t for L in lens], THETA)
+        per_token.append(sc)
+    want = np.max(np.stack(per_token), axis=0)
+    for i in range(B):
+        assert np.allclose(got[i, :, :jf[i]], want[i, :, :jf[i]], rtol=0, atol=1e-13)
+        assert np.all(got[i, :, jf[i]:] == 0.0)
+    # a single token: the single-token routine itself
+    one = oracle.scores_multi(_bits(qn[:, :1]), _bits(w), _bits(kc), lens, b, THETA)
+    ref, _ = oracle.scores(_bits(qn[:, 0]), _bits(w), _bits(kc), [(int(L) - 1) // b for L in lens],
+                           [int(L) - 1 for L in lens], THETA)
+    assert np.array_equal(one, ref)

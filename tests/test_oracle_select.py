@@ -134,3 +134,45 @@ def test_threshold_closed_forms_and_truncation():
     # a single block: nothing to normalise over
     idx, cnt, _ = oracle.select_threshold(sc3, [3], 4, 0.1, 4)
     assert list(idx[0, 0]) == [0, -1, -1, -1] and cnt[0, 0] == 1
+
+
+# ---- selection for several query tokens: the blocks holding the query tokens are forced ----------
+
+def test_multi_token_selection_with_one_token_is_the_single_token_selection():
+    r = np.random.default_rng(11)
+    sc = r.normal(size=(3, 2, 40)).astype(np.float32)
+    lens = np.array([40 * 16, 17 * 16 - 5, 3], np.int32)
+    for budget, max_sel in [(16 * 7, 12), (16 * 100, 40), (0, 4)]:
+        a = oracle.select(sc, lens, 16, budget, max_sel)
+        m = oracle.select_multi(sc, lens, 16, budget, 1, max_sel)
+        assert np.array_equal(a[0], m[0]) and np.array_equal(a[1], m[1])
+
+
+@pytest.mark.parametrize("T", [2, 5, 8])
+def test_multi_token_selection_against_lexsort_with_forced_blocks(T):
+    r = np.random.default_rng(20 + T)
+    B, Hkv, b, max_blocks, max_sel = 5, 2, 16, 40, 12
+    # 640: the T tokens sit in the last block; 16*17+3: they straddle two blocks (for T > 3);
+    # 16*9: exactly at a block end; 4: shorter than a block; 2: shorter than T for T > 2
+    lens = np.array([640, 16 * 17 + 3, 16 * 9, 4, 2], np.int32)
+    sc = np.round(r.normal(size=(B, Hkv, max_blocks)).astype(np.float32) * 3) / 3
+    for budget in (16 * 7, 16 * 2, 16, 16 * 100):
+        idx, cnt = oracle.select_multi(sc, lens, b, budget, T, max_sel)
+        for i in range(B):
+            L = int(lens[i])
+            n = -(-L // b)
+            jf = max(0, L - T) // b
+            forced = list(range(jf, n))
+            k = min(max(1, budget // b), n, max_sel)
+            need = min(max(0, k - len(forced)), jf)
+            for h in range(Hkv):
+                order = np.lexsort((np.arange(jf), -sc[i, h, :jf].astype(np.float64)))
+                want = sorted(list(order[:need]) + forced)
+                assert cnt[i, h] == len(want)
+                assert list(idx[i, h, :len(want)]) == want
+                assert np.all(idx[i, h, len(want):] == -1)
+                # every query token's own block is there
+                for t in range(T):
+                    pos = L - T + t
+                    if pos >= 0:
+                        assert pos // b in want

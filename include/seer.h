@@ -208,6 +208,26 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
                              float* scores_out, void* stream);
 
 /*
+ * The gate for q_len query tokens per sequence (the newest q_len cached tokens, as in
+ * seer_sparse_decode_multi), producing the one block list per (sequence, KV head) that the
+ * multi-token decode takes.  The paper has no gate for several decode-time queries (Sec. 6 only
+ * names the direction); this library's reading: every query token t gets its own gate query,
+ * rotated at its own position L_i - q_len + t (Eq. 1a); a block's score is the largest of the
+ * q_len tokens' scores (Eq. 1c without the softmax), over the blocks that lie wholly before the
+ * first query token, j < j_f = floor((L_i - q_len) / b); the blocks that hold a query token's own
+ * position, j_f .. n_i - 1 (one or two), are always selected and count against the budget;
+ * the other min(max(1, budget/b), n_i, max_sel) - (n_i - j_f) come from [0, j_f) by (score
+ * descending, index ascending).  q_len = 1 is seer_gate_select.
+ *  q_nope [B,q_len,Hq,d] bf16 (ignored when scores_in is given: selection only, scores_in holding
+ *  the per-block maxima).  1 <= q_len <= 8; with scores_in == NULL, gate->max_blocks <= 8192.
+ * Other arguments, outputs and errors as in seer_gate_select.
+ */
+seer_status seer_gate_select_multi(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                                   const int32_t* seq_lens, const void* q_nope, const float* scores_in,
+                                   int q_len, int token_budget, int32_t* block_idx, int32_t* block_cnt,
+                                   int max_sel, float* scores_out, void* stream);
+
+/*
  * The threshold method of Sec. 3.1: the scores are normalised by a softmax over the blocks
  * that have a compressed key (Eq. 1c; blocks [0, n_i - 1)), and the blocks whose probability
  * exceeds `threshold` are selected -- a different number for every (sequence, KV head).  The

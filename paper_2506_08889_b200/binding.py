@@ -31,7 +31,7 @@ EXPORTS = [
     "seer_get_device_status", "seer_workspace_bytes", "seer_launch_count",
     "seer_dense_decode", "seer_sparse_decode", "seer_gate_select", "seer_kcomp_append",
     "seer_gate_select_static", "seer_decode_step", "seer_gate_select_threshold",
-    "seer_sparse_decode_multi", "seer_dense_decode_multi",
+    "seer_sparse_decode_multi", "seer_dense_decode_multi", "seer_gate_select_multi",
 ]
 
 
@@ -99,6 +99,9 @@ def lib() -> ctypes.CDLL:
                                            i32, vp, vp, vp]
     L.seer_dense_decode_multi.restype = i32
     L.seer_dense_decode_multi.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), vp, i32, vp, vp, vp]
+    L.seer_gate_select_multi.restype = i32
+    L.seer_gate_select_multi.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, vp, i32, i32,
+                                         vp, vp, i32, vp, vp]
     L.seer_gate_select.restype = i32
     L.seer_gate_select.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, vp, i32,
                                    vp, vp, i32, vp, vp]
@@ -222,6 +225,13 @@ class Context:
         self._check(lib().seer_gate_select(self._h, ctypes.byref(shape), ctypes.byref(gate), _ptr(seq_lens),
                                            _ptr(q_nope), _ptr(scores_in), int(token_budget), _ptr(block_idx),
                                            _ptr(block_cnt), int(max_sel), _ptr(scores_out), _stream(stream)))
+
+    def seer_gate_select_multi(self, shape: SeerShape, gate: SeerGate, seq_lens, q_nope, scores_in, q_len,
+                               token_budget, block_idx, block_cnt, max_sel, scores_out=None, stream=None):
+        self._check(lib().seer_gate_select_multi(self._h, ctypes.byref(shape), ctypes.byref(gate), _ptr(seq_lens),
+                                                 _ptr(q_nope), _ptr(scores_in), int(q_len), int(token_budget),
+                                                 _ptr(block_idx), _ptr(block_cnt), int(max_sel), _ptr(scores_out),
+                                                 _stream(stream)))
 
     def seer_gate_select_threshold(self, shape: SeerShape, gate: SeerGate, seq_lens, q_nope, scores_in, threshold,
                                    block_idx, block_cnt, max_sel, scores_out=None, stream=None):

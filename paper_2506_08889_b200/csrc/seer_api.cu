@@ -388,7 +388,8 @@ seer_status seer_dense_decode_multi(seer_ctx* ctx, const seer_shape* shape, cons
 static seer_status gate_select_common(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
                                       const int32_t* seq_lens, const void* q_nope, const float* scores_in,
                                       int token_budget, int threshold_mode, float threshold, int32_t* block_idx,
-                                      int32_t* block_cnt, int max_sel, float* scores_out, void* stream) {
+                                      int32_t* block_cnt, int max_sel, float* scores_out, void* stream,
+                                      int q_len = 1) {
     if (!ctx) return SEER_ERR_INVALID_ARG;
     seer_status st = check_shape(ctx, shape);
     if (st != SEER_OK) return st;
@@ -396,6 +397,10 @@ static seer_status gate_select_common(seer_ctx* ctx, const seer_shape* shape, co
         return fail(ctx, SEER_ERR_INVALID_ARG, "NULL pointer among gate/seq_lens/block_idx/block_cnt");
     if (max_sel <= 0 || gate->max_blocks <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_sel and max_blocks must be positive");
     if (token_budget < 0) return fail(ctx, SEER_ERR_INVALID_ARG, "token_budget is negative");
+    if (q_len < 1 || q_len > 8) return fail(ctx, SEER_ERR_UNSUPPORTED, "q_len %d (supported 1..8)", q_len);
+    if (q_len > 1 && !scores_in && !gate_one_kernel(gate->max_blocks))
+        return fail(ctx, SEER_ERR_UNSUPPORTED, "q_len > 1 with max_blocks %d (the multi-token gate holds at most 8192 keys per unit)",
+                    gate->max_blocks);
     if (!scores_in) {
         if (!q_nope || !gate->w_q || !gate->kcomp)
             return fail(ctx, SEER_ERR_INVALID_ARG, "q_nope, w_q and kcomp are needed when scores_in is NULL");
@@ -433,6 +438,7 @@ static seer_status gate_select_common(seer_ctx* ctx, const seer_shape* shape, co
     p.max_blocks = gate->max_blocks;
     p.max_sel = max_sel;
     p.token_budget = token_budget;
+    p.q_len = q_len;
     p.threshold_mode = threshold_mode;
     p.threshold = threshold;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
@@ -453,6 +459,14 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
                              int32_t* block_cnt, int max_sel, float* scores_out, void* stream) {
     return gate_select_common(ctx, shape, gate, seq_lens, q_nope, scores_in, token_budget, 0, 0.f, block_idx, block_cnt,
                               max_sel, scores_out, stream);
+}
+
+seer_status seer_gate_select_multi(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                                   const int32_t* seq_lens, const void* q_nope, const float* scores_in, int q_len,
+                                   int token_budget, int32_t* block_idx, int32_t* block_cnt, int max_sel,
+                                   float* scores_out, void* stream) {
+    return gate_select_common(ctx, shape, gate, seq_lens, q_nope, scores_in, token_budget, 0, 0.f, block_idx, block_cnt,
+                              max_sel, scores_out, stream, q_len);
 }
 
 seer_status seer_gate_select_threshold(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,

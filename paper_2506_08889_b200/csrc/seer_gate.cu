@@ -17,6 +17,7 @@ namespace seer {
 namespace {
 
 constexpr int kGateThreads = 512;
+constexpr int kMaxQLen = 8;                 // query tokens per sequence the gate takes
 constexpr int kProjThreads = 256;
 
 __device__ __forceinline__ float dot8(const uint4& a, const float* x) {
@@ -94,8 +95,12 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
     }
     int k = max(p.token_budget / p.block_size, 1);
     k = min(k, min(n_i, p.max_sel));
-    const int n_cand = min(n_i - 1, p.max_blocks);
-    int need = min(k - 1, n_cand);                   // candidates to take besides the last block
+    // The blocks that hold a query token's own position, j_f .. n_i - 1, are always taken (one block,
+    // the last, for a single query token); the candidates are the blocks before them.
+    const int j_f = max(0, L - p.q_len) / p.block_size;
+    const int n_forced = min(n_i - j_f, p.max_sel);
+    const int n_cand = min(j_f, p.max_blocks);
+    int need = max(0, min(k - n_forced, n_cand));    // candidates to take besides the forced blocks
     const int E = (n_cand + NT - 1) / NT;
     const int j_lo = min(n_cand, tid * E), j_hi = min(n_cand, j_lo + E);
 
@@ -146,7 +151,7 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
         float cnt_above = 0.f;
         for_each_score([&](float v) { cnt_above += (__expf(v - mx) > p.threshold * z) ? 1.f : 0.f; });
         const int above = (int)(block_reduce(cnt_above, false) + 0.5f);
-        need = min(min(above, p.max_sel - 1), n_cand);
+        need = max(0, min(min(above, p.max_sel - n_forced), n_cand));
     }
 
     uint32_t thr = 0u;                               // key of the need-th best candidate
@@ -357,11 +362,9 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
             }
         }
     }
-    if (tid == 0) {
-        dst[need] = n_i - 1;                         // the last block is always active
-        p.block_cnt[u] = need + 1;
-    }
-    for (int e = need + 1 + tid; e < p.max_sel; e += NT) dst[e] = -1;
+    if (tid < n_forced) dst[need + tid] = n_i - n_forced + tid;      // the always-active last block(s)
+    if (tid == 0) p.block_cnt[u] = need + n_forced;
+    for (int e = need + n_forced + tid; e < p.max_sel; e += NT) dst[e] = -1;
 }
 
 template <int NT, bool SMEM>
@@ -526,10 +529,11 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
 //   3. The first CTA runs the selection on the scores in its shared memory.
 // Between the steps the cluster meets at its hardware barrier; nothing goes through global memory
 // and nobody takes tickets.  NIT = 16-byte pieces of a W_q row per lane.
-template <int NIT>
+template <int NIT, bool MULTI>
 __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const GateParams p, int per) {
     extern __shared__ __align__(16) float sc_all[];    // scores [max_blocks] (used in the first CTA), staged keys
-    __shared__ float qg[kMaxDGate];
+    __shared__ float qg[MULTI ? kMaxQLen : 1][kMaxDGate];   // gate queries of the unit's query tokens
+    const int q_len = MULTI ? p.q_len : 1;             // (a compile-time 1 for plain decoding)
     __shared__ SelectSmem sm;
     cg::cluster_group cluster = cg::this_cluster();
     const int S = (int)cluster.num_blocks(), slice = (int)cluster.block_rank();
@@ -537,15 +541,17 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = p.group * kHeadDim, chunks = n / 8, half = p.d_gate / 2;
     const int gw = slice * (kGateThreads / 32) + warp, n_gw = S * (kGateThreads / 32);
-    // W_q rows of this warp's first rotary pair: constants, requested before the wait
+    // Work items of the projection: (query token t, rotary pair c), item = t * half + c, dealt to the
+    // cluster's warps round robin.  W_q rows of this warp's first item: constants, requested before the wait.
+    const int n_items = q_len * half;
     uint4 wv[2][NIT];
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
-        const uint4* wrow = reinterpret_cast<const uint4*>(p.w_q + ((size_t)h * p.d_gate + min(gw, half - 1) + k * half) * n);
+        const uint4* wrow = reinterpret_cast<const uint4*>(p.w_q + ((size_t)h * p.d_gate + gw % half + k * half) * n);
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
             const int ch = lane + 32 * it;
-            wv[k][it] = (gw < half && ch < chunks) ? __ldg(wrow + ch) : make_uint4(0u, 0u, 0u, 0u);
+            wv[k][it] = (gw < n_items && ch < chunks) ? __ldg(wrow + ch) : make_uint4(0u, 0u, 0u, 0u);
         }
     }
     // The slice's compressed keys are asked into L2 meanwhile (a hint only; they are read after the
@@ -577,18 +583,19 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
         const int pc = k * kGateThreads + tid;
         if (pc < total) cp_async16(staged + pc, kc + pc);
     }
-    const uint4* xsrc = reinterpret_cast<const uint4*>(
-        p.q_nope + ((size_t)i * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
-    uint4 xv[NIT];
-#pragma unroll
-    for (int it = 0; it < NIT; ++it) {
-        const int ch = lane + 32 * it;
-        xv[it] = ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u);
-    }
     const int L = __ldg(p.seq_lens + i);
-    // ---- 1. gate query ------------------------------------------------------------------------
-    for (int c = gw; c < half; c += n_gw) {
-        if (c != gw) {
+    // ---- 1. gate queries --------------------------------------------------------------------------
+    for (int item = gw; item < n_items; item += n_gw) {
+        const int t = item / half, c = item - t * half;
+        const uint4* xsrc = reinterpret_cast<const uint4*>(
+            p.q_nope + (((size_t)i * q_len + t) * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
+        uint4 xv[NIT];
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int ch = lane + 32 * it;
+            xv[it] = ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        if (item != gw) {
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
                 const uint4* wrow = reinterpret_cast<const uint4*>(p.w_q + ((size_t)h * p.d_gate + c + k * half) * n);
@@ -607,11 +614,12 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
             a += __shfl_xor_sync(0xffffffffu, a, off);
             b += __shfl_xor_sync(0xffffffffu, b, off);
         }
+        // query token t sits at position L - q_len + t
         float sn, cs;
-        rope_sincos((double)(L > 0 ? L - 1 : 0), p.inv_freq[c], &sn, &cs);
+        rope_sincos((double)max(L - q_len + t, 0), p.inv_freq[c], &sn, &cs);
         const float ra = a * cs - b * sn, rb = b * cs + a * sn;
         if (lane < S) {                                // lane r stores into CTA r of the cluster
-            float* dst = cluster.map_shared_rank(qg, lane);
+            float* dst = cluster.map_shared_rank(&qg[0][0], lane) + t * kMaxDGate;
             dst[c] = ra;
             dst[c + half] = rb;
         }
@@ -627,51 +635,67 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     cluster.sync();
     GATE_STAMP(3);
     // ---- 2. scores of this slice, into the first CTA's shared memory ---------------------------
-    const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
-    const int n_cand = max(0, min(n_i - 1, p.max_blocks));
+    const int n_cand = min(max(0, L - q_len) / p.block_size, p.max_blocks);   // blocks before the query tokens' own
     float* sc0 = cluster.map_shared_rank(sc_all, 0);
     float* sc_user = p.scores_user ? p.scores_user + (size_t)u * p.max_blocks : nullptr;
-    float qsub[8];
-#pragma unroll
-    for (int c = 0; c < 8; ++c) qsub[c] = qg[8 * csub + c];
     const float inv = rsqrtf((float)p.d_gate);
-    // adds up the lanes of a key and stores its score; acc[k] belongs to piece cb + k * 512 + tid
-    auto finish_batch = [&](float (&acc)[kBatch], int cb) {
+    // A key's score is the largest of its dot products with the query tokens' gate queries; the lanes
+    // that hold a key's pieces add up by shuffles.  best[k] belongs to piece cb + k * 512 + tid.
+    auto score_batch = [&](auto&& piece, int cb) {
+        float best[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) best[k] = -INFINITY;
+        for (int t = 0; t < q_len; ++t) {
+            float qsub[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) qsub[c] = qg[t][8 * csub + c];
+            float acc[kBatch];
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) acc[k] = dot8(piece(k), qsub);
+            for (int off = lpk >> 1; off > 0; off >>= 1) {
+#pragma unroll
+                for (int k = 0; k < kBatch; ++k) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
+            }
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) best[k] = MULTI ? fmaxf(best[k], acc[k]) : acc[k];
+        }
 #pragma unroll
         for (int k = 0; k < kBatch; ++k) {
-            for (int off = lpk >> 1; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
             const int c = cb + k * kGateThreads + tid;
             const int j = j0 + c / lpk;
             if (c < total && csub == 0 && j < n_cand) {
-                const float v = acc[k] * inv;
+                const float v = best[k] * inv;
                 sc0[j] = v;
                 if (sc_user) sc_user[j] = v;
             }
         }
     };
-    {
-        // the staged batch (each thread reads back the pieces it copied itself)
+    // Batches alternate between the staged area (each thread reads back the pieces it copied itself)
+    // and the registers; while one is scored the one after the next is on its way into the place
+    // that has just been freed.
+    constexpr int kPieces = kGateThreads * kBatch;
+    for (int cb = 0;;) {
         cp_async_wait_all();
-        float acc[kBatch];
-#pragma unroll
-        for (int k = 0; k < kBatch; ++k) {
-            const int pc = k * kGateThreads + tid;
-            acc[k] = pc < total ? dot8(staged[pc], qsub) : 0.f;
-        }
-        finish_batch(acc, 0);
-    }
-    for (int cb = kGateThreads * kBatch; cb < total; cb += kGateThreads * kBatch) {
-        float acc[kBatch];
-#pragma unroll
-        for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
-        if (cb + kGateThreads * kBatch < total) {      // next batch on its way while this one reduces
+        score_batch([&](int k) { const int pc = cb + k * kGateThreads + tid; return pc < total ? staged[pc - cb] : make_uint4(0u, 0u, 0u, 0u); }, cb);
+        cb += kPieces;
+        if (cb >= total) break;
+        if (cb + kPieces < total) {
 #pragma unroll
             for (int k = 0; k < kBatch; ++k) {
-                const int c = cb + (kBatch + k) * kGateThreads + tid;
-                kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
+                const int pc = cb + kPieces + k * kGateThreads + tid;
+                if (pc < total) cp_async16(staged + (pc - cb - kPieces), kc + pc);
             }
         }
-        finish_batch(acc, cb);
+        score_batch([&](int k) { return kv[k]; }, cb);
+        cb += kPieces;
+        if (cb >= total) break;
+        if (cb + kPieces < total) {
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                const int pc = cb + kPieces + k * kGateThreads + tid;
+                kv[k] = pc < total ? __ldg(kc + pc) : make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
     }
     GATE_STAMP(4);
     cluster.sync();
@@ -685,11 +709,11 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
 constexpr int kClusterStageBytes = 8 * kGateThreads * 16;   // the staged first batch of a slice's keys
 constexpr int kClusterMaxBlocks = 8192;     // compressed keys per unit the cluster kernel holds in shared memory
 
-template <int NIT>
+template <int NIT, bool MULTI>
 cudaError_t launch_gate_cluster(const GateParams& p, int S, int per, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(gate_cluster_kernel<NIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        const cudaError_t e = cudaFuncSetAttribute(gate_cluster_kernel<NIT, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    kClusterMaxBlocks * (int)sizeof(float) + kClusterStageBytes);
         if (e != cudaSuccess) return e;
         configured = true;
@@ -708,10 +732,12 @@ cudaError_t launch_gate_cluster(const GateParams& p, int S, int per, cudaStream_
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, gate_cluster_kernel<NIT>, p, per);
+    return cudaLaunchKernelEx(&cfg, gate_cluster_kernel<NIT, MULTI>, p, per);
 }
 
 }  // namespace
+
+bool gate_one_kernel(int max_blocks) { return max_blocks <= kClusterMaxBlocks; }
 
 cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* launched) {
     const int U = p.batch * p.num_kv_heads;
@@ -727,11 +753,12 @@ cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* la
         int S = (p.max_blocks + 511) / 512;
         S = S < 1 ? 1 : (S > 8 ? 8 : S);
         const int per = (p.max_blocks + S - 1) / S;
+        const bool multi = p.q_len > 1;
         switch (nit) {
-            case 1: e = launch_gate_cluster<1>(p, S, per, stream); break;
-            case 2: e = launch_gate_cluster<2>(p, S, per, stream); break;
-            case 3: e = launch_gate_cluster<3>(p, S, per, stream); break;
-            default: e = launch_gate_cluster<4>(p, S, per, stream); break;
+            case 1: e = multi ? launch_gate_cluster<1, true>(p, S, per, stream) : launch_gate_cluster<1, false>(p, S, per, stream); break;
+            case 2: e = multi ? launch_gate_cluster<2, true>(p, S, per, stream) : launch_gate_cluster<2, false>(p, S, per, stream); break;
+            case 3: e = multi ? launch_gate_cluster<3, true>(p, S, per, stream) : launch_gate_cluster<3, false>(p, S, per, stream); break;
+            default: e = multi ? launch_gate_cluster<4, true>(p, S, per, stream) : launch_gate_cluster<4, false>(p, S, per, stream); break;
         }
         *launched = 1;
         return e;
@@ -859,6 +886,7 @@ extern "C" seer_status seer_gate_select_static(int device, const seer_shape* sha
     p.max_blocks = gate->max_blocks;
     p.max_sel = max_sel;
     p.token_budget = token_budget;
+    p.q_len = 1;
     p.status = nullptr;
     p.tickets = reinterpret_cast<int*>(base);
     for (int c = 0; c < gate->d_gate / 2; ++c)

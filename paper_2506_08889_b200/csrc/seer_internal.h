@@ -91,6 +91,7 @@ struct GateParams {
     int32_t* block_cnt;
     int batch, num_q_heads, num_kv_heads, group, block_size;
     int d_gate, max_blocks, max_sel, token_budget;
+    int q_len;                      // query tokens per sequence (1 for plain decoding); q_nope is [B,q_len,Hq,d]
     int threshold_mode;             // 0: token budget, 1: softmax probability above `threshold`
     float threshold;
     unsigned int* status;
@@ -100,6 +101,9 @@ struct GateParams {
 // Launches the scoring kernels (unless scores_in is given) and the selection kernel.
 // Returns the number of kernels launched through *launched.
 cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* launched);
+// Whether a gate over max_blocks compressed keys per unit runs as the one cluster kernel (the only
+// path that takes several query tokens).
+bool gate_one_kernel(int max_blocks);
 
 struct KcompParams {
     const __nv_bfloat16* k_nope;

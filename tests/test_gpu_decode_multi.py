@@ -144,3 +144,106 @@ def test_multi_rejects_unsupported_q_len(ctx):
     for bad in (0, 9):
         with pytest.raises(binding.SeerError):
             ctx.seer_dense_decode_multi(shape, kv, q, bad, out)
+
+
+# ---- the gate for several query tokens -------------------------------------------------------------
+
+THETA = 1.0e6
+
+
+@pytest.mark.parametrize("g,T,b,dg", [(5, 3, 64, 128), (4, 8, 64, 64), (8, 2, 128, 128), (1, 5, 64, 256)])
+def test_gate_multi_scores_and_selection(ctx, g, T, b, dg):
+    B, Hkv, d = 4, 2, 128
+    Hq = g * Hkv
+    nbmax = 700
+    # full; the T tokens straddle two blocks; exactly at a block end; shorter than T tokens
+    lens = np.array([nbmax * b, 333 * b + 2, 100 * b, 3], np.int32)
+    qn = synth.normal_bf16((B, T, Hq, d), 60 + T, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, g * d), 60 + T, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nbmax, dg), 60 + T, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    max_sel = 70
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nbmax), dtype=torch.float32, device=DEV)
+    ctx.seer_gate_select_multi(shape, gate, lens_t, qn, None, T, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    want_sc = oracle.scores_multi(bits(qn), bits(wq), bits(kc), lens, b, THETA)
+    got_sc = sc.cpu().numpy()
+    for i in range(B):
+        jf = max(0, int(lens[i]) - T) // b
+        if jf:
+            assert np.abs(got_sc[i, :, :jf] - want_sc[i, :, :jf]).max() <= 1e-3
+    # the selection is exact on the scores the GPU produced, for several budgets
+    for budget in (max_sel * b, 3 * b, b, 0):
+        ctx.seer_gate_select_multi(shape, gate, lens_t, qn, None, T, budget, idx, cnt, max_sel)
+        torch.cuda.synchronize()
+        want_idx, want_cnt = oracle.select_multi(got_sc, lens, b, budget, T, max_sel)
+        assert np.array_equal(cnt.cpu().numpy(), want_cnt), budget
+        assert np.array_equal(idx.cpu().numpy(), want_idx), budget
+    # selection only, on given scores
+    ctx.seer_gate_select_multi(shape, binding.make_gate(dg, THETA, None, None, None, nbmax), lens_t, None, sc, T, 20 * b,
+                               idx, cnt, max_sel)
+    torch.cuda.synchronize()
+    want_idx, want_cnt = oracle.select_multi(got_sc, lens, b, 20 * b, T, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx) and np.array_equal(cnt.cpu().numpy(), want_cnt)
+    assert ctx.device_status() == binding.SEER_OK
+
+
+def test_gate_multi_with_one_token_is_bitwise_the_single_token_gate(ctx):
+    B, Hq, Hkv, d, dg, b, nbmax = 3, 40, 8, 128, 128, 64, 2048
+    lens = np.array([nbmax * b, 1000 * b + 17, 64], np.int32)
+    qn = synth.normal_bf16((B, 1, Hq, d), 70, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, 5 * d), 70, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nbmax, dg), 70, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    res = []
+    for multi in (False, True):
+        idx = torch.zeros((B, Hkv, 205), dtype=torch.int32, device=DEV)
+        cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+        sc = torch.zeros((B, Hkv, nbmax), dtype=torch.float32, device=DEV)
+        if multi:
+            ctx.seer_gate_select_multi(shape, gate, lens_t, qn, None, 1, 205 * b, idx, cnt, 205, scores_out=sc)
+        else:
+            ctx.seer_gate_select(shape, gate, lens_t, qn[:, 0].contiguous(), None, 205 * b, idx, cnt, 205, scores_out=sc)
+        torch.cuda.synchronize()
+        res.append((idx, cnt, sc))
+    for a, c in zip(res[0], res[1]):
+        assert torch.equal(a, c)
+
+
+def test_multi_token_step_gate_then_decode(ctx):
+    # three query tokens per sequence through the gate and the decode kernel, 14B head counts
+    B, T, Hq, Hkv, d, dg, b, L = 2, 3, 40, 8, 128, 128, 64, 16384
+    nb = L // b
+    lens = np.array([L, L - 1000], np.int32)
+    q, k, v = _make(B, T, Hq, Hkv, L, 90)
+    qn = synth.normal_bf16((B, T, Hq, d), 90, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, 5 * d), 90, "wq", DEV, std=0.02)
+    wk = synth.normal_bf16((Hkv, dg, 3 * d), 90, "wk", DEV, std=0.02)
+    kc = torch.zeros((B, Hkv, nb, dg), dtype=torch.bfloat16, device=DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    gate = binding.make_gate(dg, THETA, wq, wk, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    ctx.seer_kcomp_append(shape, gate, lens_t, k, first_block=0, num_blocks=nb)
+    max_sel = 26                                                  # s = 0.9
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nb), dtype=torch.float32, device=DEV)
+    ctx.seer_gate_select_multi(shape, gate, lens_t, qn, None, T, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+    kv = binding.make_kv(k, v, lens_t)
+    out = torch.full((B, T, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, T, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    ctx.seer_sparse_decode_multi(shape, kv, q, T, idx, cnt, max_sel, out, lse)
+    torch.cuda.synchronize()
+    want_idx, want_cnt = oracle.select_multi(sc.cpu().numpy(), lens, b, max_sel * b, T, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx) and np.array_equal(cnt.cpu().numpy(), want_cnt)
+    ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, want_idx, want_cnt, b, 0.0884)
+    check_attention(out, lse, *ref, what="multi step", strict=True)
+    # every query token sees at least itself: its own block is in the list
+    assert np.isfinite(ref[1]).all()
+    assert ctx.device_status() == binding.SEER_OK

@@ -362,7 +362,11 @@ def run_ours(args):
                          "algorithmic_bytes_per_launch": decode_bytes, "us_per_launch": round(sparse_ms * 1e3, 2),
                          "traffic": (int(NCU_READ_BYTES_PER_2_SEQUENCES * B / 2 * (1.0 - args.sparsity) / 0.1
                                          + NCU_WRITE_BYTES_PER_LAUNCH) if abs(args.sparsity - 0.9) < 1e-9 else None),
-                         "traffic_note": "ncu capture at batch 2, scaled by the units processed"},
+                         "traffic_note": "ncu capture at batch 2, scaled by the units processed",
+                         # the same kernel launched back to back (no event between launches, so that each
+                         # launch's set-up overlaps its predecessor's tail as it does inside the step)
+                         "us_per_launch_back_to_back": round(sparse_b2b_ms * 1e3, 2),
+                         "frac_back_to_back": round(decode_bytes / (sparse_b2b_ms * 1e-3) / 1e9 / peak, 4)},
             "extra": {
                 "tokens_per_s_per_layer": round(world * B / (step_ms * 1e-3), 1),
                 "selected_kv_bytes_per_step": sel_kv_bytes,

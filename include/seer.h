@@ -258,6 +258,9 @@ seer_status seer_gate_select_threshold(seer_ctx* ctx, const seer_shape* shape, c
  *  first_block == -1: per sequence, write the block that has just filled,
  *          j = L_i/b - 1, if L_i % b == 0 and L_i > 0; otherwise nothing
  *          (num_blocks is ignored) -- the once-per-b-tokens update of decoding.
+ *  first_block == -t, 2 <= t <= 8: the same after t tokens were appended at once
+ *          (multi-token decoding): block j = floor(L_i/b) - 1 is written if its last
+ *          row is among the t newest tokens, i.e. L_i >= b and L_i % b < t.
  */
 seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
                               const int32_t* seq_lens, const void* k_nope,
@@ -282,6 +285,19 @@ seer_status seer_decode_step(seer_ctx* ctx, const seer_shape* shape, const seer_
                              int k_nope_rows_block_local, int token_budget,
                              int32_t* block_idx, int32_t* block_cnt, int max_sel,
                              void* out, float* lse, void* stream);
+
+/*
+ * The same step for q_len query tokens per sequence (1 <= q_len <= 8; the sequences have just grown
+ * by q_len tokens): seer_kcomp_append(.., first_block = -q_len) ; seer_gate_select_multi ;
+ * seer_sparse_decode_multi, on `stream`.  q, q_nope: [B,q_len,Hq,d]; out: [B,q_len,Hq,d];
+ * lse: [B,q_len,Hq] or NULL.  Other arguments as in seer_decode_step.
+ */
+seer_status seer_decode_step_multi(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const seer_gate* gate,
+                                   const void* q, const void* q_nope, int q_len, const void* k_nope,
+                                   int64_t k_nope_stride_batch, int64_t k_nope_stride_head,
+                                   int64_t k_nope_stride_token, int k_nope_rows_block_local, int token_budget,
+                                   int32_t* block_idx, int32_t* block_cnt, int max_sel, void* out, float* lse,
+                                   void* stream);
 
 /*
  * seer_gate_select without a context and without any allocation.  (The paper has no counterpart:

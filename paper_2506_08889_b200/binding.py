@@ -31,7 +31,7 @@ EXPORTS = [
     "seer_get_device_status", "seer_workspace_bytes", "seer_launch_count",
     "seer_dense_decode", "seer_sparse_decode", "seer_gate_select", "seer_kcomp_append",
     "seer_gate_select_static", "seer_decode_step", "seer_gate_select_threshold",
-    "seer_sparse_decode_multi", "seer_dense_decode_multi", "seer_gate_select_multi",
+    "seer_sparse_decode_multi", "seer_dense_decode_multi", "seer_gate_select_multi", "seer_decode_step_multi",
 ]
 
 
@@ -111,6 +111,9 @@ def lib() -> ctypes.CDLL:
     L.seer_gate_select_threshold.restype = i32
     L.seer_gate_select_threshold.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, vp,
                                              ctypes.c_float, vp, vp, i32, vp, vp]
+    L.seer_decode_step_multi.restype = i32
+    L.seer_decode_step_multi.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), ctypes.POINTER(SeerGate),
+                                         vp, vp, i32, vp, i64, i64, i64, i32, i32, vp, vp, i32, vp, vp, vp]
     L.seer_decode_step.restype = i32
     L.seer_decode_step.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), ctypes.POINTER(SeerGate),
                                    vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, i32, vp, vp, vp]
@@ -260,6 +263,21 @@ class Context:
                                            _ptr(q), _ptr(q_nope), _ptr(k_nope), sb, sh, st,
                                            int(bool(rows_block_local)), int(token_budget), _ptr(block_idx),
                                            _ptr(block_cnt), int(max_sel), _ptr(out), _ptr(lse), _stream(stream)))
+
+
+    def seer_decode_step_multi(self, shape: SeerShape, kv: SeerKV, gate: SeerGate, q, q_nope, q_len, k_nope,
+                               token_budget, block_idx, block_cnt, max_sel, out, lse=None, rows_block_local=False,
+                               stream=None):
+        """The step for q_len query tokens per sequence (q, q_nope, out: [B,q_len,Hq,d])."""
+        sb = sh = st = 0
+        if k_nope is not None:
+            assert k_nope.dtype == torch.bfloat16 and k_nope.stride(3) == 1
+            sb, sh, st = k_nope.stride(0), k_nope.stride(1), k_nope.stride(2)
+        self._check(lib().seer_decode_step_multi(self._h, ctypes.byref(shape), ctypes.byref(kv), ctypes.byref(gate),
+                                                 _ptr(q), _ptr(q_nope), int(q_len), _ptr(k_nope), sb, sh, st,
+                                                 int(bool(rows_block_local)), int(token_budget), _ptr(block_idx),
+                                                 _ptr(block_cnt), int(max_sel), _ptr(out), _ptr(lse),
+                                                 _stream(stream)))
 
 
 STATIC_SCRATCH_BYTES = 1 << 20

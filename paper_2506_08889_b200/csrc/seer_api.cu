@@ -496,7 +496,7 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
     if (stride_batch % 8 || stride_head % 8 || stride_token % 8 || stride_token < kHeadDim || stride_batch < 0 ||
         stride_head < 0)
         return fail(ctx, SEER_ERR_INVALID_ARG, "k_nope strides must be multiples of 8 elements");
-    if (first_block < -1) return fail(ctx, SEER_ERR_INVALID_ARG, "first_block must be >= -1");
+    if (first_block < -8) return fail(ctx, SEER_ERR_INVALID_ARG, "first_block must be >= -8");
     if (first_block >= 0 && num_blocks < 0) return fail(ctx, SEER_ERR_INVALID_ARG, "num_blocks is negative");
     if (first_block >= 0 && rows_block_local && num_blocks > 1)
         return fail(ctx, SEER_ERR_INVALID_ARG, "a block-local buffer holds one block only");
@@ -545,6 +545,26 @@ seer_status seer_decode_step(seer_ctx* ctx, const seer_shape* shape, const seer_
                           nullptr, stream);
     if (st != SEER_OK) return st;
     return seer_sparse_decode(ctx, shape, kv, q, block_idx, block_cnt, max_sel, out, lse, stream);
+}
+
+seer_status seer_decode_step_multi(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const seer_gate* gate,
+                                   const void* q, const void* q_nope, int q_len, const void* k_nope,
+                                   int64_t k_nope_stride_batch, int64_t k_nope_stride_head, int64_t k_nope_stride_token,
+                                   int k_nope_rows_block_local, int token_budget, int32_t* block_idx,
+                                   int32_t* block_cnt, int max_sel, void* out, float* lse, void* stream) {
+    if (!ctx) return SEER_ERR_INVALID_ARG;
+    if (!kv || !kv->seq_lens) return fail(ctx, SEER_ERR_INVALID_ARG, "kv or kv->seq_lens is NULL");
+    if (q_len < 1 || q_len > 8) return fail(ctx, SEER_ERR_UNSUPPORTED, "q_len %d (supported 1..8)", q_len);
+    seer_status st;
+    if (k_nope) {
+        st = seer_kcomp_append(ctx, shape, gate, kv->seq_lens, k_nope, k_nope_stride_batch, k_nope_stride_head,
+                               k_nope_stride_token, k_nope_rows_block_local, -q_len, 1, stream);
+        if (st != SEER_OK) return st;
+    }
+    st = seer_gate_select_multi(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, q_len, token_budget, block_idx, block_cnt,
+                                max_sel, nullptr, stream);
+    if (st != SEER_OK) return st;
+    return seer_sparse_decode_multi(ctx, shape, kv, q, q_len, block_idx, block_cnt, max_sel, out, lse, stream);
 }
 
 }  // extern "C"

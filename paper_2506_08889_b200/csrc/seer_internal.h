@@ -112,7 +112,7 @@ struct KcompParams {
     const int32_t* seq_lens;
     int64_t stride_batch, stride_head, stride_token;
     int rows_block_local;
-    int first_block, num_blocks;    // first_block == -1: the block that just filled
+    int first_block, num_blocks;    // first_block == -t (1..8): the block that filled while the last t tokens were appended
     int batch, num_kv_heads, block_size, d_gate, max_blocks;
     double inv_freq[kMaxDGate / 2];
 };

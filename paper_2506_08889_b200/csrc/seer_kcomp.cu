@@ -50,8 +50,9 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
     int nb = 0;                                       // blocks this CTA really handles
     int j_first;
     if (p.first_block < 0) {
+        // the sequence has just grown by -first_block tokens: the block whose last row is among them
         j_first = complete - 1;
-        nb = (blockIdx.x == 0 && L > 0 && L % b == 0 && j_first < p.max_blocks) ? 1 : 0;
+        nb = (blockIdx.x == 0 && complete > 0 && L % b < -p.first_block && j_first < p.max_blocks) ? 1 : 0;
     } else {
         j_first = p.first_block + blockIdx.x * NB;
         const int j_end = min(min(p.first_block + p.num_blocks, complete), p.max_blocks);

@@ -247,3 +247,52 @@ def test_multi_token_step_gate_then_decode(ctx):
     # every query token sees at least itself: its own block is in the list
     assert np.isfinite(ref[1]).all()
     assert ctx.device_status() == binding.SEER_OK
+
+
+def test_multi_token_step_call_appends_the_block_that_filled_among_the_new_tokens(ctx):
+    # q_len = 4 tokens have just been appended; lengths: a block boundary crossed two tokens ago
+    # (L % b = 2 < 4: block L/b - 1 is written), exactly at a boundary, and no boundary crossed
+    B, T, Hq, Hkv, d, dg, b, S = 3, 4, 32, 8, 128, 128, 64, 4096
+    nb = S // b
+    lens = np.array([40 * b + 2, 64 * b, 50 * b + 9], np.int32)
+    q, k, v = _make(B, T, Hq, Hkv, S, 95)
+    qn = synth.normal_bf16((B, T, Hq, d), 95, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, 4 * d), 95, "wq", DEV, std=0.02)
+    wk = synth.normal_bf16((Hkv, dg, 3 * d), 95, "wk", DEV, std=0.02)
+    kc = torch.zeros((B, Hkv, nb, dg), dtype=torch.bfloat16, device=DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    gate = binding.make_gate(dg, THETA, wq, wk, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    # the cache as it stood before these T tokens: every block complete by then
+    before = torch.as_tensor(lens - T, device=DEV)
+    ctx.seer_kcomp_append(shape, gate, before, k, first_block=0, num_blocks=nb)
+    torch.cuda.synchronize()
+    kc_before = kc.clone()
+    kv = binding.make_kv(k, v, lens_t)
+    max_sel = 8
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    out = torch.full((B, T, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, T, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    ctx.seer_decode_step_multi(shape, kv, gate, q, qn, T, k, max_sel * b, idx, cnt, max_sel, out, lse)
+    torch.cuda.synchronize()
+    # compressed keys: sequences 0 and 1 got the entry of the block that filled, sequence 2 nothing
+    _, want = oracle.kcomp(bits(k), bits(wk), b, 0, nb, nb, THETA)
+    got = synth.bits_to_bf16(bits(kc)).to(torch.float64).numpy()
+    for i, j in ((0, 39), (1, 63)):
+        assert (kc_before[i, :, j] == 0).all()
+        tol = np.abs(want[i, :, j]) * 2.0 ** -7 + 1e-5 * np.abs(want).max()
+        assert (np.abs(got[i, :, j] - want[i, :, j]) <= tol).all()
+    changed = (kc != kc_before).any(dim=3).cpu().numpy()
+    assert changed[0, :, 39].all() and changed[1, :, 63].all() and changed.sum() == 2 * Hkv
+    # the lists and the attention are what the separate calls give on the updated cache
+    sc = torch.zeros((B, Hkv, nb), dtype=torch.float32, device=DEV)
+    idx2, cnt2 = torch.zeros_like(idx), torch.zeros_like(cnt)
+    ctx.seer_gate_select_multi(shape, gate, lens_t, qn, None, T, max_sel * b, idx2, cnt2, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    assert torch.equal(idx, idx2) and torch.equal(cnt, cnt2)
+    want_idx, want_cnt = oracle.select_multi(sc.cpu().numpy(), lens, b, max_sel * b, T, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx) and np.array_equal(cnt.cpu().numpy(), want_cnt)
+    ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, want_idx, want_cnt, b, 0.0884)
+    check_attention(out, lse, *ref, what="multi step call")
+    assert ctx.device_status() == binding.SEER_OK

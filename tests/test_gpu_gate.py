@@ -125,6 +125,49 @@ def test_gate_scores_and_selection(ctx, g, b):
     assert torch.equal(idx, idx2) and torch.equal(cnt, cnt2)
 
 
+@pytest.mark.parametrize("nbmax,dg,g", [(6000, 128, 2), (8192, 256, 1), (5000, 64, 4)])
+def test_gate_largest_clusters_several_key_batches_per_cta(ctx, nbmax, dg, g):
+    # 4097..8192 compressed keys per unit: clusters of 8 CTAs, three or more key batches per CTA
+    # (staged, registers, staged again ...), candidates of the selection read from shared memory
+    B, Hkv, d, b = 2, 2, 128, 64
+    Hq = g * Hkv
+    lens = np.array([nbmax * b, (nbmax - 700) * b + 5], np.int32)
+    qn = synth.normal_bf16((B, Hq, d), 19, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, g * d), 19, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nbmax, dg), 19, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    max_sel = 600
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nbmax), dtype=torch.float32, device=DEV)
+    before = ctx.launch_count()
+    ctx.seer_gate_select(shape, gate, lens_t, qn, None, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    assert ctx.launch_count() - before == 1
+    n = [-(-int(L) // b) for L in lens]
+    want_sc, _ = oracle.scores(bits(qn), bits(wq), bits(kc), [x - 1 for x in n], [int(L) - 1 for L in lens], THETA)
+    got_sc = sc.cpu().numpy()
+    for i in range(B):
+        assert np.abs(got_sc[i, :, :n[i] - 1] - want_sc[i, :, :n[i] - 1]).max() <= 1e-3
+    want_idx, want_cnt = oracle.select(got_sc, lens, b, max_sel * b, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx) and np.array_equal(cnt.cpu().numpy(), want_cnt)
+    # several query tokens on the same size
+    T = 3
+    qn3 = synth.normal_bf16((B, T, Hq, d), 19, "qn3", DEV)
+    ctx.seer_gate_select_multi(shape, gate, lens_t, qn3, None, T, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    got_sc = sc.cpu().numpy()
+    want_sc = oracle.scores_multi(bits(qn3), bits(wq), bits(kc), lens, b, THETA)
+    for i in range(B):
+        jf = (int(lens[i]) - T) // b
+        assert np.abs(got_sc[i, :, :jf] - want_sc[i, :, :jf]).max() <= 1e-3
+    want_idx, want_cnt = oracle.select_multi(got_sc, lens, b, max_sel * b, T, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx) and np.array_equal(cnt.cpu().numpy(), want_cnt)
+    assert ctx.device_status() == binding.SEER_OK
+
+
 def test_gate_more_keys_than_one_cluster_holds(ctx):
     # above 8192 compressed keys per unit the gate runs as projection + score/selection kernels
     B, Hkv, g, d, dg, b = 1, 2, 2, 128, 64, 64

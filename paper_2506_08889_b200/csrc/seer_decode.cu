@@ -1085,16 +1085,17 @@ cudaError_t configure() {
 
 template <bool SPARSE, bool PAGED, int NT>
 int occupancy() {
-    static int cached = -1;
-    if (cached < 0) {
+    static int cached[kMaxDevices] = {};             // 0: not asked yet on that device
+    const int slot = current_device_slot();
+    if (cached[slot] <= 0) {
         if (configure<SPARSE, PAGED, NT>() != cudaSuccess) return 0;
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<SPARSE, PAGED, NT>, kThreads,
                                                           decode_smem_bytes()) != cudaSuccess)
             return 0;
-        cached = n;
+        cached[slot] = n;
     }
-    return cached;
+    return cached[slot];
 }
 
 template <bool SPARSE, bool PAGED, int NT>

@@ -711,12 +711,13 @@ constexpr int kClusterMaxBlocks = 8192;     // compressed keys per unit the clus
 
 template <int NIT, bool MULTI>
 cudaError_t launch_gate_cluster(const GateParams& p, int S, int per, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {};
+    const int slot = current_device_slot();
+    if (!configured[slot]) {
         const cudaError_t e = cudaFuncSetAttribute(gate_cluster_kernel<NIT, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    kClusterMaxBlocks * (int)sizeof(float) + kClusterStageBytes);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[slot] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S, p.batch * p.num_kv_heads);
@@ -799,7 +800,7 @@ namespace {
 // One copy per GPU that loads the library, held until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[SEER_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
+using seer::kMaxDevices;
 std::mutex g_static_mutex;
 unsigned char* g_static_ptr[kMaxDevices];     // device address of g_static_scratch, per device
 

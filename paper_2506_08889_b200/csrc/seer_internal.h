@@ -14,6 +14,16 @@ constexpr int kMaxGroup = 8;        // query heads per KV head handled by one MM
 constexpr int kMaxDGate = 256;      // gate width: 64, 128 or 256
 constexpr int kMaxRounds = 12;      // halving rounds of the decode kernels' dynamic tile pool
 
+// Kernel attributes (the opt-in to more dynamic shared memory) are per device: index of the current
+// device into per-device "already configured" tables (processes here use one GPU, the library does
+// not assume it).
+constexpr int kMaxDevices = 64;
+inline int current_device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
+    return dev % kMaxDevices;
+}
+
 // Launch with the programmatic-stream-serialisation attribute (see pdl_wait in seer_device.cuh).
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,

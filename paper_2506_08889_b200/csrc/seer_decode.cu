@@ -749,14 +749,18 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 // a row that has seen nothing so far keeps max = -inf; exponents are then taken against 0
                 const float mb0 = mn0 == -INFINITY ? 0.f : mn0, mb1 = mn1 == -INFINITY ? 0.f : mn1;
                 const float al0 = fast_exp2(m_run[nt][0] - mb0), al1 = fast_exp2(m_run[nt][1] - mb1);
+                // the running maxima rarely move after a piece's first tiles: then nothing is rescaled
+                const bool same_max = __all_sync(0xffffffffu, m_run[nt][0] == mn0 && m_run[nt][1] == mn1);
                 m_run[nt][0] = mn0; m_run[nt][1] = mn1;
                 const float p0 = fast_exp2(s[0] - mb0), p1 = fast_exp2(s[1] - mb1);
                 const float p2 = fast_exp2(s[2] - mb0), p3 = fast_exp2(s[3] - mb1);
                 l_run[nt][0] = l_run[nt][0] * al0 + (p0 + p2);
                 l_run[nt][1] = l_run[nt][1] * al1 + (p1 + p3);
+                if (!same_max) {
 #pragma unroll
-                for (int a = 0; a < 8; ++a) {
-                    o[nt][a][0] *= al0; o[nt][a][1] *= al1; o[nt][a][2] *= al0; o[nt][a][3] *= al1;
+                    for (int a = 0; a < 8; ++a) {
+                        o[nt][a][0] *= al0; o[nt][a][1] *= al1; o[nt][a][2] *= al0; o[nt][a][3] *= al1;
+                    }
                 }
                 pb[nt][0] = movmatrix_trans(pack_bf16x2(p0, p1));   // tokens 0-7 of the slice
                 pb[nt][1] = movmatrix_trans(pack_bf16x2(p2, p3));   // tokens 8-15

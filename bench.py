@@ -686,7 +686,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="kernel-only sparsity sweep instead of the step benchmark")
     ap.add_argument("--grid", action="store_true", help="the paper's 64/8-head kernel grid (seq len x batch x sparsity)")
     ap.add_argument("--multi", action="store_true", help="multi-query-token decode: q_len 1..8, kernel-only")
-    ap.add_argument("--block-size", type=int, default=64, help="block size for --grid (64 or 128)")
+    ap.add_argument("--block-size", type=int, default=64, help="block size for --grid (16, 32, 64 or 128)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()

@@ -20,8 +20,10 @@
  *  - A context serialises its calls through its workspace: calls that share a
  *    context must be ordered on one stream (or by events).  Use one context
  *    per concurrent stream.
- *  - Supported: head_dim 128; block_size 64 or 128; group size
- *    num_q_heads / num_kv_heads in 1..8; bf16 inputs, fp32 accumulation.
+ *  - Supported: head_dim 128; block_size 16, 32, 64 or 128 (the range of the
+ *    paper's block-size study, Sec. 5 "Block Size for Sparse Attention"; 64 is
+ *    its default); group size num_q_heads / num_kv_heads in 1..8; bf16 inputs,
+ *    fp32 accumulation.
  *
  * Notation: B batch, Hq query heads, Hkv KV heads, g = Hq / Hkv, d head_dim,
  * b block_size, L_i KV length of sequence i INCLUDING the token being decoded,
@@ -55,7 +57,7 @@ typedef struct {
     int num_q_heads;    /* Hq */
     int num_kv_heads;   /* Hkv, divides Hq */
     int head_dim;       /* d = 128 */
-    int block_size;     /* b = 64 or 128 (sparsity block of the gate, Sec. 2.2 / 3.1) */
+    int block_size;     /* b = 16, 32, 64 or 128 (sparsity block of the gate, Sec. 2.2 / 3.1) */
     float sm_scale;     /* softmax scale applied to <q,k>, e.g. 1/sqrt(d) */
 } seer_shape;
 

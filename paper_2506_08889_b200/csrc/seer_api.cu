@@ -26,6 +26,7 @@ struct MapKey {
     const void* base;
     uint64_t dims[4];
     uint64_t strides[3];
+    uint64_t box_rows;
     bool operator==(const MapKey& o) const { return memcmp(this, &o, sizeof(MapKey)) == 0; }
 };
 
@@ -107,8 +108,8 @@ seer_status check_shape(seer_ctx* ctx, const seer_shape* s) {
     if (s->batch <= 0 || s->num_q_heads <= 0 || s->num_kv_heads <= 0)
         return fail(ctx, SEER_ERR_INVALID_ARG, "batch/head counts must be positive");
     if (s->head_dim != kHeadDim) return fail(ctx, SEER_ERR_UNSUPPORTED, "head_dim %d (only 128)", s->head_dim);
-    if (s->block_size != 64 && s->block_size != 128)
-        return fail(ctx, SEER_ERR_UNSUPPORTED, "block_size %d (only 64 or 128)", s->block_size);
+    if (s->block_size != 16 && s->block_size != 32 && s->block_size != 64 && s->block_size != 128)
+        return fail(ctx, SEER_ERR_UNSUPPORTED, "block_size %d (only 16, 32, 64 or 128)", s->block_size);
     if (s->num_q_heads % s->num_kv_heads != 0)
         return fail(ctx, SEER_ERR_INVALID_ARG, "num_q_heads %d not a multiple of num_kv_heads %d",
                     s->num_q_heads, s->num_kv_heads);
@@ -127,12 +128,13 @@ void fill_inv_freq(double* dst, int d_gate, float theta) {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 seer_status get_map(seer_ctx* ctx, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
-                    const CUtensorMap** out) {
+                    int box_rows, const CUtensorMap** out) {
     MapKey key;
     memset(&key, 0, sizeof key);
     key.base = base;
     for (int a = 0; a < 4; ++a) key.dims[a] = dims[a];
     for (int a = 0; a < 3; ++a) key.strides[a] = strides_bytes[a];
+    key.box_rows = (uint64_t)box_rows;
     for (int a = 0; a < ctx->map_used; ++a)
         if (ctx->map_keys[a] == key) { *out = &ctx->maps[a]; return SEER_OK; }
     int slot;
@@ -140,7 +142,7 @@ seer_status get_map(seer_ctx* ctx, const void* base, const uint64_t dims[4], con
     else { slot = ctx->map_next; ctx->map_next = (ctx->map_next + 1) % kMapCache; }
     cuuint64_t gd[4] = {dims[0], dims[1], dims[2], dims[3]};
     cuuint64_t gs[3] = {strides_bytes[0], strides_bytes[1], strides_bytes[2]};
-    cuuint32_t box[4] = {64, (cuuint32_t)kTileTokens, 1, 1};       // 64 channels (128 B) x 64 tokens
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};          // 64 channels (128 B) x 64 tokens (or one small block)
     cuuint32_t es[4] = {1, 1, 1, 1};
     CUresult r = ctx->encode(&ctx->maps[slot], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gd, gs,
                              box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -183,7 +185,9 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
         if (max_sel <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_sel must be positive");
     }
     const int U = shape->batch * shape->num_kv_heads;
-    const int tpb = shape->block_size / kTileTokens;
+    // blocks of 64 or 128 tokens are one or two tiles; blocks of 16 or 32 tokens are gathered 4 or 2 to a tile
+    const int bpt = shape->block_size < kTileTokens ? kTileTokens / shape->block_size : 1;
+    const int tpb = bpt > 1 ? 1 : shape->block_size / kTileTokens;
 
     cudaError_t ce = cudaSetDevice(ctx->device);
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
@@ -194,7 +198,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     const int n_tiles = tok_per_launch * group > 8 ? 2 : 1;
     const int per_sm = decode_ctas_per_sm(sparse, paged, n_tiles);
     if (per_sm <= 0) return fail(ctx, SEER_ERR_CUDA, "decode kernel cannot be resident (shared memory)");
-    long long max_tiles = sparse ? (long long)U * max_sel * tpb
+    long long max_tiles = sparse ? (long long)U * ((max_sel + bpt - 1) / bpt) * tpb
                                  : (long long)U * ((kv->max_seq_len + kTileTokens - 1) / kTileTokens);
     int grid = ctx->num_sms * per_sm;
     if (grid > kMaxGridCtas) grid = kMaxGridCtas;
@@ -211,10 +215,11 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     const uint64_t strides[3] = {(uint64_t)kv->stride_token * 2, (uint64_t)kv->stride_head * 2,
                                  (uint64_t)kv->stride_batch * 2};
     const CUtensorMap *mk, *mv;
-    st = get_map(ctx, kv->k, dims, strides, &mk);
+    const int box_rows = sparse && bpt > 1 ? shape->block_size : kTileTokens;
+    st = get_map(ctx, kv->k, dims, strides, box_rows, &mk);
     if (st != SEER_OK) return st;
     const CUtensorMap mk_copy = *mk;       // the second lookup may evict the first
-    st = get_map(ctx, kv->v, dims, strides, &mv);
+    st = get_map(ctx, kv->v, dims, strides, box_rows, &mv);
     if (st != SEER_OK) return st;
 
     DecodeParams p;
@@ -237,6 +242,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.q_len = q_len;
     p.block_size = shape->block_size;
     p.tiles_per_block = tpb;
+    p.blocks_per_tile = bpt;
     p.num_units = U;
     p.max_blocks_cap = (kv->max_seq_len + kTileTokens - 1) / kTileTokens;
     p.pool_div = ctx->pool_div;

@@ -52,7 +52,8 @@ constexpr int kMinChunk = 2;                               // smallest dynamic c
 constexpr int kMinStaticTilesPerCta = 8;                   // below this everything is static
 
 struct StageMeta {
-    int nvalid;        // cached tokens from the tile's first row on, capped at 64 + 7 (0 = nothing was loaded); -1 = end of stream
+    int nvalid;        // cached tokens from the tile's first row on, capped at 64 + 7 (0 = nothing was loaded); -1 = end of
+                       // stream.  Blocks of 16 or 32 tokens: one such count per gathered block, 8 bits each (capped at b + 7)
     int unit;          // (sequence, KV head) index
     int flags;         // bit 0: first tile of a piece
     int unit_first;    // global index of the unit's first tile
@@ -109,13 +110,13 @@ __device__ __forceinline__ void trace_stamp(const DecodeParams& p, int slot) {
 #define SEER_STAMP(slot) ((void)0)
 #endif
 
-template <bool SPARSE>
+template <bool SPARSE, bool SMALL = false>
 __device__ __forceinline__ int tiles_of(const DecodeParams& p, int u) {
     const int L = p.seq_lens[u / p.num_kv_heads];
     if (SPARSE) {
         int c = p.block_cnt ? p.block_cnt[u] : p.max_sel;     // not behind the test on L: both loads in flight
         c = max(0, min(c, p.max_sel));
-        return L <= 0 ? 0 : c * p.tiles_per_block;
+        return L <= 0 ? 0 : (SMALL ? (c + p.blocks_per_tile - 1) / p.blocks_per_tile : c * p.tiles_per_block);
     } else {
         if (L <= 0) return 0;
         int t = (L + kTileTokens - 1) / kTileTokens;
@@ -312,7 +313,7 @@ __device__ __forceinline__ int scan_valid_slots(const DecodeParams& p, int first
     return n;
 }
 
-template <bool SPARSE, bool PAGED, int NT>
+template <bool SPARSE, bool PAGED, int NT, bool SMALL>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const DecodeParams p) {
@@ -355,7 +356,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         const int u_lo = min(U, lane * per), u_hi = min(U, u_lo + per);
         int mine = 0;
         for (int u = u_lo; u < u_hi; ++u) {
-            const int t = tiles_of<SPARSE>(p, u);
+            const int t = tiles_of<SPARSE, SMALL>(p, u);
             if (t == 0 && cta == 0) write_zero_unit(p, u);   // units without work: zeros, -inf
             mine += t;
         }
@@ -377,7 +378,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         {
             int acc = incl - mine;
             for (int u = u_lo; u < u_hi; ++u) {
-                const int t = tiles_of<SPARSE>(p, u);
+                const int t = tiles_of<SPARSE, SMALL>(p, u);
                 if (sc.R > 0) p.prefix[u] = acc;
                 if (t_begin < t_end && t > 0 && acc <= t_begin && t_begin < acc + t) {
                     my_start_u = u;
@@ -397,7 +398,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 const int src = __ffs(m) - 1;
                 cu = __shfl_sync(0xffffffffu, my_start_u, src);
                 cpu = t_begin - __shfl_sync(0xffffffffu, my_start_off, src);
-                cut = tiles_of<SPARSE>(p, cu);
+                cut = tiles_of<SPARSE, SMALL>(p, cu);
             } else {
                 t_end = t_begin;                         // (no static share)
             }
@@ -490,7 +491,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                         ++cu;
                         ce = 0;
                         if (cu >= U) { cut = 0; break; }
-                        cut = tiles_of<SPARSE>(p, cu);
+                        cut = tiles_of<SPARSE, SMALL>(p, cu);
                         continue;
                     }
                     int take = min(avail, n_chunk - base);
@@ -500,38 +501,72 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     base += take;
                     ce += take;
                 }
-                // per-lane tile descriptor
-                int nvalid = 0, row = 0, outer = 0, head = 0, flags = 0;
+                // per-lane tile descriptor (row/outer: TMA coordinates of the tile, or of each gathered block)
+                const int bpt = SMALL ? p.blocks_per_tile : 1;           // (a compile-time 1 for blocks of 64 or 128 tokens)
+                int nvalid = 0, head = 0, flags = 0;
+                int row[4] = {0, 0, 0, 0}, outer[4] = {0, 0, 0, 0};
                 if (my_u >= 0) {
                     const int i = my_u / p.num_kv_heads;
                     head = my_u % p.num_kv_heads;
                     const int L = p.seq_lens[i];
-                    int tok0 = 0;
-                    if (SPARSE) {
-                        const int blk = p.block_idx[(size_t)my_u * p.max_sel + my_e / p.tiles_per_block];
+                    if (SMALL) {
+                        // a tile gathers the next bpt listed blocks of the unit
                         const int n_i = (L + p.block_size - 1) / p.block_size;
-                        if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
-                        if (blk >= 0 && blk < n_i) {
-                            tok0 = blk * p.block_size + (my_e % p.tiles_per_block) * kTileTokens;
+                        int cnt_u = p.block_cnt ? p.block_cnt[my_u] : p.max_sel;
+                        cnt_u = max(0, min(cnt_u, p.max_sel));
+#pragma unroll
+                        for (int sb = 0; sb < 4; ++sb) {
+                            const int e = my_e * bpt + sb;
+                            if (sb < bpt && e < cnt_u) {
+                                const int blk = p.block_idx[(size_t)my_u * p.max_sel + e];
+                                if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
+                                if (blk >= 0 && blk < n_i) {
+                                    const int tok0 = blk * p.block_size;
+                                    int nv = max(0, min(p.block_size + 7, L - tok0));
+                                    if (PAGED && nv > 0) {
+                                        const int pg = p.page_table[(size_t)i * p.page_table_stride + tok0 / p.page_size];
+                                        if (pg < 0 || pg >= p.num_pages) {
+                                            raise_status(p.status, DEV_BAD_INDEX);
+                                            nv = 0;
+                                        }
+                                        outer[sb] = pg;
+                                        row[sb] = tok0 % p.page_size;
+                                    } else {
+                                        outer[sb] = i;
+                                        row[sb] = tok0;
+                                    }
+                                    nvalid |= nv << (8 * sb);
+                                }
+                            }
+                        }
+                    } else {
+                        int tok0 = 0;
+                        if (SPARSE) {
+                            const int blk = p.block_idx[(size_t)my_u * p.max_sel + my_e / p.tiles_per_block];
+                            const int n_i = (L + p.block_size - 1) / p.block_size;
+                            if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
+                            if (blk >= 0 && blk < n_i) {
+                                tok0 = blk * p.block_size + (my_e % p.tiles_per_block) * kTileTokens;
+                                nvalid = max(0, min(kTileTokens + 7, L - tok0));
+                            }
+                        } else {
+                            tok0 = my_e * kTileTokens;
                             nvalid = max(0, min(kTileTokens + 7, L - tok0));
                         }
-                    } else {
-                        tok0 = my_e * kTileTokens;
-                        nvalid = max(0, min(kTileTokens + 7, L - tok0));
-                    }
-                    if (PAGED) {
-                        if (nvalid > 0) {
-                            const int pg = p.page_table[(size_t)i * p.page_table_stride + tok0 / p.page_size];
-                            if (pg < 0 || pg >= p.num_pages) {
-                                raise_status(p.status, DEV_BAD_INDEX);
-                                nvalid = 0;
+                        if (PAGED) {
+                            if (nvalid > 0) {
+                                const int pg = p.page_table[(size_t)i * p.page_table_stride + tok0 / p.page_size];
+                                if (pg < 0 || pg >= p.num_pages) {
+                                    raise_status(p.status, DEV_BAD_INDEX);
+                                    nvalid = 0;
+                                }
+                                outer[0] = pg;
+                                row[0] = tok0 % p.page_size;
                             }
-                            outer = pg;
-                            row = tok0 % p.page_size;
+                        } else {
+                            outer[0] = i;
+                            row[0] = tok0;
                         }
-                    } else {
-                        outer = i;
-                        row = tok0;
                     }
                     // bit 0: first tile of a piece; (the piece's end is found by the consumers)
                     flags = (my_e == 0 || (fresh && t + lane == 0)) ? 1 : 0;
@@ -542,27 +577,49 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 }
                 for (int s = 0; s < n_chunk; ++s, ++it) {
                     const int s_nvalid = __shfl_sync(0xffffffffu, nvalid, s);
-                    const int s_row = __shfl_sync(0xffffffffu, row, s);
-                    const int s_outer = __shfl_sync(0xffffffffu, outer, s);
                     const int s_head = __shfl_sync(0xffffffffu, head, s);
                     const int s_flags = __shfl_sync(0xffffffffu, flags, s);
                     const int s_u = __shfl_sync(0xffffffffu, my_u, s);
                     const int s_pu = __shfl_sync(0xffffffffu, my_pu, s);
                     const int s_ut = __shfl_sync(0xffffffffu, my_ut, s);
+                    int s_row[4], s_outer[4];
+#pragma unroll
+                    for (int sb = 0; sb < 4; ++sb) {
+                        s_row[sb] = (sb == 0 || SMALL) ? __shfl_sync(0xffffffffu, row[sb], s) : 0;
+                        s_outer[sb] = (sb == 0 || SMALL) ? __shfl_sync(0xffffffffu, outer[sb], s) : 0;
+                    }
                     if (lane == 0) {
                         const int st = it % kStages;
                         if (!mbar_wait(&sm.empty[st], ((it / kStages) & 1) ^ 1, p.status)) return;
                         sm.meta[st] = StageMeta{s_nvalid, s_u, s_flags, s_pu, s_ut, iv_id};
                         __threadfence_block();
                         sm.issued = it + 1;                  // consumers may look ahead at this tile
-                        if (s_nvalid > 0) {
-                            unsigned char* dst = sm.stage[st];
+                        unsigned char* dst = sm.stage[st];
+                        if (SMALL && s_nvalid > 0) {
+                            // one box of b rows per gathered block, at its place in the 64-row tile
+                            const int sub_bytes = p.block_size * 128;        // one half (64 channels) of one block
+                            int n_sub = 0;
+#pragma unroll
+                            for (int sb = 0; sb < 4; ++sb) n_sub += ((s_nvalid >> (8 * sb)) & 0xff) ? 1 : 0;
+                            mbar_arrive_expect_tx(&sm.full[st], (uint32_t)(n_sub * 4 * sub_bytes));
+#pragma unroll
+                            for (int sb = 0; sb < 4; ++sb) {
+                                if ((s_nvalid >> (8 * sb)) & 0xff) {
+                                    unsigned char* d2 = dst + sb * sub_bytes;
+                                    tma_load_4d(d2, &map_k, &sm.full[st], 0, s_row[sb], s_head, s_outer[sb]);
+                                    tma_load_4d(d2 + kHalfTileBytes, &map_k, &sm.full[st], 64, s_row[sb], s_head, s_outer[sb]);
+                                    tma_load_4d(d2 + kTileBytes, &map_v, &sm.full[st], 0, s_row[sb], s_head, s_outer[sb]);
+                                    tma_load_4d(d2 + kTileBytes + kHalfTileBytes, &map_v, &sm.full[st], 64, s_row[sb],
+                                                s_head, s_outer[sb]);
+                                }
+                            }
+                        } else if (s_nvalid > 0) {
                             mbar_arrive_expect_tx(&sm.full[st], kStageBytes);
-                            tma_load_4d(dst, &map_k, &sm.full[st], 0, s_row, s_head, s_outer);
-                            tma_load_4d(dst + kHalfTileBytes, &map_k, &sm.full[st], 64, s_row, s_head, s_outer);
-                            tma_load_4d(dst + kTileBytes, &map_v, &sm.full[st], 0, s_row, s_head, s_outer);
-                            tma_load_4d(dst + kTileBytes + kHalfTileBytes, &map_v, &sm.full[st], 64, s_row,
-                                        s_head, s_outer);
+                            tma_load_4d(dst, &map_k, &sm.full[st], 0, s_row[0], s_head, s_outer[0]);
+                            tma_load_4d(dst + kHalfTileBytes, &map_k, &sm.full[st], 64, s_row[0], s_head, s_outer[0]);
+                            tma_load_4d(dst + kTileBytes, &map_v, &sm.full[st], 0, s_row[0], s_head, s_outer[0]);
+                            tma_load_4d(dst + kTileBytes + kHalfTileBytes, &map_v, &sm.full[st], 64, s_row[0],
+                                        s_head, s_outer[0]);
                         } else {
                             mbar_arrive(&sm.full[st]);
                         }
@@ -642,6 +699,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     const int v_csel = (lane >> 3) & 1;
     const int sw = lane & 7;
 
+    // blocks of 16 or 32 tokens: which of a tile's gathered blocks this warp's rows belong to, and where in it
+    constexpr bool small_blocks = SMALL;
+    const int sub_w = p.block_size == 16 ? w : (w >> 1), off_w = p.block_size == 16 ? 0 : (w & 1) * 16;
     // the first tile's metadata
     if (!mbar_wait(&sm.full[0], 0, p.status)) return;
     if (tid == 0) SEER_STAMP(10);
@@ -688,18 +748,20 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         }
         ++piece_tiles;
         // mt.nvalid counts the cached tokens from the tile's first row on (up to 7 beyond the tile, so
-        // that earlier query tokens can be cut off); nvalid is the part of the tile that exists
-        const int nvalid = min(mt.nvalid, kTileTokens);
-        if (nvalid > 16 * w) {
+        // that earlier query tokens can be cut off); nvw is the same count taken from this warp's first
+        // row (with blocks of 16 or 32 tokens: from the count of the gathered block the warp's 16 rows
+        // belong to)
+        const int nvw = small_blocks ? ((mt.nvalid >> (8 * sub_w)) & 0xff) - off_w : mt.nvalid - 16 * w;
+        if (nvw > 0) {
             const uint32_t kbase = smem_u32(sm.stage[st]);
             const uint32_t vbase = kbase + kTileBytes;
-            if (nvalid < 16 * w + 16) {
+            if (nvw < 16) {
                 // ragged tail: rows past the sequence end may hold anything; clear this warp's
                 // V rows so that 0-probability times garbage cannot produce NaN
                 unsigned char* vt = sm.stage[st] + kTileBytes;
                 for (int x = lane; x < 16 * 32; x += 32) {
                     int r = 16 * w + (x >> 5), part = x & 31;      // 32 x 8-byte pieces per row
-                    if (r >= nvalid) {
+                    if ((x >> 5) >= nvw) {
                         int half = part >> 4, off = (part & 15) * 8;
                         *reinterpret_cast<uint2*>(vt + half * kHalfTileBytes + r * 128 + off) =
                             make_uint2(0u, 0u);
@@ -725,15 +787,15 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     else        mma_bf16_16816(sa[nt], a, bq[nt][ks][0], bq[nt][ks][1]);
                 }
             }
-            const int r0 = 16 * w + rw;
+            const int r0 = rw;                         // row within the warp's 16
             uint32_t pb[NT][2];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 float s[4];
 #pragma unroll
                 for (int x = 0; x < 4; ++x) s[x] = (sa[nt][x] + sb[nt][x]) * p.scale_log2;
-                // a row's token sees the first mt.nvalid - back cached tokens counted from this tile's start
-                const int lim0 = mt.nvalid - back[nt][0], lim1 = mt.nvalid - back[nt][1];
+                // a row's token sees the first nvw - back cached tokens counted from this warp's first row
+                const int lim0 = nvw - back[nt][0], lim1 = nvw - back[nt][1];
                 if (r0 >= lim0) s[0] = -INFINITY;
                 if (r0 >= lim1) s[1] = -INFINITY;
                 if (r0 + 8 >= lim0) s[2] = -INFINITY;
@@ -1081,20 +1143,20 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 
 size_t decode_smem_bytes() { return sizeof(Smem) + 1024; }
 
-template <bool SPARSE, bool PAGED, int NT>
+template <bool SPARSE, bool PAGED, int NT, bool SMALL>
 cudaError_t configure() {
-    return cudaFuncSetAttribute(decode_kernel<SPARSE, PAGED, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(decode_kernel<SPARSE, PAGED, NT, SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)decode_smem_bytes());
 }
 
-template <bool SPARSE, bool PAGED, int NT>
+template <bool SPARSE, bool PAGED, int NT, bool SMALL>
 int occupancy() {
     static int cached[kMaxDevices] = {};             // 0: not asked yet on that device
     const int slot = current_device_slot();
     if (cached[slot] <= 0) {
-        if (configure<SPARSE, PAGED, NT>() != cudaSuccess) return 0;
+        if (configure<SPARSE, PAGED, NT, SMALL>() != cudaSuccess) return 0;
         int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<SPARSE, PAGED, NT>, kThreads,
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<SPARSE, PAGED, NT, SMALL>, kThreads,
                                                           decode_smem_bytes()) != cudaSuccess)
             return 0;
         cached[slot] = n;
@@ -1102,27 +1164,31 @@ int occupancy() {
     return cached[slot];
 }
 
-template <bool SPARSE, bool PAGED, int NT>
+template <bool SPARSE, bool PAGED, int NT, bool SMALL>
 cudaError_t launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& p, int grid,
                    cudaStream_t stream) {
-    if (occupancy<SPARSE, PAGED, NT>() <= 0) return cudaErrorInvalidConfiguration;
-    return launch_pdl(decode_kernel<SPARSE, PAGED, NT>, dim3(grid), dim3(kThreads), decode_smem_bytes(), stream, mk, mv,
-                      p);
+    if (occupancy<SPARSE, PAGED, NT, SMALL>() <= 0) return cudaErrorInvalidConfiguration;
+    return launch_pdl(decode_kernel<SPARSE, PAGED, NT, SMALL>, dim3(grid), dim3(kThreads), decode_smem_bytes(), stream,
+                      mk, mv, p);
 }
 
+// (blocks of 16 or 32 tokens use the same resources: the occupancy of the 64-token variant stands for both)
 template <int NT>
 int occupancy_of(bool sparse, bool paged) {
-    if (sparse) return paged ? occupancy<true, true, NT>() : occupancy<true, false, NT>();
-    return paged ? occupancy<false, true, NT>() : occupancy<false, false, NT>();
+    if (sparse) return paged ? occupancy<true, true, NT, false>() : occupancy<true, false, NT, false>();
+    return paged ? occupancy<false, true, NT, false>() : occupancy<false, false, NT, false>();
 }
 
 template <int NT>
 cudaError_t launch_of(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
                       const DecodeParams& p, int grid, cudaStream_t stream) {
-    if (sparse) return paged ? launch<true, true, NT>(map_k, map_v, p, grid, stream)
-                             : launch<true, false, NT>(map_k, map_v, p, grid, stream);
-    return paged ? launch<false, true, NT>(map_k, map_v, p, grid, stream)
-                 : launch<false, false, NT>(map_k, map_v, p, grid, stream);
+    if (sparse && p.blocks_per_tile > 1)
+        return paged ? launch<true, true, NT, true>(map_k, map_v, p, grid, stream)
+                     : launch<true, false, NT, true>(map_k, map_v, p, grid, stream);
+    if (sparse) return paged ? launch<true, true, NT, false>(map_k, map_v, p, grid, stream)
+                             : launch<true, false, NT, false>(map_k, map_v, p, grid, stream);
+    return paged ? launch<false, true, NT, false>(map_k, map_v, p, grid, stream)
+                 : launch<false, false, NT, false>(map_k, map_v, p, grid, stream);
 }
 
 }  // namespace

@@ -823,10 +823,11 @@ extern "C" seer_status seer_gate_select_static(int device, const seer_shape* sha
         gate->max_blocks <= 0 || token_budget < 0 || shape->num_q_heads % shape->num_kv_heads != 0)
         return static_fail(err, err_len, SEER_ERR_INVALID_ARG, "sizes must be positive and num_q_heads a multiple of num_kv_heads");
     const int group = shape->num_q_heads / shape->num_kv_heads;
-    if (shape->head_dim != kHeadDim || (shape->block_size != 64 && shape->block_size != 128) || group > kMaxGroup ||
+    const int bs = shape->block_size;
+    if (shape->head_dim != kHeadDim || (bs != 16 && bs != 32 && bs != 64 && bs != 128) || group > kMaxGroup ||
         (gate->d_gate != 64 && gate->d_gate != 128 && gate->d_gate != 256))
         return static_fail(err, err_len, SEER_ERR_UNSUPPORTED,
-                           "supported: head_dim 128, block_size 64/128, group size <= 8, d_gate 64/128/256");
+                           "supported: head_dim 128, block_size 16/32/64/128, group size <= 8, d_gate 64/128/256");
     if (!(gate->rope_theta > 0.f)) return static_fail(err, err_len, SEER_ERR_INVALID_ARG, "rope_theta must be positive");
     if (((uintptr_t)q_nope | (uintptr_t)gate->w_q | (uintptr_t)gate->kcomp) & 15u)
         return static_fail(err, err_len, SEER_ERR_INVALID_ARG, "q_nope, w_q and kcomp must be 16-byte aligned");

@@ -207,7 +207,7 @@ def test_host_side_argument_checks(ctx):
     kv = binding.make_kv(k, v, lens_t)
     for bad_shape, status in [
         (binding.make_shape(B, Hq, Hkv, 64, 64, 0.1), binding.SEER_ERR_UNSUPPORTED),
-        (binding.make_shape(B, Hq, Hkv, d, 32, 0.1), binding.SEER_ERR_UNSUPPORTED),
+        (binding.make_shape(B, Hq, Hkv, d, 48, 0.1), binding.SEER_ERR_UNSUPPORTED),
         (binding.make_shape(B, 9, 2, d, 64, 0.1), binding.SEER_ERR_INVALID_ARG),
         (binding.make_shape(B, 32, 2, d, 64, 0.1), binding.SEER_ERR_UNSUPPORTED),
         (binding.make_shape(0, Hq, Hkv, d, 64, 0.1), binding.SEER_ERR_INVALID_ARG),

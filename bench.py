@@ -282,6 +282,17 @@ def run_ours(args):
     s1.record()
     barrier()
     sparse_b2b_ms = s0.elapsed_time(s1) / K
+    # the step without the compressed-K update (63 steps of 64 in a real decode: a block fills once per b tokens)
+    n0, n1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    n0.record()
+    for s in range(K):
+        lay = layers[s % n_layers]
+        ctx.seer_decode_step(shape, lay["kv"], lay["gate"], lay["q"], lay["qn"], None, budget, idx, cnt, k_sel, out,
+                             stream=stream)
+    n1.record()
+    barrier()
+    step_noappend_ms = n0.elapsed_time(n1) / K
     clocks = sampler.stop()
 
     # ---- end to end through the same API with host buffers ----------------------------------
@@ -334,8 +345,8 @@ def run_ours(args):
     assert ctx.device_status() == binding.SEER_OK
 
     # ---- reduce over ranks -------------------------------------------------------------------
-    step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms = max_over_ranks(
-        [step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms], dev)
+    step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms, step_noappend_ms = max_over_ranks(
+        [step_ms, sparse_ms, dense_ms, sparse_b2b_ms, e2e_ms, step_noappend_ms], dev)
 
     result = None
     if rank == 0:
@@ -376,6 +387,7 @@ def run_ours(args):
                 "dense_kernel_GBps": round(dense_bytes / (dense_ms * 1e-3) / 1e9, 1),
                 "dense_frac_of_measured_peak": round(dense_bytes / (dense_ms * 1e-3) / 1e9 / peak, 4),
                 "gate_plus_kcomp_us": round((step_ms - sparse_ms) * 1e3, 2),
+                "step_without_append_us": round(step_noappend_ms * 1e3, 2),
                 "speedup_vs_dense_kernel": round(dense_ms / sparse_b2b_ms, 3),
                 "speedup_vs_dense_step": round(dense_ms / step_ms, 3),
                 "ideal_speedup": round(n_blocks / k_sel, 3),

@@ -1050,8 +1050,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     };
     // stage the n listed partials, kLand per round, and add them to ms (all consumer threads call)
     auto accumulate_list = [&](MergeState<NT>& ms, const int* slots, int n) -> bool {
-        if (n > 0 && n <= kDirect) {
-            merge_accumulate_direct<NT>(p, ms, slots, n, tid);
+        if (n > 0 && n <= 2 * kDirect) {
+            // up to two rounds of direct loads beat staging (one round trip each, no barrier)
+            merge_accumulate_direct<NT>(p, ms, slots, min(n, kDirect), tid);
+            if (n > kDirect) merge_accumulate_direct<NT>(p, ms, slots + kDirect, n - kDirect, tid);
             return true;
         }
         for (int s0 = 0; s0 < n; s0 += n_land) {

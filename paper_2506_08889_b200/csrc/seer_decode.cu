@@ -302,13 +302,22 @@ __device__ __forceinline__ void merge_finalize(const DecodeParams& p, const Merg
 template <int NT>
 __device__ __forceinline__ int scan_valid_slots(const DecodeParams& p, int first, int n_slots, int* list, int lane) {
     int n = 0;
-    for (int s0 = 0; s0 < n_slots; s0 += 32) {
-        const int sl = first + s0 + lane;
-        const bool ok = s0 + lane < n_slots &&
-                        __float_as_uint(__ldcg(p.part_ml + (size_t)sl * (kMlStride * NT) + 16 * NT)) == p.generation;
-        const unsigned m = __ballot_sync(0xffffffffu, ok);
-        if (ok) list[n + __popc(m & ((1u << lane) - 1u))] = sl;
-        n += __popc(m);
+    // four stamps per lane in flight: the scan costs one round trip per 128 candidate slots
+    for (int s0 = 0; s0 < n_slots; s0 += 128) {
+        unsigned int stamp[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int x = s0 + 32 * k + lane;
+            stamp[k] = x < n_slots ? __float_as_uint(__ldcg(p.part_ml + (size_t)(first + x) * (kMlStride * NT) + 16 * NT))
+                                   : ~p.generation;
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool ok = stamp[k] == p.generation;
+            const unsigned m = __ballot_sync(0xffffffffu, ok);
+            if (ok) list[n + __popc(m & ((1u << lane) - 1u))] = first + s0 + 32 * k + lane;
+            n += __popc(m);
+        }
     }
     return n;
 }

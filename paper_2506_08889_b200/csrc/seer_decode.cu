@@ -50,6 +50,7 @@ constexpr int kLandBytes = 2 * kStageBytes;                 // landing area for 
 constexpr int kMaxSteals = 14;                             // chunks a CTA may take from other ranges
 constexpr int kMinChunk = 2;                               // smallest dynamic chunk, in tiles
 constexpr int kMinStaticTilesPerCta = 8;                   // below this everything is static
+constexpr int kBigFirstLen = 32;                           // ranges at least this long order their chunks big to small
 
 struct StageMeta {
     int nvalid;        // cached tokens from the tile's first row on, capped at 64 + 7 (0 = nothing was loaded); -1 = end of
@@ -72,7 +73,10 @@ struct Piece {
 // [c*T/G, (c+1)*T/G); with len its length, b its end and ts = b - (len>>2) the start of its
 // tail, its intervals are
 //   0: [a, ts)   1: [ts, ts + (len>>(R+1)))   2: [.., ts + (len>>R))  ...  R: [ts + (len>>3), b),
-// i.e. the tail's chunks double in size towards the end of the range.
+// i.e. the tail's chunks double in size towards the end of the range.  Ranges of kBigFirstLen tiles or
+// more use the mirror image, 1: [ts, b - (len>>3))  2: [.., b - (len>>4)) ... R: [b - (len>>(R+1)), b):
+// the owner (front) meets the big chunks first and thieves (back) pick up small ones, which leaves
+// less to wait for at the very end when a range is long; short ranges do better the other way round.
 struct Schedule {
     int T, G;                      // tiles, ranges (G <= T)
     int R;                         // dynamic chunks per range (0: everything is static)
@@ -149,6 +153,11 @@ __device__ __forceinline__ void interval_range(const Schedule& s, int c, int j, 
     if (s.R == 0) { *begin = a; *end = b; return; }
     const int ts = b - (len >> 2);                  // the tail: last quarter of the range
     if (j == 0) { *begin = a; *end = ts; return; }
+    if (len >= kBigFirstLen) {                      // long ranges: the big chunks first
+        *begin = b - (len >> (j + 1));
+        *end = j == s.R ? b : b - (len >> (j + 2));
+        return;
+    }
     *begin = j == 1 ? ts : ts + (len >> (s.R + 3 - j));
     *end = ts + (len >> (s.R + 2 - j));
 }
@@ -161,7 +170,11 @@ __device__ __forceinline__ int interval_of(const Schedule& s, int t) {
     const int off = t - (b - (len >> 2));           // position inside the tail
     if (off < 0) return c * (s.R + 1);
     int j = 1;
-    while (j < s.R && off >= (len >> (s.R + 2 - j))) ++j;
+    if (len >= kBigFirstLen) {
+        while (j < s.R && t >= b - (len >> (j + 2))) ++j;
+    } else {
+        while (j < s.R && off >= (len >> (s.R + 2 - j))) ++j;
+    }
     return c * (s.R + 1) + j;
 }
 

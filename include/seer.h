@@ -122,7 +122,9 @@ const char* seer_status_string(seer_status s);
  * owned by the context, valid until the next call). */
 const char* seer_last_error(const seer_ctx* ctx);
 /* Synchronises `stream`, returns the sticky device-side status (SEER_OK,
- * SEER_ERR_BAD_INDEX or SEER_ERR_TIMEOUT) and clears it. */
+ * SEER_ERR_BAD_INDEX or SEER_ERR_TIMEOUT) and clears it.  After SEER_ERR_TIMEOUT the
+ * results of the calls since the last check are invalid; the context's counters are
+ * reset by this call and the context can be used again. */
 seer_status seer_get_device_status(seer_ctx* ctx, void* stream);
 /* Workspace bytes a context needs for calls of this shape (upper bound);
  * max_blocks = largest number of blocks per sequence. */

@@ -5,10 +5,10 @@
 // 64-token tiles of its selected blocks (sparse) or of its whole sequence (dense).  All
 // units' tile lists are laid end to end (T tiles) and cut into one equal contiguous range per
 // CTA.  The first three quarters of a range are its CTA's static share; the last quarter is
-// cut into chunks that double in size towards the end of the range (two tiles ... 1/8 of the
-// range).  The owner of a range claims its chunks from the front, so its work stays one
+// cut into chunks of geometrically varying size (two tiles ... 1/8 of the range; see Schedule for
+// their order).  The owner of a range claims its chunks from the front, so its work stays one
 // contiguous run; a CTA that has finished its own range steals other ranges' chunks from the
-// back, the big ones first, as in steal-half work stealing.
+// back.
 // SMs that get less memory bandwidth than others thus shed work to faster ones and all finish
 // together, while a unit is cut into few pieces.  Claims are single atomic adds on a per-range
 // counter; nobody ever waits for another CTA.
@@ -29,6 +29,11 @@
 //     P^T -> bf16, transposed in registers (movmatrix) into the B operand
 //     O^T (128 x 8)        += V_slice^T (128 x 16) . P^T (16 x 8)       mma.sync m16n8k16
 // The g <= 8 query heads of the group sit on the MMA's N = 8 side, tokens on M.
+//
+// Template variants.  NT = 2 puts up to 16 rows on the N side (two N-tiles per warp): several query
+// tokens per sequence, row = (token, head), each row cut off causally at its own position.  SMALL
+// gathers four or two listed blocks of 16 or 32 tokens into one 64-token tile (one TMA box per
+// block, one valid-token count per block); blocks of 64 or 128 tokens are one or two tiles.
 #include "seer_device.cuh"
 #include "seer_internal.h"
 

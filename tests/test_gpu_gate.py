@@ -9,7 +9,7 @@ import torch
 
 import oracle
 from paper_2506_08889_b200 import binding, synth
-from util import bits
+from util import bits, check_attention, make_qkv
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -351,3 +351,36 @@ def test_threshold_selection(ctx, tau):
     assert np.array_equal(idx2.cpu().numpy(), w2) and np.array_equal(cnt2.cpu().numpy(), c2)
     with pytest.raises(binding.SeerError):
         ctx.seer_gate_select_threshold(shape, gate, lens_t, None, torch.as_tensor(sc, device=DEV), 1.5, idx2, cnt2, small)
+
+
+@pytest.mark.parametrize("b", [16, 64, 128])
+def test_step_call_on_ragged_lengths_budget_above_and_below_the_block_counts(ctx, b):
+    # the step call on sequences shorter than the budget, empty ones, one block only
+    B, Hq, Hkv, d, dg, S = 6, 8, 2, 128, 128, 4096
+    nb = S // b
+    lens = np.array([S, (nb * 5 // 8) * b + 3, 5 * b, b, 7, 0], np.int32)
+    q, k, v = make_qkv(B, Hq, Hkv, S, d, 77 + b, DEV)
+    qn = synth.normal_bf16((B, Hq, d), 77 + b, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, 4 * d), 77 + b, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nb, dg), 77 + b, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    kv = binding.make_kv(k, v, lens_t)
+    for budget, max_sel in [(12 * b, 12), (12 * b, 9), (b, 4), (0, 3), (1000 * b, nb)]:
+        idx = torch.full((B, Hkv, max_sel), 55, dtype=torch.int32, device=DEV)
+        cnt = torch.full((B, Hkv), 55, dtype=torch.int32, device=DEV)
+        out = torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+        lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV)
+        ctx.seer_decode_step(shape, kv, gate, q, qn, None, budget, idx, cnt, max_sel, out, lse)
+        torch.cuda.synchronize()
+        sc = torch.zeros((B, Hkv, nb), dtype=torch.float32, device=DEV)
+        idx2, cnt2 = torch.zeros_like(idx), torch.zeros_like(cnt)
+        ctx.seer_gate_select(shape, gate, lens_t, qn, None, budget, idx2, cnt2, max_sel, scores_out=sc)
+        torch.cuda.synchronize()
+        assert torch.equal(idx, idx2) and torch.equal(cnt, cnt2)
+        want_idx, want_cnt = oracle.select(sc.cpu().numpy(), lens, b, budget, max_sel)
+        assert np.array_equal(cnt.cpu().numpy(), want_cnt) and np.array_equal(idx.cpu().numpy(), want_idx)
+        ref = oracle.sparse(bits(q), bits(k), bits(v), lens, want_idx, want_cnt, b, 0.0884)
+        check_attention(out, lse, *ref, what=f"step b={b} budget={budget}")
+    assert ctx.device_status() == binding.SEER_OK

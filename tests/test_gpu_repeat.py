@@ -1,0 +1,85 @@
+"""The same call repeated a few thousand times: work stealing and the in-kernel combine make the
+order of the floating-point merges vary from launch to launch, never the set of tiles.  Every
+repetition must stay within the parity bound of the oracle result; the gate's lists must be
+identical every time (the selection is exact)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_08889_b200 import binding, synth
+from util import bits, check_attention, make_qkv
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("T", [1, 3])
+def test_sparse_decode_repeated_launches_agree(ctx, T):
+    B, Hq, Hkv, d, b, S = 2, 40, 8, 128, 64, 32768
+    lens = np.array([S, S - 1234], np.int32)
+    q = synth.normal_bf16((B, T, Hq, d), 501, "q", DEV)
+    k = synth.normal_bf16((B, Hkv, S, d), 501, "k", DEV)
+    v = synth.normal_bf16((B, Hkv, S, d), 501, "v", DEV)
+    n = [-(-int(L) // b) for L in lens]
+    keep = [x // 2 for x in n]
+    idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max(keep), 501)
+    ref_o, ref_l = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.0884)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    kv = binding.make_kv(k, v, lens_t)
+    idx_t, cnt_t = torch.as_tensor(idx, device=DEV), torch.as_tensor(cnt, device=DEV)
+    out = torch.empty((B, T, Hq, d), dtype=torch.bfloat16, device=DEV)
+    lse = torch.empty((B, T, Hq), dtype=torch.float32, device=DEV)
+    ctx.seer_sparse_decode_multi(shape, kv, q, T, idx_t, cnt_t, idx.shape[2], out, lse)
+    torch.cuda.synchronize()
+    check_attention(out, lse, ref_o, ref_l, what="first launch", strict=True)
+    first_o, first_l = out.float().clone(), lse.clone()
+    worst_o = torch.zeros((), device=DEV)
+    worst_l = torch.zeros((), device=DEV)
+    for rep in range(1500):
+        out.fill_(float("nan"))
+        lse.fill_(float("nan"))
+        ctx.seer_sparse_decode_multi(shape, kv, q, T, idx_t, cnt_t, idx.shape[2], out, lse)
+        worst_o = torch.maximum(worst_o, (out.float() - first_o).abs().nan_to_num(nan=1e9).max())
+        worst_l = torch.maximum(worst_l, (lse - first_l).abs().nan_to_num(nan=1e9).max())
+    torch.cuda.synchronize()
+    # bf16 outputs of magnitude < 0.25 differ by a few units in the last place at most
+    assert float(worst_o) <= 2e-3 and float(worst_l) <= 1e-4, (float(worst_o), float(worst_l))
+    assert ctx.device_status() == binding.SEER_OK
+
+
+def test_gate_repeated_launches_give_identical_lists(ctx):
+    B, Hq, Hkv, d, dg, b, nb = 4, 40, 8, 128, 128, 64, 2048
+    lens = np.array([nb * b, nb * b - 77, 1000 * b, 64 * b + 1], np.int32)
+    qn = synth.normal_bf16((B, Hq, d), 502, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, 5 * d), 502, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nb, dg), 502, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, 1.0e6, wq, None, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    max_sel = 205
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nb), dtype=torch.float32, device=DEV)
+    ctx.seer_gate_select(shape, gate, lens_t, qn, None, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    want_idx, want_cnt = oracle.select(sc.cpu().numpy(), lens, b, max_sel * b, max_sel)
+    assert np.array_equal(idx.cpu().numpy(), want_idx) and np.array_equal(cnt.cpu().numpy(), want_cnt)
+    first_idx, first_cnt, first_sc = idx.clone(), cnt.clone(), sc.clone()
+    bad = torch.zeros((), dtype=torch.int64, device=DEV)
+    for rep in range(1500):
+        idx.fill_(-7)
+        cnt.fill_(-7)
+        ctx.seer_gate_select(shape, gate, lens_t, qn, None, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+        bad += (idx != first_idx).sum() + (cnt != first_cnt).sum() + (sc != first_sc).sum()
+    torch.cuda.synchronize()
+    assert int(bad) == 0
+    assert ctx.device_status() == binding.SEER_OK

@@ -83,3 +83,45 @@ def test_gate_repeated_launches_give_identical_lists(ctx):
     torch.cuda.synchronize()
     assert int(bad) == 0
     assert ctx.device_status() == binding.SEER_OK
+
+
+def test_calls_of_different_shapes_interleaved_on_one_context(ctx):
+    # different unit counts, block sizes, query-token counts, gate and decode calls share one workspace
+    cases = []
+    for (B, Hkv, g, b, S, T, seed) in [(1, 8, 5, 64, 8192, 1, 601), (3, 2, 8, 32, 4096, 2, 602), (2, 4, 4, 128, 16384, 3, 603),
+                                       (5, 1, 1, 16, 2048, 8, 604)]:
+        Hq = g * Hkv
+        lens = synth.ragged_lengths(B, S // 2, S, b, seed) - np.int32(seed % 7)       # partial last blocks
+        q = synth.normal_bf16((B, T, Hq, 128), seed, "q", DEV)
+        k = synth.normal_bf16((B, Hkv, S, 128), seed, "k", DEV)
+        v = synth.normal_bf16((B, Hkv, S, 128), seed, "v", DEV)
+        n = [-(-int(L) // b) for L in lens]
+        keep = [max(1, x // 3) for x in n]
+        idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max(keep), seed, shuffle=True)
+        ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
+        lens_t = torch.as_tensor(lens, device=DEV)
+        cases.append(dict(shape=binding.make_shape(B, Hq, Hkv, 128, b, 0.09), kv=binding.make_kv(k, v, lens_t), q=q, T=T,
+                          idx=torch.as_tensor(idx, device=DEV), cnt=torch.as_tensor(cnt, device=DEV), ref=ref,
+                          out=torch.empty((B, T, Hq, 128), dtype=torch.bfloat16, device=DEV),
+                          lse=torch.empty((B, T, Hq), dtype=torch.float32, device=DEV), keep=(k, v, lens_t)))
+    # a gate call of yet another shape in between
+    gB, gHkv, gnb = 2, 4, 1500
+    sc = synth.normal_f32((gB, gHkv, gnb), 605, "scores", DEV)
+    glens = torch.tensor([gnb * 64, 900 * 64], dtype=torch.int32, device=DEV)
+    gshape = binding.make_shape(gB, gHkv * 2, gHkv, 128, 64, 0.1)
+    ggate = binding.make_gate(128, 1.0e6, None, None, None, gnb)
+    gidx = torch.zeros((gB, gHkv, 100), dtype=torch.int32, device=DEV)
+    gcnt = torch.zeros((gB, gHkv), dtype=torch.int32, device=DEV)
+    want_gidx, want_gcnt = oracle.select(sc.cpu().numpy(), glens.cpu().numpy(), 64, 100 * 64, 100)
+    for rep in range(60):
+        for c in cases:
+            c["out"].fill_(float("nan"))
+            ctx.seer_sparse_decode_multi(c["shape"], c["kv"], c["q"], c["T"], c["idx"], c["cnt"], c["idx"].shape[2],
+                                         c["out"], c["lse"])
+            ctx.seer_gate_select(gshape, ggate, glens, None, sc, 100 * 64, gidx, gcnt, 100)
+        if rep % 20 == 19:
+            torch.cuda.synchronize()
+            for ci, c in enumerate(cases):
+                check_attention(c["out"], c["lse"], *c["ref"], what=f"interleaved case {ci} rep {rep}")
+            assert np.array_equal(gidx.cpu().numpy(), want_gidx) and np.array_equal(gcnt.cpu().numpy(), want_gcnt)
+    assert ctx.device_status() == binding.SEER_OK

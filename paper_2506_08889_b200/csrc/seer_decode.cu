@@ -1052,6 +1052,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (lane == 0) mbar_arrive(&sm.end_bar);
     if (!mbar_wait(&sm.end_bar, 0, p.status)) return;
     const int n_owed = sm.pieces_n;
+    if (n_owed == 0) {                                 // nothing to combine: make room for the next kernel at once
+        if (tid == 0) SEER_STAMP(7);
+        return;
+    }
 #ifdef SEER_DECODE_TRACE
     if (tid == 0 && n_owed > 0) { SEER_STAMP(2); p.trace[(size_t)blockIdx.x * 16 + 4] = n_owed; }
 #endif

@@ -619,7 +619,7 @@ def cpu_baseline(w, lay, k_sel, budget, sel_kv_bytes, seconds=15.0):
     nbytes = oracle_step(w, host, 1, H, budget, k_sel)
     one = time.perf_counter() - t0
     n_seq = int(max(1, min(w.batch, seconds / max(one, 1e-3))))
-    reps = int(max(1, min(5, seconds / max(one * n_seq, 1e-3))))
+    reps = int(max(1, min(100, seconds / max(one * n_seq, 1e-3))))
     t0 = time.perf_counter()
     for _ in range(reps):
         nbytes = oracle_step(w, host, n_seq, H, budget, k_sel)

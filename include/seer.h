@@ -318,10 +318,13 @@ seer_status seer_decode_step_multi(seer_ctx* ctx, const seer_shape* shape, const
  * is used holds one copy of that array from first use until the process exits.
  *
  *  - It calls no cudaMalloc / cudaFree and no allocating library routine.
- *  - A call whose scratch need, 4*B*Hkv + 4*B*Hkv*d_gate (+ 4*B*Hkv*max_blocks without scores_out),
- *    each part rounded up to 256 bytes, exceeds the array returns SEER_ERR_WORKSPACE and launches
- *    nothing; `err` says how much was needed.  (Example that fits: B*Hkv = 64, d_gate 128,
- *    max_blocks 2048.)
+ *  - Up to 8192 compressed keys per unit (max_blocks <= 8192) the gate is one kernel that keeps its
+ *    intermediate results in shared memory; the array is then not needed and any B*Hkv is accepted.
+ *    Beyond that the gate runs as two kernels that pass the gate query and the scores through the
+ *    array.  Such a call needs 256 + 4*B*Hkv + 4*B*Hkv*d_gate (+ 4*B*Hkv*max_blocks without
+ *    scores_out) bytes, each part rounded up to 256; if that exceeds the array the call returns
+ *    SEER_ERR_WORKSPACE and launches nothing, and `err` says how much was needed.  (Example that
+ *    fits: B*Hkv = 16, d_gate 128, max_blocks 16000.)
  *  - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
  *    that device made current).  Make that first call outside any stream capture.
  *  - All calls on a device share the one array, and it keeps the previous call's contents.  The

@@ -836,10 +836,14 @@ extern "C" seer_status seer_gate_select_static(int device, const seer_shape* sha
     const long long U = (long long)shape->batch * shape->num_kv_heads;
     if (U > 65535) return static_fail(err, err_len, SEER_ERR_UNSUPPORTED, "batch * num_kv_heads above 65535");
 
-    // layout of the scratch: [tickets U ints][gate query U*d_gate floats][scores U*max_blocks floats]
-    const size_t off_qg = ((size_t)U * sizeof(int) + 255) / 256 * 256;
+    // Layout of the scratch: [status word, 256 B][tickets U ints][gate query U*d_gate floats]
+    // [scores U*max_blocks floats].  Only the two-kernel path (more compressed keys per unit than the
+    // cluster kernel holds in shared memory) uses anything beyond the status word.
+    const bool split = !gate_one_kernel(gate->max_blocks);
+    const size_t off_tk = 256;
+    const size_t off_qg = off_tk + ((size_t)U * sizeof(int) + 255) / 256 * 256;
     const size_t off_sc = off_qg + ((size_t)U * gate->d_gate * sizeof(float) + 255) / 256 * 256;
-    const size_t need = off_sc + (scores_out ? 0 : (size_t)U * gate->max_blocks * sizeof(float));
+    const size_t need = !split ? off_tk : off_sc + (scores_out ? 0 : (size_t)U * gate->max_blocks * sizeof(float));
     if (need > (size_t)SEER_STATIC_SCRATCH_BYTES)
         return static_fail(err, err_len, SEER_ERR_WORKSPACE,
                            "this call needs %lld bytes of scratch, the built-in array holds %lld "
@@ -863,9 +867,12 @@ extern "C" seer_status seer_gate_select_static(int device, const seer_shape* sha
         base = g_static_ptr[device];
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // the tickets must start at zero; everything else is written before it is read
-    ce = cudaMemsetAsync(base, 0, (size_t)U * sizeof(int), s);
-    if (ce != cudaSuccess) return static_fail(err, err_len, SEER_ERR_CUDA, "cudaMemsetAsync failed (code %lld)", (long long)ce);
+    // the tickets must start at zero (an earlier call may have been cut short); everything else is
+    // written before it is read
+    if (split) {
+        ce = cudaMemsetAsync(base + off_tk, 0, (size_t)U * sizeof(int), s);
+        if (ce != cudaSuccess) return static_fail(err, err_len, SEER_ERR_CUDA, "cudaMemsetAsync failed (code %lld)", (long long)ce);
+    }
 
     GateParams p;
     memset(&p, 0, sizeof p);
@@ -889,8 +896,8 @@ extern "C" seer_status seer_gate_select_static(int device, const seer_shape* sha
     p.max_sel = max_sel;
     p.token_budget = token_budget;
     p.q_len = 1;
-    p.status = nullptr;
-    p.tickets = reinterpret_cast<int*>(base);
+    p.status = reinterpret_cast<unsigned int*>(base);
+    p.tickets = reinterpret_cast<int*>(base + off_tk);
     for (int c = 0; c < gate->d_gate / 2; ++c)
         p.inv_freq[c] = pow((double)gate->rope_theta, -2.0 * (double)c / (double)gate->d_gate);
     int launched = 0;

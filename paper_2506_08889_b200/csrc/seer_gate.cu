@@ -52,6 +52,10 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+// Split cluster barrier (all threads of all CTAs of the cluster execute both halves).
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
 constexpr int kUnitThreads = 1024;          // most threads a CTA that runs the selection may have
 
 // Inverse of score_key (NaN came out as key 0 and goes back as -inf).
@@ -67,6 +71,8 @@ struct SelectSmem {
     int hist[3][kSelBins];                  // one histogram per pass (at most ceil(32 / 11) passes)
     unsigned long long warp_tot[kUnitThreads / 32];
     uint32_t warp_min[kUnitThreads / 32], warp_max[kUnitThreads / 32];
+    float red[kUnitThreads / 32];           // block reductions of the threshold method (its own array: the
+                                            // selection that follows writes warp_min while slower warps still read)
     uint32_t prefix;
     int rem;
     int bin_cnt;                            // one-pass path: candidates in the boundary bin ...
@@ -123,12 +129,12 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
                 v = is_max ? fmaxf(v, o) : v + o;
             }
             __syncthreads();                                   // the scratch may still be in use
-            if (lane == 0) sm.warp_min[warp] = __float_as_uint(v);
+            if (lane == 0) sm.red[warp] = v;
             __syncthreads();
             float r = is_max ? -INFINITY : 0.f;
 #pragma unroll
             for (int w2 = 0; w2 < NT / 32; ++w2) {
-                const float o = __uint_as_float(sm.warp_min[w2]);
+                const float o = sm.red[w2];
                 r = is_max ? fmaxf(r, o) : r + o;
             }
             return r;
@@ -541,6 +547,9 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = p.group * kHeadDim, chunks = n / 8, half = p.d_gate / 2;
     const int gw = slice * (kGateThreads / 32) + warp, n_gw = S * (kGateThreads / 32);
+    // Another CTA's shared memory may only be written once that CTA is known to be running: every
+    // CTA signals its start here and waits for the others just before step 1's remote stores.
+    cluster_arrive();
     // Work items of the projection: (query token t, rotary pair c), item = t * half + c, dealt to the
     // cluster's warps round robin.  W_q rows of this warp's first item: constants, requested before the wait.
     const int n_items = q_len * half;
@@ -584,6 +593,7 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
         if (pc < total) cp_async16(staged + pc, kc + pc);
     }
     const int L = __ldg(p.seq_lens + i);
+    cluster_wait();                                    // every CTA of the cluster has started
     // ---- 1. gate queries --------------------------------------------------------------------------
     for (int item = gw; item < n_items; item += n_gw) {
         const int t = item / half, c = item - t * half;

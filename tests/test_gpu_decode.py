@@ -6,7 +6,7 @@ import torch
 
 import oracle
 from paper_2506_08889_b200 import binding, synth
-from util import bits, check_attention, make_qkv, to_paged
+from util import bits, check_attention, make_qkv, to_paged, ref_sparse, ref_dense
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -56,7 +56,7 @@ def test_tiny_workload_every_element(ctx):
     assert idx[0, 0, -1] == 63 and cnt[0, 0] == 8
     out, lse = _run_sparse(ctx, q, k, v, lens, idx, cnt, w.block_size, w.sm_scale)
     ref_o, ref_l = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, w.block_size, w.sm_scale)
-    check_attention(out, lse, ref_o, ref_l, "tiny", strict=True)
+    check_attention(out, lse, ref_o, ref_l, what="tiny", strict=True)
     assert ctx.device_status() == binding.SEER_OK
 
 
@@ -71,7 +71,7 @@ def test_sparse_ragged_shuffled_lists(ctx, g, Hkv, b, token_major):
     keep = [max(1, x // 3) for x in n]
     max_sel = max(keep) + 3
     idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max_sel, 100 + g, shuffle=True)
-    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
+    ref = ref_sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
     out, lse = _run_sparse(ctx, q, k, v, lens, idx, cnt, b, 0.09)
     check_attention(out, lse, *ref, what=f"g={g}")
     # same lists without counts: the -1 padding is skipped
@@ -91,10 +91,10 @@ def test_rows_past_the_length_are_never_used(ctx):
     k[0, :, 310] = 1e30
     idx, cnt = synth.random_block_lists(lens, Hkv, b, [3, 2], 4, 7)
     kh, vh = torch.nan_to_num(k, nan=0.0).cpu(), torch.nan_to_num(v, nan=0.0).cpu()
-    ref = oracle.sparse(bits(q), bits(kh), bits(vh), lens, idx, cnt, b, 0.1)
+    ref = ref_sparse(bits(q), bits(kh), bits(vh), lens, idx, cnt, b, 0.1)
     out, lse = _run_sparse(ctx, q, k, v, lens, idx, cnt, b, 0.1)
     check_attention(out, lse, *ref, what="nan tail sparse")
-    refd = oracle.dense(bits(q), bits(kh), bits(vh), lens, 0.1)
+    refd = ref_dense(bits(q), bits(kh), bits(vh), lens, 0.1)
     outd, lsed = _run_dense(ctx, q, k, v, lens, b, 0.1)
     check_attention(outd, lsed, *refd, what="nan tail dense")
 
@@ -104,7 +104,7 @@ def test_dense_ragged_lengths(ctx, b):
     B, Hq, Hkv, d, S = 6, 10, 2, 128, 1536
     lens = np.array([1, 64, 65, 1536, 0, 777], np.int32)
     q, k, v = make_qkv(B, Hq, Hkv, S, d, 33, DEV)
-    ref = oracle.dense(bits(q), bits(k), bits(v), lens, 0.0884)
+    ref = ref_dense(bits(q), bits(k), bits(v), lens, 0.0884)
     out, lse = _run_dense(ctx, q, k, v, lens, b, 0.0884)
     check_attention(out, lse, *ref, what="dense ragged")
     assert torch.all(out[4] == 0) and torch.all(torch.isneginf(lse[4]))
@@ -150,11 +150,11 @@ def test_paged_cache(ctx, b, page_size):
     kp, vp, table = to_paged(k, v, page_size, 66)
     n = [-(-int(L) // b) for L in lens]
     idx, cnt = synth.random_block_lists(lens, Hkv, b, [max(1, x // 2) for x in n], max(n), 66, shuffle=True)
-    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.0884)
+    ref = ref_sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.0884)
     out, lse = _run_sparse(ctx, q, kp, vp, lens, idx, cnt, b, 0.0884, page_table=table, page_size=page_size,
                            max_seq_len=S)
     check_attention(out, lse, *ref, what="paged sparse")
-    refd = oracle.dense(bits(q), bits(k), bits(v), lens, 0.0884)
+    refd = ref_dense(bits(q), bits(k), bits(v), lens, 0.0884)
     outd, lsed = _run_dense(ctx, q, kp, vp, lens, b, 0.0884, page_table=table, page_size=page_size, max_seq_len=S)
     check_attention(outd, lsed, *refd, what="paged dense")
     assert ctx.device_status() == binding.SEER_OK
@@ -166,7 +166,7 @@ def test_bad_entries_are_skipped_and_flagged(ctx):
     q, k, v = make_qkv(B, Hq, Hkv, S, d, 77, DEV)
     idx = np.array([[[3, 16, 9, -1, 15, 400], [-1, -1, 2, 15, 1 << 30, -5]]], np.int32)
     cnt = np.array([[6, 6]], np.int32)
-    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.1)      # oracle ignores them
+    ref = ref_sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.1)      # oracle ignores them
     out, lse = _run_sparse(ctx, q, k, v, lens, idx, cnt, b, 0.1)
     check_attention(out, lse, *ref, what="bad entries")
     assert ctx.device_status() == binding.SEER_ERR_BAD_INDEX
@@ -177,7 +177,7 @@ def test_bad_entries_are_skipped_and_flagged(ctx):
     table2[0, 3] = kp.shape[0] + 5
     good = np.array([[[3, 9, 15, -1, -1, -1], [2, 15, -1, -1, -1, -1]]], np.int32)
     without3 = np.array([[[9, 15, -1, -1, -1, -1], [2, 15, -1, -1, -1, -1]]], np.int32)
-    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, without3, None, b, 0.1)
+    ref = ref_sparse(bits(q), bits(k), bits(v), lens, without3, None, b, 0.1)
     out, lse = _run_sparse(ctx, q, kp, vp, lens, good, None, b, 0.1, page_table=table2, page_size=64,
                            max_seq_len=S, use_cnt=False)
     check_attention(out, lse, *ref, what="bad page")
@@ -193,7 +193,7 @@ def test_empty_lists_give_zero_and_minus_inf(ctx):
     cnt = np.zeros((B, Hkv), np.int32)
     cnt[1, 1] = 2
     cnt[0, 1] = 3                                          # counted but all padding
-    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.1)
+    ref = ref_sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.1)
     out, lse = _run_sparse(ctx, q, k, v, lens, idx, cnt, b, 0.1)
     check_attention(out, lse, *ref, what="empty")
     assert torch.all(out[0] == 0) and torch.all(torch.isneginf(lse[0]))

@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from paper_2506_08889_b200 import binding, synth
-from util import bits, check_attention
+from util import bits, check_attention, ref_sparse, ref_dense
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -56,11 +56,11 @@ def _largest_unit_count(small_ctx, ctx, B, Hq, Hkv, d, b, S):
     assert err.value.status == binding.SEER_ERR_WORKSPACE
     ctx.seer_sparse_decode(shape, kv, q, idx_t, cnt_t, 3, out, lse)
     torch.cuda.synchronize()
-    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
+    ref = ref_sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
     check_attention(out, lse, *ref, what="65528 units sparse")
     ctx.seer_dense_decode(shape, kv, q, out, lse)
     torch.cuda.synchronize()
-    refd = oracle.dense(bits(q), bits(k), bits(v), lens, 0.09)
+    refd = ref_dense(bits(q), bits(k), bits(v), lens, 0.09)
     check_attention(out, lse, *refd, what="65528 units dense")
     assert ctx.device_status() == binding.SEER_OK
     # one more sequence takes the call over the limit: refused on the host, nothing launched

@@ -8,7 +8,7 @@ import torch
 
 import oracle
 from paper_2506_08889_b200 import binding, synth
-from util import bits, check_attention, to_paged
+from util import bits, check_attention, to_paged, ref_sparse_multi
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -71,11 +71,11 @@ def test_random_configuration(ctx, case):
         full = np.full((B, Hkv, max(max(n), 1)), -1, np.int32)
         for i in range(B):
             full[i, :, :n[i]] = np.arange(n[i])
-        ref = oracle.sparse_multi(bits(q), kh, vh, lens, full, None, b, scale)
+        ref = ref_sparse_multi(bits(q), kh, vh, lens, full, None, b, scale)
     else:
         cnt_t = torch.as_tensor(cnt, device=DEV) if c["use_cnt"] else None
         ctx.seer_sparse_decode_multi(shape, kv, q, T, torch.as_tensor(idx, device=DEV), cnt_t, max_sel, out, lse)
-        ref = oracle.sparse_multi(bits(q), kh, vh, lens, idx, cnt if c["use_cnt"] else None, b, scale)
+        ref = ref_sparse_multi(bits(q), kh, vh, lens, idx, cnt if c["use_cnt"] else None, b, scale)
     torch.cuda.synchronize()
     check_attention(out, lse, *ref, what=f"case {case}: {c}")
     assert ctx.device_status() == binding.SEER_OK

@@ -8,7 +8,7 @@ import torch
 
 import oracle
 from paper_2506_08889_b200 import binding, synth
-from util import bits, check_attention, make_qkv
+from util import bits, check_attention, make_qkv, ref_sparse_multi
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -98,7 +98,7 @@ def test_calls_of_different_shapes_interleaved_on_one_context(ctx):
         n = [-(-int(L) // b) for L in lens]
         keep = [max(1, x // 3) for x in n]
         idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max(keep), seed, shuffle=True)
-        ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
+        ref = ref_sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
         lens_t = torch.as_tensor(lens, device=DEV)
         cases.append(dict(shape=binding.make_shape(B, Hq, Hkv, 128, b, 0.09), kv=binding.make_kv(k, v, lens_t), q=q, T=T,
                           idx=torch.as_tensor(idx, device=DEV), cnt=torch.as_tensor(cnt, device=DEV), ref=ref,

@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from paper_2506_08889_b200 import binding, synth
-from util import bits, check_attention, make_qkv, to_paged
+from util import bits, check_attention, make_qkv, to_paged, ref_sparse, ref_dense, ref_sparse_multi, bf16_ulp
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -46,7 +46,7 @@ def test_sparse_small_blocks_ragged_shuffled_lists(ctx, b, g, Hkv):
     keep = [max(1, x // 3) for x in n]                  # counts that are not multiples of the blocks per tile
     max_sel = max(keep) + 3
     idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max_sel, 300 + b, shuffle=True)
-    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
+    ref = ref_sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
     out, lse = _sparse(ctx, q, k, v, lens, idx, cnt, b, 0.09)
     check_attention(out, lse, *ref, what=f"b={b} g={g}")
     out2, lse2 = _sparse(ctx, q, k, v, lens, idx, None, b, 0.09)          # -1 padding instead of counts
@@ -80,12 +80,12 @@ def test_small_blocks_full_selection_is_dense_and_bad_entries_are_flagged(ctx, b
     idx = np.full((B, Hkv, max(n) + 2), -1, np.int32)
     for i in range(B):
         idx[i, :, :n[i]] = np.arange(n[i])
-    refd = oracle.dense(bits(q), bits(k), bits(v), lens, 0.09)
+    refd = ref_dense(bits(q), bits(k), bits(v), lens, 0.09)
     out, lse = _sparse(ctx, q, k, v, lens, idx, None, b, 0.09)
     check_attention(out, lse, *refd, what=f"b={b} all blocks")
     assert ctx.device_status() == binding.SEER_OK
     idx[1, 0, 3] = n[1] + 5                                    # past the end: skipped and flagged
-    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, None, b, 0.09)
+    ref = ref_sparse(bits(q), bits(k), bits(v), lens, idx, None, b, 0.09)
     out, lse = _sparse(ctx, q, k, v, lens, idx, None, b, 0.09)
     check_attention(out, lse, *ref, what=f"b={b} bad entry")
     assert ctx.device_status() == binding.SEER_ERR_BAD_INDEX
@@ -102,7 +102,7 @@ def test_small_blocks_several_query_tokens(ctx, b, T):
     n = [-(-int(L) // b) for L in lens]
     keep = [max(2, x // 2) for x in n]
     idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max(keep) + 1, 360 + b, shuffle=True)
-    ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
+    ref = ref_sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.09)
     shape = binding.make_shape(B, Hq, Hkv, d, b, 0.09)
     lens_t = torch.as_tensor(lens, device=DEV)
     kv = binding.make_kv(k, v, lens_t)
@@ -142,7 +142,7 @@ def test_small_blocks_kcomp_gate_and_step(ctx, b):
     got = synth.bits_to_bf16(bits(kc)).to(torch.float64).numpy()
     for i in range(B):
         n_i = int(lens[i]) // b
-        tol = np.abs(kc_want[i, :, :n_i]) * 2.0 ** -7 + 1e-5 * np.abs(kc_want).max()
+        tol = bf16_ulp(kc_want[i, :, :n_i]) + 1e-5 * np.abs(kc_want).max()
         assert (np.abs(got[i, :, :n_i] - kc_want[i, :, :n_i]) <= tol).all()
         assert (got[i, :, n_i:] == 0).all()
     sc = torch.zeros((B, Hkv, nb), dtype=torch.float32, device=DEV)

@@ -10,7 +10,7 @@ import torch
 
 import oracle
 from paper_2506_08889_b200 import binding, synth
-from util import bits, check_attention, to_paged
+from util import bits, check_attention, to_paged, kc_tolerance
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -118,7 +118,7 @@ def test_qwen3_14b_shape_gate_then_decode(ctx):
     _, kc_want = oracle.kcomp(kh, bits(wk), b, 0, nb, nb, w.rope_theta)
     got_kc = bits(kc)
     got = synth.bits_to_bf16(got_kc).to(torch.float64).numpy()
-    tol = np.abs(kc_want) * 2.0 ** -7 + 1e-5 * np.abs(kc_want).max()
+    tol = kc_tolerance(kc_want)
     assert (np.abs(got - kc_want) <= tol).all()
     # stage 2: scores on the GPU's compressed keys
     want_sc, _ = oracle.scores(bits(qn), bits(wq), got_kc, [nb - 1] * B, [L - 1] * B, w.rope_theta)

@@ -243,6 +243,13 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.block_size = shape->block_size;
     p.tiles_per_block = tpb;
     p.blocks_per_tile = bpt;
+    p.bs_shift = shape->block_size == 16 ? 4 : shape->block_size == 32 ? 5 : shape->block_size == 64 ? 6 : 7;
+    p.tpb_shift = tpb == 2 ? 1 : 0;
+    p.bpt_shift = bpt == 4 ? 2 : bpt == 2 ? 1 : 0;
+    p.kvh_magic = shape->num_kv_heads == 1 ? 0u
+                                           : (unsigned int)((0x100000000ull + (unsigned long long)shape->num_kv_heads - 1) /
+                                                            (unsigned long long)shape->num_kv_heads);
+    p.group_magic = (65536 + group - 1) / group;
     p.num_units = U;
     p.max_blocks_cap = (kv->max_seq_len + kTileTokens - 1) / kTileTokens;
     p.pool_div = ctx->pool_div;

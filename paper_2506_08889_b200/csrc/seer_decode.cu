@@ -53,6 +53,7 @@ constexpr int kMaxPieces = 32;                             // partial pieces a C
 constexpr int kListInts = kStageBytes / 4 - 64;              // slot numbers that fit in one stage buffer (less 64 counts)
 constexpr int kLandBytes = 2 * kStageBytes;                 // landing area for staged partials: two stage buffers
 constexpr int kMaxSteals = 14;                             // chunks a CTA may take from other ranges
+constexpr int kSmemUnits = 128;                            // units whose tile-count prefix sums fit in shared memory
 constexpr int kMinChunk = 2;                               // smallest dynamic chunk, in tiles
 constexpr int kMinStaticTilesPerCta = 8;                   // below this everything is static
 constexpr int kBigFirstLen = 32;                           // ranges at least this long order their chunks big to small
@@ -67,15 +68,15 @@ struct StageMeta {
     int interval;      // interval this tile belongs to
 };
 
-// A partial this CTA wrote (unit, tiles, unit_first, unit_tiles, interval it went to); after the
-// counts are taken the same records list the units this CTA has to combine
+// A partial this CTA wrote (unit, tiles, first candidate slot of the unit, number of candidate slots,
+// tiles of the unit); after the stream the same records list the units this CTA has to combine
 // (unit, -, first_slot, n_slots, mask of valid slots or 0 if unknown).
 struct Piece {
     int unit, tiles, unit_first, unit_tiles, extra;
 };
 
-// Geometry of the intervals, identical in every CTA (derived from T and gridDim.x).  Range c is
-// [c*T/G, (c+1)*T/G); with len its length, b its end and ts = b - (len>>2) the start of its
+// Geometry of the intervals, identical in every CTA (derived from T and gridDim.x).  With range c
+// = [a, b), len its length, b its end and ts = b - (len>>2) the start of its
 // tail, its intervals are
 //   0: [a, ts)   1: [ts, ts + (len>>(R+1)))   2: [.., ts + (len>>R))  ...  R: [ts + (len>>3), b),
 // i.e. the tail's chunks double in size towards the end of the range.  Ranges of kBigFirstLen tiles or
@@ -85,6 +86,7 @@ struct Piece {
 struct Schedule {
     int T, G;                      // tiles, ranges (G <= T)
     int R;                         // dynamic chunks per range (0: everything is static)
+    int q, r;                      // T = q * G + r
 };
 
 struct __align__(1024) Smem {
@@ -98,6 +100,8 @@ struct __align__(1024) Smem {
     uint64_t list_bar;               // all consumer warps: the lists of valid slots are written
     uint64_t land_bar;               // bulk copies of partials into the landing area have arrived
     volatile int issued;             // tiles whose metadata the producer has written so far
+    volatile int first_unit;         // unit of the CTA's first tile (-1: none yet known, -2: not yet decided)
+    int upfx[kSmemUnits + 1];        // prefix sums of the units' tile counts (when there are at most kSmemUnits units)
     StageMeta meta[kStages];
     Schedule sched;
     Piece pieces[kMaxPieces];
@@ -109,23 +113,31 @@ struct __align__(1024) Smem {
 static_assert(sizeof(Smem) + 1024 <= 113 * 1024, "decode kernel no longer fits two CTAs per SM");
 
 #ifdef SEER_DECODE_TRACE
+// diagnostic builds: per CTA, slots 0..15 are named stamps, slots 16.. the arrival time of every tile
+constexpr int kTraceSlots = 128;
 __device__ __forceinline__ void trace_stamp(const DecodeParams& p, int slot) {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    p.trace[(size_t)blockIdx.x * 16 + slot] = t;
+    p.trace[(size_t)blockIdx.x * kTraceSlots + slot] = t;
 }
 #define SEER_STAMP(slot) trace_stamp(p, slot)
 #else
 #define SEER_STAMP(slot) ((void)0)
 #endif
 
+// Sequence of unit u (u / num_kv_heads by a multiplication: kvh_magic = ceil(2^32 / num_kv_heads), exact
+// for the 16-bit unit numbers the library takes; 0 stands for one KV head).
+__device__ __forceinline__ int unit_seq(const DecodeParams& p, int u) {
+    return p.kvh_magic ? (int)__umulhi((unsigned int)u, p.kvh_magic) : u;
+}
+
 template <bool SPARSE, bool SMALL = false>
 __device__ __forceinline__ int tiles_of(const DecodeParams& p, int u) {
-    const int L = p.seq_lens[u / p.num_kv_heads];
+    const int L = p.seq_lens[unit_seq(p, u)];
     if (SPARSE) {
         int c = p.block_cnt ? p.block_cnt[u] : p.max_sel;     // not behind the test on L: both loads in flight
         c = max(0, min(c, p.max_sel));
-        return L <= 0 ? 0 : (SMALL ? (c + p.blocks_per_tile - 1) / p.blocks_per_tile : c * p.tiles_per_block);
+        return L <= 0 ? 0 : (SMALL ? (c + p.blocks_per_tile - 1) >> p.bpt_shift : c << p.tpb_shift);
     } else {
         if (L <= 0) return 0;
         int t = (L + kTileTokens - 1) / kTileTokens;
@@ -133,18 +145,22 @@ __device__ __forceinline__ int tiles_of(const DecodeParams& p, int u) {
     }
 }
 
-// Range that owns tile t when T tiles are cut into G equal contiguous ranges
-// (range c = [floor(c*T/G), floor((c+1)*T/G)) ).
-__device__ __forceinline__ int range_of(long long t, long long T, long long G) {
-    return (int)(((t + 1) * G - 1) / T);
+// T tiles are cut into G contiguous ranges of q = T / G tiles, the first r = T % G of them one tile
+// longer: range c begins at c*q + min(c, r).
+__device__ __forceinline__ int range_begin(const Schedule& s, int c) { return c * s.q + min(c, s.r); }
+__device__ __forceinline__ int range_of(const Schedule& s, int t) {
+    const int long_part = s.r * (s.q + 1);
+    return t < long_part ? (int)((unsigned int)t / (unsigned int)(s.q + 1))
+                         : s.r + (int)((unsigned int)(t - long_part) / (unsigned int)s.q);
 }
-__device__ __forceinline__ int range_begin(const Schedule& s, int c) { return (int)(((long long)c * s.T) / s.G); }
 
-__device__ void build_schedule(Schedule& s, int T, int grid, int pool_div) {
+__device__ __forceinline__ void build_schedule(Schedule& s, int T, int grid, int pool_div) {
     s.T = T;
     s.G = max(1, min(grid, T));
+    s.q = (int)((unsigned int)T / (unsigned int)s.G);   // shortest range (>= 1 whenever T > 0)
+    s.r = T - s.q * s.G;
     s.R = 0;
-    const int len = T / s.G;                        // shortest range
+    const int len = s.q;
     if (pool_div > 0 && len >= kMinStaticTilesPerCta) {
         int R = 1;
         while (R < kMaxRounds && (len >> (R + 2)) >= kMinChunk) ++R;
@@ -169,7 +185,7 @@ __device__ __forceinline__ void interval_range(const Schedule& s, int c, int j, 
 
 // Number (c * (R+1) + j, increasing with the tile position) of the interval that holds tile t.
 __device__ __forceinline__ int interval_of(const Schedule& s, int t) {
-    const int c = range_of(t, s.T, s.G);
+    const int c = range_of(s, t);
     if (s.R == 0) return c;
     const int a = range_begin(s, c), b = range_begin(s, c + 1), len = b - a;
     const int off = t - (b - (len >> 2));           // position inside the tail
@@ -186,8 +202,8 @@ __device__ __forceinline__ int interval_of(const Schedule& s, int t) {
 // Output row of row r on a unit's MMA N side: query token t_base + r / group, head r % group of
 // the KV head's group; rows of q, out and lse are laid out [sequence][token][query head].
 __device__ __forceinline__ size_t unit_row(const DecodeParams& p, int u, int r) {
-    const int i = u / p.num_kv_heads, h = u % p.num_kv_heads;
-    const int tl = r / p.group, gi = r - tl * p.group;
+    const int i = unit_seq(p, u), h = u - i * p.num_kv_heads;
+    const int tl = (r * p.group_magic) >> 16, gi = r - tl * p.group;      // r / group for r < 16
     return ((size_t)i * p.q_len + p.t_base + tl) * p.num_q_heads + (size_t)h * p.group + gi;
 }
 
@@ -224,8 +240,8 @@ __device__ __forceinline__ void merge_init(MergeState<NT>& st) {
 // cheapest way for a few partials).
 constexpr int kDirect = 8;
 template <int NT>
-__device__ __forceinline__ void merge_accumulate_direct(const DecodeParams& p, MergeState<NT>& st, const int* slots,
-                                                        int n, int t) {
+__device__ __forceinline__ void merge_accumulate_direct(const DecodeParams& p, MergeState<NT>& st,
+                                                        const int (&slots)[kDirect], int n, int t) {
     const int d0 = 8 * (t & 15);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -234,7 +250,7 @@ __device__ __forceinline__ void merge_accumulate_direct(const DecodeParams& p, M
         float4 va[kDirect], vb[kDirect];
 #pragma unroll
         for (int k = 0; k < kDirect; ++k) {
-            const size_t sl = (size_t)slots[min(k, n - 1)];
+            const size_t sl = (size_t)slots[k];            // (entries from n on repeat a valid slot)
             const float* pm = p.part_ml + sl * (kMlStride * NT);
             const float4* qo = reinterpret_cast<const float4*>(p.part_o + sl * (8 * NT * kHeadDim) + hh * kHeadDim + d0);
             ms[k] = __ldcg(pm + hh);
@@ -363,6 +379,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         mbar_init(&sm.land_bar, 1);
         mbar_fence_init();
         sm.issued = 0;
+        sm.first_unit = -2;
         sm.pieces_n = 0;
     }
     if (warp == kConsumerWarps && lane == 0) {
@@ -370,6 +387,13 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         tma_prefetch_desc(&map_v);
     }
 
+#ifdef SEER_DECODE_TRACE
+    if (tid == 0) {
+        unsigned int smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        p.trace[(size_t)blockIdx.x * kTraceSlots + 15] = smid;
+    }
+#endif
     if (tid == 0) SEER_STAMP(8);
     __syncthreads();                                 // barriers initialised
     pdl_wait();
@@ -378,13 +402,18 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (warp == kConsumerWarps) {
         // =========================== producer warp ====================================
         // The warp first sums the units' tile counts by itself (the consumer warps do not need the
-        // result to start waiting), derives the schedule and finds where its static share starts.
+        // result to start waiting) and derives the schedule.  The prefix sums of the counts, by which
+        // the unit that holds a given tile is found, stay in shared memory for up to kSmemUnits units
+        // and go through global memory beyond that.
         const int per = (U + 31) / 32;
         const int u_lo = min(U, lane * per), u_hi = min(U, u_lo + per);
+        const bool smem_pfx = U <= kSmemUnits;
         int mine = 0;
+#pragma unroll 1
         for (int u = u_lo; u < u_hi; ++u) {
             const int t = tiles_of<SPARSE, SMALL>(p, u);
-            if (t == 0 && cta == 0) write_zero_unit(p, u);   // units without work: zeros, -inf
+            if (t == 0 && cta == 0) write_zero_unit(p, u);       // units without work: zeros, -inf
+            if (smem_pfx) sm.upfx[u + 1] = t;                      // (the count for now)
             mine += t;
         }
         int incl = mine;
@@ -394,54 +423,90 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             if (lane >= o) incl += v;
         }
         const int T = __shfl_sync(0xffffffffu, incl, 31);
+        if (lane == 0) SEER_STAMP(11);
         Schedule sc;
         build_schedule(sc, T, gridDim.x, p.pool_div);
         if (lane == 0) sm.sched = sc;                    // the consumers use it when a piece ends
-        int t_begin = 0, t_end = 0;                      // this CTA's static share
-        if (T > 0 && cta < sc.G) interval_range(sc, cta, 0, &t_begin, &t_end);
-        // prefix sums of the tile counts, for locating a tile's unit later (every CTA writes the
-        // same values; a CTA only relies on its own writes), and the unit holding tile t_begin
-        int my_start_u = -1, my_start_off = 0;
+        const int R = sc.R, G = sc.G;
         {
             int acc = incl - mine;
-            for (int u = u_lo; u < u_hi; ++u) {
-                const int t = tiles_of<SPARSE, SMALL>(p, u);
-                if (sc.R > 0) p.prefix[u] = acc;
-                if (t_begin < t_end && t > 0 && acc <= t_begin && t_begin < acc + t) {
-                    my_start_u = u;
-                    my_start_off = t_begin - acc;
-                }
-                acc += t;
+            if (smem_pfx) {
+                if (lane == 0) sm.upfx[0] = 0;
+#pragma unroll 1
+                for (int u = u_lo; u < u_hi; ++u) { acc += sm.upfx[u + 1]; sm.upfx[u + 1] = acc; }
+            } else if (R > 0) {
+                // (every CTA writes the same values; a CTA only relies on its own writes)
+#pragma unroll 1
+                for (int u = u_lo; u < u_hi; ++u) { p.prefix[u] = acc; acc += tiles_of<SPARSE, SMALL>(p, u); }
+                if (lane == 0) p.prefix[U] = T;
             }
-            if (sc.R > 0 && lane == 0) p.prefix[U] = T;
+            __syncwarp();
         }
-        __syncwarp();
-        // position in the units' tile lists: unit cu, whose first tile is global tile cpu and
-        // which has cut tiles
+        // Unit cu that holds global tile t, with the global index cpu of its first tile and its tile
+        // count cut.  false: no unit holds it (the counts changed under us).
         int cu = 0, cpu = 0, cut = 0;
-        {
-            const unsigned m = __ballot_sync(0xffffffffu, my_start_u >= 0);
-            if (m) {
-                const int src = __ffs(m) - 1;
-                cu = __shfl_sync(0xffffffffu, my_start_u, src);
-                cpu = t_begin - __shfl_sync(0xffffffffu, my_start_off, src);
-                cut = tiles_of<SPARSE, SMALL>(p, cu);
+        auto locate = [&](int t, bool first) -> bool {
+            int f_u = -1, f_p = 0, f_t = 0;
+            if (smem_pfx) {
+#pragma unroll 1
+                for (int u = u_lo; u < u_hi; ++u) {
+                    const int lo = sm.upfx[u], hi = sm.upfx[u + 1];
+                    if (lo <= t && t < hi) { f_u = u; f_p = lo; f_t = hi - lo; }
+                }
+            } else if (first) {
+                int acc = incl - mine;
+#pragma unroll 1
+                for (int u = u_lo; u < u_hi; ++u) {
+                    const int n = tiles_of<SPARSE, SMALL>(p, u);
+                    if (acc <= t && t < acc + n) { f_u = u; f_p = acc; f_t = n; }
+                    acc += n;
+                }
             } else {
-                t_end = t_begin;                         // (no static share)
+                // 32-ary search in the prefix sums
+                int lo = 0, hi = U;                       // prefix[lo] <= t < prefix[hi]
+                while (hi - lo > 1) {
+                    const int step = (hi - lo + 31) / 32;
+                    const int cand = lo + min((lane + 1) * step, hi - lo);
+                    const int pv = cand < hi ? __ldcg(p.prefix + cand) : 0x7fffffff;
+                    const unsigned m = __ballot_sync(0xffffffffu, pv > t);
+                    const int f = __ffs(m) - 1;             // the last lane always votes yes
+                    const int new_hi = __shfl_sync(0xffffffffu, cand, f);
+                    const int new_lo = f == 0 ? lo : __shfl_sync(0xffffffffu, cand, f - 1);
+                    hi = new_hi;
+                    lo = new_lo;
+                }
+                f_p = __ldcg(p.prefix + lo);
+                f_t = __ldcg(p.prefix + lo + 1) - f_p;
+                f_u = (t >= f_p && t < f_p + f_t) ? lo : -1;
             }
-        }
+            const unsigned m = __ballot_sync(0xffffffffu, f_u >= 0);
+            if (!m) return false;
+            const int src = __ffs(m) - 1;
+            cu = __shfl_sync(0xffffffffu, f_u, src);
+            cpu = __shfl_sync(0xffffffffu, f_p, src);
+            cut = __shfl_sync(0xffffffffu, f_t, src);
+            return true;
+        };
         int it = 0;
-        int iv_begin = t_begin, iv_end = t_end, iv_id = cta * (sc.R + 1);
-        bool have = t_begin < t_end;
-        bool own = cta < sc.G;           // still claiming chunks of the own range
-        bool contiguous = true;          // the next interval continues the previous one
+        int iv_begin = 0, iv_end = 0, iv_id = 0;
+        bool first = true;               // the static share has not been taken yet
+        bool own = cta < G;              // still claiming chunks of the own range
+        bool contiguous = false;         // the next interval continues the previous one
         int fails = 0, steals = 0;
-        const int R = sc.R, G = sc.G;
         for (;;) {
-            if (!have) {
-                if (R == 0 || T == 0) break;
+            {
                 int c, j;
-                if (own) {
+                if (first) {
+                    // the static share: the head of the own range
+                    if (T == 0 || cta >= G) {
+                        if (lane == 0) sm.first_unit = -1;
+                        break;
+                    }
+                    c = cta;
+                    j = 0;
+                } else if (R == 0) {
+                    break;
+                } else if (own) {
                     // own range, from the front: low half of the counter counts front claims
                     int old = 0;
                     if (lane == 0) old = atomicAdd(&p.steal[cta], 1);
@@ -455,14 +520,25 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     // and go for the one with the most chunks left (its owner is the furthest
                     // behind); ties are broken differently by every thief.
                     if (fails >= 3 || steals >= kMaxSteals) break;
+                    // (all of a lane's counters are requested before any is looked at: one round trip)
                     int best = -1;
-                    for (int c0 = 0; c0 < G; c0 += 32) {
-                        const int cc = c0 + lane;
-                        if (cc < G && cc != cta) {
-                            const int st = __ldcg(p.steal + cc);
-                            const int left = R - (st & 0xffff) - (st >> 16);
-                            if (left > 0) {
-                                const int rot = (cc - cta + G) % G;          // this thief's order of preference
+                    // (a range's last chunk is left to its owner: by the time a thief's loads came
+                    // back the owner would have been there)
+                    const int min_left = min(2, R);
+                    constexpr int kScan = 10;                 // counters per lane and round: 320 ranges a round
+                    for (int c0 = 0; c0 < G; c0 += 32 * kScan) {
+                        int st[kScan];
+#pragma unroll
+                        for (int k = 0; k < kScan; ++k) {
+                            const int cc = c0 + 32 * k + lane;
+                            st[k] = cc < G ? __ldcg(p.steal + cc) : (R << 16);
+                        }
+#pragma unroll
+                        for (int k = 0; k < kScan; ++k) {
+                            const int cc = c0 + 32 * k + lane;
+                            const int left = R - (st[k] & 0xffff) - (st[k] >> 16);
+                            if (cc < G && cc != cta && left >= min_left) {
+                                const int rot = cc - cta + (cc < cta ? G : 0);   // this thief's order of preference
                                 best = max(best, (left << 20) | (0xfffff - min(rot, 0xfffff)));
                             }
                         }
@@ -470,7 +546,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 #pragma unroll
                     for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
                     if (best < 0) break;                                  // nothing left anywhere
-                    c = (cta + (0xfffff - (best & 0xfffff))) % G;
+                    c = cta + (0xfffff - (best & 0xfffff));
+                    if (c >= G) c -= G;
                     int old = 0;
                     if (lane == 0) old = atomicAdd(&p.steal[c], 1 << 16);
                     old = __shfl_sync(0xffffffffu, old, 0);
@@ -483,27 +560,19 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 interval_range(sc, c, j, &iv_begin, &iv_end);
                 iv_id = c * (R + 1) + j;
                 if (!contiguous) {
-                    // unit that holds tile iv_begin: 32-ary search in the prefix sums
-                    int lo = 0, hi = U;                       // prefix[lo] <= iv_begin < prefix[hi]
-                    while (hi - lo > 1) {
-                        const int step = (hi - lo + 31) / 32;
-                        const int cand = lo + min((lane + 1) * step, hi - lo);
-                        const int pv = cand < hi ? __ldcg(p.prefix + cand) : 0x7fffffff;
-                        const unsigned m = __ballot_sync(0xffffffffu, pv > iv_begin);
-                        const int f = __ffs(m) - 1;             // the last lane always votes yes
-                        const int new_hi = __shfl_sync(0xffffffffu, cand, f);
-                        const int new_lo = f == 0 ? lo : __shfl_sync(0xffffffffu, cand, f - 1);
-                        hi = new_hi;
-                        lo = new_lo;
+                    const bool found = iv_begin < iv_end && locate(iv_begin, first);
+                    if (first) {
+                        // the consumers request this unit's queries now, ahead of the tile loads that
+                        // are about to fill the memory system's queues
+                        if (lane == 0) { sm.first_unit = found ? cu : -1; SEER_STAMP(12); }
+                        first = false;
+                        if (!found) break;
+                    } else if (!found) {
+                        break;                                // counts changed under us
                     }
-                    cu = lo;
-                    cpu = __ldcg(p.prefix + lo);
-                    cut = __ldcg(p.prefix + lo + 1) - cpu;
-                    if (iv_begin < cpu || iv_begin >= cpu + cut) break;   // counts changed under us
                 }
             }
-            const bool fresh = have || !contiguous;  // this interval starts a new piece
-            have = false;
+            const bool fresh = !contiguous;          // this interval starts a new piece
             int ce = iv_begin - cpu;                  // offset of the next tile inside unit cu
             const int n_tiles = iv_end - iv_begin;
             for (int t = 0; t < n_tiles; t += 32) {
@@ -533,12 +602,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 int nvalid = 0, head = 0, flags = 0;
                 int row[4] = {0, 0, 0, 0}, outer[4] = {0, 0, 0, 0};
                 if (my_u >= 0) {
-                    const int i = my_u / p.num_kv_heads;
-                    head = my_u % p.num_kv_heads;
+                    const int i = unit_seq(p, my_u);
+                    head = my_u - i * p.num_kv_heads;
                     const int L = p.seq_lens[i];
                     if (SMALL) {
                         // a tile gathers the next bpt listed blocks of the unit
-                        const int n_i = (L + p.block_size - 1) / p.block_size;
+                        const int n_i = (L + p.block_size - 1) >> p.bs_shift;
                         int cnt_u = p.block_cnt ? p.block_cnt[my_u] : p.max_sel;
                         cnt_u = max(0, min(cnt_u, p.max_sel));
 #pragma unroll
@@ -569,11 +638,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     } else {
                         int tok0 = 0;
                         if (SPARSE) {
-                            const int blk = p.block_idx[(size_t)my_u * p.max_sel + my_e / p.tiles_per_block];
-                            const int n_i = (L + p.block_size - 1) / p.block_size;
+                            const int blk = p.block_idx[(size_t)my_u * p.max_sel + (my_e >> p.tpb_shift)];
+                            const int n_i = (L + p.block_size - 1) >> p.bs_shift;
                             if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
                             if (blk >= 0 && blk < n_i) {
-                                tok0 = blk * p.block_size + (my_e % p.tiles_per_block) * kTileTokens;
+                                tok0 = (blk << p.bs_shift) + (my_e & (p.tiles_per_block - 1)) * kTileTokens;
                                 nvalid = max(0, min(kTileTokens + 7, L - tok0));
                             }
                         } else {
@@ -617,6 +686,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     }
                     if (lane == 0) {
                         const int st = it % kStages;
+#ifdef SEER_DECODE_TRACE
+                        if (it == 0) SEER_STAMP(13);
+                        if (it == 1) SEER_STAMP(14);
+#endif
                         if (!mbar_wait(&sm.empty[st], ((it / kStages) & 1) ^ 1, p.status)) return;
                         sm.meta[st] = StageMeta{s_nvalid, s_u, s_flags, s_pu, s_ut, iv_id};
                         __threadfence_block();
@@ -654,8 +727,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 }
             }
         }
-#ifdef SEER_DECODE_TRACE
-#endif
         if (lane == 0) {
             // end-of-stream marker for the consumers
             const int st = it % kStages;
@@ -684,6 +755,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     float o[NT][8][4];                  // O^T accumulators: 8 m-tiles over d per N-tile
     float m_run[NT][2], l_run[NT][2];
     int seg = 0;                        // merge rounds finished so far (NT per piece)
+    unsigned long long tk_before = 0ull; // warp 0, lane k: what the unit's counter held before the k-th held piece was added
+    unsigned int tk_bit = 0u;            // ... and that piece's bit
     int piece_tiles = 0, piece_iv = 0;  // tiles in the current piece, interval it started in
     // Query token of this thread's two columns in every N-tile, as the number of newest cached
     // tokens it may not see (q_len - 1 - token): column c of N-tile nt is row 8*nt + c of the unit,
@@ -694,7 +767,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
             const int r = 8 * nt + 2 * qd + c;
-            back[nt][c] = r < p.rows ? p.q_len - 1 - (p.t_base + r / p.group) : 0;
+            back[nt][c] = r < p.rows ? p.q_len - 1 - (p.t_base + ((r * p.group_magic) >> 16)) : 0;
         }
     // B fragment of N-tile nt: this thread supplies row 8*nt + rw of the unit's queries
     auto load_q = [&](uint32_t (&dst)[8][2], int unit, int nt) {
@@ -709,14 +782,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     };
     int pre_unit = -1;
     if (NT == 1) {
-        // the first tile's unit is known as soon as the producer has issued it, well before its data
-        // lands: request that unit's queries in the meantime
-        for (int spin = 0; spin < (1 << 22) && sm.issued < 1; ++spin) __nanosleep(32);
-        __threadfence_block();
-        if (sm.issued >= 1) {
-            const int u0 = *reinterpret_cast<volatile int*>(&sm.meta[0].unit);
-            if (u0 >= 0) { load_q(bq_pre, u0, 0); pre_unit = u0; }
-        }
+        // the first tile's unit is known as soon as the producer has found where its share starts,
+        // well before the first tile is even requested: ask for that unit's queries at once
+        for (int spin = 0; spin < (1 << 22) && sm.first_unit == -2; ++spin) __nanosleep(20);
+        const int u0 = sm.first_unit;
+        if (u0 >= 0) { load_q(bq_pre, u0, 0); pre_unit = u0; }
     }
 
     // lane-constant parts of the ldmatrix addresses (swizzle: 16-B chunk ^= row & 7)
@@ -735,6 +805,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     StageMeta mt = sm.meta[0];
     for (int it = 0; mt.nvalid >= 0; ++it) {
         const int st = it % kStages;
+#ifdef SEER_DECODE_TRACE
+        if (tid == 0 && it < kTraceSlots - 16) SEER_STAMP(16 + it);
+#endif
         if (NT == 1) {
             // look ahead: request the queries of the next unit as soon as the producer has issued a
             // tile of it (its metadata is stable from then until we release that stage)
@@ -966,8 +1039,24 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     }
                     if (lane == 0) {
                         pm[16 * NT] = __uint_as_float(p.generation);
-                        sm.pieces[n_held] = Piece{u, piece_tiles, mt.unit_first, mt.unit_tiles, piece_iv};
                         sm.pieces_n = n_held + 1;
+                    }
+                    // Make the piece count at once (not at the end of the stream, which may be far off
+                    // when this CTA goes on to take other ranges' chunks): the partial is made visible,
+                    // then one 64-bit add on the unit's counter -- high half: tiles done; low half: one
+                    // bit per piece, its slot's place among the unit's candidate slots, when there are at
+                    // most 32 of those.  Lane k makes the add for the k-th piece held and keeps the
+                    // answer in a register until the stream is over; nothing waits for it here.
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == n_held) {
+                        const int iv_first = interval_of(sm.sched, mt.unit_first);
+                        const int iv_last = interval_of(sm.sched, mt.unit_first + mt.unit_tiles - 1);
+                        const int n_slots = iv_last - iv_first + 1;
+                        const unsigned int bit = n_slots <= 32 ? 1u << (piece_iv - iv_first) : 0u;
+                        sm.pieces[n_held] = Piece{u, piece_tiles, iv_first + u, n_slots, mt.unit_tiles};
+                        tk_bit = bit;
+                        tk_before = atomicAdd(&p.tickets[u], ((unsigned long long)piece_tiles << 32) | bit);
                     }
                     __syncwarp();
                 } else if (piece_tiles >= mt.unit_tiles) {
@@ -1013,30 +1102,19 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (tid == 0) SEER_STAMP(6);
     if (w == 0) {
         const int n_held = sm.pieces_n;
-#ifdef SEER_DECODE_TRACE
-#endif
-        __threadfence();                               // the partials above are visible from here on
-        __syncwarp();
+        // Every piece was added to its unit's counter when it ended.  Whoever completed a unit's tile
+        // count learns from the same word which slots hold the unit's partials.
         if (lane == 0) SEER_STAMP(0);
-        // One 64-bit add per piece on its unit's counter: the high half counts tiles, the low half
-        // collects one bit per piece (its slot's place among the unit's candidate slots, when there
-        // are at most 32 of those).  Whoever completes the tile count learns from the same word
-        // which slots hold the unit's partials.
         bool owe = false;
         Piece pc = Piece{0, 0, 0, 0, 0};
         int first_slot = 0, n_slots = 0;
         unsigned int mask = 0u;
         if (lane < n_held) {
-            pc = sm.pieces[lane];
-            const int iv_first = interval_of(sm.sched, pc.unit_first);
-            const int iv_last = interval_of(sm.sched, pc.unit_first + pc.unit_tiles - 1);
-            first_slot = iv_first + pc.unit;
-            n_slots = iv_last - iv_first + 1;
-            const unsigned int bit = n_slots <= 32 ? 1u << (pc.extra - iv_first) : 0u;
-            const unsigned long long before =
-                atomicAdd(&p.tickets[pc.unit], ((unsigned long long)pc.tiles << 32) | bit);
-            owe = (int)(before >> 32) + pc.tiles == pc.unit_tiles;     // this piece completed the unit's count
-            mask = (unsigned int)before | bit;
+            pc = sm.pieces[lane];                      // (unit, tiles, first slot, slots, tiles of the unit)
+            first_slot = pc.unit_first;
+            n_slots = pc.unit_tiles;
+            owe = (int)(tk_before >> 32) + pc.tiles == pc.extra;     // this piece completed the unit's count
+            mask = (unsigned int)tk_before | tk_bit;
         }
         // rewrite the list: the units this CTA has to combine, with their candidate slots
         const unsigned m = __ballot_sync(0xffffffffu, owe);
@@ -1057,15 +1135,18 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         return;
     }
 #ifdef SEER_DECODE_TRACE
-    if (tid == 0 && n_owed > 0) { SEER_STAMP(2); p.trace[(size_t)blockIdx.x * 16 + 4] = n_owed; }
+    if (tid == 0 && n_owed > 0) { SEER_STAMP(2); p.trace[(size_t)blockIdx.x * kTraceSlots + 4] = n_owed; }
 #endif
-    // The combines use the stage buffers as scratch (the stream is over, nothing is in flight).  The
-    // slots that really hold a partial of a unit are found by looking at the generation stamps of
-    // the unit's candidate slots (lists, in the third stage buffer); the partials themselves are
-    // brought in by bulk copies, kLand at a time, into the first two stage buffers, and added up.
-    int* lists = reinterpret_cast<int*>(sm.stage[2]);            // kListInts slot numbers
-    int* counts = lists + kListInts;                             // per owed unit (or per warp)
-    // only the unit's real rows are brought in: rows x 512 B + 128 B * NT per partial, one per lane
+    // The combines use the stage buffers as scratch (the stream is over, nothing is in flight).  Which
+    // of a unit's candidate slots hold a partial of this launch is known from the start when the split
+    // is static (all of them) or the unit has at most 32 candidates (the ticket word said which);
+    // otherwise the four warps look at the generation stamps of a quarter of the candidates each and
+    // list the valid ones in the third stage buffer.  Up to 2 * kDirect partials are added straight
+    // from global memory; more are brought in by bulk copies, n_land at a time, into the first two
+    // stage buffers (only the unit's real rows: rows x 512 B + 128 B * NT per partial, one per lane).
+    constexpr int kSeg = kListInts / kConsumerWarps;             // slot numbers a warp can list per window
+    int* lists = reinterpret_cast<int*>(sm.stage[2]);            // [4][kSeg] slot numbers
+    int* counts = lists + kListInts;                             // [4]
     constexpr int kMl = kMlStride * NT;                          // floats per (max, sum, stamp) record
     const int o_stride = p.rows * kHeadDim;                      // floats per staged partial
     const int n_land = min(32, kLandBytes / (o_stride * 4 + kMl * 4));
@@ -1079,97 +1160,84 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         ++sync_phase;
         return ok;
     };
-    // stage the n listed partials, kLand per round, and add them to ms (all consumer threads call)
-    auto accumulate_list = [&](MergeState<NT>& ms, const int* slots, int n) -> bool {
-        if (n > 0 && n <= 2 * kDirect) {
-            // up to two rounds of direct loads beat staging (one round trip each, no barrier)
-            merge_accumulate_direct<NT>(p, ms, slots, min(n, kDirect), tid);
-            if (n > kDirect) merge_accumulate_direct<NT>(p, ms, slots + kDirect, n - kDirect, tid);
-            return true;
-        }
-        for (int s0 = 0; s0 < n; s0 += n_land) {
-            const int m = min(n_land, n - s0);
-            if (w == 0) {
-                // warp 0 issues the copies, one partial per lane
-                if (lane == 0) {
-                    fence_proxy_async_smem();        // earlier plain accesses to the landing area are done
-                    mbar_arrive_expect_tx(&sm.land_bar, (uint32_t)m * (o_stride * 4 + kMl * 4));
-                }
-                __syncwarp();
-                if (lane < m) {
-                    const size_t sl = (size_t)slots[s0 + lane];
-                    bulk_load(land_o + lane * o_stride, p.part_o + sl * (8 * NT * kHeadDim), o_stride * 4, &sm.land_bar);
-                    bulk_load(land_ml + lane * kMl, p.part_ml + sl * kMl, kMl * 4, &sm.land_bar);
-                }
-            }
-            if (!mbar_wait(&sm.land_bar, land_phase & 1, p.status)) return false;
-#ifdef SEER_DECODE_TRACE
-            if (tid == 0 && land_phase == 0) SEER_STAMP(5);
-#endif
-            ++land_phase;
-            merge_accumulate_staged<NT>(ms, land_o, o_stride, land_ml, m, p.rows, tid);
-            if (!sync_consumers()) return false;     // everybody has read the landing area
-#ifdef SEER_DECODE_TRACE
-            if (tid == 0 && land_phase == 1) SEER_STAMP(1);
-#endif
-        }
-        return true;
-    };
-    int total_cand = 0;
-    for (int e = 0; e < n_owed; ++e) total_cand += sm.pieces[e].unit_tiles;
-    if (total_cand <= kListInts) {
-        // usual case: every owed unit's candidates fit at once; warp e%4 lists unit e's valid slots.
-        // With a static split every candidate slot holds a partial; with at most 32 candidates the
-        // ticket word said which ones do; otherwise the generation stamps are looked at.
-        int base = 0;
-        for (int e = 0; e < n_owed; ++e) {
-            if ((e & (kConsumerWarps - 1)) == w) {
-                const int first = sm.pieces[e].unit_first, n_slots = sm.pieces[e].unit_tiles;
-                int n;
-                if (sm.sched.R == 0) {
-                    for (int x = lane; x < n_slots; x += 32) lists[base + x] = first + x;
-                    n = n_slots;
-                } else if (n_slots <= 32) {
-                    const unsigned int mk = (unsigned int)sm.pieces[e].extra;
-                    if ((mk >> lane) & 1u) lists[base + __popc(mk & ((1u << lane) - 1u))] = first + lane;
-                    n = __popc(mk);
-                } else {
-                    n = scan_valid_slots<NT>(p, first, n_slots, lists + base, lane);
-                }
-                if (lane == 0) counts[e] = n;
-            }
-            base += sm.pieces[e].unit_tiles;
-        }
-        if (!sync_consumers()) return;
-#ifdef SEER_DECODE_TRACE
-        if (tid == 0 && n_owed > 0) { SEER_STAMP(3); p.trace[(size_t)blockIdx.x * 16 + 4] = n_owed * 1000 + counts[0]; }
-#endif
-        base = 0;
-        for (int e = 0; e < n_owed; ++e) {
-            MergeState<NT> ms;
-            merge_init(ms);
-            if (!accumulate_list(ms, lists + base, counts[e])) return;
-            merge_finalize(p, ms, sm.pieces[e].unit, tid);
-            base += sm.pieces[e].unit_tiles;
-        }
-    } else {
-        // a unit cut into thousands of pieces: go through its candidates in windows
-        constexpr int kWin = kListInts / kConsumerWarps;
-        for (int e = 0; e < n_owed; ++e) {
-            MergeState<NT> ms;
-            merge_init(ms);
-            const int first = sm.pieces[e].unit_first, n_slots = sm.pieces[e].unit_tiles;
-            for (int w0 = 0; w0 < n_slots; w0 += kListInts) {
-                const int lo = w0 + w * kWin, hi = min(n_slots, min(w0 + kListInts, lo + kWin));
-                const int n = lo < hi ? scan_valid_slots<NT>(p, first + lo, hi - lo, lists + w * kWin, lane) : 0;
+    const bool all_valid = sm.sched.R == 0;
+    bool lists_in_use = false;
+#pragma unroll 1
+    for (int e = 0; e < n_owed; ++e) {
+        const int unit = sm.pieces[e].unit, first = sm.pieces[e].unit_first, n_slots = sm.pieces[e].unit_tiles;
+        const unsigned int mask = (unsigned int)sm.pieces[e].extra;
+        const bool by_mask = !all_valid && n_slots <= 32;
+        MergeState<NT> ms;
+        merge_init(ms);
+#pragma unroll 1
+        for (int w0 = 0; w0 < n_slots; w0 += kListInts) {
+            const int win = min(kListInts, n_slots - w0);
+            const bool listed = !all_valid && !by_mask;
+            if (listed) {
+                if (lists_in_use && !sync_consumers()) return;   // everybody is done with the previous lists
+                lists_in_use = true;
+                const int lo = w * kSeg, hi = min(win, lo + kSeg);
+                const int n = lo < hi ? scan_valid_slots<NT>(p, first + w0 + lo, hi - lo, lists + lo, lane) : 0;
                 if (lane == 0) counts[w] = n;
                 if (!sync_consumers()) return;
-                for (int ww = 0; ww < kConsumerWarps; ++ww)
-                    if (!accumulate_list(ms, lists + ww * kWin, counts[ww])) return;
-                if (!sync_consumers()) return;
             }
-            merge_finalize(p, ms, sm.pieces[e].unit, tid);
+#pragma unroll 1
+            for (int seg = 0; seg < (listed ? kConsumerWarps : 1); ++seg) {
+                const int n = all_valid ? win : by_mask ? __popc(mask) : counts[seg];
+                const int* seg_list = lists + seg * kSeg;
+                if (n <= 2 * kDirect) {
+                    // up to two rounds of direct loads beat staging (one round trip each, no barrier)
+                    unsigned int rem = mask;                 // bits of the valid slots not yet taken
+#pragma unroll 1
+                    for (int k0 = 0; k0 < n; k0 += kDirect) {
+                        const int m = min(kDirect, n - k0);
+                        int sl[kDirect];
+#pragma unroll
+                        for (int k = 0; k < kDirect; ++k) {
+                            const int kk = k0 + min(k, m - 1);
+                            if (by_mask) {
+                                sl[k] = first + __ffs(rem) - 1;
+                                if (k < m - 1) rem &= rem - 1;
+                            } else {
+                                sl[k] = all_valid ? first + w0 + kk : seg_list[kk];
+                            }
+                        }
+                        if (by_mask) rem &= rem - 1;
+                        merge_accumulate_direct<NT>(p, ms, sl, m, tid);
+                    }
+                    continue;
+                }
+                // the k-th valid slot of this segment
+                auto slot_at = [&](int k) -> int {
+                    return all_valid ? first + w0 + k : by_mask ? first + (int)__fns(mask, 0u, k + 1) : seg_list[k];
+                };
+#pragma unroll 1
+                for (int s0 = 0; s0 < n; s0 += n_land) {
+                    const int m = min(n_land, n - s0);
+                    if (w == 0) {
+                        // warp 0 issues the copies, one partial per lane
+                        if (lane == 0) {
+                            fence_proxy_async_smem();        // earlier plain accesses to the landing area are done
+                            mbar_arrive_expect_tx(&sm.land_bar, (uint32_t)m * (o_stride * 4 + kMl * 4));
+                        }
+                        __syncwarp();
+                        if (lane < m) {
+                            const size_t sl = (size_t)slot_at(s0 + lane);
+                            bulk_load(land_o + lane * o_stride, p.part_o + sl * (8 * NT * kHeadDim), o_stride * 4, &sm.land_bar);
+                            bulk_load(land_ml + lane * kMl, p.part_ml + sl * kMl, kMl * 4, &sm.land_bar);
+                        }
+                    }
+                    if (!mbar_wait(&sm.land_bar, land_phase & 1, p.status)) return;
+#ifdef SEER_DECODE_TRACE
+                    if (tid == 0 && land_phase == 0) SEER_STAMP(5);
+#endif
+                    ++land_phase;
+                    merge_accumulate_staged<NT>(ms, land_o, o_stride, land_ml, m, p.rows, tid);
+                    if (!sync_consumers()) return;           // everybody has read the landing area
+                }
+            }
         }
+        merge_finalize(p, ms, unit, tid);
     }
     if (tid == 0) SEER_STAMP(7);
 }

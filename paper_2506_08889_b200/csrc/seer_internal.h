@@ -56,6 +56,9 @@ struct DecodeParams {
     int num_pages;
     int batch, num_q_heads, num_kv_heads, group, block_size, tiles_per_block;
     int blocks_per_tile;            // 64 / block_size for blocks of 16 or 32 tokens (a tile gathers several listed blocks), else 1
+    int bs_shift, tpb_shift, bpt_shift;   // log2 of block_size, tiles_per_block, blocks_per_tile
+    unsigned int kvh_magic;         // ceil(2^32 / num_kv_heads), 0 for one KV head: unit / num_kv_heads by __umulhi
+    int group_magic;                // ceil(2^16 / group): r / group = (r * group_magic) >> 16 for r < 16
     int q_len;                      // query tokens per sequence (the last q_len cached tokens), 1 for plain decoding
     int t_base, t_cnt;              // this launch handles query tokens t_base .. t_base + t_cnt - 1
     int rows;                       // t_cnt * group: rows on the MMA N side, <= 8 * (N-tiles of the kernel)

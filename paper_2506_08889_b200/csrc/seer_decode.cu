@@ -53,10 +53,11 @@ constexpr int kMaxPieces = 32;                             // partial pieces a C
 constexpr int kListInts = kStageBytes / 4 - 64;              // slot numbers that fit in one stage buffer (less 64 counts)
 constexpr int kLandBytes = 2 * kStageBytes;                 // landing area for staged partials: two stage buffers
 constexpr int kMaxSteals = 14;                             // chunks a CTA may take from other ranges
+constexpr int kAheadMaxChunk = 8;                          // own chunks up to this size are claimed ahead
+constexpr int kAheadTiles = 3;                             // tiles left to issue when the next interval's claim is made
 constexpr int kSmemUnits = 128;                            // units whose tile-count prefix sums fit in shared memory
 constexpr int kMinChunk = 2;                               // smallest dynamic chunk, in tiles
 constexpr int kMinStaticTilesPerCta = 8;                   // below this everything is static
-constexpr int kBigFirstLen = 32;                           // ranges at least this long order their chunks big to small
 
 struct StageMeta {
     int nvalid;        // cached tokens from the tile's first row on, capped at 64 + 7 (0 = nothing was loaded); -1 = end of
@@ -75,18 +76,18 @@ struct Piece {
     int unit, tiles, unit_first, unit_tiles, extra;
 };
 
-// Geometry of the intervals, identical in every CTA (derived from T and gridDim.x).  With range c
-// = [a, b), len its length, b its end and ts = b - (len>>2) the start of its
-// tail, its intervals are
-//   0: [a, ts)   1: [ts, ts + (len>>(R+1)))   2: [.., ts + (len>>R))  ...  R: [ts + (len>>3), b),
-// i.e. the tail's chunks double in size towards the end of the range.  Ranges of kBigFirstLen tiles or
-// more use the mirror image, 1: [ts, b - (len>>3))  2: [.., b - (len>>4)) ... R: [b - (len>>(R+1)), b):
-// the owner (front) meets the big chunks first and thieves (back) pick up small ones, which leaves
-// less to wait for at the very end when a range is long; short ranges do better the other way round.
+// Geometry of the intervals, identical in every CTA (derived from T and gridDim.x).  Range c = [a, b)
+// is cut into its static share [a, b - off[1]) and R chunks [b - off[j], b - off[j+1]), j = 1..R
+// (off[R+1] = 0).  The chunks cover the last quarter of the range and halve towards its end (1/8, 1/16,
+// ... of the range, down to kMinChunk tiles), except that none is longer than 8 tiles (16 from ranges of
+// 512 tiles on, 32 from 1024 on, ...): longer ones are cut up.  The owner, coming from the front, meets the bigger
+// chunks, thieves take the small ones at the back first, and no chunk is so big that a slow owner who
+// has just claimed it holds everybody up.
 struct Schedule {
     int T, G;                      // tiles, ranges (G <= T)
     int R;                         // dynamic chunks per range (0: everything is static)
-    int q, r;                      // T = q * G + r
+    int q, r;                      // T = q * G + r: ranges of q tiles, the first r of them one tile longer
+    int off[kMaxRounds + 2];       // off[j]: tiles from the start of chunk j to the end of its range
 };
 
 struct __align__(1024) Smem {
@@ -154,48 +155,67 @@ __device__ __forceinline__ int range_of(const Schedule& s, int t) {
                          : s.r + (int)((unsigned int)(t - long_part) / (unsigned int)s.q);
 }
 
-__device__ __forceinline__ void build_schedule(Schedule& s, int T, int grid, int pool_div) {
+// Run by a whole warp: the scalar fields come out in every lane's copy `s`, the table is written to
+// `shared`, where all of the schedule is also left for the other warps.  Lane k takes level k of the
+// tail, [b - (q/4 >> k), b - (q/4 >> (k+1))), and cuts it into pieces of `cap` tiles (a power of two)
+// counted from its back end, the front piece taking the remainder.
+__device__ __forceinline__ void build_schedule(Schedule& s, Schedule& shared, int T, int grid, int pool_div, int lane) {
     s.T = T;
     s.G = max(1, min(grid, T));
-    s.q = (int)((unsigned int)T / (unsigned int)s.G);   // shortest range (>= 1 whenever T > 0)
-    s.r = T - s.q * s.G;
-    s.R = 0;
-    const int len = s.q;
-    if (pool_div > 0 && len >= kMinStaticTilesPerCta) {
-        int R = 1;
-        while (R < kMaxRounds && (len >> (R + 2)) >= kMinChunk) ++R;
-        s.R = R;
+    const int q = (int)((unsigned int)T / (unsigned int)s.G);   // shortest range (>= 1 whenever T > 0)
+    s.q = q;
+    s.r = T - q * s.G;
+    int R = 0;
+    if (pool_div > 0 && q >= kMinStaticTilesPerCta) {
+        const int tail = pool_div == 4 ? q >> 2 : q / pool_div;
+        // (with one piece per level there are at most kMaxRounds pieces, so the loop ends at the latest
+        // when cap exceeds the tail)
+        for (int cap_shift = 3 + max(0, 23 - __clz(q)); cap_shift < 31; ++cap_shift) {      // cap = 8, or about q/32 .. q/64
+            // level k = [b - prev, b - nxt): halves, down to kMinChunk tiles; the last level takes the rest
+            int prev = lane < kMaxRounds ? tail >> lane : 0;
+            if (lane > 0 && prev < kMinChunk) prev = 0;
+            int nxt = prev >> 1;
+            if (nxt < kMinChunk || lane == kMaxRounds - 1) nxt = 0;
+            const int size = prev - nxt;                    // (0 for the levels past the last)
+            const int parts = (size + (1 << cap_shift) - 1) >> cap_shift;
+            int incl = parts;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            R = __shfl_sync(0xffffffffu, incl, 31);
+            if (R > kMaxRounds) { R = 0; continue; }
+            // piece i of the level (front to back) starts prev tiles before the range's end for i = 0,
+            // nxt + (parts - i) * cap for the others
+            for (int i = 0; i < parts; ++i) shared.off[incl - parts + 1 + i] = i == 0 ? prev : nxt + ((parts - i) << cap_shift);
+            break;
+        }
     }
+    s.R = R;
+    if (lane == 0) {
+        shared.off[R + 1] = 0;
+        shared.T = s.T; shared.G = s.G; shared.R = R; shared.q = q; shared.r = s.r;
+    }
+    __syncwarp();
 }
 
-// Interval j (0 = static share, 1..R = chunks, small ones first) of range c.
-__device__ __forceinline__ void interval_range(const Schedule& s, int c, int j, int* begin, int* end) {
-    const int a = range_begin(s, c), b = range_begin(s, c + 1), len = b - a;
+// Interval j (0 = static share, 1..R = chunks, front to back) of range c.
+// (s: the scalar fields, possibly a register copy; off: the table in shared memory)
+__device__ __forceinline__ void interval_range(const Schedule& s, const int* off, int c, int j, int* begin, int* end) {
+    const int a = range_begin(s, c), b = range_begin(s, c + 1);
     if (s.R == 0) { *begin = a; *end = b; return; }
-    const int ts = b - (len >> 2);                  // the tail: last quarter of the range
-    if (j == 0) { *begin = a; *end = ts; return; }
-    if (len >= kBigFirstLen) {                      // long ranges: the big chunks first
-        *begin = b - (len >> (j + 1));
-        *end = j == s.R ? b : b - (len >> (j + 2));
-        return;
-    }
-    *begin = j == 1 ? ts : ts + (len >> (s.R + 3 - j));
-    *end = ts + (len >> (s.R + 2 - j));
+    *begin = j == 0 ? a : b - off[j];
+    *end = b - off[j + 1];
 }
 
 // Number (c * (R+1) + j, increasing with the tile position) of the interval that holds tile t.
 __device__ __forceinline__ int interval_of(const Schedule& s, int t) {
     const int c = range_of(s, t);
     if (s.R == 0) return c;
-    const int a = range_begin(s, c), b = range_begin(s, c + 1), len = b - a;
-    const int off = t - (b - (len >> 2));           // position inside the tail
-    if (off < 0) return c * (s.R + 1);
-    int j = 1;
-    if (len >= kBigFirstLen) {
-        while (j < s.R && t >= b - (len >> (j + 2))) ++j;
-    } else {
-        while (j < s.R && off >= (len >> (s.R + 2 - j))) ++j;
-    }
+    const int d = range_begin(s, c + 1) - t;        // tiles from t to the end of its range (>= 1)
+    int j = 0;
+    while (j < s.R && d <= s.off[j + 1]) ++j;
     return c * (s.R + 1) + j;
 }
 
@@ -424,9 +444,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         }
         const int T = __shfl_sync(0xffffffffu, incl, 31);
         if (lane == 0) SEER_STAMP(11);
-        Schedule sc;
-        build_schedule(sc, T, gridDim.x, p.pool_div);
-        if (lane == 0) sm.sched = sc;                    // the consumers use it when a piece ends
+        Schedule sc;                                     // (its table stays in shared memory)
+        build_schedule(sc, sm.sched, T, gridDim.x, p.pool_div, lane);     // (the consumers use it when a piece ends)
         const int R = sc.R, G = sc.G;
         {
             int acc = incl - mine;
@@ -490,12 +509,46 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         int it = 0;
         int iv_begin = 0, iv_end = 0, iv_id = 0;
         bool first = true;               // the static share has not been taken yet
-        bool own = cta < G;              // still claiming chunks of the own range
+        bool own = R > 0 && cta < G;     // the own range may still have chunks to claim
         bool contiguous = false;         // the next interval continues the previous one
         int fails = 0, steals = 0;
+        // What the next interval needs from global memory is asked for before the tiles of the current
+        // one are issued, so that the round trip runs under them: the claim on the own range's counter
+        // while that range lasts, afterwards the look at all ranges' counters.
+        constexpr int kScan = 10;        // counters per lane and round: 320 ranges a round
+        int next_own_tiles = 0;          // size of the own range's chunk after the current one
+        int ahead = 0;                   // 0: nothing asked for, 1: own claim (pend_old), 2: first round of counters (st)
+        int pend_old = 0;
+        int st[kScan];
+        // (a range's last chunk is left to its owner: by the time a thief's loads came back the owner
+        // would have been there)
+#ifdef SEER_EXP_MINLEFT
+        const int min_left = min(SEER_EXP_MINLEFT, R);
+#else
+        const int min_left = min(2, R);
+#endif
+        auto scan_load = [&](int c0) {
+#pragma unroll
+            for (int k = 0; k < kScan; ++k) {
+                const int cc = c0 + 32 * k + lane;
+                st[k] = cc < G ? __ldcg(p.steal + cc) : (R << 16);
+            }
+        };
+        auto scan_pick = [&](int c0, int best) -> int {
+#pragma unroll
+            for (int k = 0; k < kScan; ++k) {
+                const int cc = c0 + 32 * k + lane;
+                const int left = R - (st[k] & 0xffff) - (st[k] >> 16);
+                if (cc < G && cc != cta && left >= min_left) {
+                    const int rot = cc - cta + (cc < cta ? G : 0);   // this thief's order of preference
+                    best = max(best, (left << 20) | (0xfffff - min(rot, 0xfffff)));
+                }
+            }
+            return best;
+        };
         for (;;) {
             {
-                int c, j;
+                int c = 0, j = 0;
                 if (first) {
                     // the static share: the head of the own range
                     if (T == 0 || cta >= G) {
@@ -503,62 +556,60 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                         break;
                     }
                     c = cta;
-                    j = 0;
                 } else if (R == 0) {
                     break;
-                } else if (own) {
-                    // own range, from the front: low half of the counter counts front claims
-                    int old = 0;
-                    if (lane == 0) old = atomicAdd(&p.steal[cta], 1);
-                    old = __shfl_sync(0xffffffffu, old, 0);
-                    if ((old & 0xffff) + (old >> 16) >= R) { own = false; continue; }
-                    c = cta;
-                    j = (old & 0xffff) + 1;
-                    contiguous = true;
                 } else {
-                    // Somebody else's range, from the back.  Look at every range's claim counter
-                    // and go for the one with the most chunks left (its owner is the furthest
-                    // behind); ties are broken differently by every thief.
-                    if (fails >= 3 || steals >= kMaxSteals) break;
-                    // (all of a lane's counters are requested before any is looked at: one round trip)
-                    int best = -1;
-                    // (a range's last chunk is left to its owner: by the time a thief's loads came
-                    // back the owner would have been there)
-                    const int min_left = min(2, R);
-                    constexpr int kScan = 10;                 // counters per lane and round: 320 ranges a round
-                    for (int c0 = 0; c0 < G; c0 += 32 * kScan) {
-                        int st[kScan];
-#pragma unroll
-                        for (int k = 0; k < kScan; ++k) {
-                            const int cc = c0 + 32 * k + lane;
-                            st[k] = cc < G ? __ldcg(p.steal + cc) : (R << 16);
-                        }
-#pragma unroll
-                        for (int k = 0; k < kScan; ++k) {
-                            const int cc = c0 + 32 * k + lane;
-                            const int left = R - (st[k] & 0xffff) - (st[k] >> 16);
-                            if (cc < G && cc != cta && left >= min_left) {
-                                const int rot = cc - cta + (cc < cta ? G : 0);   // this thief's order of preference
-                                best = max(best, (left << 20) | (0xfffff - min(rot, 0xfffff)));
+                    bool got = false, done = false;
+                    while (!got && !done) {
+                        if (own) {
+                            // own range, from the front: low half of the counter counts front claims
+                            if (ahead != 1 && lane == 0) pend_old = atomicAdd(&p.steal[cta], 1);
+                            ahead = 0;
+                            const int old = __shfl_sync(0xffffffffu, pend_old, 0);
+                            const int taken = (old & 0xffff) + (old >> 16);
+                            if (taken + 1 >= R) own = false;     // the last chunk, or none left
+                            if (taken >= R) continue;
+                            c = cta;
+                            j = (old & 0xffff) + 1;
+                            contiguous = true;
+                            got = true;
+                        } else {
+                            // Somebody else's range, from the back.  Look at every range's claim counter
+                            // and go for the one with the most chunks left (its owner is the furthest
+                            // behind); ties are broken differently by every thief.  (All of a lane's
+                            // counters are requested before any is looked at: one round trip.)
+                            if (fails >= 3 || steals >= kMaxSteals) { done = true; break; }
+                            int best = -1;
+                            for (int c0 = 0; c0 < G; c0 += 32 * kScan) {
+                                if (c0 > 0 || ahead != 2) scan_load(c0);
+                                best = scan_pick(c0, best);
                             }
+                            ahead = 0;
+#pragma unroll
+                            for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+                            if (best < 0) { done = true; break; }                 // nothing left anywhere
+                            c = cta + (0xfffff - (best & 0xfffff));
+                            if (c >= G) c -= G;
+                            int old = 0;
+                            if (lane == 0) old = atomicAdd(&p.steal[c], 1 << 16);
+                            old = __shfl_sync(0xffffffffu, old, 0);
+                            if ((old & 0xffff) + (old >> 16) >= R) { ++fails; continue; }
+                            fails = 0;
+                            ++steals;
+                            j = R - (old >> 16);
+                            contiguous = false;
+                            got = true;
                         }
                     }
-#pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
-                    if (best < 0) break;                                  // nothing left anywhere
-                    c = cta + (0xfffff - (best & 0xfffff));
-                    if (c >= G) c -= G;
-                    int old = 0;
-                    if (lane == 0) old = atomicAdd(&p.steal[c], 1 << 16);
-                    old = __shfl_sync(0xffffffffu, old, 0);
-                    if ((old & 0xffff) + (old >> 16) >= R) { ++fails; continue; }
-                    fails = 0;
-                    ++steals;
-                    j = R - (old >> 16);
-                    contiguous = false;
+                    if (!got) break;
                 }
-                interval_range(sc, c, j, &iv_begin, &iv_end);
+                interval_range(sc, sm.sched.off, c, j, &iv_begin, &iv_end);
                 iv_id = c * (R + 1) + j;
+                if (own && c == cta && j < R) {
+                    int nb, ne;
+                    interval_range(sc, sm.sched.off, c, j + 1, &nb, &ne);
+                    next_own_tiles = ne - nb;
+                }
                 if (!contiguous) {
                     const bool found = iv_begin < iv_end && locate(iv_begin, first);
                     if (first) {
@@ -572,6 +623,23 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     }
                 }
             }
+            // asks for what the next interval will need (called when the last few tiles of the current
+            // interval are about to be issued: earlier, an own claim would take a chunk out of the
+            // thieves' reach long before its owner gets to it)
+            auto ask_ahead = [&]() {
+                if (R == 0) return;
+                if (own) {
+                    // (only when the chunk to come is small: a big one is worth more within the thieves'
+                    // reach than the round trip its claim costs)
+                    if (next_own_tiles <= kAheadMaxChunk) {
+                        if (lane == 0) pend_old = atomicAdd(&p.steal[cta], 1);
+                        ahead = 1;
+                    }
+                } else if (fails < 3 && steals < kMaxSteals) {
+                    scan_load(0);
+                    ahead = 2;
+                }
+            };
             const bool fresh = !contiguous;          // this interval starts a new piece
             int ce = iv_begin - cpu;                  // offset of the next tile inside unit cu
             const int n_tiles = iv_end - iv_begin;
@@ -672,6 +740,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     raise_status(p.status, DEV_BAD_INDEX);
                 }
                 for (int s = 0; s < n_chunk; ++s, ++it) {
+                    if (n_tiles - (t + s) == min(n_tiles, kAheadTiles)) ask_ahead();
                     const int s_nvalid = __shfl_sync(0xffffffffu, nvalid, s);
                     const int s_head = __shfl_sync(0xffffffffu, head, s);
                     const int s_flags = __shfl_sync(0xffffffffu, flags, s);
@@ -807,6 +876,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         const int st = it % kStages;
 #ifdef SEER_DECODE_TRACE
         if (tid == 0 && it < kTraceSlots - 16) SEER_STAMP(16 + it);
+        if (tid == 0) p.trace[(size_t)blockIdx.x * kTraceSlots + 3] = it + 1;     // tiles consumed so far
 #endif
         if (NT == 1) {
             // look ahead: request the queries of the next unit as soon as the producer has issued a

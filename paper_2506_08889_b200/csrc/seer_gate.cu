@@ -587,12 +587,26 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     const int total = (j1 - j0) * lpk;
     constexpr int kBatch = 8;
     uint4* staged = reinterpret_cast<uint4*>(sc_all + ((p.max_blocks + 3) & ~3));     // [kBatch * 512] pieces
+    // The small loads the projection waits for -- the sequence length and the pre-RoPE queries of this
+    // warp's first work item -- are requested before the keys: behind 128 KB of key requests they would
+    // come back microseconds later.
+    const int L = __ldg(p.seq_lens + i);
+    uint4 xv0[NIT];
+    {
+        const int t0 = gw / half;
+        const uint4* xsrc = reinterpret_cast<const uint4*>(
+            p.q_nope + (((size_t)i * q_len + min(t0, q_len - 1)) * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int ch = lane + 32 * it;
+            xv0[it] = ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
 #pragma unroll
     for (int k = 0; k < kBatch; ++k) {                 // entries past n_i - 1 exist in memory: harmless
         const int pc = k * kGateThreads + tid;
         if (pc < total) cp_async16(staged + pc, kc + pc);
     }
-    const int L = __ldg(p.seq_lens + i);
     cluster_wait();                                    // every CTA of the cluster has started
     // ---- 1. gate queries --------------------------------------------------------------------------
     for (int item = gw; item < n_items; item += n_gw) {
@@ -603,7 +617,7 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
             const int ch = lane + 32 * it;
-            xv[it] = ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u);
+            xv[it] = item == gw ? xv0[it] : (ch < chunks ? __ldg(xsrc + ch) : make_uint4(0u, 0u, 0u, 0u));
         }
         if (item != gw) {
 #pragma unroll

@@ -242,57 +242,58 @@ def run_ours(args):
     torch.cuda.synchronize()
     assert ctx.device_status() == binding.SEER_OK
 
-    # ---- timed region: exactly K steps, device timed, max over ranks ------------------------
+    # ---- timed region: blocks of exactly K steps, device timed, max over ranks ---------------
+    # A block of K steps is timed as one region (barrier + synchronize on both sides, events on the
+    # stream); the block is repeated until at least `min_timed_s` seconds have been timed and the
+    # median block is reported, so that a small --steps gives the same figure as a large one.
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
-    # the sparse-decode launch is bracketed by events on one step in eight only: an event record
-    # between two kernels keeps the second from starting its set-up under the first one's tail
-    ev_every = 8
-    evs = {s: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-           for s in range(0, K, ev_every)}
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_block(fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for s in range(n):
+            fn(s)
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1) / n
+
+    def repeated(fn, n, min_s=None, max_repeats=200):
+        """Median over repeated blocks of n calls (ms per call), and the number of blocks."""
+        min_s = args.min_timed_s if min_s is None else min_s
+        blocks, total = [], 0.0
+        while not blocks or (total < min_s and len(blocks) < max_repeats):
+            ms = timed_block(fn, n)
+            blocks.append(ms)
+            total += ms * n * 1e-3
+        return float(np.median(blocks)), len(blocks)
+
     launches0 = ctx.launch_count()
+    step_ms, repeats = repeated(lambda s: step(layers[s % n_layers]), K)
+    launches = (ctx.launch_count() - launches0) // repeats
+    # The sparse-decode launch bracketed by events, in a pass of its own (an event record between two
+    # kernels keeps the second from starting its set-up under the first one's tail, so bracketed steps
+    # are kept out of the step timing): at least 32 samples, median.
+    n_ev = max(32, min(K, 256))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
     barrier()
-    t0.record()
-    for s in range(K):
-        step(layers[s % n_layers], evs.get(s))
-    t1.record()
+    for s in range(n_ev):
+        step(layers[s % n_layers], evs[s])
     barrier()
-    launches = ctx.launch_count() - launches0
-    step_ms = t0.elapsed_time(t1) / K
-    sparse_ms = float(np.mean([a.elapsed_time(bq) for a, bq in evs.values()]))
+    sparse_ms = float(np.median([a.elapsed_time(bq) for a, bq in evs]))
 
     # dense decode on the same tensors (speed-up denominator), same protocol
     Kd = max(8, min(K, 200))
-    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    d0.record()
-    for s in range(Kd):
-        ctx.seer_dense_decode(shape, layers[s % n_layers]["kv"], layers[s % n_layers]["q"], out_dense)
-    d1.record()
-    barrier()
-    dense_ms = d0.elapsed_time(d1) / Kd
+    dense_ms, _ = repeated(lambda s: ctx.seer_dense_decode(shape, layers[s % n_layers]["kv"], layers[s % n_layers]["q"],
+                                                           out_dense), Kd)
     # sparse kernel alone, back to back (no events inside), for the kernel-only speed-up
-    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    s0.record()
-    for s in range(K):
-        lay = layers[s % n_layers]
-        ctx.seer_sparse_decode(shape, lay["kv"], lay["q"], idx, cnt, k_sel, out)
-    s1.record()
-    barrier()
-    sparse_b2b_ms = s0.elapsed_time(s1) / K
+    sparse_b2b_ms, _ = repeated(lambda s: ctx.seer_sparse_decode(shape, layers[s % n_layers]["kv"], layers[s % n_layers]["q"],
+                                                                 idx, cnt, k_sel, out), K)
     # the step without the compressed-K update (63 steps of 64 in a real decode: a block fills once per b tokens)
-    n0, n1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    n0.record()
-    for s in range(K):
-        lay = layers[s % n_layers]
-        ctx.seer_decode_step(shape, lay["kv"], lay["gate"], lay["q"], lay["qn"], None, budget, idx, cnt, k_sel, out,
-                             stream=stream)
-    n1.record()
-    barrier()
-    step_noappend_ms = n0.elapsed_time(n1) / K
+    step_noappend_ms, _ = repeated(lambda s: ctx.seer_decode_step(shape, layers[s % n_layers]["kv"], layers[s % n_layers]["gate"],
+                                                                  layers[s % n_layers]["q"], layers[s % n_layers]["qn"], None,
+                                                                  budget, idx, cnt, k_sel, out, stream=stream), K)
     clocks = sampler.stop()
 
     # ---- end to end through the same API with host buffers ----------------------------------
@@ -336,12 +337,16 @@ def run_ours(args):
     Ke = max(8, min(K, 300))
     for s in range(3):
         e2e_step(layers[s % n_layers])
-    barrier()
-    w0 = time.perf_counter()
-    for s in range(Ke):
-        e2e_step(layers[s % n_layers])
-    barrier()
-    e2e_ms = (time.perf_counter() - w0) * 1e3 / Ke
+    e2e_blocks, e2e_total = [], 0.0
+    while not e2e_blocks or (e2e_total < args.min_timed_s and len(e2e_blocks) < 200):
+        barrier()
+        w0 = time.perf_counter()
+        for s in range(Ke):
+            e2e_step(layers[s % n_layers])
+        barrier()
+        e2e_blocks.append((time.perf_counter() - w0) * 1e3 / Ke)
+        e2e_total += e2e_blocks[-1] * Ke * 1e-3
+    e2e_ms = float(np.median(e2e_blocks))
     assert ctx.device_status() == binding.SEER_OK
 
     # ---- reduce over ranks -------------------------------------------------------------------
@@ -355,6 +360,7 @@ def run_ours(args):
         kern_gbs = decode_bytes / (sparse_ms * 1e-3) / 1e9
         result = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "repeats": repeats,
             "ms_per_step": round(step_ms, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "batch_per_gpu": B, "num_q_heads": Hq, "num_kv_heads": Hkv,
@@ -371,6 +377,7 @@ def run_ours(args):
                          "peak": peak, "unit": "GB/s", "frac": round(kern_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
                          "frac_of_nominal_8000": round(kern_gbs / NOMINAL_HBM_GBS, 4),
                          "algorithmic_bytes_per_launch": decode_bytes, "us_per_launch": round(sparse_ms * 1e3, 2),
+                         "event_samples": n_ev,
                          "traffic": (int(NCU_READ_BYTES_PER_2_SEQUENCES * B / 2 * (1.0 - args.sparsity) / 0.1
                                          + NCU_WRITE_BYTES_PER_LAUNCH) if abs(args.sparsity - 0.9) < 1e-9 else None),
                          "traffic_note": "ncu capture at batch 2, scaled by the units processed",
@@ -588,6 +595,227 @@ def run_grid(args):
     ctx.close()
 
 
+def run_workloads(args):
+    """The other specified workloads, one GPU, one JSON document: the batch-1 8B and 14B shapes (a
+    launch moves 16 MiB, less than L2 holds and about as long as a launch takes) each timed (i) alone --
+    one call, L2 flushed before it, event-bracketed -- and (ii) as a stream over `layers` distinct
+    layer caches (more than twice L2 in total), which is the figure compared with the HBM roofline;
+    and the ragged batch of 16 at block size 128.  Beside each: the library's own dense kernel under
+    the same protocol, and the fp64 oracle's time for the same call on the host cores."""
+    import torch
+    import oracle
+    from paper_2506_08889_b200 import binding, synth
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    ctx = binding.Context(0)
+    peak, peak_kind = measured_hbm_peak()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)        # > 2 x L2
+    rows = []
+
+    def isolated(fn, n=40):
+        """Median of single calls, each after an L2 flush, bracketed by events (us)."""
+        fn(0)
+        ts = []
+        for s in range(n):
+            flush.fill_(s & 1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn(s)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts))
+
+    def streamed(fn, n):
+        """Calls back to back over the distinct layers (us per call, median of repeated blocks)."""
+        for s in range(n):
+            fn(s)
+        blocks, total = [], 0.0
+        while not blocks or (total < args.min_timed_s and len(blocks) < 100):
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for s in range(n):
+                fn(s)
+            e1.record()
+            torch.cuda.synchronize()
+            blocks.append(e0.elapsed_time(e1) / n * 1e3)
+            total += blocks[-1] * n * 1e-6
+        return float(np.median(blocks))
+
+    def row(w, what, sel_bytes, us_iso, us_stream, dense_bytes, dense_iso, dense_stream, extra):
+        r = {"workload": w.name, "call": what, "selected_kv_MB": round(sel_bytes / 1e6, 2),
+             "isolated_us": round(us_iso, 2), "streamed_us": round(us_stream, 2),
+             "streamed_GBps": round(sel_bytes / us_stream / 1e3, 1),
+             "streamed_frac_of_measured_peak": round(sel_bytes / us_stream / 1e3 / peak, 4),
+             "streamed_frac_of_8000": round(sel_bytes / us_stream / 1e3 / NOMINAL_HBM_GBS, 4),
+             "isolated_GBps": round(sel_bytes / us_iso / 1e3, 1),
+             "dense_isolated_us": round(dense_iso, 2), "dense_streamed_us": round(dense_stream, 2),
+             "dense_streamed_GBps": round(dense_bytes / dense_stream / 1e3, 1),
+             "speedup_vs_dense_streamed": round(dense_stream / us_stream, 3),
+             "speedup_vs_dense_isolated": round(dense_iso / us_iso, 3)}
+        r.update(extra)
+        rows.append(r)
+
+    # ---- batch 1, Qwen3-8B shape: selection on given scores, then sparse decode ---------------------
+    w = synth.workload(1)
+    B, Hq, Hkv, d, b, L = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size, w.seq_len
+    nb, k_sel, NL = L // b, w.keep(L // b), args.stream_layers
+    lens_t = torch.full((B,), L, dtype=torch.int32, device=dev)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, w.sm_scale)
+    lay = []
+    for l in range(NL):
+        tag = f"{w.name}:L{l}:"
+        k = synth.normal_bf16((B, Hkv, L, d), synth.BASE_SEED, tag + "k", dev)
+        v = synth.normal_bf16((B, Hkv, L, d), synth.BASE_SEED, tag + "v", dev)
+        lay.append({"kv": binding.make_kv(k, v, lens_t), "k": k, "v": v,
+                    "q": synth.normal_bf16((B, Hq, d), synth.BASE_SEED, tag + "q", dev),
+                    "sc": synth.normal_f32((B, Hkv, nb), synth.BASE_SEED, tag + "scores", dev)})
+    gate0 = binding.make_gate(w.d_gate, w.rope_theta, None, None, None, nb)
+    idx = torch.zeros((B, Hkv, k_sel), dtype=torch.int32, device=dev)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+    out = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=dev)
+    ctx.seer_gate_select(shape, gate0, lens_t, None, lay[0]["sc"], w.token_budget, idx, cnt, k_sel)
+
+    def dec(s):
+        ctx.seer_sparse_decode(shape, lay[s % NL]["kv"], lay[s % NL]["q"], idx, cnt, k_sel, out)
+
+    def sel_dec(s):
+        ctx.seer_gate_select(shape, gate0, lens_t, None, lay[s % NL]["sc"], w.token_budget, idx, cnt, k_sel)
+        ctx.seer_sparse_decode(shape, lay[s % NL]["kv"], lay[s % NL]["q"], idx, cnt, k_sel, out)
+
+    def dense(s):
+        ctx.seer_dense_decode(shape, lay[s % NL]["kv"], lay[s % NL]["q"], out)
+
+    sel_bytes = B * Hkv * k_sel * b * d * 4
+    dense_bytes = B * Hkv * L * d * 4
+    d_iso, d_str = isolated(dense), streamed(dense, NL)
+    # the oracle on the same call: all host threads, and one thread
+    hk, hv, hq = synth.bf16_bits(lay[0]["k"]), synth.bf16_bits(lay[0]["v"]), synth.bf16_bits(lay[0]["q"])
+    hsc = lay[0]["sc"].cpu().numpy()
+    lens = np.full(B, L, np.int32)
+
+    def oracle_call():
+        i2, c2 = oracle.select(hsc, lens, b, w.token_budget, k_sel)
+        oracle.sparse(hq, hk, hv, lens, i2, c2, b, w.sm_scale)
+    oracle_call()
+    t0 = time.perf_counter(); oracle_call(); o_all = time.perf_counter() - t0
+    n_thr = oracle.num_threads()
+    oracle.set_num_threads(1)
+    t0 = time.perf_counter(); oracle_call(); o_one = time.perf_counter() - t0
+    oracle.set_num_threads(n_thr)
+    row(w, "seer_sparse_decode", sel_bytes, isolated(dec), streamed(dec, NL), dense_bytes, d_iso, d_str,
+        {"layers_streamed": NL, "oracle_ms_all_threads": round(o_all * 1e3, 2), "oracle_threads": n_thr,
+         "oracle_ms_one_thread": round(o_one * 1e3, 2)})
+    row(w, "seer_gate_select(scores) + seer_sparse_decode", sel_bytes, isolated(sel_dec), streamed(sel_dec, NL),
+        dense_bytes, d_iso, d_str, {"layers_streamed": NL})
+    del lay
+    torch.cuda.empty_cache()
+
+    # ---- batch 1, Qwen3-14B shape: the whole step (append + gate + sparse decode) ---------------------
+    w = synth.workload(2)
+    B, Hq, Hkv, d, b, L = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size, w.seq_len
+    nb, k_sel = L // b, w.keep(L // b)
+    budget = k_sel * b
+    lens_t = torch.full((B,), L, dtype=torch.int32, device=dev)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, w.sm_scale)
+    layers = build_layers(w, NL, synth.BASE_SEED, dev)
+    idx = torch.zeros((B, Hkv, k_sel), dtype=torch.int32, device=dev)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+    out = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=dev)
+    for la in layers:
+        la["gate"] = binding.make_gate(w.d_gate, w.rope_theta, la["wq"], la["wk"], la["kc"], nb)
+        la["kv"] = binding.make_kv(la["k"], la["v"], lens_t)
+        ctx.seer_kcomp_append(shape, la["gate"], lens_t, la["k"], first_block=0, num_blocks=nb - 1)
+    torch.cuda.synchronize()
+
+    def step(s):
+        la = layers[s % NL]
+        ctx.seer_decode_step(shape, la["kv"], la["gate"], la["q"], la["qn"], la["k"], budget, idx, cnt, k_sel, out)
+
+    def step_noappend(s):
+        la = layers[s % NL]
+        ctx.seer_decode_step(shape, la["kv"], la["gate"], la["q"], la["qn"], None, budget, idx, cnt, k_sel, out)
+
+    def dec3(s):
+        la = layers[s % NL]
+        ctx.seer_sparse_decode(shape, la["kv"], la["q"], idx, cnt, k_sel, out)
+
+    def dense3(s):
+        la = layers[s % NL]
+        ctx.seer_dense_decode(shape, la["kv"], la["q"], out)
+
+    step(0)
+    sel_bytes = B * Hkv * k_sel * b * d * 4
+    dense_bytes = B * Hkv * L * d * 4
+    gate_bytes = B * Hkv * (nb - 1) * w.d_gate * 2 + Hkv * w.d_gate * w.group * d * 2
+    d_iso, d_str = isolated(dense3), streamed(dense3, NL)
+    host = host_copy(layers[0])
+    host["kc"], _ = oracle.kcomp(host["k"], host["wk"], b, 0, nb - 1, nb, w.rope_theta)
+    oracle_step(w, host, 1, Hkv, budget, k_sel)
+    t0 = time.perf_counter(); oracle_step(w, host, 1, Hkv, budget, k_sel); o_all = time.perf_counter() - t0
+    row(w, "seer_decode_step (append + gate + sparse decode)", sel_bytes, isolated(step), streamed(step, NL),
+        dense_bytes, d_iso, d_str, {"layers_streamed": NL, "gate_bytes_MB": round(gate_bytes / 1e6, 2),
+                                    "oracle_ms_all_threads": round(o_all * 1e3, 2), "oracle_threads": oracle.num_threads()})
+    row(w, "seer_decode_step without the append", sel_bytes, isolated(step_noappend), streamed(step_noappend, NL),
+        dense_bytes, d_iso, d_str, {"layers_streamed": NL})
+    row(w, "seer_sparse_decode", sel_bytes, isolated(dec3), streamed(dec3, NL), dense_bytes, d_iso, d_str,
+        {"layers_streamed": NL})
+    del layers, host
+    torch.cuda.empty_cache()
+
+    # ---- batch 16, ragged lengths, block size 128, 90 % of each sequence's blocks skipped ---------------
+    w = synth.workload(3)
+    B, Hq, Hkv, d, b, L = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size, w.seq_len
+    lens = w.lengths()
+    n_i = [-(-int(x) // b) for x in lens]
+    keep = [w.keep(n) for n in n_i]
+    max_sel = max(keep)
+    NL4 = 3
+    lens_t = torch.as_tensor(lens, device=dev)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, w.sm_scale)
+    shape1 = binding.make_shape(1, Hq, Hkv, d, b, w.sm_scale)
+    lay = []
+    for l in range(NL4):
+        tag = f"{w.name}:L{l}:"
+        k = synth.normal_bf16((B, Hkv, L, d), synth.BASE_SEED, tag + "k", dev)
+        v = synth.normal_bf16((B, Hkv, L, d), synth.BASE_SEED, tag + "v", dev)
+        lay.append({"kv": binding.make_kv(k, v, lens_t, max_seq_len=L), "k": k, "v": v,
+                    "q": synth.normal_bf16((B, Hq, d), synth.BASE_SEED, tag + "q", dev)})
+    scores = synth.normal_f32((B, Hkv, L // b), synth.BASE_SEED, w.name + ":scores", dev)
+    gate4 = binding.make_gate(w.d_gate, w.rope_theta, None, None, None, L // b)
+    idx = torch.full((B, Hkv, max_sel), -1, dtype=torch.int32, device=dev)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+    for i in range(B):                    # the kept count differs between sequences: one selection call each
+        ctx.seer_gate_select(shape1, gate4, lens_t[i:i + 1], None, scores[i:i + 1], keep[i] * b, idx[i:i + 1],
+                             cnt[i:i + 1], max_sel)
+    torch.cuda.synchronize()
+    out = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=dev)
+
+    def dec4(s):
+        ctx.seer_sparse_decode(shape, lay[s % NL4]["kv"], lay[s % NL4]["q"], idx, cnt, max_sel, out)
+
+    def dense4(s):
+        ctx.seer_dense_decode(shape, lay[s % NL4]["kv"], lay[s % NL4]["q"], out)
+
+    sel_tokens = sum(min(int(lens[i]) - (n_i[i] - 1) * b, b) + (keep[i] - 1) * b for i in range(B))   # (an upper figure:
+    # the forced last block may be partial; the other selected blocks are complete)
+    sel_bytes = Hkv * sel_tokens * d * 4
+    dense_bytes = Hkv * int(np.sum(lens)) * d * 4
+    hq = synth.bf16_bits(lay[0]["q"])
+    hk, hv = synth.bf16_bits(lay[0]["k"][:2]), synth.bf16_bits(lay[0]["v"][:2])
+    i2, c2 = idx[:2].cpu().numpy(), cnt[:2].cpu().numpy()
+    oracle.sparse(hq[:2], hk, hv, lens[:2], i2, c2, b, w.sm_scale)
+    t0 = time.perf_counter(); oracle.sparse(hq[:2], hk, hv, lens[:2], i2, c2, b, w.sm_scale); o2 = time.perf_counter() - t0
+    row(w, "seer_sparse_decode", sel_bytes, isolated(dec4, 20), streamed(dec4, 2 * NL4), dense_bytes,
+        isolated(dense4, 10), streamed(dense4, NL4),
+        {"layers_streamed": NL4, "lengths": [int(x) for x in lens], "selected_blocks": keep,
+         "oracle_ms_all_threads_2_of_16_sequences": round(o2 * 1e3, 2), "oracle_threads": oracle.num_threads()})
+    assert ctx.device_status() == binding.SEER_OK
+    ctx.close()
+    print(json.dumps({"peak_GBps": peak, "peak_kind": peak_kind, "rows": rows}))
+
+
 def oracle_step(w, host, n_seq, n_kv_heads, budget, k_sel):
     """The whole step on the CPU oracle for the first n_seq sequences and the first
     n_kv_heads KV heads (with their query-head groups).  Returns the selected-KV bytes."""
@@ -699,10 +927,17 @@ def main():
     ap.add_argument("--grid", action="store_true", help="the paper's 64/8-head kernel grid (seq len x batch x sparsity)")
     ap.add_argument("--multi", action="store_true", help="multi-query-token decode: q_len 1..8, kernel-only")
     ap.add_argument("--block-size", type=int, default=64, help="block size for --grid (16, 32, 64 or 128)")
+    ap.add_argument("--min-timed-s", type=float, default=0.2,
+                    help="the block of --steps steps is repeated until this many seconds have been timed (median block reported)")
+    ap.add_argument("--workloads", action="store_true",
+                    help="the other specified workloads (batch-1 8B and 14B shapes, ragged batch 16): isolated and streamed")
+    ap.add_argument("--stream-layers", type=int, default=32, help="distinct layer caches of the batch-1 streams (--workloads)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()
-    if args.grid:
+    if args.workloads:
+        run_workloads(args)
+    elif args.grid:
         run_grid(args)
     elif args.multi:
         run_multi(args)

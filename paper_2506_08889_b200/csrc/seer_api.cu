@@ -47,6 +47,7 @@ struct seer_ctx {
     uint64_t launches;
     unsigned int generation;    // stamps the partials of a decode launch
     int pool_div;               // decode scheduling: share of tiles handed out dynamically
+    int min_tiles;              // decode scheduling: fewest tiles of a CTA's range
     char err[512];
 };
 
@@ -253,6 +254,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.num_units = U;
     p.max_blocks_cap = (kv->max_seq_len + kTileTokens - 1) / kTileTokens;
     p.pool_div = ctx->pool_div;
+    p.min_tiles = ctx->min_tiles;
     p.scale_log2 = shape->sm_scale * 1.4426950408889634f;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
     p.tickets = reinterpret_cast<unsigned long long*>(ctx->ws + w.tickets);
@@ -305,6 +307,8 @@ seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes) {
     ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
     ctx->pool_div = 4;
     if (const char* e = getenv("SEER_DECODE_POOL_DIV")) ctx->pool_div = atoi(e);
+    ctx->min_tiles = 4;
+    if (const char* e = getenv("SEER_DECODE_MIN_TILES")) ctx->min_tiles = atoi(e);
     ctx->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)64 << 20;
     if (ctx->ws_bytes < 4096) ctx->ws_bytes = 4096;     // (far too small for any call: every call checks)
     if (cudaMalloc(reinterpret_cast<void**>(&ctx->ws), ctx->ws_bytes) != cudaSuccess) {

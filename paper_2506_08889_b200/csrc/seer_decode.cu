@@ -53,6 +53,7 @@ constexpr int kMaxPieces = 32;                             // partial pieces a C
 constexpr int kListInts = kStageBytes / 4 - 64;              // slot numbers that fit in one stage buffer (less 64 counts)
 constexpr int kLandBytes = 2 * kStageBytes;                 // landing area for staged partials: two stage buffers
 constexpr int kMaxSteals = 14;                             // chunks a CTA may take from other ranges
+constexpr int kFewTilesPerCta = 16;                        // up to this many tiles per CTA the number of ranges is chosen with care
 constexpr int kAheadMaxChunk = 8;                          // own chunks up to this size are claimed ahead
 constexpr int kAheadTiles = 3;                             // tiles left to issue when the next interval's claim is made
 constexpr int kSmemUnits = 128;                            // units whose tile-count prefix sums fit in shared memory
@@ -428,13 +429,15 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         const int per = (U + 31) / 32;
         const int u_lo = min(U, lane * per), u_hi = min(U, u_lo + per);
         const bool smem_pfx = U <= kSmemUnits;
-        int mine = 0;
+        int mine = 0, t_min = 0x7fffffff, t_max = 0;
 #pragma unroll 1
         for (int u = u_lo; u < u_hi; ++u) {
             const int t = tiles_of<SPARSE, SMALL>(p, u);
             if (t == 0 && cta == 0) write_zero_unit(p, u);       // units without work: zeros, -inf
             if (smem_pfx) sm.upfx[u + 1] = t;                      // (the count for now)
             mine += t;
+            t_min = min(t_min, t);
+            t_max = max(t_max, t);
         }
         int incl = mine;
 #pragma unroll
@@ -444,8 +447,32 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         }
         const int T = __shfl_sync(0xffffffffu, incl, 31);
         if (lane == 0) SEER_STAMP(11);
+        // With little work (a few tiles per CTA at most) fewer CTAs take part, kMinTiles tiles or more each:
+        // a unit is then cut into fewer pieces and its combine is short.  If, moreover, all units have
+        // the same number of tiles t, the ranges are made to divide the units evenly (P ranges of t/P
+        // tiles per unit, P the largest such divisor of t), so that no range straddles two units --
+        // provided that keeps at least 4/5 of the CTAs the plain rule would use.
+        int ranges = gridDim.x;
+        if (T > 0 && T <= kFewTilesPerCta * (int)gridDim.x && p.min_tiles > 0) {
+            ranges = max(1, min((int)gridDim.x, (T + p.min_tiles - 1) / p.min_tiles));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                t_min = min(t_min, __shfl_xor_sync(0xffffffffu, t_min, o));
+                t_max = max(t_max, __shfl_xor_sync(0xffffffffu, t_max, o));
+            }
+            if (t_min == t_max && U <= ranges) {
+                const int p_max = max(1, min(ranges / U, t_max / p.min_tiles));
+                const int cand = p_max - lane;                   // lane k tries P = p_max - k
+                const bool ok = cand >= 1 && t_max % cand == 0;
+                const unsigned m = __ballot_sync(0xffffffffu, ok);
+                if (m) {
+                    const int P = p_max - (__ffs(m) - 1);
+                    if (5 * U * P >= 4 * ranges) ranges = U * P;
+                }
+            }
+        }
         Schedule sc;                                     // (its table stays in shared memory)
-        build_schedule(sc, sm.sched, T, gridDim.x, p.pool_div, lane);     // (the consumers use it when a piece ends)
+        build_schedule(sc, sm.sched, T, ranges, p.pool_div, lane);     // (the consumers use it when a piece ends)
         const int R = sc.R, G = sc.G;
         {
             int acc = incl - mine;

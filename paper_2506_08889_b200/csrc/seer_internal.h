@@ -65,6 +65,7 @@ struct DecodeParams {
     int num_units;                  // batch * num_kv_heads
     int max_blocks_cap;             // tile-count clamp for dense: capacity in tiles
     int pool_div;                   // 1/pool_div of the tiles are handed out dynamically (0: none)
+    int min_tiles;                  // a CTA's range has at least this many tiles (fewer CTAs take part when work is short)
     float scale_log2;               // sm_scale * log2(e)
     unsigned int* status;
     unsigned long long* tickets;    // [num_units]: tiles done << 32 | valid-slot bits; zero between launches

@@ -496,9 +496,9 @@ seer_status seer_gate_select_threshold(seer_ctx* ctx, const seer_shape* shape, c
                               scores_out, stream);
 }
 
-seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,
-                              const void* k_nope, int64_t stride_batch, int64_t stride_head, int64_t stride_token,
-                              int rows_block_local, int first_block, int num_blocks, void* stream) {
+static seer_status kcomp_append_common(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,
+                                       const void* k_nope, int64_t stride_batch, int64_t stride_head, int64_t stride_token,
+                                       int rows_block_local, int first_block, int num_blocks, int wait_at_end, void* stream) {
     if (!ctx) return SEER_ERR_INVALID_ARG;
     seer_status st = check_shape(ctx, shape);
     if (st != SEER_OK) return st;
@@ -537,12 +537,20 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
     p.block_size = shape->block_size;
     p.d_gate = gate->d_gate;
     p.max_blocks = gate->max_blocks;
+    p.wait_at_end = wait_at_end;
     fill_inv_freq(p.inv_freq, gate->d_gate, gate->rope_theta);
     int launched = 0;
     ce = launch_kcomp_append(p, static_cast<cudaStream_t>(stream), &launched);
     ctx->launches += launched;
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "kcomp launch: %s", cudaGetErrorString(ce));
     return SEER_OK;
+}
+
+seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,
+                              const void* k_nope, int64_t stride_batch, int64_t stride_head, int64_t stride_token,
+                              int rows_block_local, int first_block, int num_blocks, void* stream) {
+    return kcomp_append_common(ctx, shape, gate, seq_lens, k_nope, stride_batch, stride_head, stride_token,
+                               rows_block_local, first_block, num_blocks, 0, stream);
 }
 
 seer_status seer_decode_step(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const seer_gate* gate,
@@ -552,16 +560,16 @@ seer_status seer_decode_step(seer_ctx* ctx, const seer_shape* shape, const seer_
                              float* lse, void* stream) {
     if (!ctx) return SEER_ERR_INVALID_ARG;
     if (!kv || !kv->seq_lens) return fail(ctx, SEER_ERR_INVALID_ARG, "kv or kv->seq_lens is NULL");
-    seer_status st;
-    if (k_nope) {
-        st = seer_kcomp_append(ctx, shape, gate, kv->seq_lens, k_nope, k_nope_stride_batch, k_nope_stride_head,
-                               k_nope_stride_token, k_nope_rows_block_local, -1, 1, stream);
-        if (st != SEER_OK) return st;
-    }
-    st = seer_gate_select(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, token_budget, block_idx, block_cnt, max_sel,
-                          nullptr, stream);
+    // The block that has just filled is the sequence's last block, which the gate always selects without
+    // scoring it (Sec. 3.2): its compressed key is first needed in the next step.  The append is therefore
+    // the step's last launch and does its work under the tail of the attention kernel.
+    seer_status st = seer_gate_select(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, token_budget, block_idx, block_cnt,
+                                      max_sel, nullptr, stream);
     if (st != SEER_OK) return st;
-    return seer_sparse_decode(ctx, shape, kv, q, block_idx, block_cnt, max_sel, out, lse, stream);
+    st = seer_sparse_decode(ctx, shape, kv, q, block_idx, block_cnt, max_sel, out, lse, stream);
+    if (st != SEER_OK || !k_nope) return st;
+    return kcomp_append_common(ctx, shape, gate, kv->seq_lens, k_nope, k_nope_stride_batch, k_nope_stride_head,
+                               k_nope_stride_token, k_nope_rows_block_local, -1, 1, 1, stream);
 }
 
 seer_status seer_decode_step_multi(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const seer_gate* gate,
@@ -572,16 +580,15 @@ seer_status seer_decode_step_multi(seer_ctx* ctx, const seer_shape* shape, const
     if (!ctx) return SEER_ERR_INVALID_ARG;
     if (!kv || !kv->seq_lens) return fail(ctx, SEER_ERR_INVALID_ARG, "kv or kv->seq_lens is NULL");
     if (q_len < 1 || q_len > 8) return fail(ctx, SEER_ERR_UNSUPPORTED, "q_len %d (supported 1..8)", q_len);
-    seer_status st;
-    if (k_nope) {
-        st = seer_kcomp_append(ctx, shape, gate, kv->seq_lens, k_nope, k_nope_stride_batch, k_nope_stride_head,
-                               k_nope_stride_token, k_nope_rows_block_local, -q_len, 1, stream);
-        if (st != SEER_OK) return st;
-    }
-    st = seer_gate_select_multi(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, q_len, token_budget, block_idx, block_cnt,
-                                max_sel, nullptr, stream);
+    // (the block that filled holds one of the query tokens, so it is among the blocks selected without a
+    // score: as in seer_decode_step the append comes last)
+    seer_status st = seer_gate_select_multi(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, q_len, token_budget, block_idx,
+                                            block_cnt, max_sel, nullptr, stream);
     if (st != SEER_OK) return st;
-    return seer_sparse_decode_multi(ctx, shape, kv, q, q_len, block_idx, block_cnt, max_sel, out, lse, stream);
+    st = seer_sparse_decode_multi(ctx, shape, kv, q, q_len, block_idx, block_cnt, max_sel, out, lse, stream);
+    if (st != SEER_OK || !k_nope) return st;
+    return kcomp_append_common(ctx, shape, gate, kv->seq_lens, k_nope, k_nope_stride_batch, k_nope_stride_head,
+                               k_nope_stride_token, k_nope_rows_block_local, -q_len, 1, 1, stream);
 }
 
 }  // extern "C"

@@ -128,6 +128,7 @@ struct KcompParams {
     int64_t stride_batch, stride_head, stride_token;
     int rows_block_local;
     int first_block, num_blocks;    // first_block == -t (1..8): the block that filled while the last t tokens were appended
+    int wait_at_end;                // append only: work first, wait for the preceding kernel just before the end
     int batch, num_kv_heads, block_size, d_gate, max_blocks;
     double inv_freq[kMaxDGate / 2];
 };

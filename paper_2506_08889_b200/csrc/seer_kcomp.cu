@@ -18,7 +18,7 @@ constexpr int kInChunks = 3 * kHeadDim / 8;          // 48 pieces of 16 B per W_
 // rotary pairs (c, c + d_gate/2), two at a time: their four W_k rows are requested before the
 // pooling starts.  (NB is the number of blocks per CTA; only NB = 1 is instantiated.)
 template <int NB>
-__global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) {
+__device__ __forceinline__ void kcomp_body(const KcompParams& p) {
     __shared__ float red[kKcWarps][3][kHeadDim];                   // per-warp pooled partials
     __shared__ __align__(16) float feat[NB][3 * kHeadDim];         // [max | min | avg]
 
@@ -29,8 +29,6 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
     const int pps = half / gridDim.z;                 // rotary pairs per row split
     const int pair_base = blockIdx.z * pps;
 
-    pdl_wait();
-    pdl_launch_dependents();
     // first batch of W_k rows, requested before the pooling starts
     uint4 wv[4][2];
     auto load_rows = [&](int pb) {
@@ -181,6 +179,19 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) 
             }
         }
     }
+}
+
+// The kernel normally waits for its predecessor in the stream before it touches memory.  As the last
+// kernel of a decode step (p.wait_at_end) its inputs -- the keys the caller wrote before the step --
+// are final from the start and nothing in the step reads the entry it writes, so it works at once, under
+// the tail of the attention kernel before it, and waits for that kernel only before it ends: its own
+// completion then still implies that of everything before it in the stream.
+template <int NB>
+__global__ void __launch_bounds__(kKcThreads) kcomp_kernel(const KcompParams p) {
+    if (!p.wait_at_end) pdl_wait();
+    pdl_launch_dependents();
+    kcomp_body<NB>(p);
+    if (p.wait_at_end) pdl_wait();
 }
 
 // ---- bulk build (after prefill): 16 consecutive blocks of one (sequence, KV head) per CTA --------

@@ -126,6 +126,16 @@ const char* seer_last_error(const seer_ctx* ctx);
  * results of the calls since the last check are invalid; the context's counters are
  * reset by this call and the context can be used again. */
 seer_status seer_get_device_status(seer_ctx* ctx, void* stream);
+
+/*
+ * Diagnostic: exercises the path every bounded device-side wait of the library takes when it runs out
+ * (Sec. 3.3's kernels never wait for one another; the waits are on the kernels' own copies in flight).
+ * One CTA polls `polls` times (1 .. 2^20) on a barrier that nobody arrives at, gives up, sets the sticky
+ * time-out bit and leaves a ticket and the scheduler counters non-zero, as a kernel that was cut short
+ * would.  The next seer_get_device_status then returns SEER_ERR_TIMEOUT and clears those counters, after
+ * which the context works as before.  Asynchronous on `stream`; faults nothing.
+ */
+seer_status seer_debug_wait_timeout(seer_ctx* ctx, int polls, void* stream);
 /* Workspace bytes a context needs for calls of this shape (upper bound);
  * max_blocks = largest number of blocks per sequence. */
 size_t seer_workspace_bytes(const seer_shape* shape, int max_blocks, int d_gate);

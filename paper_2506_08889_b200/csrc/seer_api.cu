@@ -30,7 +30,8 @@ struct MapKey {
     bool operator==(const MapKey& o) const { return memcmp(this, &o, sizeof(MapKey)) == 0; }
 };
 
-constexpr int kMapCache = 16;
+constexpr int kMapCache = 256;            // tensor-map cache slots (K and V of 128 layers), open addressing
+constexpr int kMapProbe = 8;              // slots looked at per lookup
 
 }  // namespace
 
@@ -42,8 +43,7 @@ struct seer_ctx {
     EncodeTiledFn encode;
     MapKey map_keys[kMapCache];
     CUtensorMap maps[kMapCache];
-    int map_used;
-    int map_next;
+    bool map_valid[kMapCache];
     uint64_t launches;
     unsigned int generation;    // stamps the partials of a decode launch
     int pool_div;               // decode scheduling: share of tiles handed out dynamically
@@ -136,11 +136,21 @@ seer_status get_map(seer_ctx* ctx, const void* base, const uint64_t dims[4], con
     for (int a = 0; a < 4; ++a) key.dims[a] = dims[a];
     for (int a = 0; a < 3; ++a) key.strides[a] = strides_bytes[a];
     key.box_rows = (uint64_t)box_rows;
-    for (int a = 0; a < ctx->map_used; ++a)
-        if (ctx->map_keys[a] == key) { *out = &ctx->maps[a]; return SEER_OK; }
-    int slot;
-    if (ctx->map_used < kMapCache) slot = ctx->map_used++;
-    else { slot = ctx->map_next; ctx->map_next = (ctx->map_next + 1) % kMapCache; }
+    // hashed on the base address (a layer's K or V cache), a few slots probed; a full neighbourhood
+    // gives up its first slot
+    const uint64_t hb = reinterpret_cast<uintptr_t>(base) >> 8;
+    const int home = (int)((hb ^ (hb >> 11) ^ (hb >> 23)) & (kMapCache - 1));
+    int slot = -1;
+    for (int a = 0; a < kMapProbe; ++a) {
+        const int c = (home + a) & (kMapCache - 1);
+        if (ctx->map_valid[c]) {
+            if (ctx->map_keys[c] == key) { *out = &ctx->maps[c]; return SEER_OK; }
+        } else if (slot < 0) {
+            slot = c;
+        }
+    }
+    if (slot < 0) slot = home;
+    ctx->map_valid[slot] = false;
     cuuint64_t gd[4] = {dims[0], dims[1], dims[2], dims[3]};
     cuuint64_t gs[3] = {strides_bytes[0], strides_bytes[1], strides_bytes[2]};
     cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};          // 64 channels (128 B) x 64 tokens (or one small block)
@@ -148,11 +158,9 @@ seer_status get_map(seer_ctx* ctx, const void* base, const uint64_t dims[4], con
     CUresult r = ctx->encode(&ctx->maps[slot], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gd, gs,
                              box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        memset(&ctx->map_keys[slot], 0, sizeof(MapKey));
-        return fail(ctx, SEER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
-    }
+    if (r != CUDA_SUCCESS) return fail(ctx, SEER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     ctx->map_keys[slot] = key;
+    ctx->map_valid[slot] = true;
     *out = &ctx->maps[slot];
     return SEER_OK;
 }
@@ -353,6 +361,42 @@ uint64_t seer_launch_count(const seer_ctx* ctx) { return ctx ? ctx->launches : 0
 void* seer_debug_trace_ptr(seer_ctx* ctx) { return ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)); }
 int seer_debug_ctas_per_sm(int sparse, int paged) { return decode_ctas_per_sm(sparse != 0, paged != 0, 1); }
 #endif
+
+namespace {
+// One CTA waits, with the given poll limit, on an mbarrier that nobody ever arrives at, gives up, raises
+// DEV_TIMEOUT as the library's kernels do, and leaves the counters that a kernel cut short would leave
+// (a ticket, the scheduler words, a claim counter) non-zero.
+__global__ void debug_wait_timeout_kernel(unsigned int* status, unsigned long long* tickets, int* sched, int* steal,
+                                          unsigned int polls) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait(&bar, 0, status, polls)) {
+        tickets[0] = (3ull << 32) | 5ull;
+        sched[0] = 7;
+        sched[1] = 2;
+        steal[1] = 1 | (1 << 16);
+    }
+}
+}  // namespace
+
+seer_status seer_debug_wait_timeout(seer_ctx* ctx, int polls, void* stream) {
+    if (!ctx) return SEER_ERR_INVALID_ARG;
+    if (polls < 1 || polls > (1 << 20)) return fail(ctx, SEER_ERR_INVALID_ARG, "polls must lie in 1 .. 2^20");
+    cudaError_t ce = cudaSetDevice(ctx->device);
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
+    const WsLayout w = ws_layout(1, 0, 0, 0);
+    debug_wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<unsigned int*>(ctx->ws), reinterpret_cast<unsigned long long*>(ctx->ws + w.tickets),
+        reinterpret_cast<int*>(ctx->ws + w.sched), reinterpret_cast<int*>(ctx->ws + w.steal), (unsigned int)polls);
+    ce = cudaGetLastError();
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "launch: %s", cudaGetErrorString(ce));
+    ctx->launches += 1;
+    return SEER_OK;
+}
 
 seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
     if (!ctx) return SEER_ERR_INVALID_ARG;

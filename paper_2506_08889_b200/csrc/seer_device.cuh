@@ -48,8 +48,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait: gives up after a fixed number of polls (well over a second of wall time),
 // raises DEV_TIMEOUT and returns false so that the caller can leave the kernel cleanly.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* status) {
-    for (uint32_t it = 0; it < (1u << 24); ++it) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* status,
+                                          uint32_t max_polls = 1u << 24) {
+    for (uint32_t it = 0; it < max_polls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it > 64) __nanosleep(64);
     }

@@ -125,3 +125,36 @@ def test_calls_of_different_shapes_interleaved_on_one_context(ctx):
                 check_attention(c["out"], c["lse"], *c["ref"], what=f"interleaved case {ci} rep {rep}")
             assert np.array_equal(gidx.cpu().numpy(), want_gidx) and np.array_equal(gcnt.cpu().numpy(), want_gcnt)
     assert ctx.device_status() == binding.SEER_OK
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(ctx):
+    # A bounded device-side wait that gives up sets the sticky time-out bit; the status call reports it once,
+    # clears the counters a kernel cut short would have left behind, and the context then decodes as before.
+    B, Hq, Hkv, d, b, S = 2, 8, 2, 128, 64, 64 * 160
+    lens = np.array([S, S - 1000], np.int32)
+    q, k, v = make_qkv(B, Hq, Hkv, S, d, 611, DEV)
+    n = [-(-int(L) // b) for L in lens]
+    idx, cnt = synth.random_block_lists(lens, Hkv, b, [x // 2 for x in n], max(n) // 2, 611)
+    ref = oracle.sparse(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.0884)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    kv = binding.make_kv(k, v, lens_t)
+    idx_t, cnt_t = torch.as_tensor(idx, device=DEV), torch.as_tensor(cnt, device=DEV)
+    out = torch.empty((B, Hq, d), dtype=torch.bfloat16, device=DEV)
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=DEV)
+
+    def decode_and_check(what):
+        out.fill_(float("nan"))
+        ctx.seer_sparse_decode(shape, kv, q, idx_t, cnt_t, idx.shape[2], out, lse)
+        torch.cuda.synchronize()
+        check_attention(out, lse, *ref, what=what, strict=True)
+
+    decode_and_check("before")
+    assert ctx.device_status() == binding.SEER_OK
+    ctx.seer_debug_wait_timeout(1000)                      # a wait on a barrier nobody arrives at, 1000 polls
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.SEER_ERR_TIMEOUT
+    assert ctx.device_status() == binding.SEER_OK          # reported once, then clear
+    decode_and_check("after the time-out")
+    decode_and_check("after the time-out, again")
+    assert ctx.device_status() == binding.SEER_OK

@@ -233,7 +233,7 @@ seer_status seer_gate_select(seer_ctx* ctx, const seer_shape* shape, const seer_
  * the other min(max(1, budget/b), n_i, max_sel) - (n_i - j_f) come from [0, j_f) by (score
  * descending, index ascending).  q_len = 1 is seer_gate_select.
  *  q_nope [B,q_len,Hq,d] bf16 (ignored when scores_in is given: selection only, scores_in holding
- *  the per-block maxima).  1 <= q_len <= 8; with scores_in == NULL, gate->max_blocks <= 8192.
+ *  the per-block maxima).  1 <= q_len <= 8.
  * Other arguments, outputs and errors as in seer_gate_select.
  */
 seer_status seer_gate_select_multi(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,

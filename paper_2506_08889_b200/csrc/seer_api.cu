@@ -97,7 +97,7 @@ WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks, int n_t
     w.part_o = d;  d = align_up(d + sizeof(float) * (size_t)slots * 8 * n_tiles * kHeadDim, 256);
     // gate view of the scratch
     size_t g = off;
-    w.q_gate = g;  g = align_up(g + sizeof(float) * (size_t)num_units * (size_t)(d_gate > 0 ? d_gate : 0), 256);
+    w.q_gate = g;  g = align_up(g + sizeof(float) * (size_t)num_units * 8 /* query tokens */ * (size_t)(d_gate > 0 ? d_gate : 0), 256);
     w.scores = g;  g = align_up(g + sizeof(float) * (size_t)num_units * (size_t)(max_blocks > 0 ? max_blocks : 0), 256);
     w.total = d > g ? d : g;
     return w;
@@ -459,9 +459,6 @@ static seer_status gate_select_common(seer_ctx* ctx, const seer_shape* shape, co
     if (max_sel <= 0 || gate->max_blocks <= 0) return fail(ctx, SEER_ERR_INVALID_ARG, "max_sel and max_blocks must be positive");
     if (token_budget < 0) return fail(ctx, SEER_ERR_INVALID_ARG, "token_budget is negative");
     if (q_len < 1 || q_len > 8) return fail(ctx, SEER_ERR_UNSUPPORTED, "q_len %d (supported 1..8)", q_len);
-    if (q_len > 1 && !scores_in && !gate_one_kernel(gate->max_blocks))
-        return fail(ctx, SEER_ERR_UNSUPPORTED, "q_len > 1 with max_blocks %d (the multi-token gate holds at most 8192 keys per unit)",
-                    gate->max_blocks);
     if (!scores_in) {
         if (!q_nope || !gate->w_q || !gate->kcomp)
             return fail(ctx, SEER_ERR_INVALID_ARG, "q_nope, w_q and kcomp are needed when scores_in is NULL");

@@ -389,7 +389,8 @@ __global__ void __launch_bounds__(kGateThreads) gate_select_only_kernel(const Ga
 }
 
 // ---- q_gate = RoPE_{L_i - 1}( W_q[h] . concat_g(Q_nope) )  (Eq. 1a) ---------------------------
-// grid (B*Hkv, d_gate/32): a CTA computes 16 rotary pairs; each of its 8 warps takes two pairs,
+// grid (B*Hkv, d_gate/32, q_len): a CTA computes 16 rotary pairs of one query token's gate query
+// (q_gate [B*Hkv][q_len][d_gate]); each of its 8 warps takes two pairs,
 // i.e. rows c, c+1, c+d_gate/2, c+1+d_gate/2, with all of their loads in flight together.
 // NIT = 16-byte pieces of a row per lane (row length g*128 bf16 = g*16 pieces over 32 lanes).
 template <int NIT>
@@ -401,8 +402,9 @@ __global__ void __launch_bounds__(kProjThreads) gate_qproj_kernel(const GatePara
     const int n = p.group * kHeadDim, chunks = n / 8, half = p.d_gate / 2;
     const int c0 = blockIdx.y * 16 + warp * 2;
     if (c0 >= half) return;
+    const int t = blockIdx.z;                          // query token (its position: L - q_len + t)
     const uint4* xsrc = reinterpret_cast<const uint4*>(
-        p.q_nope + ((size_t)i * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
+        p.q_nope + (((size_t)i * p.q_len + t) * p.num_q_heads + (size_t)h * p.group) * kHeadDim);
     const int L = __ldg(p.seq_lens + i);
     uint4 xv[NIT], wv[4][NIT];
 #pragma unroll
@@ -432,9 +434,9 @@ __global__ void __launch_bounds__(kProjThreads) gate_qproj_kernel(const GatePara
     if (lane < 2) {
         const int c = c0 + lane;
         float sn, cs;
-        rope_sincos((double)(L > 0 ? L - 1 : 0), p.inv_freq[c], &sn, &cs);
+        rope_sincos((double)max(L - p.q_len + t, 0), p.inv_freq[c], &sn, &cs);
         const float a = lane ? acc[1] : acc[0], b = lane ? acc[3] : acc[2];
-        float* dst = p.q_gate + (size_t)u * p.d_gate;
+        float* dst = p.q_gate + ((size_t)u * p.q_len + t) * p.d_gate;
         dst[c] = a * cs - b * sn;
         dst[c + half] = b * cs + a * sn;
     }
@@ -477,22 +479,39 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
     GATE_STAMP(1);
     pdl_launch_dependents();
     const int L = __ldg(p.seq_lens + i);
-    const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
-    const int n_cand = max(0, min(n_i - 1, p.max_blocks));
+    const int q_len = p.q_len;
+    // the blocks wholly before the first query token (for one token: all but the last block)
+    const int n_cand = min(max(0, L - q_len) / p.block_size, p.max_blocks);
     float* sc_out = p.scores + (size_t)u * p.max_blocks;
+    // this thread's 8 channels of every query token's gate query
+    const float* qbase = p.q_gate + (size_t)u * q_len * p.d_gate + 8 * csub;
     float qsub[8];
-    {
-        const float4 a = __ldcg(reinterpret_cast<const float4*>(p.q_gate + (size_t)u * p.d_gate + 8 * csub));
-        const float4 b = __ldcg(reinterpret_cast<const float4*>(p.q_gate + (size_t)u * p.d_gate + 8 * csub + 4));
+    auto load_q = [&](int t) {
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(qbase + (size_t)t * p.d_gate));
+        const float4 b = __ldcg(reinterpret_cast<const float4*>(qbase + (size_t)t * p.d_gate + 4));
         qsub[0] = a.x; qsub[1] = a.y; qsub[2] = a.z; qsub[3] = a.w;
         qsub[4] = b.x; qsub[5] = b.y; qsub[6] = b.z; qsub[7] = b.w;
-    }
+    };
+    load_q(0);
     const float inv = rsqrtf((float)p.d_gate);
     for (int cb = 0; cb < total; cb += kGateThreads * kBatch) {
-        float acc[kBatch];
+        // a key's score is the largest of its dot products with the query tokens' gate queries
+        float best[kBatch];
 #pragma unroll
-        for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
-        if (cb + kGateThreads * kBatch < total) {      // next batch on its way while this one reduces
+        for (int k = 0; k < kBatch; ++k) best[k] = -INFINITY;
+        for (int t = 0; t < q_len; ++t) {
+            if (q_len > 1) load_q(t);
+            float acc[kBatch];
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+                for (int off = lpk >> 1; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
+                best[k] = q_len > 1 ? fmaxf(best[k], acc[k]) : acc[k];
+            }
+        }
+        const int cb_now = cb;
+        if (cb + kGateThreads * kBatch < total) {      // next batch on its way while this one is stored
 #pragma unroll
             for (int k = 0; k < kBatch; ++k) {
                 const int c = cb + (kBatch + k) * kGateThreads + tid;
@@ -501,10 +520,9 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
         }
 #pragma unroll
         for (int k = 0; k < kBatch; ++k) {
-            for (int off = lpk >> 1; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
-            const int c = cb + k * kGateThreads + tid;
+            const int c = cb_now + k * kGateThreads + tid;
             const int j = j0 + c / lpk;
-            if (c < total && csub == 0 && j < n_cand) __stcg(sc_out + j, acc[k] * inv);
+            if (c < total && csub == 0 && j < n_cand) __stcg(sc_out + j, best[k] * inv);
         }
     }
     // ---- ticket: the last slice of the unit to finish does the selection --------------------
@@ -788,7 +806,7 @@ cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* la
         *launched = 1;
         return e;
     }
-    const dim3 pgrid(U, (p.d_gate / 2 + 15) / 16);
+    const dim3 pgrid(U, (p.d_gate / 2 + 15) / 16, p.q_len);
     switch (nit) {
         case 1: e = launch_pdl(gate_qproj_kernel<1>, pgrid, dim3(kProjThreads), 0, stream, p); break;
         case 2: e = launch_pdl(gate_qproj_kernel<2>, pgrid, dim3(kProjThreads), 0, stream, p); break;

@@ -192,6 +192,40 @@ def test_gate_multi_scores_and_selection(ctx, g, T, b, dg):
     assert ctx.device_status() == binding.SEER_OK
 
 
+@pytest.mark.parametrize("g,T,dg", [(5, 3, 128), (4, 8, 64)])
+def test_gate_multi_more_keys_than_one_cluster_holds(ctx, g, T, dg):
+    # more than 8192 compressed keys per unit: the projection kernel makes one gate query per token,
+    # the score kernel keeps per key the largest of the tokens' scores, the last slice selects
+    B, Hkv, d, b = 2, 2, 128, 64
+    Hq = g * Hkv
+    nbmax = 9000
+    lens = np.array([nbmax * b - 1, 8300 * b + 2], np.int32)     # the T tokens straddle two blocks in both
+    qn = synth.normal_bf16((B, T, Hq, d), 90 + T, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, g * d), 90 + T, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nbmax, dg), 90 + T, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    max_sel = 300
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nbmax), dtype=torch.float32, device=DEV)
+    ctx.seer_gate_select_multi(shape, gate, lens_t, qn, None, T, max_sel * b, idx, cnt, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    want_sc = oracle.scores_multi(bits(qn), bits(wq), bits(kc), lens, b, THETA)
+    got_sc = sc.cpu().numpy()
+    for i in range(B):
+        jf = max(0, int(lens[i]) - T) // b
+        assert np.abs(got_sc[i, :, :jf] - want_sc[i, :, :jf]).max() <= 1e-3
+    for budget in (max_sel * b, 17 * b):
+        ctx.seer_gate_select_multi(shape, gate, lens_t, qn, None, T, budget, idx, cnt, max_sel)
+        torch.cuda.synchronize()
+        want_idx, want_cnt = oracle.select_multi(got_sc, lens, b, budget, T, max_sel)
+        assert np.array_equal(cnt.cpu().numpy(), want_cnt), budget
+        assert np.array_equal(idx.cpu().numpy(), want_idx), budget
+    assert ctx.device_status() == binding.SEER_OK
+
+
 def test_gate_multi_with_one_token_is_bitwise_the_single_token_gate(ctx):
     B, Hq, Hkv, d, dg, b, nbmax = 3, 40, 8, 128, 128, 64, 2048
     lens = np.array([nbmax * b, 1000 * b + 17, 64], np.int32)

@@ -242,6 +242,20 @@ seer_status seer_gate_select_multi(seer_ctx* ctx, const seer_shape* shape, const
                                    int max_sel, float* scores_out, void* stream);
 
 /*
+ * The threshold method (Sec. 3.1, second method) for q_len query tokens per sequence.  The paper has
+ * neither; the reading combines the two above: the per-block scores are the maxima over the tokens'
+ * scores, the softmax runs over the candidate blocks [0, j_f), a candidate is selected when its
+ * probability exceeds `threshold`, the blocks j_f .. n_i - 1 that hold the query tokens are always
+ * selected and take no part in the normalisation, and when more candidates pass than max_sel leaves room
+ * for beside those, the highest-scoring ones are kept.  q_len = 1 is seer_gate_select_threshold.
+ * Arguments as in seer_gate_select_multi (threshold in [0, 1] in place of the token budget).
+ */
+seer_status seer_gate_select_threshold_multi(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                                             const int32_t* seq_lens, const void* q_nope, const float* scores_in,
+                                             int q_len, float threshold, int32_t* block_idx, int32_t* block_cnt,
+                                             int max_sel, float* scores_out, void* stream);
+
+/*
  * The threshold method of Sec. 3.1: the scores are normalised by a softmax over the blocks
  * that have a compressed key (Eq. 1c; blocks [0, n_i - 1)), and the blocks whose probability
  * exceeds `threshold` are selected -- a different number for every (sequence, KV head).  The

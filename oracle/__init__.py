@@ -246,6 +246,23 @@ def select_threshold(scores_f32, seq_lens, block_size, tau, max_sel):
     return idx, cnt, probs
 
 
+def select_threshold_multi(scores_f32, seq_lens, block_size, tau, q_len, max_sel):
+    """Threshold selection for q_len query tokens: softmax over the blocks wholly before the first query
+    token, the blocks holding the query tokens forced.  Returns (idx, cnt, probs f64 [B,Hkv,max_blocks])."""
+    s = np.ascontiguousarray(np.asarray(scores_f32))
+    if s.dtype != np.float32:
+        raise TypeError("selection is defined on fp32 scores")
+    B, Hkv, max_blocks = s.shape
+    seq_lens = _i32(seq_lens)
+    idx = np.zeros((B, Hkv, max_sel), np.int32)
+    cnt = np.zeros((B, Hkv), np.int32)
+    probs = np.zeros((B, Hkv, max_blocks), np.float64)
+    lib().oracle_select_threshold_multi(_p(s), _p(seq_lens), ctypes.c_int(B), ctypes.c_int(Hkv),
+                                        ctypes.c_int(block_size), ctypes.c_int(max_blocks), ctypes.c_double(tau),
+                                        ctypes.c_int(q_len), ctypes.c_int(max_sel), _p(idx), _p(cnt), _p(probs))
+    return idx, cnt, probs
+
+
 def rope(y, pos, theta):
     """Rotate one fp64 vector (length d_gate) to position ``pos``."""
     y = np.array(y, dtype=np.float64).copy()

@@ -548,3 +548,49 @@ void oracle_select_multi(const float *scores, const int32_t *seq_lens,
         }
 }
 
+/* Threshold selection for T query tokens per sequence (the reading taken for Sec. 3.1's second method
+ * when several tokens are decoded at once; the paper has no such case): the per-block scores are the
+ * maxima over the tokens (oracle_scores_multi); the softmax runs over the candidate blocks, those wholly
+ * before the first query token, [0, jf) with jf = floor((L - T) / b); a candidate is selected if its
+ * probability exceeds tau; the blocks that hold a query token, jf .. n-1, are always selected and take no
+ * part in the normalisation; if more candidates pass than the list has room for beside the forced
+ * blocks, the highest-scoring ones are kept (score descending, index ascending). */
+void oracle_select_threshold_multi(const float *scores, const int32_t *seq_lens,
+                                   int B, int Hkv, int b, int max_blocks, double tau, int T,
+                                   int max_sel, int32_t *block_idx, int32_t *block_cnt, double *probs_out)
+{
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int i = 0; i < B; ++i)
+        for (int h = 0; h < Hkv; ++h) {
+            int32_t *dst = block_idx + ((int64_t)i * Hkv + h) * max_sel;
+            for (int e = 0; e < max_sel; ++e) dst[e] = -1;
+            int L = seq_lens[i];
+            int n = (L + b - 1) / b;
+            if (n <= 0) { block_cnt[i * Hkv + h] = 0; continue; }
+            int jf = L - T > 0 ? (L - T) / b : 0;
+            int forced = n - jf;
+            if (forced > max_sel) forced = max_sel;
+            const float *s = scores + ((int64_t)i * Hkv + h) * max_blocks;
+            int ncand = jf < max_blocks ? jf : max_blocks;
+            double mx = -INFINITY, z = 0.0;
+            for (int j = 0; j < ncand; ++j) if ((double)s[j] > mx) mx = (double)s[j];
+            for (int j = 0; j < ncand; ++j) z += exp((double)s[j] - mx);
+            int above = 0;
+            for (int j = 0; j < ncand; ++j) {
+                double pj = exp((double)s[j] - mx) / z;
+                if (probs_out) probs_out[((int64_t)i * Hkv + h) * max_blocks + j] = pj;
+                if (pj > tau) ++above;
+            }
+            int need = above;
+            if (need > max_sel - forced) need = max_sel - forced;
+            cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(ncand > 0 ? ncand : 1));
+            for (int j = 0; j < ncand; ++j) { cand[j].s = s[j]; cand[j].j = j; }
+            qsort(cand, (size_t)ncand, sizeof(cand_t), cand_before);
+            int m = 0;
+            for (int e = 0; e < need && e < ncand; ++e) dst[m++] = cand[e].j;
+            for (int j = n - forced; j < n; ++j) dst[m++] = j;
+            qsort(dst, (size_t)m, sizeof(int32_t), int_asc);
+            free(cand);
+            block_cnt[i * Hkv + h] = m;
+        }
+}

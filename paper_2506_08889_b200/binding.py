@@ -32,7 +32,7 @@ EXPORTS = [
     "seer_dense_decode", "seer_sparse_decode", "seer_gate_select", "seer_kcomp_append",
     "seer_gate_select_static", "seer_decode_step", "seer_gate_select_threshold",
     "seer_sparse_decode_multi", "seer_dense_decode_multi", "seer_gate_select_multi", "seer_decode_step_multi",
-    "seer_debug_wait_timeout",
+    "seer_debug_wait_timeout", "seer_gate_select_threshold_multi",
 ]
 
 
@@ -112,6 +112,9 @@ def lib() -> ctypes.CDLL:
     L.seer_gate_select_threshold.restype = i32
     L.seer_gate_select_threshold.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, vp,
                                              ctypes.c_float, vp, vp, i32, vp, vp]
+    L.seer_gate_select_threshold_multi.restype = i32
+    L.seer_gate_select_threshold_multi.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, vp, i32,
+                                                   ctypes.c_float, vp, vp, i32, vp, vp]
     L.seer_decode_step_multi.restype = i32
     L.seer_decode_step_multi.argtypes = [vp, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerKV), ctypes.POINTER(SeerGate),
                                          vp, vp, i32, vp, i64, i64, i64, i32, i32, vp, vp, i32, vp, vp, vp]
@@ -248,6 +251,13 @@ class Context:
                                                      _ptr(seq_lens), _ptr(q_nope), _ptr(scores_in),
                                                      ctypes.c_float(threshold), _ptr(block_idx), _ptr(block_cnt),
                                                      int(max_sel), _ptr(scores_out), _stream(stream)))
+
+    def seer_gate_select_threshold_multi(self, shape: SeerShape, gate: SeerGate, seq_lens, q_nope, scores_in, q_len,
+                                         threshold, block_idx, block_cnt, max_sel, scores_out=None, stream=None):
+        self._check(lib().seer_gate_select_threshold_multi(self._h, ctypes.byref(shape), ctypes.byref(gate),
+                                                           _ptr(seq_lens), _ptr(q_nope), _ptr(scores_in), int(q_len),
+                                                           ctypes.c_float(threshold), _ptr(block_idx), _ptr(block_cnt),
+                                                           int(max_sel), _ptr(scores_out), _stream(stream)))
 
     def seer_kcomp_append(self, shape: SeerShape, gate: SeerGate, seq_lens, k_nope, rows_block_local=False,
                           first_block=-1, num_blocks=1, stream=None):

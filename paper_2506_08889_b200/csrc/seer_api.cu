@@ -587,6 +587,16 @@ static seer_status kcomp_append_common(seer_ctx* ctx, const seer_shape* shape, c
     return SEER_OK;
 }
 
+seer_status seer_gate_select_threshold_multi(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate,
+                                             const int32_t* seq_lens, const void* q_nope, const float* scores_in,
+                                             int q_len, float threshold, int32_t* block_idx, int32_t* block_cnt,
+                                             int max_sel, float* scores_out, void* stream) {
+    if (ctx && !(threshold >= 0.f && threshold <= 1.f))
+        return fail(ctx, SEER_ERR_INVALID_ARG, "threshold must lie in [0, 1] (it is compared with a softmax probability)");
+    return gate_select_common(ctx, shape, gate, seq_lens, q_nope, scores_in, 0, 1, threshold, block_idx, block_cnt, max_sel,
+                              scores_out, stream, q_len);
+}
+
 seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer_gate* gate, const int32_t* seq_lens,
                               const void* k_nope, int64_t stride_batch, int64_t stride_head, int64_t stride_token,
                               int rows_block_local, int first_block, int num_blocks, void* stream) {

@@ -226,6 +226,47 @@ def test_gate_multi_more_keys_than_one_cluster_holds(ctx, g, T, dg):
     assert ctx.device_status() == binding.SEER_OK
 
 
+@pytest.mark.parametrize("nbmax,tau,T", [(700, 2e-3, 3), (9000, 1.5e-4, 4)])
+def test_gate_multi_threshold_method(ctx, nbmax, tau, T):
+    # the threshold method with several query tokens, through both scoring paths: scores against the oracle,
+    # the selection against the oracle's rule on the GPU's own scores (only blocks whose probability is
+    # within rounding of tau may fall on either side)
+    B, Hkv, g, d, dg, b = 2, 2, 4, 128, 128, 64
+    Hq = g * Hkv
+    max_sel = nbmax // 2
+    lens = np.array([nbmax * b - 1, (nbmax // 2) * b + 2], np.int32)
+    qn = synth.normal_bf16((B, T, Hq, d), 77, "thr:qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, g * d), 77, "thr:wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nbmax, dg), 77, "thr:kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nbmax)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    idx = torch.full((B, Hkv, max_sel), 77, dtype=torch.int32, device=DEV)
+    cnt = torch.full((B, Hkv), 77, dtype=torch.int32, device=DEV)
+    sc = torch.zeros((B, Hkv, nbmax), dtype=torch.float32, device=DEV)
+    ctx.seer_gate_select_threshold_multi(shape, gate, lens_t, qn, None, T, tau, idx, cnt, max_sel, scores_out=sc)
+    torch.cuda.synchronize()
+    want_sc = oracle.scores_multi(bits(qn), bits(wq), bits(kc), lens, b, THETA)
+    got_sc = sc.cpu().numpy()
+    for i in range(B):
+        jf = max(0, int(lens[i]) - T) // b
+        assert np.abs(got_sc[i, :, :jf] - want_sc[i, :, :jf]).max() <= 1e-3
+    want_idx, want_cnt, probs = oracle.select_threshold_multi(got_sc, lens, b, tau, T, max_sel)
+    idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+    for i in range(B):
+        L = int(lens[i])
+        n, jf = -(-L // b), max(0, L - T) // b
+        for h in range(Hkv):
+            got = set(idx[i, h, :cnt[i, h]].tolist())
+            want = set(want_idx[i, h, :want_cnt[i, h]].tolist())
+            assert set(range(jf, n)) <= got and list(idx[i, h, :cnt[i, h]]) == sorted(got)
+            assert np.all(idx[i, h, cnt[i, h]:] == -1)
+            for j in got ^ want:
+                assert abs(probs[i, h, j] - tau) <= 1e-5 * tau + 1e-9, (i, h, j, probs[i, h, j])
+            assert n - jf < len(got) < n                     # the threshold cut somewhere inside
+    assert ctx.device_status() == binding.SEER_OK
+
+
 def test_gate_multi_with_one_token_is_bitwise_the_single_token_gate(ctx):
     B, Hq, Hkv, d, dg, b, nbmax = 3, 40, 8, 128, 128, 64, 2048
     lens = np.array([nbmax * b, 1000 * b + 17, 64], np.int32)

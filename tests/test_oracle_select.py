@@ -176,3 +176,59 @@ def test_multi_token_selection_against_lexsort_with_forced_blocks(T):
                     pos = L - T + t
                     if pos >= 0:
                         assert pos // b in want
+
+
+# ---- threshold selection for several query tokens ----------------------------------------------------
+
+def test_threshold_multi_with_one_token_is_the_single_token_routine():
+    r = np.random.default_rng(321)
+    B, Hkv, b, max_blocks = 3, 2, 16, 50
+    lens = np.array([50 * 16, 31 * 16 + 7, 16], np.int32)
+    sc = (r.normal(size=(B, Hkv, max_blocks)) * 2.0).astype(np.float32)
+    for tau in (0.004, 0.03):
+        for max_sel in (50, 7):
+            a = oracle.select_threshold(sc, lens, b, tau, max_sel)
+            m = oracle.select_threshold_multi(sc, lens, b, tau, 1, max_sel)
+            assert np.array_equal(a[0], m[0]) and np.array_equal(a[1], m[1])
+            assert np.allclose(a[2], m[2], rtol=0, atol=0)
+
+
+@pytest.mark.parametrize("T", [2, 5, 8])
+def test_threshold_multi_against_numpy_softmax_and_forced_range(T):
+    r = np.random.default_rng(400 + T)
+    B, Hkv, b, max_blocks, max_sel = 4, 2, 16, 40, 40
+    # the T tokens inside one block; straddling two blocks; exactly filling a block's end; fewer tokens than T
+    lens = np.array([40 * 16, 21 * 16 + 2, 30 * 16, 3], np.int32)
+    sc = (r.normal(size=(B, Hkv, max_blocks)) * 2.0).astype(np.float32)
+    tau = 0.03
+    idx, cnt, probs = oracle.select_threshold_multi(sc, lens, b, tau, T, max_sel)
+    for i in range(B):
+        L = int(lens[i])
+        n = -(-L // b)
+        jf = max(0, L - T) // b
+        forced = list(range(jf, n))
+        for h in range(Hkv):
+            got = list(idx[i, h, : cnt[i, h]])
+            if jf:
+                p = _softmax64(sc[i, h, :jf])
+                assert np.allclose(probs[i, h, :jf], p, rtol=1e-12)
+                want = sorted([j for j in range(jf) if p[j] > tau] + forced)
+            else:
+                want = forced
+            assert got == want and np.all(idx[i, h, cnt[i, h]:] == -1)
+    # the forced blocks' own scores play no role
+    sc2 = sc.copy()
+    for i in range(B):
+        jf = max(0, int(lens[i]) - T) // b
+        sc2[i, :, jf:] = 1e9
+    idx2, cnt2, _ = oracle.select_threshold_multi(sc2, lens, b, tau, T, max_sel)
+    assert np.array_equal(idx2, idx) and np.array_equal(cnt2, cnt)
+
+
+def test_threshold_multi_truncation_keeps_the_best_beside_the_forced_blocks():
+    # blocks of 4 tokens, L = 30: n = 8 blocks; T = 3 tokens at positions 27..29: jf = 6, forced {6, 7}
+    sc = np.array([[[1, 3, 2, 3, 0, 1, 9, 9]]], np.float32)
+    idx, cnt, _ = oracle.select_threshold_multi(sc, [30], 4, 1e-6, 3, 4)     # all six pass, room for two
+    assert list(idx[0, 0]) == [1, 3, 6, 7] and cnt[0, 0] == 4               # (ties: the lower index first)
+    idx, cnt, _ = oracle.select_threshold_multi(sc, [30], 4, 0.9, 3, 4)      # nothing passes: the forced only
+    assert list(idx[0, 0, :2]) == [6, 7] and cnt[0, 0] == 2

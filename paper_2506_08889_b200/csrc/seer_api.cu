@@ -202,9 +202,13 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
     // Query tokens share a launch while (tokens x group) fits the kernel's 16 rows; more tokens
     // take further launches over the same lists (each reads the selected K/V once).
+    // Up to 16 rows ride on the MMA's N side (tokens on M); more than 16 rows (with blocks of 64 or 128 tokens)
+    // take the variant with the rows on M, up to 64 a launch.
     const int group = shape->num_q_heads / shape->num_kv_heads;
-    const int tok_per_launch = q_len < 16 / group ? q_len : 16 / group;
-    const int n_tiles = tok_per_launch * group > 8 ? 2 : 1;
+    const bool wide = q_len * group > 16 && bpt == 1;
+    const int row_cap = wide ? 64 : 16;
+    const int tok_per_launch = q_len < row_cap / group ? q_len : row_cap / group;
+    const int n_tiles = wide ? 8 : tok_per_launch * group > 8 ? 2 : 1;
     const int per_sm = decode_ctas_per_sm(sparse, paged, n_tiles);
     if (per_sm <= 0) return fail(ctx, SEER_ERR_CUDA, "decode kernel cannot be resident (shared memory)");
     long long max_tiles = sparse ? (long long)U * ((max_sel + bpt - 1) / bpt) * tpb
@@ -212,8 +216,13 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     int grid = ctx->num_sms * per_sm;
     if (grid > kMaxGridCtas) grid = kMaxGridCtas;
     if (max_tiles < grid) grid = (int)(max_tiles > 0 ? max_tiles : 1);
-    const int slots = decode_max_intervals(grid) + U;
-    const WsLayout w = ws_layout(U, slots, 0, 0, n_tiles);
+    // a partial slot of the wide variant is 33 KiB: fewer dynamic chunks per range if the workspace asks for it
+    int max_rounds = kMaxRounds;
+    WsLayout w = ws_layout(U, decode_max_intervals(grid, max_rounds) + U, 0, 0, n_tiles);
+    while (w.total > ctx->ws_bytes && max_rounds > 0) {
+        --max_rounds;
+        w = ws_layout(U, decode_max_intervals(grid, max_rounds) + U, 0, 0, n_tiles);
+    }
     if (w.total > ctx->ws_bytes)
         return fail(ctx, SEER_ERR_WORKSPACE, "workspace %zu bytes, call needs %zu", ctx->ws_bytes, w.total);
 
@@ -263,6 +272,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.max_blocks_cap = (kv->max_seq_len + kTileTokens - 1) / kTileTokens;
     p.pool_div = ctx->pool_div;
     p.min_tiles = ctx->min_tiles;
+    p.max_rounds = max_rounds;
     p.scale_log2 = shape->sm_scale * 1.4426950408889634f;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
     p.tickets = reinterpret_cast<unsigned long long*>(ctx->ws + w.tickets);
@@ -421,7 +431,7 @@ seer_status seer_get_device_status(seer_ctx* ctx, void* stream) {
 size_t seer_workspace_bytes(const seer_shape* shape, int max_blocks, int d_gate) {
     if (!shape || shape->batch <= 0 || shape->num_kv_heads <= 0) return 0;
     const int U = shape->batch * shape->num_kv_heads;
-    return ws_layout(U, decode_max_intervals(kMaxGridCtas) + U, d_gate, max_blocks, 2).total;
+    return ws_layout(U, decode_max_intervals(kMaxGridCtas) + U, d_gate, max_blocks, 2).total;   // (enough for every call; more lets the 17-to-64-row decode use more dynamic chunks)
 }
 
 seer_status seer_dense_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv, const void* q, void* out,

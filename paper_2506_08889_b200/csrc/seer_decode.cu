@@ -54,6 +54,7 @@ constexpr int kListInts = kStageBytes / 4 - 64;              // slot numbers tha
 constexpr int kLandBytes = 2 * kStageBytes;                 // landing area for staged partials: two stage buffers
 constexpr int kMaxSteals = 14;                             // chunks a CTA may take from other ranges
 constexpr int kFewTilesPerCta = 16;                        // up to this many tiles per CTA the number of ranges is chosen with care
+constexpr int kWideTiles = 8;                              // N-tile count that stands for the rows-on-M variant (up to 64 rows)
 constexpr int kAheadMaxChunk = 8;                          // own chunks up to this size are claimed ahead
 constexpr int kAheadTiles = 3;                             // tiles left to issue when the next interval's claim is made
 constexpr int kSmemUnits = 128;                            // units whose tile-count prefix sums fit in shared memory
@@ -160,7 +161,8 @@ __device__ __forceinline__ int range_of(const Schedule& s, int t) {
 // `shared`, where all of the schedule is also left for the other warps.  Lane k takes level k of the
 // tail, [b - (q/4 >> k), b - (q/4 >> (k+1))), and cuts it into pieces of `cap` tiles (a power of two)
 // counted from its back end, the front piece taking the remainder.
-__device__ __forceinline__ void build_schedule(Schedule& s, Schedule& shared, int T, int grid, int pool_div, int lane) {
+__device__ __forceinline__ void build_schedule(Schedule& s, Schedule& shared, int T, int grid, int pool_div, int max_rounds,
+                                               int lane) {
     s.T = T;
     s.G = max(1, min(grid, T));
     const int q = (int)((unsigned int)T / (unsigned int)s.G);   // shortest range (>= 1 whenever T > 0)
@@ -169,14 +171,14 @@ __device__ __forceinline__ void build_schedule(Schedule& s, Schedule& shared, in
     int R = 0;
     if (pool_div > 0 && q >= kMinStaticTilesPerCta) {
         const int tail = pool_div == 4 ? q >> 2 : q / pool_div;
-        // (with one piece per level there are at most kMaxRounds pieces, so the loop ends at the latest
+        // (with one piece per level there are at most max_rounds pieces, so the loop ends at the latest
         // when cap exceeds the tail)
         for (int cap_shift = 3 + max(0, 23 - __clz(q)); cap_shift < 31; ++cap_shift) {      // cap = 8, or about q/32 .. q/64
             // level k = [b - prev, b - nxt): halves, down to kMinChunk tiles; the last level takes the rest
-            int prev = lane < kMaxRounds ? tail >> lane : 0;
+            int prev = lane < max_rounds ? tail >> lane : 0;
             if (lane > 0 && prev < kMinChunk) prev = 0;
             int nxt = prev >> 1;
-            if (nxt < kMinChunk || lane == kMaxRounds - 1) nxt = 0;
+            if (nxt < kMinChunk || lane == max_rounds - 1) nxt = 0;
             const int size = prev - nxt;                    // (0 for the levels past the last)
             const int parts = (size + (1 << cap_shift) - 1) >> cap_shift;
             int incl = parts;
@@ -186,7 +188,7 @@ __device__ __forceinline__ void build_schedule(Schedule& s, Schedule& shared, in
                 if (lane >= o) incl += v;
             }
             R = __shfl_sync(0xffffffffu, incl, 31);
-            if (R > kMaxRounds) { R = 0; continue; }
+            if (R > max_rounds) { R = 0; continue; }
             // piece i of the level (front to back) starts prev tiles before the range's end for i = 0,
             // nxt + (parts - i) * cap for the others
             for (int i = 0; i < parts; ++i) shared.off[incl - parts + 1 + i] = i == 0 ? prev : nxt + ((parts - i) << cap_shift);
@@ -393,7 +395,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             mbar_init(&sm.full[s], 1);
             mbar_init(&sm.empty[s], kConsumerWarps);
         }
-        mbar_init(&sm.merge_bar[0], kConsumerWarps - 1);
+        mbar_init(&sm.merge_bar[0], NT < kWideTiles ? kConsumerWarps - 1 : kConsumerWarps);   // (rows on M: "partial written" by all four)
         mbar_init(&sm.merge_bar[1], 1);
         mbar_init(&sm.end_bar, kConsumerWarps);
         mbar_init(&sm.list_bar, kConsumerWarps);
@@ -472,7 +474,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             }
         }
         Schedule sc;                                     // (its table stays in shared memory)
-        build_schedule(sc, sm.sched, T, ranges, p.pool_div, lane);     // (the consumers use it when a piece ends)
+        build_schedule(sc, sm.sched, T, ranges, p.max_rounds > 0 ? p.pool_div : 0, min(max(p.max_rounds, 1), kMaxRounds), lane);     // (the consumers use it when a piece ends)
         const int R = sc.R, G = sc.G;
         {
             int acc = incl - mine;
@@ -846,14 +848,16 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     const int w = warp;
     const int qd = lane & 3;            // column pair: rows 2*qd, 2*qd+1 of every N-tile
     const int rw = lane >> 2;           // row within an 8-row slab
+    unsigned long long tk_before = 0ull; // warp 0, lane k: what the unit's counter held before the k-th held piece was added
+    unsigned int tk_bit = 0u;            // ... and that piece's bit
+    int piece_tiles = 0, piece_iv = 0;  // tiles in the current piece, interval it started in
+    if constexpr (NT < kWideTiles) {
+    // ---------------- tokens on the MMA's M side, the unit's (up to 16) rows on N ----------------
     uint32_t bq[NT][8][2];              // Q^T B-fragments: NT N-tiles x 8 k-steps over d
     uint32_t bq_pre[8][2];              // NT == 1: the same for the unit expected next (prefetched)
     float o[NT][8][4];                  // O^T accumulators: 8 m-tiles over d per N-tile
     float m_run[NT][2], l_run[NT][2];
     int seg = 0;                        // merge rounds finished so far (NT per piece)
-    unsigned long long tk_before = 0ull; // warp 0, lane k: what the unit's counter held before the k-th held piece was added
-    unsigned int tk_bit = 0u;            // ... and that piece's bit
-    int piece_tiles = 0, piece_iv = 0;  // tiles in the current piece, interval it started in
     // Query token of this thread's two columns in every N-tile, as the number of newest cached
     // tokens it may not see (q_len - 1 - token): column c of N-tile nt is row 8*nt + c of the unit,
     // i.e. token t_base + row / group.  Rows past p.rows are padding (their result is never stored).
@@ -1194,6 +1198,217 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         }
         mt = nx;
     }
+    } else {
+    // ---------------- the unit's (17 to 64) rows on the MMA's M side, tokens on N ----------------
+    // Warp w owns rows 16w .. 16w+15 of the unit and goes through all 64 tokens of every tile, so its
+    // running max, sum and 16 x 128 output block are complete for its rows: nothing is folded across
+    // warps when a piece ends.
+    //     S (16 rows x 64 tok) = Q_w (16 x 128) . K^T (128 x 64)       mma.sync m16n8k16, K straight from its tile
+    //     O (16 rows x 128)   += P (16 x 64) . V (64 x 128)           P from S's registers, V through ldmatrix.trans
+    const int rA = 16 * w + rw, rB = rA + 8;                            // this thread's two rows
+    const bool realA = rA < p.rows, realB = rB < p.rows;
+    // newest cached tokens a row may not see (its query token's distance from the last one)
+    const int backA = realA ? p.q_len - 1 - (p.t_base + ((rA * p.group_magic) >> 16)) : 0;
+    const int backB = realB ? p.q_len - 1 - (p.t_base + ((rB * p.group_magic) >> 16)) : 0;
+    uint32_t qa[8][4];                  // Q A-fragments: 8 k-steps over d
+    float o[16][4];                     // O accumulators: 16 n-tiles of 8 channels
+    float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;
+    int pubs = 0;                       // partials written so far (phase of pub_bar)
+    auto load_q_wide = [&](int unit) {
+        const uint32_t* qrA = reinterpret_cast<const uint32_t*>(p.q + unit_row(p, unit, realA ? rA : 0) * kHeadDim);
+        const uint32_t* qrB = reinterpret_cast<const uint32_t*>(p.q + unit_row(p, unit, realB ? rB : 0) * kHeadDim);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            qa[ks][0] = realA ? __ldg(qrA + 8 * ks + qd) : 0u;
+            qa[ks][1] = realB ? __ldg(qrB + 8 * ks + qd) : 0u;
+            qa[ks][2] = realA ? __ldg(qrA + 8 * ks + 4 + qd) : 0u;
+            qa[ks][3] = realB ? __ldg(qrB + 8 * ks + 4 + qd) : 0u;
+        }
+    };
+    // lane-constant parts of the ldmatrix addresses (swizzle: 16-B chunk ^= row & 7)
+    const int sw = lane & 7;
+    const int k_cb = lane >> 3;                          // K: which of the four 8-channel blocks of a load
+    const int v_tok = 8 * ((lane >> 3) & 1) + (lane & 7);  // V: token within a 16-token step
+    const int v_cb = lane >> 4;                          // V: which of the two 8-channel blocks of a load
+    if (!mbar_wait(&sm.full[0], 0, p.status)) return;
+    if (tid == 0) SEER_STAMP(10);
+    StageMeta mt = sm.meta[0];
+    for (int it = 0; mt.nvalid >= 0; ++it) {
+        const int st = it % kStages;
+        if (mt.flags & 1) {
+            load_q_wide(mt.unit);
+#pragma unroll
+            for (int ct = 0; ct < 16; ++ct)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) o[ct][x] = 0.f;
+            mA = mB = -INFINITY;
+            lA = lB = 0.f;
+            piece_tiles = 0;
+            piece_iv = mt.interval;
+        }
+        ++piece_tiles;
+        const int nv = mt.nvalid;                          // cached tokens from the tile's first row on (capped at 64 + 7)
+        if (nv > 0 && w * 16 < p.rows) {
+            const uint32_t kbase = smem_u32(sm.stage[st]);
+            const uint32_t vbase = kbase + kTileBytes;
+            if (nv < kTileTokens) {
+                // ragged tail: rows past the sequence end may hold anything; every warp clears them in V for
+                // itself (the same zeros from all), so that 0-probability times garbage cannot produce NaN
+                unsigned char* vt = sm.stage[st] + kTileBytes;
+                for (int x = lane; x < (kTileTokens - nv) * 32; x += 32) {
+                    const int r = nv + (x >> 5), part = x & 31;    // 32 x 8-byte pieces per row
+                    const int half = part >> 4, off = (part & 15) * 8;
+                    *reinterpret_cast<uint2*>(vt + half * kHalfTileBytes + r * 128 + off) = make_uint2(0u, 0u);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+            }
+            // ---- S = Q . K^T ----
+            float sc[8][4];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
+                const int row = 8 * j + (lane & 7);        // (row & 7 == lane & 7 == sw)
+#pragma unroll
+                for (int kp = 0; kp < 4; ++kp) {
+                    uint32_t b[4];
+                    const int cb = 4 * kp + k_cb;          // 8-channel block 0..15
+                    ldmatrix_x4(b, kbase + (cb >> 3) * kHalfTileBytes + row * 128 + (((cb & 7) ^ sw) << 4));
+                    mma_bf16_16816(sc[j], qa[2 * kp], b[0], b[1]);
+                    mma_bf16_16816(sc[j], qa[2 * kp + 1], b[2], b[3]);
+                }
+            }
+            // ---- mask, online softmax per row (a row's 64 tokens sit in the four lanes of its quad) ----
+            const int limA = nv - backA, limB = nv - backB;
+            float mxA = -INFINITY, mxB = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int t0 = 8 * j + 2 * qd;
+                sc[j][0] = t0 < limA ? sc[j][0] * p.scale_log2 : -INFINITY;
+                sc[j][1] = t0 + 1 < limA ? sc[j][1] * p.scale_log2 : -INFINITY;
+                sc[j][2] = t0 < limB ? sc[j][2] * p.scale_log2 : -INFINITY;
+                sc[j][3] = t0 + 1 < limB ? sc[j][3] * p.scale_log2 : -INFINITY;
+                mxA = fmaxf(mxA, fmaxf(sc[j][0], sc[j][1]));
+                mxB = fmaxf(mxB, fmaxf(sc[j][2], sc[j][3]));
+            }
+            mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 1));
+            mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 1));
+            mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 2));
+            mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 2));
+            const float mnA = fmaxf(mA, mxA), mnB = fmaxf(mB, mxB);
+            // a row that has seen nothing so far keeps max = -inf; exponents are then taken against 0
+            const float mbA = mnA == -INFINITY ? 0.f : mnA, mbB = mnB == -INFINITY ? 0.f : mnB;
+            const float alA = fast_exp2(mA - mbA), alB = fast_exp2(mB - mbB);
+            const bool same_max = __all_sync(0xffffffffu, mA == mnA && mB == mnB);
+            mA = mnA; mB = mnB;
+            float sumA = 0.f, sumB = 0.f;
+            uint32_t pa[8][2];                             // P as bf16 pairs: [n-tile][row A | row B]
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float p0 = fast_exp2(sc[j][0] - mbA), p1 = fast_exp2(sc[j][1] - mbA);
+                const float p2 = fast_exp2(sc[j][2] - mbB), p3 = fast_exp2(sc[j][3] - mbB);
+                sumA += p0 + p1;
+                sumB += p2 + p3;
+                pa[j][0] = pack_bf16x2(p0, p1);
+                pa[j][1] = pack_bf16x2(p2, p3);
+            }
+            lA = lA * alA + sumA;
+            lB = lB * alB + sumB;
+            if (!same_max) {
+#pragma unroll
+                for (int ct = 0; ct < 16; ++ct) { o[ct][0] *= alA; o[ct][1] *= alA; o[ct][2] *= alB; o[ct][3] *= alB; }
+            }
+            // ---- O += P . V ----
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const uint32_t a[4] = {pa[2 * kk][0], pa[2 * kk][1], pa[2 * kk + 1][0], pa[2 * kk + 1][1]};
+                const int row = 16 * kk + v_tok;
+#pragma unroll
+                for (int cp = 0; cp < 8; ++cp) {
+                    uint32_t b[4];
+                    const int cb = 2 * cp + v_cb;
+                    ldmatrix_x4_trans(b, vbase + (cb >> 3) * kHalfTileBytes + row * 128 + (((cb & 7) ^ (row & 7)) << 4));
+                    mma_bf16_16816(o[2 * cp], a, b[0], b[1]);
+                    mma_bf16_16816(o[2 * cp + 1], a, b[2], b[3]);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[st]);
+
+        // the next tile's metadata tells whether the piece goes on
+        const int nst = (it + 1) % kStages;
+        if (!mbar_wait(&sm.full[nst], ((it + 1) / kStages) & 1, p.status)) return;
+        const StageMeta nx = sm.meta[nst];
+        if (nx.flags & 1) {
+            // ---------------- the current piece ends here: every warp stores its own rows -----------------
+            float l0 = lA, l1 = lB;
+            l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+            l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+            const int u = mt.unit;
+            if (piece_tiles < mt.unit_tiles) {
+                // part of the unit: partial into the slot of the interval the piece began in
+                const size_t slot = (size_t)piece_iv + u;
+                float* po = p.part_o + slot * (8 * NT * kHeadDim);
+                float* pm = p.part_ml + slot * (kMlStride * NT);
+#pragma unroll
+                for (int ct = 0; ct < 16; ++ct) {
+                    if (realA) *reinterpret_cast<float2*>(po + rA * kHeadDim + 8 * ct + 2 * qd) = make_float2(o[ct][0], o[ct][1]);
+                    if (realB) *reinterpret_cast<float2*>(po + rB * kHeadDim + 8 * ct + 2 * qd) = make_float2(o[ct][2], o[ct][3]);
+                }
+                if (qd == 0) {
+                    if (realA) { pm[rA] = mA; pm[8 * NT + rA] = l0; }
+                    if (realB) { pm[rB] = mB; pm[8 * NT + rB] = l1; }
+                }
+                if (tid == 0) pm[16 * NT] = __uint_as_float(p.generation);
+                // every warp makes its rows of the partial visible; then warp 0 counts the piece on the unit's
+                // ticket (as in the other variant: lane k for the k-th piece held, answer kept in a register)
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.merge_bar[0]);
+                if (w == 0) {
+                    if (!mbar_wait(&sm.merge_bar[0], pubs & 1, p.status)) return;
+                    const int n_held = sm.pieces_n;
+                    if (n_held < kMaxPieces) {
+                        if (lane == n_held) {
+                            const int iv_first = interval_of(sm.sched, mt.unit_first);
+                            const int iv_last = interval_of(sm.sched, mt.unit_first + mt.unit_tiles - 1);
+                            const int n_slots = iv_last - iv_first + 1;
+                            const unsigned int bit = n_slots <= 32 ? 1u << (piece_iv - iv_first) : 0u;
+                            sm.pieces[n_held] = Piece{u, piece_tiles, iv_first + u, n_slots, mt.unit_tiles};
+                            tk_bit = bit;
+                            tk_before = atomicAdd(&p.tickets[u], ((unsigned long long)piece_tiles << 32) | bit);
+                        }
+                        __syncwarp();
+                        if (lane == 0) sm.pieces_n = n_held + 1;
+                    } else {
+                        raise_status(p.status, DEV_TIMEOUT);   // (cannot happen with the schedule's bound on pieces per CTA)
+                    }
+                }
+                ++pubs;
+            } else {
+                // the whole unit in one piece: final output
+                const float invA = l0 > 0.f ? 1.f / l0 : 0.f, invB = l1 > 0.f ? 1.f / l1 : 0.f;
+                const size_t rowA = unit_row(p, u, realA ? rA : 0), rowB = unit_row(p, u, realB ? rB : 0);
+                uint32_t* oA = reinterpret_cast<uint32_t*>(p.out + rowA * kHeadDim);
+                uint32_t* oB = reinterpret_cast<uint32_t*>(p.out + rowB * kHeadDim);
+#pragma unroll
+                for (int ct = 0; ct < 16; ++ct) {
+                    if (realA) oA[4 * ct + qd] = pack_bf16x2(o[ct][0] * invA, o[ct][1] * invA);
+                    if (realB) oB[4 * ct + qd] = pack_bf16x2(o[ct][2] * invB, o[ct][3] * invB);
+                }
+                if (p.lse && qd == 0) {
+                    const float ln2 = 0.6931471805599453f;
+                    if (realA) p.lse[rowA] = l0 > 0.f ? (mA + log2f(l0)) * ln2 : -INFINITY;
+                    if (realB) p.lse[rowB] = l1 > 0.f ? (mB + log2f(l1)) * ln2 : -INFINITY;
+                }
+            }
+        }
+        mt = nx;
+    }
+    }
     // ---- the stream is over: make this CTA's partials count, and do the combines it owes ------
     pdl_launch_dependents();
     if (tid == 0) SEER_STAMP(6);
@@ -1380,9 +1595,11 @@ int occupancy_of(bool sparse, bool paged) {
 template <int NT>
 cudaError_t launch_of(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
                       const DecodeParams& p, int grid, cudaStream_t stream) {
-    if (sparse && p.blocks_per_tile > 1)
-        return paged ? launch<true, true, NT, true>(map_k, map_v, p, grid, stream)
-                     : launch<true, false, NT, true>(map_k, map_v, p, grid, stream);
+    if constexpr (NT < kWideTiles) {            // (the rows-on-M variant takes blocks of 64 or 128 tokens only)
+        if (sparse && p.blocks_per_tile > 1)
+            return paged ? launch<true, true, NT, true>(map_k, map_v, p, grid, stream)
+                         : launch<true, false, NT, true>(map_k, map_v, p, grid, stream);
+    }
     if (sparse) return paged ? launch<true, true, NT, false>(map_k, map_v, p, grid, stream)
                              : launch<true, false, NT, false>(map_k, map_v, p, grid, stream);
     return paged ? launch<false, true, NT, false>(map_k, map_v, p, grid, stream)
@@ -1392,16 +1609,19 @@ cudaError_t launch_of(bool sparse, bool paged, const CUtensorMap& map_k, const C
 }  // namespace
 
 int decode_ctas_per_sm(bool sparse, bool paged, int n_tiles) {
-    return n_tiles == 1 ? occupancy_of<1>(sparse, paged) : occupancy_of<2>(sparse, paged);
+    return n_tiles == 1 ? occupancy_of<1>(sparse, paged) : n_tiles == 2 ? occupancy_of<2>(sparse, paged)
+                                                                         : occupancy_of<kWideTiles>(sparse, paged);
 }
 
-int decode_max_intervals(int grid) { return grid * (kMaxRounds + 1) + 1; }
+int decode_max_intervals(int grid, int max_rounds) { return grid * (max_rounds + 1) + 1; }
 
 cudaError_t launch_decode(bool sparse, bool paged, int n_tiles, const CUtensorMap& map_k, const CUtensorMap& map_v,
                           const DecodeParams& p, int grid, cudaStream_t stream) {
-    if (n_tiles < 1 || n_tiles > 2 || p.rows > 8 * n_tiles) return cudaErrorInvalidValue;
+    if ((n_tiles != 1 && n_tiles != 2 && n_tiles != kWideTiles) || p.rows > 8 * n_tiles) return cudaErrorInvalidValue;
+    if (n_tiles == kWideTiles && p.blocks_per_tile > 1) return cudaErrorInvalidValue;
     return n_tiles == 1 ? launch_of<1>(sparse, paged, map_k, map_v, p, grid, stream)
-                        : launch_of<2>(sparse, paged, map_k, map_v, p, grid, stream);
+           : n_tiles == 2 ? launch_of<2>(sparse, paged, map_k, map_v, p, grid, stream)
+                          : launch_of<kWideTiles>(sparse, paged, map_k, map_v, p, grid, stream);
 }
 
 }  // namespace seer

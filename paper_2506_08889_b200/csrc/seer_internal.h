@@ -66,6 +66,7 @@ struct DecodeParams {
     int max_blocks_cap;             // tile-count clamp for dense: capacity in tiles
     int pool_div;                   // 1/pool_div of the tiles are handed out dynamically (0: none)
     int min_tiles;                  // a CTA's range has at least this many tiles (fewer CTAs take part when work is short)
+    int max_rounds;                 // most dynamic chunks per range (<= kMaxRounds; 0: none) -- bounds the partial slots
     float scale_log2;               // sm_scale * log2(e)
     unsigned int* status;
     unsigned long long* tickets;    // [num_units]: tiles done << 32 | valid-slot bits; zero between launches
@@ -88,8 +89,9 @@ struct DecodeLaunch {
 // Returns resident CTAs per SM for the decode kernel (queried once).
 int decode_ctas_per_sm(bool sparse, bool paged, int n_tiles);
 // Upper bound on the number of work intervals (static ranges + dynamic chunks) of a launch.
-int decode_max_intervals(int grid);
-// n_tiles: MMA N-tiles of 8 rows (1 or 2); p.rows <= 8 * n_tiles.
+int decode_max_intervals(int grid, int max_rounds = kMaxRounds);
+// n_tiles: MMA N-tiles of 8 rows (1 or 2: tokens on M), or 8 for the variant with the unit's (up to 64) rows on M;
+// p.rows <= 8 * n_tiles.
 cudaError_t launch_decode(bool sparse, bool paged, int n_tiles, const CUtensorMap& map_k, const CUtensorMap& map_v,
                           const DecodeParams& p, int grid, cudaStream_t stream);
 

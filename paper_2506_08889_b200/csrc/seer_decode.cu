@@ -1263,73 +1263,80 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 fence_proxy_async_smem();
                 __syncwarp();
             }
-            // ---- S = Q . K^T ----
-            float sc[8][4];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
-                const int row = 8 * j + (lane & 7);        // (row & 7 == lane & 7 == sw)
-#pragma unroll
-                for (int kp = 0; kp < 4; ++kp) {
-                    uint32_t b[4];
-                    const int cb = 4 * kp + k_cb;          // 8-channel block 0..15
-                    ldmatrix_x4(b, kbase + (cb >> 3) * kHalfTileBytes + row * 128 + (((cb & 7) ^ sw) << 4));
-                    mma_bf16_16816(sc[j], qa[2 * kp], b[0], b[1]);
-                    mma_bf16_16816(sc[j], qa[2 * kp + 1], b[2], b[3]);
-                }
-            }
-            // ---- mask, online softmax per row (a row's 64 tokens sit in the four lanes of its quad) ----
+            // The tile's 64 tokens are taken in two halves of 32, each a complete online-softmax step (scores,
+            // running max and sum, P . V): half as many score and probability registers are live at a time.
             const int limA = nv - backA, limB = nv - backB;
-            float mxA = -INFINITY, mxB = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int t0 = 8 * j + 2 * qd;
-                sc[j][0] = t0 < limA ? sc[j][0] * p.scale_log2 : -INFINITY;
-                sc[j][1] = t0 + 1 < limA ? sc[j][1] * p.scale_log2 : -INFINITY;
-                sc[j][2] = t0 < limB ? sc[j][2] * p.scale_log2 : -INFINITY;
-                sc[j][3] = t0 + 1 < limB ? sc[j][3] * p.scale_log2 : -INFINITY;
-                mxA = fmaxf(mxA, fmaxf(sc[j][0], sc[j][1]));
-                mxB = fmaxf(mxB, fmaxf(sc[j][2], sc[j][3]));
-            }
-            mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 1));
-            mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 1));
-            mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 2));
-            mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 2));
-            const float mnA = fmaxf(mA, mxA), mnB = fmaxf(mB, mxB);
-            // a row that has seen nothing so far keeps max = -inf; exponents are then taken against 0
-            const float mbA = mnA == -INFINITY ? 0.f : mnA, mbB = mnB == -INFINITY ? 0.f : mnB;
-            const float alA = fast_exp2(mA - mbA), alB = fast_exp2(mB - mbB);
-            const bool same_max = __all_sync(0xffffffffu, mA == mnA && mB == mnB);
-            mA = mnA; mB = mnB;
-            float sumA = 0.f, sumB = 0.f;
-            uint32_t pa[8][2];                             // P as bf16 pairs: [n-tile][row A | row B]
+            for (int hb = 0; hb < 2; ++hb) {
+                if (32 * hb >= nv) break;                  // (nothing cached in the second half)
+                // ---- S = Q . K^T ----
+                float sc[4][4];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float p0 = fast_exp2(sc[j][0] - mbA), p1 = fast_exp2(sc[j][1] - mbA);
-                const float p2 = fast_exp2(sc[j][2] - mbB), p3 = fast_exp2(sc[j][3] - mbB);
-                sumA += p0 + p1;
-                sumB += p2 + p3;
-                pa[j][0] = pack_bf16x2(p0, p1);
-                pa[j][1] = pack_bf16x2(p2, p3);
-            }
-            lA = lA * alA + sumA;
-            lB = lB * alB + sumB;
-            if (!same_max) {
+                for (int jj = 0; jj < 4; ++jj) sc[jj][0] = sc[jj][1] = sc[jj][2] = sc[jj][3] = 0.f;
 #pragma unroll
-                for (int ct = 0; ct < 16; ++ct) { o[ct][0] *= alA; o[ct][1] *= alA; o[ct][2] *= alB; o[ct][3] *= alB; }
-            }
-            // ---- O += P . V ----
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int row = 8 * (4 * hb + jj) + (lane & 7);        // (row & 7 == lane & 7 == sw)
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                const uint32_t a[4] = {pa[2 * kk][0], pa[2 * kk][1], pa[2 * kk + 1][0], pa[2 * kk + 1][1]};
-                const int row = 16 * kk + v_tok;
+                    for (int kp = 0; kp < 4; ++kp) {
+                        uint32_t b[4];
+                        const int cb = 4 * kp + k_cb;      // 8-channel block 0..15
+                        ldmatrix_x4(b, kbase + (cb >> 3) * kHalfTileBytes + row * 128 + (((cb & 7) ^ sw) << 4));
+                        mma_bf16_16816(sc[jj], qa[2 * kp], b[0], b[1]);
+                        mma_bf16_16816(sc[jj], qa[2 * kp + 1], b[2], b[3]);
+                    }
+                }
+                // ---- mask, online softmax per row (a row's tokens sit in the four lanes of its quad) ----
+                float mxA = -INFINITY, mxB = -INFINITY;
 #pragma unroll
-                for (int cp = 0; cp < 8; ++cp) {
-                    uint32_t b[4];
-                    const int cb = 2 * cp + v_cb;
-                    ldmatrix_x4_trans(b, vbase + (cb >> 3) * kHalfTileBytes + row * 128 + (((cb & 7) ^ (row & 7)) << 4));
-                    mma_bf16_16816(o[2 * cp], a, b[0], b[1]);
-                    mma_bf16_16816(o[2 * cp + 1], a, b[2], b[3]);
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int t0 = 8 * (4 * hb + jj) + 2 * qd;
+                    sc[jj][0] = t0 < limA ? sc[jj][0] * p.scale_log2 : -INFINITY;
+                    sc[jj][1] = t0 + 1 < limA ? sc[jj][1] * p.scale_log2 : -INFINITY;
+                    sc[jj][2] = t0 < limB ? sc[jj][2] * p.scale_log2 : -INFINITY;
+                    sc[jj][3] = t0 + 1 < limB ? sc[jj][3] * p.scale_log2 : -INFINITY;
+                    mxA = fmaxf(mxA, fmaxf(sc[jj][0], sc[jj][1]));
+                    mxB = fmaxf(mxB, fmaxf(sc[jj][2], sc[jj][3]));
+                }
+                mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 1));
+                mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 1));
+                mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 2));
+                mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 2));
+                const float mnA = fmaxf(mA, mxA), mnB = fmaxf(mB, mxB);
+                // a row that has seen nothing so far keeps max = -inf; exponents are then taken against 0
+                const float mbA = mnA == -INFINITY ? 0.f : mnA, mbB = mnB == -INFINITY ? 0.f : mnB;
+                const float alA = fast_exp2(mA - mbA), alB = fast_exp2(mB - mbB);
+                const bool same_max = __all_sync(0xffffffffu, mA == mnA && mB == mnB);
+                mA = mnA; mB = mnB;
+                float sumA = 0.f, sumB = 0.f;
+                uint32_t pa[4][2];                         // P as bf16 pairs: [n-tile][row A | row B]
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const float p0 = fast_exp2(sc[jj][0] - mbA), p1 = fast_exp2(sc[jj][1] - mbA);
+                    const float p2 = fast_exp2(sc[jj][2] - mbB), p3 = fast_exp2(sc[jj][3] - mbB);
+                    sumA += p0 + p1;
+                    sumB += p2 + p3;
+                    pa[jj][0] = pack_bf16x2(p0, p1);
+                    pa[jj][1] = pack_bf16x2(p2, p3);
+                }
+                lA = lA * alA + sumA;
+                lB = lB * alB + sumB;
+                if (!same_max) {
+#pragma unroll
+                    for (int ct = 0; ct < 16; ++ct) { o[ct][0] *= alA; o[ct][1] *= alA; o[ct][2] *= alB; o[ct][3] *= alB; }
+                }
+                // ---- O += P . V ----
+#pragma unroll
+                for (int k2 = 0; k2 < 2; ++k2) {
+                    const uint32_t a[4] = {pa[2 * k2][0], pa[2 * k2][1], pa[2 * k2 + 1][0], pa[2 * k2 + 1][1]};
+                    const int row = 16 * (2 * hb + k2) + v_tok;
+#pragma unroll
+                    for (int cp = 0; cp < 8; ++cp) {
+                        uint32_t b[4];
+                        const int cb = 2 * cp + v_cb;
+                        ldmatrix_x4_trans(b, vbase + (cb >> 3) * kHalfTileBytes + row * 128 + (((cb & 7) ^ (row & 7)) << 4));
+                        mma_bf16_16816(o[2 * cp], a, b[0], b[1]);
+                        mma_bf16_16816(o[2 * cp + 1], a, b[2], b[3]);
+                    }
                 }
             }
         }

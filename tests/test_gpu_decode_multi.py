@@ -56,9 +56,11 @@ def _all_blocks(lens, Hkv, b):
 
 # (Hq, Hkv, q_len): rows on the MMA N side and launches per call
 #   (32,8,2): 8 rows, one N-tile      (40,8,3): 15 rows, two N-tiles     (64,8,2): 16 rows
-#   (40,8,8): 3 + 3 + 2 tokens in three launches   (8,8,8): 8 rows   (16,8,8): 16 rows   (40,8,1): plain decode
+#   (8,8,8): 8 rows   (16,8,8): 16 rows   (40,8,1): plain decode
+# more than 16 rows take the variant with the rows on the MMA's M side, one launch for up to 64 rows:
+#   (40,8,8): 40 rows   (64,8,8): 64 rows   (6,2,6): 18 rows   (56,8,8): 56 rows   (40,8,4): 20 rows
 @pytest.mark.parametrize("Hq,Hkv,T", [(32, 8, 2), (40, 8, 3), (64, 8, 2), (40, 8, 8), (8, 8, 8), (16, 8, 8),
-                                      (40, 8, 1), (6, 2, 5)])
+                                      (40, 8, 1), (6, 2, 5), (64, 8, 8), (6, 2, 6), (56, 8, 8), (40, 8, 4)])
 def test_sparse_multi_ragged_lengths_and_boundaries(ctx, Hq, Hkv, T):
     B, S, b = 6, 1536, 64
     # 1536: full blocks; 1025: the last block holds one token, the others' own tokens sit in the block before;
@@ -115,6 +117,31 @@ def test_multi_long_lists_split_over_ctas_and_paged(ctx):
     kp, vp, table = to_paged(k, v, b, 820)
     outp, lsep = _run(ctx, q, kp, vp, lens, idx, cnt, b, 0.0884, page_table=table, page_size=b, max_seq_len=S)
     check_attention(outp, lsep, *ref, what="multi long paged", strict=True)
+    assert ctx.device_status() == binding.SEER_OK
+
+
+@pytest.mark.parametrize("Hq,T", [(40, 8), (64, 8), (56, 7)])
+def test_multi_many_rows_long_lists_dense_and_paged(ctx, Hq, T):
+    # 17 to 64 rows per unit in one launch (rows on the MMA's M side): long lists cut into pieces and combined,
+    # the dense call, and the same cache behind a page table, at the bound stated for long contexts
+    B, Hkv, S, b = 2, 8, 16384, 64
+    lens = np.array([16384, 12345], np.int32)
+    q, k, v = _make(B, T, Hq, Hkv, S, 870 + T)
+    n = [-(-int(L) // b) for L in lens]
+    keep = [x // 2 for x in n]
+    idx, cnt = synth.random_block_lists(lens, Hkv, b, keep, max(keep), 870 + T)
+    ref = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, idx, cnt, b, 0.0884)
+    launches = ctx.launch_count()
+    out, lse = _run(ctx, q, k, v, lens, idx, cnt, b, 0.0884)
+    assert ctx.launch_count() - launches == 1
+    check_attention(out, lse, *ref, what="many rows sparse", strict=True)
+    kp, vp, table = to_paged(k, v, b, 870)
+    outp, lsep = _run(ctx, q, kp, vp, lens, idx, cnt, b, 0.0884, page_table=table, page_size=b, max_seq_len=S)
+    check_attention(outp, lsep, *ref, what="many rows paged", strict=True)
+    full_idx, full_cnt = _all_blocks(lens, Hkv, b)
+    refd = oracle.sparse_multi(bits(q), bits(k), bits(v), lens, full_idx, full_cnt, b, 0.0884)
+    outd, lsed = _run(ctx, q, k, v, lens, None, None, b, 0.0884, dense=True)
+    check_attention(outd, lsed, *refd, what="many rows dense", strict=True)
     assert ctx.device_status() == binding.SEER_OK
 
 

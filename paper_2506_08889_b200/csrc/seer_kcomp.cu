@@ -206,7 +206,7 @@ constexpr int kBulkBlocks = 16;
 constexpr int kFeatStride = 3 * kHeadDim + 8;         // bf16 per block row (+8: conflict-free fragment reads)
 constexpr int kLoStride = kHeadDim + 8;
 
-__global__ void __launch_bounds__(kKcThreads) kcomp_bulk_kernel(const KcompParams p) {
+__global__ void __launch_bounds__(kKcThreads, 4) kcomp_bulk_kernel(const KcompParams p) {
     __shared__ __align__(16) __nv_bfloat16 feat_hi[kBulkBlocks][kFeatStride];   // [max | min | avg]
     __shared__ __align__(16) __nv_bfloat16 feat_lo[kBulkBlocks][kLoStride];     // avg - bf16(avg)
     __shared__ float ybuf[kBulkBlocks][kMaxDGate];
@@ -237,16 +237,29 @@ __global__ void __launch_bounds__(kKcThreads) kcomp_bulk_kernel(const KcompParam
         for (int c = 0; c < 8; ++c) sm[c] = 0.f;
         if (q < nb) {
             const __nv_bfloat16* src = p.k_nope + base + (size_t)(j_first + q) * b * p.stride_token + 8 * cchunk;
-#pragma unroll 16
-            for (int r = rsel; r < b; r += 2) {
-                const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + (size_t)r * p.stride_token));
-                const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&v);
+            // 16 rows per lane (32 rows of the block, 8 KiB per warp) are requested before any is looked at: the
+            // kernel lives on the bytes it has in flight
+            constexpr int kInFlight = 8;
+            for (int r0 = 0; r0 < b; r0 += 2 * kInFlight) {
+                uint4 buf[kInFlight];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    mx[c] = __hmax2(mx[c], hh[c]);
-                    mn[c] = __hmin2(mn[c], hh[c]);
-                    const float2 f = __bfloat1622float2(hh[c]);
-                    sm[2 * c] += f.x; sm[2 * c + 1] += f.y;
+                for (int k = 0; k < kInFlight; ++k) {
+                    const int r = r0 + 2 * k + rsel;
+                    buf[k] = r < b ? __ldg(reinterpret_cast<const uint4*>(src + (size_t)r * p.stride_token))
+                                   : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int k = 0; k < kInFlight; ++k) {
+                    if (r0 + 2 * k + rsel < b) {
+                        const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&buf[k]);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            mx[c] = __hmax2(mx[c], hh[c]);
+                            mn[c] = __hmin2(mn[c], hh[c]);
+                            const float2 f = __bfloat1622float2(hh[c]);
+                            sm[2 * c] += f.x; sm[2 * c + 1] += f.y;
+                        }
+                    }
                 }
             }
 #pragma unroll

@@ -589,6 +589,8 @@ static seer_status kcomp_append_common(seer_ctx* ctx, const seer_shape* shape, c
     p.d_gate = gate->d_gate;
     p.max_blocks = gate->max_blocks;
     p.wait_at_end = wait_at_end;
+    p.sm_count = ctx->num_sms;
+    p.status = reinterpret_cast<unsigned int*>(ctx->ws);
     fill_inv_freq(p.inv_freq, gate->d_gate, gate->rope_theta);
     int launched = 0;
     ce = launch_kcomp_append(p, static_cast<cudaStream_t>(stream), &launched);

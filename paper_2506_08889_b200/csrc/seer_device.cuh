@@ -111,6 +111,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// A bf16 is the upper half of the fp32 with the same value: the pair is widened with a shift and a mask
+// (the conversion instruction goes through the slow special-function pipe).
+__device__ __forceinline__ float2 bf16x2_to_float2(uint32_t v) {
+    return make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+}
+__device__ __forceinline__ float2 bf16x2_to_float2(const __nv_bfloat162& h) {
+    return bf16x2_to_float2(*reinterpret_cast<const uint32_t*>(&h));
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
     return *reinterpret_cast<uint32_t*>(&v);

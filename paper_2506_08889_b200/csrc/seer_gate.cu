@@ -25,7 +25,7 @@ __device__ __forceinline__ float dot8(const uint4& a, const float* x) {
     float acc = 0.f;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        float2 f = __bfloat1622float2(h[k]);
+        float2 f = bf16x2_to_float2(h[k]);
         acc = fmaf(f.x, x[2 * k], acc);
         acc = fmaf(f.y, x[2 * k + 1], acc);
     }
@@ -37,7 +37,7 @@ __device__ __forceinline__ float dot8(const uint4& a, const uint4& b) {
     float acc = 0.f;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        const float2 f = __bfloat1622float2(h[k]), e = __bfloat1622float2(g[k]);
+        const float2 f = bf16x2_to_float2(h[k]), e = bf16x2_to_float2(g[k]);
         acc = fmaf(f.x, e.x, acc);
         acc = fmaf(f.y, e.y, acc);
     }

@@ -132,6 +132,8 @@ struct KcompParams {
     int first_block, num_blocks;    // first_block == -t (1..8): the block that filled while the last t tokens were appended
     int wait_at_end;                // append only: work first, wait for the preceding kernel just before the end
     int batch, num_kv_heads, block_size, d_gate, max_blocks;
+    int sm_count;                   // bulk build: one persistent CTA per SM
+    unsigned int* status;           // sticky device status word (bounded waits report here)
     double inv_freq[kMaxDGate / 2];
 };
 cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* launched);

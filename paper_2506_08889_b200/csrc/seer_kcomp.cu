@@ -75,7 +75,7 @@ __device__ __forceinline__ void kcomp_body(const KcompParams& p) {
             const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&v);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const float2 f = __bfloat1622float2(hh[c]);
+                const float2 f = bf16x2_to_float2(hh[c]);
                 mx[2 * c] = fmaxf(mx[2 * c], f.x); mx[2 * c + 1] = fmaxf(mx[2 * c + 1], f.y);
                 mn[2 * c] = fminf(mn[2 * c], f.x); mn[2 * c + 1] = fminf(mn[2 * c + 1], f.y);
                 sm[2 * c] += f.x; sm[2 * c + 1] += f.y;
@@ -137,7 +137,7 @@ __device__ __forceinline__ void kcomp_body(const KcompParams& p) {
                 float wf[8];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const float2 f = __bfloat1622float2(hh[c]);
+                    const float2 f = bf16x2_to_float2(hh[c]);
                     wf[2 * c] = f.x; wf[2 * c + 1] = f.y;
                 }
 #pragma unroll
@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(kKcThreads, 4) kcomp_bulk_kernel(const KcompPa
                         for (int c = 0; c < 4; ++c) {
                             mx[c] = __hmax2(mx[c], hh[c]);
                             mn[c] = __hmin2(mn[c], hh[c]);
-                            const float2 f = __bfloat1622float2(hh[c]);
+                            const float2 f = bf16x2_to_float2(hh[c]);
                             sm[2 * c] += f.x; sm[2 * c + 1] += f.y;
                         }
                     }
@@ -343,6 +343,274 @@ __global__ void __launch_bounds__(kKcThreads, 4) kcomp_bulk_kernel(const KcompPa
     }
 }
 
+
+// ---- bulk build, streaming variant (b = 64, d_gate <= 128) ----------------------------------------
+// One persistent CTA per SM, three kinds of warps that meet only through mbarriers:
+//   producer (1 warp)    keeps a ring of 64-row stages (one block each, 16 KiB) full with bulk copies, so
+//                        the bytes in flight do not depend on what the other warps are doing;
+//   pooling (6 warps)    each takes one stage at a time out of shared memory and leaves the block's
+//                        3*128 features (bf16; the mean as high part + correction) in one of two
+//                        feature buffers;
+//   projection (8 warps) warp w holds rows 16w .. 16w+15 of W_k as mma A fragments (96 registers) and,
+//                        once 16 blocks are pooled, multiplies them in (64 mma, nothing to fetch),
+//                        rotates and stores - while the pooling warps are already on the next item.
+// An item is 16 consecutive blocks of one (sequence, KV head); items are numbered head-major and dealt
+// round-robin, so a CTA changes head a handful of times per launch.
+//
+// Stage number n of a CTA (counted over all its items) lives in ring slot n % kStreamStages and is pooled
+// by warp n % kPoolWarps.  kStreamStages is a multiple of kPoolWarps, so a slot is always read by the same
+// warp, which goes through its stages in order: a wait on a slot's barrier is then never more than one
+// phase away from the barrier's own, which is what a parity wait needs to be unambiguous.  (With a
+// block-of-the-item -> warp rule a fast warp could ask for a slot's next use before the slot's current use
+// had landed for another warp, and the parity test would pass on stale data.)
+#ifndef SEER_KC_STAGES
+#define SEER_KC_STAGES 12
+#endif
+#ifndef SEER_KC_POOLWARPS
+#define SEER_KC_POOLWARPS 6
+#endif
+constexpr int kStreamStages = SEER_KC_STAGES;
+constexpr int kStreamRows = 64;
+constexpr int kStageBytes = kStreamRows * kHeadDim * 2;
+constexpr int kStreamDGate = 128;
+constexpr int kPoolWarps = SEER_KC_POOLWARPS;
+constexpr int kProjWarps = kStreamDGate / 16;
+constexpr int kProjThreads = 32 * kProjWarps;
+constexpr int kStreamThreads = 32 * (kProjWarps + kPoolWarps + 1);
+static_assert(kStreamStages % kPoolWarps == 0, "a ring slot must always be read by the same pooling warp");
+
+struct StreamSmem {
+    alignas(128) unsigned char ring[kStreamStages][kStageBytes];
+    // [max | min | avg]; once a buffer's features have been multiplied in, its start holds the 16 x 128
+    // fp32 products until they are rotated and stored
+    alignas(16) __nv_bfloat16 feat_hi[2][kBulkBlocks][kFeatStride];
+    alignas(16) __nv_bfloat16 feat_lo[2][kBulkBlocks][kLoStride];     // avg - bf16(avg)
+    uint64_t full[kStreamStages], empty[kStreamStages];
+    uint64_t feat_full[2], feat_empty[2];
+};
+static_assert(sizeof(float) * kBulkBlocks * kStreamDGate <= sizeof(__nv_bfloat16) * kBulkBlocks * kFeatStride,
+              "the products must fit in the feature buffer they replace");
+static_assert(sizeof(StreamSmem) <= 227 * 1024, "one CTA's shared memory");
+
+__device__ __forceinline__ void proj_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kProjThreads) : "memory"); }
+
+__global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const KcompParams p) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        for (int s = 0; s < kStreamStages; ++s) {
+            mbar_init(&sm.full[s], 1);
+            mbar_init(&sm.empty[s], 1);
+        }
+        for (int f = 0; f < 2; ++f) {
+            mbar_init(&sm.feat_full[f], kPoolWarps);
+            mbar_init(&sm.feat_empty[f], kProjWarps);
+        }
+        mbar_fence_init();
+    }
+    __syncthreads();
+    pdl_wait();
+    pdl_launch_dependents();
+
+    const int b = p.block_size;                        // == kStreamRows
+    const int groups = (p.num_blocks + kBulkBlocks - 1) / kBulkBlocks;
+    const int per_head = groups * p.batch;
+    const int n_items = per_head * p.num_kv_heads;
+    bool dead = false;                                 // a wait ran out: stop waiting, finish the motions
+
+    // item -> (head, sequence, first block) and the number of complete blocks of it that exist
+    auto item_blocks = [&](int item, int& h, int& i, int& j_first) {
+        h = item / per_head;
+        const int rem = item - h * per_head;
+        const int g = rem / p.batch;
+        i = rem - g * p.batch;
+        const int L = p.seq_lens[i];
+        const int complete = L > 0 ? L / b : 0;
+        j_first = p.first_block + g * kBulkBlocks;
+        const int j_end = min(min(p.first_block + p.num_blocks, complete), p.max_blocks);
+        return max(0, min(kBulkBlocks, j_end - j_first));
+    };
+
+    if (warp == kProjWarps + kPoolWarps) {
+        // ---- producer ----
+        const bool rows_adjacent = p.stride_token == kHeadDim;
+        uint32_t stage_no = 0;                         // stages this CTA has been through so far
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            int h, i, j_first;
+            const int nb = item_blocks(item, h, i, j_first);
+            const __nv_bfloat16* src0 = p.k_nope + (size_t)i * p.stride_batch + (size_t)h * p.stride_head;
+            for (int q = 0; q < nb; ++q, ++stage_no) {
+                const int s = stage_no % kStreamStages;
+                const uint32_t use = stage_no / kStreamStages;
+                if (!dead && !mbar_wait(&sm.empty[s], (use & 1u) ^ 1u, p.status)) dead = true;
+                if (dead) continue;
+                const __nv_bfloat16* src = src0 + (size_t)(j_first + q) * b * p.stride_token;
+                if (lane == 0) mbar_arrive_expect_tx(&sm.full[s], kStageBytes);
+                __syncwarp();
+                if (rows_adjacent) {
+                    if (lane == 0) bulk_load(sm.ring[s], src, kStageBytes, &sm.full[s]);
+                } else {
+                    for (int r = lane; r < kStreamRows; r += 32)
+                        bulk_load(sm.ring[s] + r * (kHeadDim * 2), src + (size_t)r * p.stride_token, kHeadDim * 2,
+                                  &sm.full[s]);
+                }
+            }
+        }
+    } else if (warp >= kProjWarps) {
+        // ---- pooling ----
+        const int pw = warp - kProjWarps;
+        const int cchunk = lane & 15;
+        uint32_t stage_no = 0, n_done = 0;
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            int h, i, j_first;
+            const int nb = item_blocks(item, h, i, j_first);
+            if (nb == 0) continue;
+            const int fb = n_done & 1;
+            if (!dead && !mbar_wait(&sm.feat_empty[fb], ((n_done >> 1) & 1u) ^ 1u, p.status)) dead = true;
+            for (int q = 0; q < kBulkBlocks; ++q) {
+                if ((stage_no + q) % kPoolWarps != (uint32_t)pw) continue;
+                __nv_bfloat162 mx[4], mn[4];
+                float sum[8];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    mx[c] = __float2bfloat162_rn(-INFINITY);
+                    mn[c] = __float2bfloat162_rn(INFINITY);
+                }
+#pragma unroll
+                for (int c = 0; c < 8; ++c) sum[c] = 0.f;
+                if (q < nb) {
+                    const uint32_t sn = stage_no + q;
+                    const int s = sn % kStreamStages;
+                    if (!dead && !mbar_wait(&sm.full[s], (sn / kStreamStages) & 1u, p.status)) dead = true;
+                    // lane: 16-byte column piece (lane & 15) of rows 2k + (lane >> 4)
+                    const uint4* st = reinterpret_cast<const uint4*>(sm.ring[s]) + lane;
+#pragma unroll 8
+                    for (int k = 0; k < kStreamRows / 2; ++k) {
+                        const uint4 v = st[k * 32];
+                        const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            mx[c] = __hmax2(mx[c], hh[c]);
+                            mn[c] = __hmin2(mn[c], hh[c]);
+                            const float2 f = bf16x2_to_float2(hh[c]);
+                            sum[2 * c] += f.x; sum[2 * c + 1] += f.y;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.empty[s]);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t xm = *reinterpret_cast<uint32_t*>(&mx[c]), xn = *reinterpret_cast<uint32_t*>(&mn[c]);
+                        uint32_t ym = __shfl_xor_sync(0xffffffffu, xm, 16), yn = __shfl_xor_sync(0xffffffffu, xn, 16);
+                        mx[c] = __hmax2(mx[c], *reinterpret_cast<__nv_bfloat162*>(&ym));
+                        mn[c] = __hmin2(mn[c], *reinterpret_cast<__nv_bfloat162*>(&yn));
+                    }
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) sum[c] += __shfl_xor_sync(0xffffffffu, sum[c], 16);
+                }
+                if (lane < 16) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const __nv_bfloat162 zero = __float2bfloat162_rn(0.f);
+                        *reinterpret_cast<__nv_bfloat162*>(&sm.feat_hi[fb][q][8 * cchunk + 2 * c]) = q < nb ? mx[c] : zero;
+                        *reinterpret_cast<__nv_bfloat162*>(&sm.feat_hi[fb][q][kHeadDim + 8 * cchunk + 2 * c]) =
+                            q < nb ? mn[c] : zero;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const float av = q < nb ? sum[c] / (float)b : 0.f;
+                        const __nv_bfloat16 av_hi = __float2bfloat16(av);
+                        sm.feat_hi[fb][q][2 * kHeadDim + 8 * cchunk + c] = av_hi;
+                        sm.feat_lo[fb][q][8 * cchunk + c] = __float2bfloat16(av - __bfloat162float(av_hi));
+                    }
+                }
+            }
+            stage_no += nb;
+            ++n_done;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.feat_full[fb]);
+        }
+    } else {
+        // ---- projection, rotation, store ----
+        const int g = lane >> 2, t4 = lane & 3;
+        const bool projects = warp < p.d_gate / 16;
+        uint32_t wa[3 * kHeadDim / 16][4];            // this warp's 16 rows of W_k as A fragments
+        int h_held = -1;
+        uint32_t n_done = 0;
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            int h, i, j_first;
+            const int nb = item_blocks(item, h, i, j_first);
+            if (nb == 0) continue;
+            if (h != h_held && projects) {
+                const uint32_t* w0 =
+                    reinterpret_cast<const uint32_t*>(p.w_k + ((size_t)h * p.d_gate + 16 * warp + g) * 3 * kHeadDim);
+                const uint32_t* w1 = w0 + 8 * (3 * kHeadDim / 2);
+#pragma unroll
+                for (int ks = 0; ks < 3 * kHeadDim / 16; ++ks) {
+                    wa[ks][0] = __ldg(w0 + 8 * ks + t4);
+                    wa[ks][1] = __ldg(w1 + 8 * ks + t4);
+                    wa[ks][2] = __ldg(w0 + 8 * ks + 4 + t4);
+                    wa[ks][3] = __ldg(w1 + 8 * ks + 4 + t4);
+                }
+            }
+            h_held = h;
+            const int fb = n_done & 1;
+            if (!dead && !mbar_wait(&sm.feat_full[fb], (n_done >> 1) & 1u, p.status)) dead = true;
+            ++n_done;
+            float acc[2][4];
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) acc[n][x] = 0.f;
+            if (projects) {
+#pragma unroll
+                for (int ks = 0; ks < 3 * kHeadDim / 16; ++ks) {
+#pragma unroll
+                    for (int n = 0; n < 2; ++n) {
+                        const __nv_bfloat16* fr = &sm.feat_hi[fb][8 * n + g][16 * ks + 2 * t4];
+                        mma_bf16_16816(acc[n], wa[ks], *reinterpret_cast<const uint32_t*>(fr),
+                                       *reinterpret_cast<const uint32_t*>(fr + 8));
+                        if (ks >= 2 * kHeadDim / 16) {        // the mean's correction term
+                            const __nv_bfloat16* fl = &sm.feat_lo[fb][8 * n + g][16 * ks - 2 * kHeadDim + 2 * t4];
+                            mma_bf16_16816(acc[n], wa[ks], *reinterpret_cast<const uint32_t*>(fl),
+                                           *reinterpret_cast<const uint32_t*>(fl + 8));
+                        }
+                    }
+                }
+            }
+            proj_sync();                                    // every warp is done with the features
+            float (*ybuf)[kStreamDGate] = reinterpret_cast<float (*)[kStreamDGate]>(&sm.feat_hi[fb][0][0]);
+            if (projects) {
+#pragma unroll
+                for (int n = 0; n < 2; ++n) {
+                    ybuf[8 * n + 2 * t4][16 * warp + g] = acc[n][0];
+                    ybuf[8 * n + 2 * t4 + 1][16 * warp + g] = acc[n][1];
+                    ybuf[8 * n + 2 * t4][16 * warp + g + 8] = acc[n][2];
+                    ybuf[8 * n + 2 * t4 + 1][16 * warp + g + 8] = acc[n][3];
+                }
+            }
+            proj_sync();
+            const int half = p.d_gate / 2;
+            const int u = i * p.num_kv_heads + h;
+            for (int x = tid; x < nb * half; x += kProjThreads) {
+                const int q = x / half, c = x % half;
+                const int j = j_first + q;
+                float sn, cs;
+                rope_sincos((double)j * (double)b, p.inv_freq[c], &sn, &cs);
+                const float a = ybuf[q][c], bb = ybuf[q][c + half];
+                __nv_bfloat16* dst = p.kcomp + ((size_t)u * p.max_blocks + j) * p.d_gate;
+                dst[c] = __float2bfloat16(a * cs - bb * sn);
+                dst[c + half] = __float2bfloat16(bb * cs + a * sn);
+            }
+            // the buffer may be refilled once all eight warps have read their products out of it; the next
+            // item's features and products are in the other buffer
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.feat_empty[fb]);
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* launched) {
@@ -357,6 +625,22 @@ cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* 
     } else {
         const int gx = (p.num_blocks + kBulkBlocks - 1) / kBulkBlocks;
         if (gx <= 0) return cudaSuccess;
+        if (p.block_size == kStreamRows && p.d_gate <= kStreamDGate && !p.rows_block_local && gx * U >= 2 * p.sm_count) {
+            static bool attr_set[64] = {};
+            int dev = 0;
+            cudaError_t e = cudaGetDevice(&dev);
+            if (e != cudaSuccess) return e;
+            if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+                e = cudaFuncSetAttribute(kcomp_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)sizeof(StreamSmem));
+                if (e != cudaSuccess) return e;
+                if (dev >= 0 && dev < 64) attr_set[dev] = true;
+            }
+            e = launch_pdl(kcomp_stream_kernel, dim3(min(p.sm_count, gx * U), 1, 1), dim3(kStreamThreads),
+                           sizeof(StreamSmem), stream, p);
+            *launched = 1;
+            return e;
+        }
         cudaError_t e = launch_pdl(kcomp_bulk_kernel, dim3(gx, U, 1), dim3(kKcThreads), 0, stream, p);
         *launched = 1;
         return e;

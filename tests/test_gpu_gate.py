@@ -61,6 +61,39 @@ def test_kcomp_bulk_build(ctx, b, dg, token_major):
     assert np.all(got2[:, :, :3] == 0) and np.all(got2[:, :, 8:] == 0)
 
 
+@pytest.mark.parametrize("dg,token_major,first", [(128, False, 0), (64, True, 0), (128, True, 37)])
+def test_kcomp_bulk_build_large_enough_for_the_streaming_kernel(ctx, dg, token_major, first):
+    """From 2 * (SM count) work items of 16 blocks on (block size 64, d_gate <= 128) the bulk build runs as
+    the persistent kernel with a ring of stages and specialised warps: 3 x 4 units x 26 groups = 312 items
+    here, ragged lengths (one sequence ends inside a group, one has a single group), four heads (a CTA
+    changes W_k slice several times), both K layouts, and a build that starts in the middle of a group."""
+    B, Hkv, d, b = 3, 4, 128, 64
+    nb = 416
+    S = nb * b
+    lens = np.array([S, 333 * b + 17, 9 * b], np.int32)
+    n_complete = [nb, 333, 9]
+    if token_major:
+        kn = synth.normal_bf16((B, S, Hkv, d), 6, "kn", DEV).permute(0, 2, 1, 3)
+    else:
+        kn = synth.normal_bf16((B, Hkv, S, d), 6, "kn", DEV)
+    wk = synth.normal_bf16((Hkv, dg, 3 * d), 6, "wk", DEV, std=0.02)
+    kc = torch.zeros((B, Hkv, nb, dg), dtype=torch.bfloat16, device=DEV)
+    shape = binding.make_shape(B, Hkv * 2, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, None, wk, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    for _ in range(2):                                    # the second launch overlaps the first one's tail
+        ctx.seer_kcomp_append(shape, gate, lens_t, kn, first_block=first, num_blocks=nb - first)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.SEER_OK
+    _, want = oracle.kcomp(bits(kn), bits(wk), b, 0, nb, nb, THETA)
+    got = bits(kc)
+    for i in range(B):
+        if n_complete[i] > first:
+            _bf16_ulp_close(got[i, :, first:n_complete[i]], want[i, :, first:n_complete[i]])
+        assert np.all(got[i, :, max(first, n_complete[i]):] == 0)     # incomplete blocks are not written
+        assert np.all(got[i, :, :first] == 0)             # nor blocks before the first one asked for
+
+
 def test_kcomp_append_when_a_block_fills(ctx):
     B, Hkv, d, dg, b, nb = 3, 2, 128, 128, 64, 8
     lens = np.array([5 * b, 5 * b + 1, 3 * b], np.int32)  # sequences 0 and 2 just filled a block

@@ -591,9 +591,21 @@ static seer_status kcomp_append_common(seer_ctx* ctx, const seer_shape* shape, c
     p.wait_at_end = wait_at_end;
     p.sm_count = ctx->num_sms;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
+#ifdef SEER_DECODE_TRACE
+    p.trace = reinterpret_cast<unsigned long long*>(ctx->ws + (ctx->ws_bytes - (size_t)(1 << 20)));
+#endif
     fill_inv_freq(p.inv_freq, gate->d_gate, gate->rope_theta);
+    const CUtensorMap* map_k = nullptr;
+    if (kcomp_bulk_streams(p)) {
+        // (channel, token row, head, sequence); the row extent is the last row the build may touch
+        const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)(first_block + num_blocks) * (uint64_t)shape->block_size,
+                                  (uint64_t)shape->num_kv_heads, (uint64_t)shape->batch};
+        const uint64_t strides[3] = {(uint64_t)stride_token * 2, (uint64_t)stride_head * 2, (uint64_t)stride_batch * 2};
+        st = get_map(ctx, k_nope, dims, strides, kKcompStageRows, &map_k);
+        if (st != SEER_OK) return st;
+    }
     int launched = 0;
-    ce = launch_kcomp_append(p, static_cast<cudaStream_t>(stream), &launched);
+    ce = launch_kcomp_append(p, map_k, static_cast<cudaStream_t>(stream), &launched);
     ctx->launches += launched;
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "kcomp launch: %s", cudaGetErrorString(ce));
     return SEER_OK;

@@ -134,8 +134,16 @@ struct KcompParams {
     int batch, num_kv_heads, block_size, d_gate, max_blocks;
     int sm_count;                   // bulk build: one persistent CTA per SM
     unsigned int* status;           // sticky device status word (bounded waits report here)
+#ifdef SEER_DECODE_TRACE
+    unsigned long long* trace;      // diagnostic builds: per-warp cycle counters of the bulk build
+#endif
     double inv_freq[kMaxDGate / 2];
 };
-cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* launched);
+// True when the bulk build of these parameters runs as the persistent streaming kernel, which reads the keys
+// through a tensor map (channel, token row, head, sequence) with a box of 64 channels x kKcompStageRows rows,
+// 128-byte swizzle; launch_kcomp_append falls back to the plain-load kernel when it is given no map.
+constexpr int kKcompStageRows = 64;
+bool kcomp_bulk_streams(const KcompParams& p);
+cudaError_t launch_kcomp_append(const KcompParams& p, const CUtensorMap* map_k, cudaStream_t stream, int* launched);
 
 }  // namespace seer

@@ -346,9 +346,9 @@ __global__ void __launch_bounds__(kKcThreads, 4) kcomp_bulk_kernel(const KcompPa
 
 // ---- bulk build, streaming variant (b = 64, d_gate <= 128) ----------------------------------------
 // One persistent CTA per SM, three kinds of warps that meet only through mbarriers:
-//   producer (1 warp)    keeps a ring of 64-row stages (one block each, 16 KiB) full with bulk copies, so
+//   producer (1 warp)    keeps a ring of 64-row stages (one block, 16 KiB) full with tiled copies, so
 //                        the bytes in flight do not depend on what the other warps are doing;
-//   pooling (6 warps)    each takes one stage at a time out of shared memory and leaves the block's
+//   pooling (7 warps)    each takes one block at a time out of shared memory and leaves the block's
 //                        3*128 features (bf16; the mean as high part + correction) in one of two
 //                        feature buffers;
 //   projection (8 warps) warp w holds rows 16w .. 16w+15 of W_k as mma A fragments (96 registers) and,
@@ -357,46 +357,60 @@ __global__ void __launch_bounds__(kKcThreads, 4) kcomp_bulk_kernel(const KcompPa
 // An item is 16 consecutive blocks of one (sequence, KV head); items are numbered head-major and dealt
 // round-robin, so a CTA changes head a handful of times per launch.
 //
-// Stage number n of a CTA (counted over all its items) lives in ring slot n % kStreamStages and is pooled
-// by warp n % kPoolWarps.  kStreamStages is a multiple of kPoolWarps, so a slot is always read by the same
+// A block comes in kStagesPerBlock stages (a stage is freed as soon as it has been read, and what is free
+// is in flight again).  Block number n of a CTA (counted over all its items) is pooled by warp
+// n % kPoolWarps and its stages live in ring slots (n * kStagesPerBlock + part) % kStreamStages;
+// kStreamStages is a multiple of kStagesPerBlock * kPoolWarps, so a slot is always read by the same
 // warp, which goes through its stages in order: a wait on a slot's barrier is then never more than one
 // phase away from the barrier's own, which is what a parity wait needs to be unambiguous.  (With a
 // block-of-the-item -> warp rule a fast warp could ask for a slot's next use before the slot's current use
 // had landed for another warp, and the parity test would pass on stale data.)
-#ifndef SEER_KC_STAGES
-#define SEER_KC_STAGES 12
-#endif
-#ifndef SEER_KC_POOLWARPS
-#define SEER_KC_POOLWARPS 6
-#endif
-constexpr int kStreamStages = SEER_KC_STAGES;
-constexpr int kStreamRows = 64;
-constexpr int kStageBytes = kStreamRows * kHeadDim * 2;
+constexpr int kStreamStages = 7;                       // 112 KiB in flight per SM
+constexpr int kStreamRows = 64;                        // the block size this kernel is written for
+constexpr int kStageRows = kKcompStageRows;
+constexpr int kStagesPerBlock = kStreamRows / kStageRows;
+constexpr int kStageBytes = kStageRows * kHeadDim * 2;
 constexpr int kStreamDGate = 128;
-constexpr int kPoolWarps = SEER_KC_POOLWARPS;
+constexpr int kLensCache = 2048;                       // sequences whose length is kept in shared memory
+constexpr int kPoolWarps = 7;                        // with 8 + 1 others: 16 warps, 128 registers each
 constexpr int kProjWarps = kStreamDGate / 16;
 constexpr int kProjThreads = 32 * kProjWarps;
 constexpr int kStreamThreads = 32 * (kProjWarps + kPoolWarps + 1);
-static_assert(kStreamStages % kPoolWarps == 0, "a ring slot must always be read by the same pooling warp");
+static_assert(kStreamStages <= 32, "one producer lane per ring slot");
+static_assert(kStreamStages % (kStagesPerBlock * kPoolWarps) == 0,
+              "a ring slot must always be read by the same pooling warp");
 
-struct StreamSmem {
-    alignas(128) unsigned char ring[kStreamStages][kStageBytes];
+struct __align__(1024) StreamSmem {
+    // a stage: channels 0..63 of its 32 rows (128 B per row, 16-byte pieces swizzled by row as the copy engine
+    // lays them out), then channels 64..127
+    unsigned char ring[kStreamStages][kStageBytes];
     // [max | min | avg]; once a buffer's features have been multiplied in, its start holds the 16 x 128
     // fp32 products until they are rotated and stored
     alignas(16) __nv_bfloat16 feat_hi[2][kBulkBlocks][kFeatStride];
     alignas(16) __nv_bfloat16 feat_lo[2][kBulkBlocks][kLoStride];     // avg - bf16(avg)
     uint64_t full[kStreamStages], empty[kStreamStages];
     uint64_t feat_full[2], feat_empty[2];
+    int lens[kLensCache];                                             // seq_lens, read once
 };
 static_assert(sizeof(float) * kBulkBlocks * kStreamDGate <= sizeof(__nv_bfloat16) * kBulkBlocks * kFeatStride,
               "the products must fit in the feature buffer they replace");
-static_assert(sizeof(StreamSmem) <= 227 * 1024, "one CTA's shared memory");
+static_assert(sizeof(StreamSmem) + 1024 <= 227 * 1024, "one CTA's shared memory");
+static_assert(kStageBytes % 2048 == 0, "both halves of a stage start on a swizzle-pattern boundary");
+
+#ifdef SEER_DECODE_TRACE
+#define KC_T(var) const long long var = clock64()
+#define KC_ACC(slot, t0, t1) tr[slot] += (unsigned long long)((t1) - (t0))
+#else
+#define KC_T(var)
+#define KC_ACC(slot, t0, t1)
+#endif
 
 __device__ __forceinline__ void proj_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kProjThreads) : "memory"); }
 
-__global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const KcompParams p) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
+__global__ void __launch_bounds__(kStreamThreads, 1)
+kcomp_stream_kernel(const __grid_constant__ CUtensorMap map_k, const KcompParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    StreamSmem& sm = *reinterpret_cast<StreamSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
         for (int s = 0; s < kStreamStages; ++s) {
@@ -409,15 +423,22 @@ __global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const K
         }
         mbar_fence_init();
     }
-    __syncthreads();
     pdl_wait();
     pdl_launch_dependents();
+    // A small load issued while the copies flood the memory system waits microseconds behind them: the
+    // lengths are fetched once, before any copy is in flight.
+    for (int x = tid; x < min(p.batch, kLensCache); x += kStreamThreads) sm.lens[x] = p.seq_lens[x];
+    __syncthreads();
 
     const int b = p.block_size;                        // == kStreamRows
     const int groups = (p.num_blocks + kBulkBlocks - 1) / kBulkBlocks;
     const int per_head = groups * p.batch;
     const int n_items = per_head * p.num_kv_heads;
     bool dead = false;                                 // a wait ran out: stop waiting, finish the motions
+#ifdef SEER_DECODE_TRACE
+    unsigned long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const long long t_begin = clock64();
+#endif
 
     // item -> (head, sequence, first block) and the number of complete blocks of it that exist
     auto item_blocks = [&](int item, int& h, int& i, int& j_first) {
@@ -425,7 +446,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const K
         const int rem = item - h * per_head;
         const int g = rem / p.batch;
         i = rem - g * p.batch;
-        const int L = p.seq_lens[i];
+        const int L = i < kLensCache ? sm.lens[i] : p.seq_lens[i];
         const int complete = L > 0 ? L / b : 0;
         j_first = p.first_block + g * kBulkBlocks;
         const int j_end = min(min(p.first_block + p.num_blocks, complete), p.max_blocks);
@@ -434,42 +455,69 @@ __global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const K
 
     if (warp == kProjWarps + kPoolWarps) {
         // ---- producer ----
-        const bool rows_adjacent = p.stride_token == kHeadDim;
-        uint32_t stage_no = 0;                         // stages this CTA has been through so far
-        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-            int h, i, j_first;
-            const int nb = item_blocks(item, h, i, j_first);
-            const __nv_bfloat16* src0 = p.k_nope + (size_t)i * p.stride_batch + (size_t)h * p.stride_head;
-            for (int q = 0; q < nb; ++q, ++stage_no) {
-                const int s = stage_no % kStreamStages;
-                const uint32_t use = stage_no / kStreamStages;
-                if (!dead && !mbar_wait(&sm.empty[s], (use & 1u) ^ 1u, p.status)) dead = true;
-                if (dead) continue;
-                const __nv_bfloat16* src = src0 + (size_t)(j_first + q) * b * p.stride_token;
-                if (lane == 0) mbar_arrive_expect_tx(&sm.full[s], kStageBytes);
-                __syncwarp();
-                if (rows_adjacent) {
-                    if (lane == 0) bulk_load(sm.ring[s], src, kStageBytes, &sm.full[s]);
-                } else {
-                    for (int r = lane; r < kStreamRows; r += 32)
-                        bulk_load(sm.ring[s] + r * (kHeadDim * 2), src + (size_t)r * p.stride_token, kHeadDim * 2,
-                                  &sm.full[s]);
+        // Lane l owns ring slot l: it walks the CTA's items for the stages l, l + kStreamStages, ... and
+        // re-arms its slot the moment the slot is free.  The lanes poll in lockstep (one look at the slot's
+        // barrier per turn, no waiting inside), so slots that are freed together are refilled together
+        // instead of one barrier round trip after the other.
+        if (lane == 0) tma_prefetch_desc(&map_k);
+        uint32_t cursor = lane;                        // the stage this lane arms next
+        uint32_t item_first = 0;                       // stage number of the first stage of `item`
+        int item = blockIdx.x, h = 0, i = 0, j_first = 0;
+        int nb = item < n_items ? item_blocks(item, h, i, j_first) : 0;
+        uint32_t idle = 0;
+        while (true) {
+            while (item < n_items && cursor >= item_first + (uint32_t)(nb * kStagesPerBlock)) {
+                item_first += nb * kStagesPerBlock;
+                item += gridDim.x;
+                nb = item < n_items ? item_blocks(item, h, i, j_first) : 0;
+            }
+            const bool have = lane < kStreamStages && item < n_items;
+            if (!__any_sync(0xffffffffu, have)) break;
+            const bool go = have && mbar_test_wait(&sm.empty[lane], ((cursor / kStreamStages) & 1u) ^ 1u);
+            if (go) {
+                const uint32_t rel = cursor - item_first;
+                const int q = rel / kStagesPerBlock, part = rel % kStagesPerBlock;
+                const int row0 = (j_first + q) * b + part * kStageRows;
+                mbar_arrive_expect_tx(&sm.full[lane], kStageBytes);
+                tma_load_4d(sm.ring[lane], &map_k, &sm.full[lane], 0, row0, h, i);
+                tma_load_4d(sm.ring[lane] + kStageBytes / 2, &map_k, &sm.full[lane], 64, row0, h, i);
+                cursor += kStreamStages;
+            }
+            const uint32_t went = __ballot_sync(0xffffffffu, go);
+#ifdef SEER_DECODE_TRACE
+            tr[0] += 1; tr[1] += __popc(went);
+#endif
+            if (went) {
+                idle = 0;
+            } else if (++idle > 64) {
+                if (idle > (1u << 22)) {               // seconds: nothing will free these slots any more
+                    raise_status(p.status, DEV_TIMEOUT);
+                    break;
                 }
+                __nanosleep(32);
             }
         }
     } else if (warp >= kProjWarps) {
         // ---- pooling ----
         const int pw = warp - kProjWarps;
         const int cchunk = lane & 15;
-        uint32_t stage_no = 0, n_done = 0;
+        // where this lane's piece sits in rows 2k + (lane >> 4) for k = 0..3 mod 4 (see the read below)
+        const int lane_off = (cchunk >> 3) * (kStageBytes / 2) + (lane >> 4) * 128;
+        int piece_off[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) piece_off[m] = (((cchunk & 7) ^ (lane >> 4)) ^ (2 * m)) << 4;
+        uint32_t block_no = 0, n_done = 0;                 // blocks and items this CTA has been through
         for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
             int h, i, j_first;
             const int nb = item_blocks(item, h, i, j_first);
             if (nb == 0) continue;
             const int fb = n_done & 1;
+            KC_T(t_fe0);
             if (!dead && !mbar_wait(&sm.feat_empty[fb], ((n_done >> 1) & 1u) ^ 1u, p.status)) dead = true;
+            KC_T(t_fe1);
+            KC_ACC(0, t_fe0, t_fe1);
             for (int q = 0; q < kBulkBlocks; ++q) {
-                if ((stage_no + q) % kPoolWarps != (uint32_t)pw) continue;
+                if ((block_no + q) % kPoolWarps != (uint32_t)pw) continue;
                 __nv_bfloat162 mx[4], mn[4];
                 float sum[8];
 #pragma unroll
@@ -480,25 +528,37 @@ __global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const K
 #pragma unroll
                 for (int c = 0; c < 8; ++c) sum[c] = 0.f;
                 if (q < nb) {
-                    const uint32_t sn = stage_no + q;
-                    const int s = sn % kStreamStages;
-                    if (!dead && !mbar_wait(&sm.full[s], (sn / kStreamStages) & 1u, p.status)) dead = true;
-                    // lane: 16-byte column piece (lane & 15) of rows 2k + (lane >> 4)
-                    const uint4* st = reinterpret_cast<const uint4*>(sm.ring[s]) + lane;
+#pragma unroll 1
+                    for (int part = 0; part < kStagesPerBlock; ++part) {
+                        const uint32_t sn = (block_no + q) * kStagesPerBlock + part;
+                        const int s = sn % kStreamStages;
+                        KC_T(t_w0);
+                        if (!dead && !mbar_wait(&sm.full[s], (sn / kStreamStages) & 1u, p.status)) dead = true;
+                        KC_T(t_w1);
+                        KC_ACC(1, t_w0, t_w1);
+                        // lane: 16-byte column piece (lane & 15) of rows 2k + (lane >> 4); piece c of row r of a
+                        // 64-channel half sits at position c ^ (r & 7) of the row's 128 bytes
+                        const unsigned char* st = sm.ring[s] + lane_off;
 #pragma unroll 8
-                    for (int k = 0; k < kStreamRows / 2; ++k) {
-                        const uint4 v = st[k * 32];
-                        const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&v);
+                        for (int k = 0; k < kStageRows / 2; ++k) {
+                            const uint4 v = *reinterpret_cast<const uint4*>(st + k * 256 + piece_off[k & 3]);
+                            const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&v);
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            mx[c] = __hmax2(mx[c], hh[c]);
-                            mn[c] = __hmin2(mn[c], hh[c]);
-                            const float2 f = bf16x2_to_float2(hh[c]);
-                            sum[2 * c] += f.x; sum[2 * c + 1] += f.y;
+                            for (int c = 0; c < 4; ++c) {
+                                mx[c] = __hmax2(mx[c], hh[c]);
+                                mn[c] = __hmin2(mn[c], hh[c]);
+                                const float2 f = bf16x2_to_float2(hh[c]);
+                                sum[2 * c] += f.x; sum[2 * c + 1] += f.y;
+                            }
                         }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sm.empty[s]);
+                        KC_T(t_w2);
+                        KC_ACC(2, t_w1, t_w2);
+#ifdef SEER_DECODE_TRACE
+                        tr[3] += 1;
+#endif
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.empty[s]);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t xm = *reinterpret_cast<uint32_t*>(&mx[c]), xn = *reinterpret_cast<uint32_t*>(&mn[c]);
@@ -519,17 +579,20 @@ __global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const K
                     }
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        const float av = q < nb ? sum[c] / (float)b : 0.f;
+                        const float av = q < nb ? sum[c] * (1.f / kStreamRows) : 0.f;
                         const __nv_bfloat16 av_hi = __float2bfloat16(av);
                         sm.feat_hi[fb][q][2 * kHeadDim + 8 * cchunk + c] = av_hi;
                         sm.feat_lo[fb][q][8 * cchunk + c] = __float2bfloat16(av - __bfloat162float(av_hi));
                     }
                 }
             }
-            stage_no += nb;
+            block_no += nb;
             ++n_done;
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.feat_full[fb]);
+#ifdef SEER_DECODE_TRACE
+            { const long long t_e = clock64(); tr[4] += (unsigned long long)(t_e - t_fe0); }
+#endif
         }
     } else {
         // ---- projection, rotation, store ----
@@ -556,7 +619,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const K
             }
             h_held = h;
             const int fb = n_done & 1;
+            KC_T(t_p0);
             if (!dead && !mbar_wait(&sm.feat_full[fb], (n_done >> 1) & 1u, p.status)) dead = true;
+            KC_T(t_p1);
+            KC_ACC(0, t_p0, t_p1);
             ++n_done;
             float acc[2][4];
 #pragma unroll
@@ -579,6 +645,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const K
                     }
                 }
             }
+            KC_T(t_pa);
+            KC_ACC(2, t_p1, t_pa);
             proj_sync();                                    // every warp is done with the features
             float (*ybuf)[kStreamDGate] = reinterpret_cast<float (*)[kStreamDGate]>(&sm.feat_hi[fb][0][0]);
             if (projects) {
@@ -591,29 +659,61 @@ __global__ void __launch_bounds__(kStreamThreads, 1) kcomp_stream_kernel(const K
                 }
             }
             proj_sync();
+            KC_T(t_pb);
+            KC_ACC(3, t_pa, t_pb);
             const int half = p.d_gate / 2;
             const int u = i * p.num_kv_heads + h;
-            for (int x = tid; x < nb * half; x += kProjThreads) {
-                const int q = x / half, c = x % half;
+            // eight rotary pairs per thread: two 16-byte stores instead of sixteen 2-byte ones (a store, too,
+            // queues behind the copies)
+            for (int x = tid; x < nb * (half / 8); x += kProjThreads) {
+                const int q = x / (half / 8), c0 = 8 * (x % (half / 8));
                 const int j = j_first + q;
-                float sn, cs;
-                rope_sincos((double)j * (double)b, p.inv_freq[c], &sn, &cs);
-                const float a = ybuf[q][c], bb = ybuf[q][c + half];
-                __nv_bfloat16* dst = p.kcomp + ((size_t)u * p.max_blocks + j) * p.d_gate;
-                dst[c] = __float2bfloat16(a * cs - bb * sn);
-                dst[c + half] = __float2bfloat16(bb * cs + a * sn);
+                uint32_t lo[4], hi[4];
+#pragma unroll
+                for (int e = 0; e < 8; e += 2) {
+                    float r0[2], r1[2];
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        float sn, cs;
+                        rope_sincos((double)j * (double)b, p.inv_freq[c0 + e + k], &sn, &cs);
+                        const float a = ybuf[q][c0 + e + k], bb = ybuf[q][c0 + e + k + half];
+                        r0[k] = a * cs - bb * sn;
+                        r1[k] = bb * cs + a * sn;
+                    }
+                    lo[e / 2] = pack_bf16x2(r0[0], r0[1]);
+                    hi[e / 2] = pack_bf16x2(r1[0], r1[1]);
+                }
+                __nv_bfloat16* dst = p.kcomp + ((size_t)u * p.max_blocks + j) * p.d_gate + c0;
+                *reinterpret_cast<uint4*>(dst) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                *reinterpret_cast<uint4*>(dst + half) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
             }
             // the buffer may be refilled once all eight warps have read their products out of it; the next
             // item's features and products are in the other buffer
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.feat_empty[fb]);
+            KC_T(t_p2);
+            KC_ACC(1, t_p1, t_p2);
+            KC_ACC(4, t_pb, t_p2);
         }
     }
+#ifdef SEER_DECODE_TRACE
+    if (lane == 0) {
+        tr[7] = (unsigned long long)(clock64() - t_begin);
+        for (int k = 0; k < 8; ++k) p.trace[((size_t)blockIdx.x * (kStreamThreads / 32) + warp) * 8 + k] = tr[k];
+    }
+#endif
 }
 
 }  // namespace
 
-cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* launched) {
+bool kcomp_bulk_streams(const KcompParams& p) {
+    const int U = p.batch * p.num_kv_heads;
+    const int gx = (p.num_blocks + kBulkBlocks - 1) / kBulkBlocks;
+    return p.first_block >= 0 && p.block_size == kStreamRows && p.d_gate <= kStreamDGate && !p.rows_block_local &&
+           (long long)gx * U >= 2LL * p.sm_count;
+}
+
+cudaError_t launch_kcomp_append(const KcompParams& p, const CUtensorMap* map_k, cudaStream_t stream, int* launched) {
     const int U = p.batch * p.num_kv_heads;
     *launched = 0;
     if (U <= 0) return cudaSuccess;
@@ -625,19 +725,19 @@ cudaError_t launch_kcomp_append(const KcompParams& p, cudaStream_t stream, int* 
     } else {
         const int gx = (p.num_blocks + kBulkBlocks - 1) / kBulkBlocks;
         if (gx <= 0) return cudaSuccess;
-        if (p.block_size == kStreamRows && p.d_gate <= kStreamDGate && !p.rows_block_local && gx * U >= 2 * p.sm_count) {
+        if (map_k && kcomp_bulk_streams(p)) {
             static bool attr_set[64] = {};
             int dev = 0;
             cudaError_t e = cudaGetDevice(&dev);
             if (e != cudaSuccess) return e;
             if (dev < 0 || dev >= 64 || !attr_set[dev]) {
                 e = cudaFuncSetAttribute(kcomp_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)sizeof(StreamSmem));
+                                         (int)sizeof(StreamSmem) + 1024);
                 if (e != cudaSuccess) return e;
                 if (dev >= 0 && dev < 64) attr_set[dev] = true;
             }
             e = launch_pdl(kcomp_stream_kernel, dim3(min(p.sm_count, gx * U), 1, 1), dim3(kStreamThreads),
-                           sizeof(StreamSmem), stream, p);
+                           sizeof(StreamSmem) + 1024, stream, *map_k, p);
             *launched = 1;
             return e;
         }

@@ -48,6 +48,7 @@ struct seer_ctx {
     unsigned int generation;    // stamps the partials of a decode launch
     int pool_div;               // decode scheduling: share of tiles handed out dynamically
     int min_tiles;              // decode scheduling: fewest tiles of a CTA's range
+    int wide_variant;           // kernel variant code for more than 16 rows per unit: 16 (tcgen05) or 8 (mma.sync)
     char err[512];
 };
 
@@ -208,8 +209,9 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     const bool wide = q_len * group > 16 && bpt == 1;
     const int row_cap = wide ? 64 : 16;
     const int tok_per_launch = q_len < row_cap / group ? q_len : row_cap / group;
-    const int n_tiles = wide ? 8 : tok_per_launch * group > 8 ? 2 : 1;
-    const int per_sm = decode_ctas_per_sm(sparse, paged, n_tiles);
+    const int n_tiles = wide ? 8 : tok_per_launch * group > 8 ? 2 : 1;    // (sizes the partial slots: 8 rows each)
+    const int variant = wide ? ctx->wide_variant : n_tiles;               // (the kernel: 16 = rows on M by tcgen05)
+    const int per_sm = decode_ctas_per_sm(sparse, paged, variant);
     if (per_sm <= 0) return fail(ctx, SEER_ERR_CUDA, "decode kernel cannot be resident (shared memory)");
     long long max_tiles = sparse ? (long long)U * ((max_sel + bpt - 1) / bpt) * tpb
                                  : (long long)U * ((kv->max_seq_len + kTileTokens - 1) / kTileTokens);
@@ -290,7 +292,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
         p.t_cnt = q_len - t0 < tok_per_launch ? q_len - t0 : tok_per_launch;
         p.rows = p.t_cnt * group;
         p.generation = ++ctx->generation;
-        ce = launch_decode(sparse, paged, n_tiles, mk_copy, *mv, p, grid, static_cast<cudaStream_t>(stream));
+        ce = launch_decode(sparse, paged, variant, mk_copy, *mv, p, grid, static_cast<cudaStream_t>(stream));
         if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "decode launch: %s", cudaGetErrorString(ce));
         ctx->launches += 1;
     }
@@ -327,6 +329,8 @@ seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes) {
     if (const char* e = getenv("SEER_DECODE_POOL_DIV")) ctx->pool_div = atoi(e);
     ctx->min_tiles = 4;
     if (const char* e = getenv("SEER_DECODE_MIN_TILES")) ctx->min_tiles = atoi(e);
+    ctx->wide_variant = 8;
+    if (const char* e = getenv("SEER_DECODE_WIDE_VARIANT")) ctx->wide_variant = atoi(e) == 16 ? 16 : 8;
     ctx->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)64 << 20;
     if (ctx->ws_bytes < 4096) ctx->ws_bytes = 4096;     // (far too small for any call: every call checks)
     if (cudaMalloc(reinterpret_cast<void**>(&ctx->ws), ctx->ws_bytes) != cudaSuccess) {

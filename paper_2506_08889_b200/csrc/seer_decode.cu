@@ -51,10 +51,17 @@ constexpr int kStageBytes = 2 * kTileBytes;                // K + V
 constexpr int kMergeStride = 132;                          // floats per head row (bank spread)
 constexpr int kMaxPieces = 32;                             // partial pieces a CTA can hold back to its end
 constexpr int kListInts = kStageBytes / 4 - 64;              // slot numbers that fit in one stage buffer (less 64 counts)
-constexpr int kLandBytes = 2 * kStageBytes;                 // landing area for staged partials: two stage buffers
 constexpr int kMaxSteals = 14;                             // chunks a CTA may take from other ranges
 constexpr int kFewTilesPerCta = 16;                        // up to this many tiles per CTA the number of ranges is chosen with care
 constexpr int kWideTiles = 8;                              // N-tile count that stands for the rows-on-M variant (up to 64 rows)
+// The rows-on-M variant on the fifth-generation tensor cores (TC): one CTA per SM, a deeper ring, an extra
+// warp that issues the MMAs; S, P and O live in tensor memory.
+constexpr int kTcTilesCode = 16;                           // what the host passes as n_tiles to ask for it
+constexpr int kTcStages = 8;                               // V buffers (16 KiB each) = tiles between landing and product
+constexpr int kTcKStages = 4;                              // K buffers (16 KiB each): a K tile is free once its scores are computed
+constexpr int kTcThreads = kThreads + 32;
+constexpr int kTcRows = 128;                               // M of the MMAs (rows past the unit's are zero)
+constexpr int kTcCols = 256;                               // tensor-memory columns: S/P twice 64, O 128
 constexpr int kAheadMaxChunk = 8;                          // own chunks up to this size are claimed ahead
 constexpr int kAheadTiles = 3;                             // tiles left to issue when the next interval's claim is made
 constexpr int kSmemUnits = 128;                            // units whose tile-count prefix sums fit in shared memory
@@ -92,12 +99,33 @@ struct Schedule {
     int off[kMaxRounds + 2];       // off[j]: tiles from the start of chunk j to the end of its range
 };
 
-struct __align__(1024) Smem {
-    unsigned char stage[kStages][kStageBytes];
+// What only one kind of variant needs: the cross-warp merge scratch of the mma.sync variants, or the barriers of
+// the tensor-memory variant.
+template <bool TC>
+struct VariantPart {
     float merge_o[kConsumerWarps - 1][kMaxGroup][kMergeStride];   // warps 1..3 -> warp 0
     float merge_ml[kConsumerWarps - 1][2][kMaxGroup];
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+};
+template <>
+struct VariantPart<true> {
+    uint64_t bar_s[2];               // S of an even / odd tile is complete (the MMA warp's commit)
+    uint64_t bar_p[2];               // P of an even / odd tile is written (one arrival per row warp with real rows)
+    uint64_t bar_o[2];               // O includes an even / odd tile's product (commit)
+    uint64_t tmem_done;              // the row warps have made their last tensor-memory access
+    uint64_t empty_k[kTcKStages];    // a K buffer's scores have been computed (commit)
+    uint32_t tmem_base;
+};
+
+template <bool TC>
+struct __align__(1024) SmemT {
+    static constexpr int kS = TC ? kTcStages : kStages;
+    // The K/V ring.  The tensor-memory variant cuts the same memory differently: kTcStages V buffers, then
+    // kTcKStages K buffers (16 KiB each), then the unit's queries, [64-channel half][128 rows][128 B] with
+    // 16-byte pieces swizzled by row.
+    static constexpr int kBufs = TC ? (kTcStages + kTcKStages) / 2 + 1 : kStages;
+    unsigned char stage[kBufs][kStageBytes];
+    uint64_t full[kS];
+    uint64_t empty[kS];
     uint64_t merge_bar[2];           // [0]: scratch filled (3 arrivals), [1]: scratch free again / end sync
     uint64_t end_bar;                // all consumer warps: streams over, the list of combines is final
     uint64_t list_bar;               // all consumer warps: the lists of valid slots are written
@@ -105,11 +133,15 @@ struct __align__(1024) Smem {
     volatile int issued;             // tiles whose metadata the producer has written so far
     volatile int first_unit;         // unit of the CTA's first tile (-1: none yet known, -2: not yet decided)
     int upfx[kSmemUnits + 1];        // prefix sums of the units' tile counts (when there are at most kSmemUnits units)
-    StageMeta meta[kStages];
+    StageMeta meta[kS];
     Schedule sched;
     Piece pieces[kMaxPieces];
     int pieces_n;
+    VariantPart<TC> v;
 };
+static_assert(2 * kTcRows * 128 == kStageBytes, "the query tile takes one stage buffer");
+using Smem = SmemT<false>;
+static_assert(sizeof(SmemT<true>) + 1024 <= 227 * 1024, "the tensor-memory variant's shared memory");
 
 // two CTAs per SM: 2 * (sizeof(Smem) + 1 KiB alignment slack + 1 KiB reserved by the system) must
 // fit in the SM's 228 KiB
@@ -379,23 +411,39 @@ __device__ __forceinline__ int scan_valid_slots(const DecodeParams& p, int first
     return n;
 }
 
-template <bool SPARSE, bool PAGED, int NT, bool SMALL>
-__global__ void __launch_bounds__(kThreads, 2)
+template <bool SPARSE, bool PAGED, int NT, bool SMALL, bool TC = false>
+__global__ void __launch_bounds__(TC ? kTcThreads : kThreads, TC ? 1 : 2)
 decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const DecodeParams p) {
+    static_assert(!TC || (NT == kWideTiles && !SMALL), "the tensor-memory variant is the rows-on-M variant");
+    using SmemK = SmemT<TC>;
+    constexpr int kS = SmemK::kS;    // stages of the K/V ring
     extern __shared__ unsigned char smem_raw[];
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    SmemK& sm = *reinterpret_cast<SmemK*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int U = p.num_units;
     const int cta = blockIdx.x;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        // row warps that hold real rows of the unit (tensor-memory variant: lane = row, 32 rows per warp)
+        const int tc_row_warps = min(kConsumerWarps, (p.rows + 31) / 32);
+        for (int s = 0; s < kS; ++s) {
             mbar_init(&sm.full[s], 1);
-            mbar_init(&sm.empty[s], kConsumerWarps);
+            // a stage is free once every consumer warp has arrived; tensor-memory variant: once the MMAs that read
+            // it have completed (one commit) and every row warp has taken the tile's metadata
+            mbar_init(&sm.empty[s], TC ? 1 + tc_row_warps : kConsumerWarps);
         }
-        mbar_init(&sm.merge_bar[0], NT < kWideTiles ? kConsumerWarps - 1 : kConsumerWarps);   // (rows on M: "partial written" by all four)
+        if constexpr (TC) {
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(&sm.v.bar_s[b], 1);
+                mbar_init(&sm.v.bar_p[b], tc_row_warps);
+                mbar_init(&sm.v.bar_o[b], 1);
+            }
+            mbar_init(&sm.v.tmem_done, tc_row_warps);
+            for (int b = 0; b < kTcKStages; ++b) mbar_init(&sm.v.empty_k[b], 1);
+        }
+        mbar_init(&sm.merge_bar[0], TC ? tc_row_warps : NT < kWideTiles ? kConsumerWarps - 1 : kConsumerWarps);   // (rows on M: "partial written" by every warp with rows)
         mbar_init(&sm.merge_bar[1], 1);
         mbar_init(&sm.end_bar, kConsumerWarps);
         mbar_init(&sm.list_bar, kConsumerWarps);
@@ -418,7 +466,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     }
 #endif
     if (tid == 0) SEER_STAMP(8);
+    if constexpr (TC) {
+        if (warp == kConsumerWarps + 1) tmem_alloc(&sm.v.tmem_base, kTcCols);
+        tc_fence_before_sync();
+    }
     __syncthreads();                                 // barriers initialised
+    if constexpr (TC) tc_fence_after_sync();
     pdl_wait();
     if (tid == 0) SEER_STAMP(9);
 
@@ -783,12 +836,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                         s_outer[sb] = (sb == 0 || SMALL) ? __shfl_sync(0xffffffffu, outer[sb], s) : 0;
                     }
                     if (lane == 0) {
-                        const int st = it % kStages;
+                        const int st = it % kS;
 #ifdef SEER_DECODE_TRACE
                         if (it == 0) SEER_STAMP(13);
                         if (it == 1) SEER_STAMP(14);
 #endif
-                        if (!mbar_wait(&sm.empty[st], ((it / kStages) & 1) ^ 1, p.status)) return;
+                        if (!mbar_wait(&sm.empty[st], ((it / kS) & 1) ^ 1, p.status)) return;
                         sm.meta[st] = StageMeta{s_nvalid, s_u, s_flags, s_pu, s_ut, iv_id};
                         __threadfence_block();
                         sm.issued = it + 1;                  // consumers may look ahead at this tile
@@ -811,6 +864,23 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                                                 s_head, s_outer[sb]);
                                 }
                             }
+                        } else if (TC) {
+                            // K and V go to rings of their own: the K buffer has to be free as well
+                            if constexpr (TC) {
+                                const int sk = it % kTcKStages;
+                                if (!mbar_wait(&sm.v.empty_k[sk], ((it / kTcKStages) & 1) ^ 1, p.status)) return;
+                                if (s_nvalid > 0) {
+                                    unsigned char* dk = sm.stage[0] + (size_t)(kTcStages + sk) * kTileBytes;
+                                    unsigned char* dv = sm.stage[0] + (size_t)st * kTileBytes;
+                                    mbar_arrive_expect_tx(&sm.full[st], kStageBytes);
+                                    tma_load_4d(dk, &map_k, &sm.full[st], 0, s_row[0], s_head, s_outer[0]);
+                                    tma_load_4d(dk + kHalfTileBytes, &map_k, &sm.full[st], 64, s_row[0], s_head, s_outer[0]);
+                                    tma_load_4d(dv, &map_v, &sm.full[st], 0, s_row[0], s_head, s_outer[0]);
+                                    tma_load_4d(dv + kHalfTileBytes, &map_v, &sm.full[st], 64, s_row[0], s_head, s_outer[0]);
+                                } else {
+                                    mbar_arrive(&sm.full[st]);
+                                }
+                            }
                         } else if (s_nvalid > 0) {
                             mbar_arrive_expect_tx(&sm.full[st], kStageBytes);
                             tma_load_4d(dst, &map_k, &sm.full[st], 0, s_row[0], s_head, s_outer[0]);
@@ -827,8 +897,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         }
         if (lane == 0) {
             // end-of-stream marker for the consumers
-            const int st = it % kStages;
-            if (!mbar_wait(&sm.empty[st], ((it / kStages) & 1) ^ 1, p.status)) return;
+            const int st = it % kS;
+            if (!mbar_wait(&sm.empty[st], ((it / kS) & 1) ^ 1, p.status)) return;
             sm.meta[st] = StageMeta{-1, -1, 1, 0, 0, 0};
             __threadfence_block();
             sm.issued = it + 1;
@@ -844,6 +914,154 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         return;
     }
 
+    if constexpr (TC) {
+    if (warp == kConsumerWarps + 1) {
+        // =========================== MMA warp (tensor-memory variant) ====================
+        // Lane 0 issues, per tile, S = Q . K^T (8 MMAs of K = 16 over the 128 channels; Q and the K tile
+        // K-major in shared memory) and, once the row warps have written the tile's probabilities,
+        // O (+)= P . V (4 MMAs over the 64 tokens; P from tensor memory, the V tile MN-major).  The product
+        // of a tile is issued after the scores of the next one, so the tensor cores work on S(t + 1)
+        // while the row warps are busy with S(t).  The whole warp brings a unit's queries into shared
+        // memory (zero rows past the unit's) and clears the rows of a ragged last tile of V.
+        const uint32_t tbase = sm.v.tmem_base;
+        const uint32_t t_o = tbase + 128;
+        constexpr uint32_t idesc_qk = tc_idesc_bf16(kTcRows, kTileTokens, false);
+        constexpr uint32_t idesc_pv = tc_idesc_bf16(kTcRows, kHeadDim, true);
+        const uint32_t q_addr = smem_u32(sm.stage[SmemK::kBufs - 1]);
+        bool dead = false;                         // a wait ran out: stop issuing, free the tensor memory, leave
+        int ct = 0, piece_ct = 0;                  // computed tiles so far (of the CTA, of the piece)
+        int q_unit = -1;
+#ifdef SEER_DECODE_TRACE
+        unsigned long long mm_tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const long long mm_t0 = clock64();
+#endif
+        // Two kinds of work, taken as they become possible: the scores of the next tile once it has landed
+        // (at most two tiles may be between their scores and their product: S is double-buffered), and the
+        // product of the oldest such tile once its probabilities are written.  A stage is released by the
+        // commit behind its product, so it is held no longer than the row warps need for its tile.
+        int pend_n = 0;                            // tiles whose product is still to be issued (0..2)
+        int pend_stage[2] = {0, 0};
+        bool pend_acc[2] = {false, false};         // indexed by the tile's parity (ct & 1)
+        int it = 0;                                // next tile of the stream
+        bool ended = false;
+        uint32_t idle = 0;
+        // rows of the query tile past the unit's stay zero for the whole launch
+        for (int x = p.rows * 16 + lane; x < kTcRows * 16; x += 32) {
+            const int r = x >> 4, c16 = x & 15;
+            *reinterpret_cast<uint4*>(sm.stage[SmemK::kBufs - 1] + (c16 >> 3) * (kTcRows * 128) + r * 128 + ((c16 & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        __syncwarp();
+        while (!dead && (!ended || pend_n > 0)) {
+            bool did = false;
+            if (pend_n > 0) {
+                const int c = ct - pend_n, b = c & 1;
+                if (__shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.v.bar_p[b], (c >> 1) & 1) : 0, 0)) {
+                    __syncwarp();
+                    if (lane == 0) {
+                        tc_fence_after_sync();
+                        const uint32_t v_addr = smem_u32(sm.stage[0]) + pend_stage[b] * kTileBytes;
+#pragma unroll
+                        for (int ks = 0; ks < kTileTokens / 16; ++ks)
+                            tc_mma_ts(t_o, tbase + 64 * b + 8 * ks, tc_smem_desc(v_addr + ks * 2048, kHalfTileBytes, 1024), idesc_pv,
+                                      pend_acc[b] || ks > 0);
+                        tc_commit(&sm.empty[pend_stage[b]]);   // the stage's K and V have been read
+                        tc_commit(&sm.v.bar_o[b]);
+                    }
+                    __syncwarp();
+                    --pend_n;
+                    did = true;
+                }
+            }
+            if (!ended && pend_n < 2) {
+                const int st = it % kS;
+                if (__shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.full[st], (it / kS) & 1) : 0, 0)) {
+                    // (every lane reads the metadata after lane 0 has seen the barrier's phase complete)
+                    mbar_try_wait(&sm.full[st], (it / kS) & 1);
+                    __syncwarp();
+                    const StageMeta mt = sm.meta[st];
+                    did = true;
+                    if (mt.nvalid < 0) {
+                        ended = true;
+                    } else {
+                        if (mt.flags & 1) piece_ct = 0;
+                        const int nv = mt.nvalid;
+                        if (nv > 0) {
+                            if (q_unit != mt.unit) {
+                                // every earlier S has been computed before the queries change
+                                if (ct > 0 && !mbar_wait(&sm.v.bar_s[(ct - 1) & 1], ((ct - 1) >> 1) & 1, p.status)) { dead = true; break; }
+                                // the unit's real rows, by asynchronous 16-byte copies all issued before any is waited for
+                                // (the rows past them were cleared once and stay zero)
+                                for (int x = lane; x < p.rows * 16; x += 32) {
+                                    const int r = x >> 4, c16 = x & 15;
+                                    cp_async16(sm.stage[SmemK::kBufs - 1] + (c16 >> 3) * (kTcRows * 128) + r * 128 + (((c16 & 7) ^ (r & 7)) << 4),
+                                               reinterpret_cast<const uint4*>(p.q + unit_row(p, mt.unit, r) * kHeadDim) + c16);
+                                }
+                                cp_async_wait_all();
+                                q_unit = mt.unit;
+                                fence_proxy_async_smem();
+                                __syncwarp();
+                            }
+                            if (nv < kTileTokens) {
+                                // ragged tail: rows past the sequence end may hold anything; cleared in V so that a
+                                // zero probability times garbage cannot produce NaN
+                                unsigned char* vt = sm.stage[0] + (size_t)st * kTileBytes;
+                                for (int x = lane; x < (kTileTokens - nv) * 16; x += 32) {
+                                    const int r = nv + (x >> 4), part = x & 15;
+                                    *reinterpret_cast<uint4*>(vt + (part >> 3) * kHalfTileBytes + r * 128 + ((part & 7) << 4)) =
+                                        make_uint4(0u, 0u, 0u, 0u);
+                                }
+                                fence_proxy_async_smem();
+                                __syncwarp();
+                            }
+                            const int b = ct & 1;
+                            if (lane == 0) {
+                                tc_fence_after_sync();
+                                const uint32_t k_addr = smem_u32(sm.stage[0]) + (kTcStages + it % kTcKStages) * kTileBytes;
+#pragma unroll
+                                for (int ks = 0; ks < kHeadDim / 16; ++ks)
+                                    tc_mma_ss(tbase + 64 * b, tc_smem_desc(q_addr + (ks >> 2) * (kTcRows * 128) + (ks & 3) * 32, 16, 1024),
+                                              tc_smem_desc(k_addr + (ks >> 2) * kHalfTileBytes + (ks & 3) * 32, 16, 1024), idesc_qk, ks > 0);
+                                tc_commit(&sm.v.bar_s[b]);
+                                tc_commit(&sm.v.empty_k[it % kTcKStages]);   // the K buffer has been read
+                            }
+                            __syncwarp();
+                            pend_stage[b] = st;
+                            pend_acc[b] = piece_ct > 0;
+                            ++pend_n;
+                            ++ct;
+                            ++piece_ct;
+                        } else {
+                            if (lane == 0) {                               // nothing was loaded: the buffers go straight back
+                                mbar_arrive(&sm.empty[st]);
+                                mbar_arrive(&sm.v.empty_k[it % kTcKStages]);
+                            }
+                        }
+                        ++it;
+                    }
+                }
+            }
+            if (did) {
+                idle = 0;
+            } else if (++idle > 64) {
+                if (idle > (1u << 23)) {               // seconds: whatever this warp waits for will not come
+                    raise_status(p.status, DEV_TIMEOUT);
+                    dead = true;
+                }
+                __nanosleep(32);
+            }
+        }
+#ifdef SEER_DECODE_TRACE
+        mm_tr[3] = (unsigned long long)(clock64() - mm_t0);
+        if (lane == 0) for (int k = 0; k < 8; ++k) p.trace[(size_t)blockIdx.x * kTraceSlots + 64 + k] = mm_tr[k];
+#endif
+        // the tensor memory goes back once the row warps are done with it (or a wait has run out)
+        mbar_wait(&sm.v.tmem_done, 0, p.status);
+        __syncwarp();
+        tmem_dealloc(tbase, kTcCols);
+        return;
+    }
+    }
+
     // =============================== consumer warps =====================================
     const int w = warp;
     const int qd = lane & 3;            // column pair: rows 2*qd, 2*qd+1 of every N-tile
@@ -851,7 +1069,230 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     unsigned long long tk_before = 0ull; // warp 0, lane k: what the unit's counter held before the k-th held piece was added
     unsigned int tk_bit = 0u;            // ... and that piece's bit
     int piece_tiles = 0, piece_iv = 0;  // tiles in the current piece, interval it started in
-    if constexpr (NT < kWideTiles) {
+    if constexpr (TC) {
+    // ---------------- the unit's rows on M, on the fifth-generation tensor cores ----------------
+    // Thread t of the four row warps is row t of the unit and lane t of tensor memory; warps whose 32 rows
+    // are all padding have nothing to do until the stream is over.  Per tile a row thread reads its 64 scores
+    // (S, fp32), masks, exponentiates against the row's reference maximum, adds up, and writes the 64
+    // probabilities back over S as bf16 pairs (P) for the MMA warp's second product.  The reference maximum
+    // only moves when the true one has grown by more than 2^8 since (probabilities stay below 2^8, exact in
+    // bf16's range); O, which accumulates in tensor memory, is rescaled on those occasions only.
+    //     S (128 x 64 tok) = Q (128 x 128) . K^T      tcgen05.mma, Q and K K-major in shared memory
+    //     O (128 x 128)   += P (128 x 64) . V          P from tensor memory, V MN-major in shared memory
+    constexpr float kSlack = 8.f;
+#ifdef SEER_DECODE_TRACE
+    unsigned long long tc_tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#define TC_T(v) const long long v = clock64()
+#define TC_ACC(k, a, b) tc_tr[k] += (unsigned long long)((b) - (a))
+#else
+#define TC_T(v)
+#define TC_ACC(k, a, b)
+#endif
+    const int row = tid;
+    const bool real = row < p.rows;
+    // newest cached tokens the row may not see (its query token's distance from the last one)
+    const int back = real ? p.q_len - 1 - (p.t_base + ((row * p.group_magic) >> 16)) : 0;
+    int pubs = 0;                       // partials written so far (phase of merge_bar[0])
+    if (32 * w < p.rows) {
+        const uint32_t tbase = sm.v.tmem_base + ((uint32_t)(32 * w) << 16);
+        const uint32_t t_o = tbase + 128;
+        float m_ref = -INFINITY, l_run = 0.f;
+        int ct = 0, piece_ct = 0;       // computed tiles so far (of the CTA, of the piece)
+        if (!mbar_wait(&sm.full[0], 0, p.status)) return;
+        if (tid == 0) SEER_STAMP(10);
+        StageMeta mt = sm.meta[0];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[0]);              // metadata taken
+        for (int it = 0; mt.nvalid >= 0; ++it) {
+            if (mt.flags & 1) {
+                m_ref = -INFINITY;
+                l_run = 0.f;
+                piece_tiles = 0;
+                piece_iv = mt.interval;
+                piece_ct = 0;
+            }
+            ++piece_tiles;
+            const int nv = mt.nvalid;                          // cached tokens from the tile's first row on (capped at 64 + 7)
+            if (nv > 0) {
+                const int b = ct & 1;
+                TC_T(t_a);
+                if (!mbar_wait(&sm.v.bar_s[b], (ct >> 1) & 1, p.status)) return;
+                __syncwarp();
+                tc_fence_after_sync();
+                TC_T(t_b);
+                TC_ACC(0, t_a, t_b);
+                uint32_t sr[2][32];
+                tmem_ld32(tbase + 64 * b, sr[0]);
+                tmem_ld32(tbase + 64 * b + 32, sr[1]);
+                tmem_wait_ld();
+                TC_T(t_c);
+                TC_ACC(1, t_b, t_c);
+                // tokens the row may see: the first `lim` of the tile; hidden ones get a score of -inf.  (Only the
+                // newest tiles of a sequence have any, so the test is skipped when the whole warp sees all 64.)
+                const int lim = nv - back;
+                if (!__all_sync(0xffffffffu, lim >= kTileTokens)) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (32 * h + c >= lim) sr[h][c] = 0xff800000u;
+                }
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};       // (four short chains instead of one long)
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(sr[h][c]));
+                // (the scale is positive: the largest raw score is the largest scaled one)
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+                const float m_new = fmaxf(m_ref, mx);
+                const bool grow = m_new > m_ref + kSlack;      // (also: the row's first visible token)
+                if (__any_sync(0xffffffffu, grow)) {
+#ifdef SEER_DECODE_TRACE
+                    tc_tr[4] += 1;
+#endif
+                    float alpha = 1.f;
+                    if (grow) {
+                        alpha = m_ref == -INFINITY ? 0.f : fast_exp2(m_ref - m_new);
+                        m_ref = m_new;
+                        l_run *= alpha;
+                    }
+                    if (piece_ct > 0) {
+                        // O holds the earlier tiles' products: all of them are in once the last one is
+                        const int c = ct - 1;
+                        if (!mbar_wait(&sm.v.bar_o[c & 1], (c >> 1) & 1, p.status)) return;
+                        __syncwarp();
+                        tc_fence_after_sync();
+#pragma unroll 1
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            uint32_t orow[32];
+                            tmem_ld32(t_o + 32 * q4, orow);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c2 = 0; c2 < 32; ++c2) orow[c2] = __float_as_uint(__uint_as_float(orow[c2]) * alpha);
+                            tmem_st32(t_o + 32 * q4, orow);
+                        }
+                    }
+                }
+                // a row that has seen nothing so far keeps max = -inf; exponents are then taken against 0
+                const float mb = m_ref == -INFINITY ? 0.f : m_ref;
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t pk[32];
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[h][c]), p.scale_log2, -mb));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[h][c + 1]), p.scale_log2, -mb));
+                        sum4[(c >> 1) & 3] += p0 + p1;
+                        pk[(32 * h + c) >> 1] = pack_bf16x2(p0, p1);
+                    }
+                const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                l_run += sum;
+                tmem_st32(tbase + 64 * b, pk);                 // P over the first half of S's columns
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.v.bar_p[b]);
+                TC_T(t_d);
+                TC_ACC(2, t_c, t_d);
+                ++ct;
+                ++piece_ct;
+            }
+            // the next tile's metadata tells whether the piece goes on
+            const int nst = (it + 1) % kS;
+            TC_T(t_e);
+            if (!mbar_wait(&sm.full[nst], ((it + 1) / kS) & 1, p.status)) return;
+            const StageMeta nx = sm.meta[nst];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[nst]);        // metadata taken
+            TC_T(t_f);
+            TC_ACC(3, t_e, t_f);
+            if (nx.flags & 1) {
+                // ---------------- the current piece ends here: every row thread stores its row -----------------
+                const int u = mt.unit;
+                const bool partial = piece_tiles < mt.unit_tiles;
+                if (piece_ct > 0) {
+                    const int c = ct - 1;
+                    if (!mbar_wait(&sm.v.bar_o[c & 1], (c >> 1) & 1, p.status)) return;
+                    __syncwarp();
+                    tc_fence_after_sync();
+                }
+                const size_t slot = (size_t)piece_iv + u;
+                float* po = p.part_o + slot * (8 * NT * kHeadDim) + row * kHeadDim;
+                float* pm = p.part_ml + slot * (kMlStride * NT);
+                const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+                const size_t orow_g = unit_row(p, u, real ? row : 0);
+#pragma unroll 1
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t orow[32];
+                    if (piece_ct > 0) {
+                        tmem_ld32(t_o + 32 * q4, orow);
+                        tmem_wait_ld();
+                    } else {
+#pragma unroll
+                        for (int c2 = 0; c2 < 32; ++c2) orow[c2] = 0u;
+                    }
+                    if (real) {
+                        if (partial) {
+#pragma unroll
+                            for (int c2 = 0; c2 < 32; c2 += 4)
+                                *reinterpret_cast<uint4*>(po + 32 * q4 + c2) = make_uint4(orow[c2], orow[c2 + 1], orow[c2 + 2], orow[c2 + 3]);
+                        } else {
+                            uint4* ob = reinterpret_cast<uint4*>(p.out + orow_g * kHeadDim + 32 * q4);
+#pragma unroll
+                            for (int c2 = 0; c2 < 32; c2 += 8) {
+                                ob[c2 >> 3] = make_uint4(
+                                    pack_bf16x2(__uint_as_float(orow[c2]) * inv, __uint_as_float(orow[c2 + 1]) * inv),
+                                    pack_bf16x2(__uint_as_float(orow[c2 + 2]) * inv, __uint_as_float(orow[c2 + 3]) * inv),
+                                    pack_bf16x2(__uint_as_float(orow[c2 + 4]) * inv, __uint_as_float(orow[c2 + 5]) * inv),
+                                    pack_bf16x2(__uint_as_float(orow[c2 + 6]) * inv, __uint_as_float(orow[c2 + 7]) * inv));
+                            }
+                        }
+                    }
+                }
+                if (partial) {
+                    if (real) { pm[row] = m_ref; pm[8 * NT + row] = l_run; }
+                    if (tid == 0) pm[16 * NT] = __uint_as_float(p.generation);
+                    // every row warp makes its rows of the partial visible; then warp 0 counts the piece on the unit's
+                    // ticket (lane k for the k-th piece held, answer kept in a register)
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.merge_bar[0]);
+                    if (w == 0) {
+                        if (!mbar_wait(&sm.merge_bar[0], pubs & 1, p.status)) return;
+                        const int n_held = sm.pieces_n;
+                        if (n_held < kMaxPieces) {
+                            if (lane == n_held) {
+                                const int iv_first = interval_of(sm.sched, mt.unit_first);
+                                const int iv_last = interval_of(sm.sched, mt.unit_first + mt.unit_tiles - 1);
+                                const int n_slots = iv_last - iv_first + 1;
+                                const unsigned int bit = n_slots <= 32 ? 1u << (piece_iv - iv_first) : 0u;
+                                sm.pieces[n_held] = Piece{u, piece_tiles, iv_first + u, n_slots, mt.unit_tiles};
+                                tk_bit = bit;
+                                tk_before = atomicAdd(&p.tickets[u], ((unsigned long long)piece_tiles << 32) | bit);
+                            }
+                            __syncwarp();
+                            if (lane == 0) sm.pieces_n = n_held + 1;
+                        } else {
+                            raise_status(p.status, DEV_TIMEOUT);   // (cannot happen with the schedule's bound on pieces per CTA)
+                        }
+                    }
+                    ++pubs;
+                } else if (p.lse && real) {
+                    p.lse[orow_g] = l_run > 0.f ? (m_ref + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+                }
+            }
+            mt = nx;
+        }
+#ifdef SEER_DECODE_TRACE
+        if (lane == 0) for (int k = 0; k < 8; ++k) p.trace[(size_t)blockIdx.x * kTraceSlots + 32 + 8 * w + k] = tc_tr[k];
+#endif
+        // the last access to tensor memory is behind this warp: the MMA warp may give the columns back
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.v.tmem_done);
+    }
+    } else if constexpr (NT < kWideTiles) {
     // ---------------- tokens on the MMA's M side, the unit's (up to 16) rows on N ----------------
     uint32_t bq[NT][8][2];              // Q^T B-fragments: NT N-tiles x 8 k-steps over d
     uint32_t bq_pre[8][2];              // NT == 1: the same for the unit expected next (prefetched)
@@ -904,7 +1345,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (tid == 0) SEER_STAMP(10);
     StageMeta mt = sm.meta[0];
     for (int it = 0; mt.nvalid >= 0; ++it) {
-        const int st = it % kStages;
+        const int st = it % kS;
 #ifdef SEER_DECODE_TRACE
         if (tid == 0 && it < kTraceSlots - 16) SEER_STAMP(16 + it);
         if (tid == 0) p.trace[(size_t)blockIdx.x * kTraceSlots + 3] = it + 1;     // tiles consumed so far
@@ -915,9 +1356,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             const int iss = sm.issued;
             __threadfence_block();
 #pragma unroll
-            for (int look = 1; look < kStages; ++look) {
+            for (int look = 1; look < kS; ++look) {
                 if (it + look < iss) {
-                    const int u2 = *reinterpret_cast<volatile int*>(&sm.meta[(it + look) % kStages].unit);
+                    const int u2 = *reinterpret_cast<volatile int*>(&sm.meta[(it + look) % kS].unit);
                     if (u2 >= 0 && u2 != mt.unit && u2 != pre_unit) {
                         load_q(bq_pre, u2, 0);
                         pre_unit = u2;
@@ -1042,8 +1483,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         if (lane == 0) mbar_arrive(&sm.empty[st]);
 
         // the next tile's metadata tells whether the piece goes on
-        const int nst = (it + 1) % kStages;
-        if (!mbar_wait(&sm.full[nst], ((it + 1) / kStages) & 1, p.status)) return;
+        const int nst = (it + 1) % kS;
+        if (!mbar_wait(&sm.full[nst], ((it + 1) / kS) & 1, p.status)) return;
         const StageMeta nx = sm.meta[nst];
         if (nx.flags & 1) {
             // ---------------- the current piece ends here ------------------------------------
@@ -1063,16 +1504,16 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 #pragma unroll
                     for (int a = 0; a < 8; ++a) {
                         const int d0 = 16 * a + rw;
-                        sm.merge_o[w - 1][2 * qd][d0] = o[nt][a][0];
-                        sm.merge_o[w - 1][2 * qd + 1][d0] = o[nt][a][1];
-                        sm.merge_o[w - 1][2 * qd][d0 + 8] = o[nt][a][2];
-                        sm.merge_o[w - 1][2 * qd + 1][d0 + 8] = o[nt][a][3];
+                        sm.v.merge_o[w - 1][2 * qd][d0] = o[nt][a][0];
+                        sm.v.merge_o[w - 1][2 * qd + 1][d0] = o[nt][a][1];
+                        sm.v.merge_o[w - 1][2 * qd][d0 + 8] = o[nt][a][2];
+                        sm.v.merge_o[w - 1][2 * qd + 1][d0 + 8] = o[nt][a][3];
                     }
                     if (rw == 0) {
-                        sm.merge_ml[w - 1][0][2 * qd] = m_run[nt][0];
-                        sm.merge_ml[w - 1][0][2 * qd + 1] = m_run[nt][1];
-                        sm.merge_ml[w - 1][1][2 * qd] = l0;
-                        sm.merge_ml[w - 1][1][2 * qd + 1] = l1;
+                        sm.v.merge_ml[w - 1][0][2 * qd] = m_run[nt][0];
+                        sm.v.merge_ml[w - 1][0][2 * qd + 1] = m_run[nt][1];
+                        sm.v.merge_ml[w - 1][1][2 * qd] = l0;
+                        sm.v.merge_ml[w - 1][1][2 * qd + 1] = l1;
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.merge_bar[0]);
@@ -1082,8 +1523,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     m_all[nt][0] = m_run[nt][0]; m_all[nt][1] = m_run[nt][1];
 #pragma unroll
                     for (int ww = 0; ww < kConsumerWarps - 1; ++ww) {
-                        mw[ww][0] = sm.merge_ml[ww][0][2 * qd]; mw[ww][1] = sm.merge_ml[ww][0][2 * qd + 1];
-                        lw[ww][0] = sm.merge_ml[ww][1][2 * qd]; lw[ww][1] = sm.merge_ml[ww][1][2 * qd + 1];
+                        mw[ww][0] = sm.v.merge_ml[ww][0][2 * qd]; mw[ww][1] = sm.v.merge_ml[ww][0][2 * qd + 1];
+                        lw[ww][0] = sm.v.merge_ml[ww][1][2 * qd]; lw[ww][1] = sm.v.merge_ml[ww][1][2 * qd + 1];
                         m_all[nt][0] = fmaxf(m_all[nt][0], mw[ww][0]); m_all[nt][1] = fmaxf(m_all[nt][1], mw[ww][1]);
                     }
                     const float f0 = (m_run[nt][0] == -INFINITY) ? 0.f : fast_exp2(m_run[nt][0] - m_all[nt][0]);
@@ -1101,10 +1542,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 #pragma unroll
                         for (int a = 0; a < 8; ++a) {
                             const int d0 = 16 * a + rw;
-                            o[nt][a][0] += g0 * sm.merge_o[ww][2 * qd][d0];
-                            o[nt][a][1] += g1 * sm.merge_o[ww][2 * qd + 1][d0];
-                            o[nt][a][2] += g0 * sm.merge_o[ww][2 * qd][d0 + 8];
-                            o[nt][a][3] += g1 * sm.merge_o[ww][2 * qd + 1][d0 + 8];
+                            o[nt][a][0] += g0 * sm.v.merge_o[ww][2 * qd][d0];
+                            o[nt][a][1] += g1 * sm.v.merge_o[ww][2 * qd + 1][d0];
+                            o[nt][a][2] += g0 * sm.v.merge_o[ww][2 * qd][d0 + 8];
+                            o[nt][a][3] += g1 * sm.v.merge_o[ww][2 * qd + 1][d0 + 8];
                         }
                     }
                     __syncwarp();
@@ -1234,7 +1675,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (tid == 0) SEER_STAMP(10);
     StageMeta mt = sm.meta[0];
     for (int it = 0; mt.nvalid >= 0; ++it) {
-        const int st = it % kStages;
+        const int st = it % kS;
         if (mt.flags & 1) {
             load_q_wide(mt.unit);
 #pragma unroll
@@ -1344,8 +1785,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         if (lane == 0) mbar_arrive(&sm.empty[st]);
 
         // the next tile's metadata tells whether the piece goes on
-        const int nst = (it + 1) % kStages;
-        if (!mbar_wait(&sm.full[nst], ((it + 1) / kStages) & 1, p.status)) return;
+        const int nst = (it + 1) % kS;
+        if (!mbar_wait(&sm.full[nst], ((it + 1) / kS) & 1, p.status)) return;
         const StageMeta nx = sm.meta[nst];
         if (nx.flags & 1) {
             // ---------------- the current piece ends here: every warp stores its own rows -----------------
@@ -1464,11 +1905,13 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     // from global memory; more are brought in by bulk copies, n_land at a time, into the first two
     // stage buffers (only the unit's real rows: rows x 512 B + 128 B * NT per partial, one per lane).
     constexpr int kSeg = kListInts / kConsumerWarps;             // slot numbers a warp can list per window
-    int* lists = reinterpret_cast<int*>(sm.stage[2]);            // [4][kSeg] slot numbers
+    int* lists = reinterpret_cast<int*>(sm.stage[SmemK::kBufs - 1]);   // [4][kSeg] slot numbers
     int* counts = lists + kListInts;                             // [4]
     constexpr int kMl = kMlStride * NT;                          // floats per (max, sum, stamp) record
     const int o_stride = p.rows * kHeadDim;                      // floats per staged partial
-    const int n_land = min(32, kLandBytes / (o_stride * 4 + kMl * 4));
+    // (the landing area is every stage buffer but the last: two of them, six in the tensor-memory variant)
+    constexpr int kLand = (SmemK::kBufs - 1) * kStageBytes;
+    const int n_land = min(32, kLand / (o_stride * 4 + kMl * 4));
     float* land_o = reinterpret_cast<float*>(sm.stage[0]);       // [n_land][rows][128]
     float* land_ml = land_o + n_land * o_stride;                 // [n_land][32 * NT]
     int sync_phase = 0, land_phase = 0;
@@ -1504,8 +1947,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             for (int seg = 0; seg < (listed ? kConsumerWarps : 1); ++seg) {
                 const int n = all_valid ? win : by_mask ? __popc(mask) : counts[seg];
                 const int* seg_list = lists + seg * kSeg;
-                if (n <= 2 * kDirect) {
-                    // up to two rounds of direct loads beat staging (one round trip each, no barrier)
+                if ((NT < kWideTiles || n_land < 2) && n <= 2 * kDirect) {
+                    // up to two rounds of direct loads beat staging (one round trip each, no barrier); with the
+                    // rows on M a thread's share of a partial is eight such round trips, and staging wins as
+                    // long as more than one partial fits the landing area
                     unsigned int rem = mask;                 // bits of the valid slots not yet taken
 #pragma unroll 1
                     for (int k0 = 0; k0 < n; k0 += kDirect) {
@@ -1561,74 +2006,82 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if (tid == 0) SEER_STAMP(7);
 }
 
-size_t decode_smem_bytes() { return sizeof(Smem) + 1024; }
+template <bool TC>
+constexpr size_t decode_smem_bytes() { return sizeof(SmemT<TC>) + 1024; }
 
-template <bool SPARSE, bool PAGED, int NT, bool SMALL>
+template <bool SPARSE, bool PAGED, int NT, bool SMALL, bool TC = false>
 cudaError_t configure() {
-    return cudaFuncSetAttribute(decode_kernel<SPARSE, PAGED, NT, SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)decode_smem_bytes());
+    return cudaFuncSetAttribute(decode_kernel<SPARSE, PAGED, NT, SMALL, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)decode_smem_bytes<TC>());
 }
 
-template <bool SPARSE, bool PAGED, int NT, bool SMALL>
+template <bool SPARSE, bool PAGED, int NT, bool SMALL, bool TC = false>
 int occupancy() {
     static int cached[kMaxDevices] = {};             // 0: not asked yet on that device
     const int slot = current_device_slot();
     if (cached[slot] <= 0) {
-        if (configure<SPARSE, PAGED, NT, SMALL>() != cudaSuccess) return 0;
+        if (configure<SPARSE, PAGED, NT, SMALL, TC>() != cudaSuccess) return 0;
         int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<SPARSE, PAGED, NT, SMALL>, kThreads,
-                                                          decode_smem_bytes()) != cudaSuccess)
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<SPARSE, PAGED, NT, SMALL, TC>,
+                                                          TC ? kTcThreads : kThreads, decode_smem_bytes<TC>()) != cudaSuccess)
             return 0;
         cached[slot] = n;
     }
     return cached[slot];
 }
 
-template <bool SPARSE, bool PAGED, int NT, bool SMALL>
+template <bool SPARSE, bool PAGED, int NT, bool SMALL, bool TC = false>
 cudaError_t launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& p, int grid,
                    cudaStream_t stream) {
-    if (occupancy<SPARSE, PAGED, NT, SMALL>() <= 0) return cudaErrorInvalidConfiguration;
-    return launch_pdl(decode_kernel<SPARSE, PAGED, NT, SMALL>, dim3(grid), dim3(kThreads), decode_smem_bytes(), stream,
-                      mk, mv, p);
+    if (occupancy<SPARSE, PAGED, NT, SMALL, TC>() <= 0) return cudaErrorInvalidConfiguration;
+    return launch_pdl(decode_kernel<SPARSE, PAGED, NT, SMALL, TC>, dim3(grid), dim3(TC ? kTcThreads : kThreads),
+                      decode_smem_bytes<TC>(), stream, mk, mv, p);
 }
 
 // (blocks of 16 or 32 tokens use the same resources: the occupancy of the 64-token variant stands for both)
-template <int NT>
+template <int NT, bool TC = false>
 int occupancy_of(bool sparse, bool paged) {
-    if (sparse) return paged ? occupancy<true, true, NT, false>() : occupancy<true, false, NT, false>();
-    return paged ? occupancy<false, true, NT, false>() : occupancy<false, false, NT, false>();
+    if (sparse) return paged ? occupancy<true, true, NT, false, TC>() : occupancy<true, false, NT, false, TC>();
+    return paged ? occupancy<false, true, NT, false, TC>() : occupancy<false, false, NT, false, TC>();
 }
 
-template <int NT>
+template <int NT, bool TC = false>
 cudaError_t launch_of(bool sparse, bool paged, const CUtensorMap& map_k, const CUtensorMap& map_v,
                       const DecodeParams& p, int grid, cudaStream_t stream) {
-    if constexpr (NT < kWideTiles) {            // (the rows-on-M variant takes blocks of 64 or 128 tokens only)
+    if constexpr (NT < kWideTiles) {            // (the rows-on-M variants take blocks of 64 or 128 tokens only)
         if (sparse && p.blocks_per_tile > 1)
             return paged ? launch<true, true, NT, true>(map_k, map_v, p, grid, stream)
                          : launch<true, false, NT, true>(map_k, map_v, p, grid, stream);
     }
-    if (sparse) return paged ? launch<true, true, NT, false>(map_k, map_v, p, grid, stream)
-                             : launch<true, false, NT, false>(map_k, map_v, p, grid, stream);
-    return paged ? launch<false, true, NT, false>(map_k, map_v, p, grid, stream)
-                 : launch<false, false, NT, false>(map_k, map_v, p, grid, stream);
+    if (sparse) return paged ? launch<true, true, NT, false, TC>(map_k, map_v, p, grid, stream)
+                             : launch<true, false, NT, false, TC>(map_k, map_v, p, grid, stream);
+    return paged ? launch<false, true, NT, false, TC>(map_k, map_v, p, grid, stream)
+                 : launch<false, false, NT, false, TC>(map_k, map_v, p, grid, stream);
 }
 
 }  // namespace
 
+// n_tiles: 1 or 2 (the unit's rows on the MMA's N side), 8 (rows on M, mma.sync), 16 (rows on M, tcgen05:
+// the same 64-row partial slots as 8)
 int decode_ctas_per_sm(bool sparse, bool paged, int n_tiles) {
-    return n_tiles == 1 ? occupancy_of<1>(sparse, paged) : n_tiles == 2 ? occupancy_of<2>(sparse, paged)
-                                                                         : occupancy_of<kWideTiles>(sparse, paged);
+    return n_tiles == 1   ? occupancy_of<1>(sparse, paged)
+           : n_tiles == 2 ? occupancy_of<2>(sparse, paged)
+           : n_tiles == kTcTilesCode ? occupancy_of<kWideTiles, true>(sparse, paged)
+                                     : occupancy_of<kWideTiles>(sparse, paged);
 }
 
 int decode_max_intervals(int grid, int max_rounds) { return grid * (max_rounds + 1) + 1; }
 
 cudaError_t launch_decode(bool sparse, bool paged, int n_tiles, const CUtensorMap& map_k, const CUtensorMap& map_v,
                           const DecodeParams& p, int grid, cudaStream_t stream) {
-    if ((n_tiles != 1 && n_tiles != 2 && n_tiles != kWideTiles) || p.rows > 8 * n_tiles) return cudaErrorInvalidValue;
-    if (n_tiles == kWideTiles && p.blocks_per_tile > 1) return cudaErrorInvalidValue;
-    return n_tiles == 1 ? launch_of<1>(sparse, paged, map_k, map_v, p, grid, stream)
+    const int slot_tiles = n_tiles == kTcTilesCode ? kWideTiles : n_tiles;
+    if ((n_tiles != 1 && n_tiles != 2 && n_tiles != kWideTiles && n_tiles != kTcTilesCode) || p.rows > 8 * slot_tiles)
+        return cudaErrorInvalidValue;
+    if (slot_tiles == kWideTiles && p.blocks_per_tile > 1) return cudaErrorInvalidValue;
+    return n_tiles == 1   ? launch_of<1>(sparse, paged, map_k, map_v, p, grid, stream)
            : n_tiles == 2 ? launch_of<2>(sparse, paged, map_k, map_v, p, grid, stream)
-                          : launch_of<kWideTiles>(sparse, paged, map_k, map_v, p, grid, stream);
+           : n_tiles == kTcTilesCode ? launch_of<kWideTiles, true>(sparse, paged, map_k, map_v, p, grid, stream)
+                                     : launch_of<kWideTiles>(sparse, paged, map_k, map_v, p, grid, stream);
 }
 
 }  // namespace seer

@@ -12,9 +12,21 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-@pytest.fixture(scope="module")
-def ctx():
-    c = binding.Context(0)
+@pytest.fixture(scope="module", params=["mma.sync", "tcgen05"])
+def ctx(request):
+    """Every test of this file runs twice: units of 17 to 64 rows take the rows-on-M kernel, which exists as an
+    mma.sync variant (the default) and as a tcgen05 variant (S, P and O in tensor memory) that a context picks
+    up from SEER_DECODE_WIDE_VARIANT=16 when it is created.  Up to 16 rows both runs take the same kernels."""
+    import os
+    old = os.environ.get("SEER_DECODE_WIDE_VARIANT")
+    os.environ["SEER_DECODE_WIDE_VARIANT"] = "16" if request.param == "tcgen05" else "8"
+    try:
+        c = binding.Context(0)
+    finally:
+        if old is None:
+            del os.environ["SEER_DECODE_WIDE_VARIANT"]
+        else:
+            os.environ["SEER_DECODE_WIDE_VARIANT"] = old
     yield c
     c.close()
 

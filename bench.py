@@ -297,7 +297,7 @@ def run_ours(args):
     # the bulk build of the compressed-K cache after prefill (all blocks but the last), one layer per launch
     bulk_ms, _ = repeated(lambda s: ctx.seer_kcomp_append(shape, layers[s % n_layers]["gate"], lens_t, layers[s % n_layers]["k"],
                                                           first_block=0, num_blocks=n_blocks - 1, stream=stream),
-                          max(4, min(K, 2 * n_layers)))
+                          max(4, min(K, 8 * n_layers)))
     clocks = sampler.stop()
 
     # ---- end to end through the same API with host buffers ----------------------------------

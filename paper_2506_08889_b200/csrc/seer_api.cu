@@ -48,6 +48,7 @@ struct seer_ctx {
     unsigned int generation;    // stamps the partials of a decode launch
     int pool_div;               // decode scheduling: share of tiles handed out dynamically
     int min_tiles;              // decode scheduling: fewest tiles of a CTA's range
+    int sel_from_lens;          // set by seer_decode_step around its attention call (see DecodeParams)
     int wide_variant;           // kernel variant code for more than 16 rows per unit: 16 (tcgen05) or 8 (mma.sync)
     char err[512];
 };
@@ -253,6 +254,7 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.page_table = kv->page_table;
     p.page_table_stride = kv->page_table_stride;
     p.max_sel = max_sel;
+    p.sel_from_lens = sparse && q_len == 1 ? ctx->sel_from_lens : 0;
     p.page_size = kv->page_size;
     p.num_pages = kv->num_pages;
     p.batch = shape->batch;
@@ -645,7 +647,14 @@ seer_status seer_decode_step(seer_ctx* ctx, const seer_shape* shape, const seer_
     seer_status st = seer_gate_select(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, token_budget, block_idx, block_cnt,
                                       max_sel, nullptr, stream);
     if (st != SEER_OK) return st;
+    // With the token budget every list has min(budget in blocks, blocks of the sequence) entries (as long as the
+    // compressed-key cache covers the longest sequence): the attention kernel then counts its tiles from the
+    // lengths, before the gate has finished, and waits for the gate only when it reads the lists.
+    const int k_blocks = token_budget / shape->block_size > 1 ? token_budget / shape->block_size : 1;
+    const bool covered = (long long)gate->max_blocks * shape->block_size >= (long long)kv->max_seq_len;
+    ctx->sel_from_lens = covered ? (k_blocks < max_sel ? k_blocks : max_sel) : 0;
     st = seer_sparse_decode(ctx, shape, kv, q, block_idx, block_cnt, max_sel, out, lse, stream);
+    ctx->sel_from_lens = 0;
     if (st != SEER_OK || !k_nope) return st;
     return kcomp_append_common(ctx, shape, gate, kv->seq_lens, k_nope, k_nope_stride_batch, k_nope_stride_head,
                                k_nope_stride_token, k_nope_rows_block_local, -1, 1, 1, stream);

@@ -170,7 +170,12 @@ template <bool SPARSE, bool SMALL = false>
 __device__ __forceinline__ int tiles_of(const DecodeParams& p, int u) {
     const int L = p.seq_lens[unit_seq(p, u)];
     if (SPARSE) {
-        int c = p.block_cnt ? p.block_cnt[u] : p.max_sel;     // not behind the test on L: both loads in flight
+        int c;
+        if (p.sel_from_lens > 0) {
+            c = min(p.sel_from_lens, (L + p.block_size - 1) >> p.bs_shift);     // (the lists are not final yet)
+        } else {
+            c = p.block_cnt ? p.block_cnt[u] : p.max_sel;     // not behind the test on L: both loads in flight
+        }
         c = max(0, min(c, p.max_sel));
         return L <= 0 ? 0 : (SMALL ? (c + p.blocks_per_tile - 1) >> p.bpt_shift : c << p.tpb_shift);
     } else {
@@ -472,7 +477,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     }
     __syncthreads();                                 // barriers initialised
     if constexpr (TC) tc_fence_after_sync();
-    pdl_wait();
+    // The producer warp puts its wait off when the lists' lengths follow from the sequence lengths: it then
+    // makes the schedule and finds its first unit while the kernel that writes the lists is still running, and
+    // waits just before it reads a list.  (Everything it touches before that was final before that kernel began.)
+    bool producer_waited = !(SPARSE && p.sel_from_lens > 0 && warp == kConsumerWarps);
+    if (producer_waited) pdl_wait();
     if (tid == 0) SEER_STAMP(9);
 
     if (warp == kConsumerWarps) {
@@ -722,6 +731,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     ahead = 2;
                 }
             };
+            if (!producer_waited) {                  // the lists are read from here on
+                pdl_wait();
+                producer_waited = true;
+            }
             const bool fresh = !contiguous;          // this interval starts a new piece
             int ce = iv_begin - cpu;                  // offset of the next tile inside unit cu
             const int n_tiles = iv_end - iv_begin;
@@ -758,7 +771,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     if (SMALL) {
                         // a tile gathers the next bpt listed blocks of the unit
                         const int n_i = (L + p.block_size - 1) >> p.bs_shift;
-                        int cnt_u = p.block_cnt ? p.block_cnt[my_u] : p.max_sel;
+                        int cnt_u = p.sel_from_lens > 0 ? min(p.sel_from_lens, n_i) : p.block_cnt ? p.block_cnt[my_u] : p.max_sel;
                         cnt_u = max(0, min(cnt_u, p.max_sel));
 #pragma unroll
                         for (int sb = 0; sb < 4; ++sb) {
@@ -895,6 +908,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 }
             }
         }
+        if (!producer_waited) pdl_wait();            // (a CTA without tiles: the counters below belong to this launch only after the wait)
         if (lane == 0) {
             // end-of-stream marker for the consumers
             const int st = it % kS;

@@ -68,6 +68,9 @@ struct DecodeParams {
     int min_tiles;                  // a CTA's range has at least this many tiles (fewer CTAs take part when work is short)
     int max_rounds;                 // most dynamic chunks per range (<= kMaxRounds; 0: none) -- bounds the partial slots
     float scale_log2;               // sm_scale * log2(e)
+    int sel_from_lens;              // > 0: every unit's list holds min(this, blocks of its sequence) entries, so the
+                                    // counts follow from the lengths and the schedule can be made before the kernel
+                                    // that writes the lists has finished (0: read block_cnt)
     unsigned int* status;
     unsigned long long* tickets;    // [num_units]: tiles done << 32 | valid-slot bits; zero between launches
     int* sched;                     // [2]: theft cursor, exit counter; zero between launches

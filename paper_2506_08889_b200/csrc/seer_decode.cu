@@ -613,11 +613,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         int st[kScan];
         // (a range's last chunk is left to its owner: by the time a thief's loads came back the owner
         // would have been there)
-#ifdef SEER_EXP_MINLEFT
-        const int min_left = min(SEER_EXP_MINLEFT, R);
-#else
         const int min_left = min(2, R);
-#endif
         auto scan_load = [&](int c0) {
 #pragma unroll
             for (int k = 0; k < kScan; ++k) {

@@ -94,6 +94,34 @@ def test_kcomp_bulk_build_large_enough_for_the_streaming_kernel(ctx, dg, token_m
         assert np.all(got[i, :, :first] == 0)             # nor blocks before the first one asked for
 
 
+def test_kcomp_bulk_build_more_sequences_than_the_length_cache_holds(ctx):
+    """The streaming bulk build keeps the first 2048 sequence lengths in shared memory and reads the others from
+    global memory: 2100 sequences of one KV head, 16 blocks each (2100 work items), lengths that differ on both
+    sides of that boundary."""
+    B, Hkv, d, b, dg = 2100, 1, 128, 64, 128
+    nb = 16
+    S = nb * b
+    lens = np.full(B, S, np.int32)
+    lens[5] = 3 * b + 1
+    lens[2047] = 7 * b
+    lens[2048] = 2 * b + 63
+    lens[2099] = 11 * b
+    kn = synth.normal_bf16((B, Hkv, S, d), 8, "kn", DEV)
+    wk = synth.normal_bf16((Hkv, dg, 3 * d), 8, "wk", DEV, std=0.02)
+    kc = torch.zeros((B, Hkv, nb, dg), dtype=torch.bfloat16, device=DEV)
+    shape = binding.make_shape(B, Hkv * 4, Hkv, d, b, 0.1)
+    gate = binding.make_gate(dg, THETA, None, wk, kc, nb)
+    ctx.seer_kcomp_append(shape, gate, torch.as_tensor(lens, device=DEV), kn, first_block=0, num_blocks=nb)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.SEER_OK
+    got = bits(kc)
+    for i in (0, 5, 2046, 2047, 2048, 2049, 2099):
+        _, want = oracle.kcomp(bits(kn[i:i + 1]), bits(wk), b, 0, nb, nb, THETA)
+        n = int(lens[i]) // b
+        _bf16_ulp_close(got[i, :, :n], want[0, :, :n])
+        assert np.all(got[i, :, n:] == 0)
+
+
 def test_kcomp_append_when_a_block_fills(ctx):
     B, Hkv, d, dg, b, nb = 3, 2, 128, 128, 64, 8
     lens = np.array([5 * b, 5 * b + 1, 3 * b], np.int32)  # sequences 0 and 2 just filled a block

@@ -210,7 +210,7 @@ __device__ __forceinline__ void build_schedule(Schedule& s, Schedule& shared, in
         const int tail = pool_div == 4 ? q >> 2 : q / pool_div;
         // (with one piece per level there are at most max_rounds pieces, so the loop ends at the latest
         // when cap exceeds the tail)
-        for (int cap_shift = 3 + max(0, 23 - __clz(q)); cap_shift < 31; ++cap_shift) {      // cap = 8, or about q/32 .. q/64
+                for (int cap_shift = 3 + max(0, 23 - __clz(q)); cap_shift < 31; ++cap_shift) {      // cap = 8, or about q/32 .. q/64
             // level k = [b - prev, b - nxt): halves, down to kMinChunk tiles; the last level takes the rest
             int prev = lane < max_rounds ? tail >> lane : 0;
             if (lane > 0 && prev < kMinChunk) prev = 0;

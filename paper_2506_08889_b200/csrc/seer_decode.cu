@@ -61,7 +61,7 @@ constexpr int kTcStages = 8;                               // V buffers (16 KiB 
 constexpr int kTcKStages = 4;                              // K buffers (16 KiB each): a K tile is free once its scores are computed
 constexpr int kTcThreads = kThreads + 32;
 constexpr int kTcRows = 128;                               // M of the MMAs (rows past the unit's are zero)
-constexpr int kTcCols = 256;                               // tensor-memory columns: S/P twice 64, O 128
+constexpr int kTcCols = 512;                               // tensor-memory columns: S/P twice 64, O 128, Q 64 (320, as a power of two)
 constexpr int kAheadMaxChunk = 8;                          // own chunks up to this size are claimed ahead
 constexpr int kAheadTiles = 3;                             // tiles left to issue when the next interval's claim is made
 constexpr int kSmemUnits = 128;                            // units whose tile-count prefix sums fit in shared memory
@@ -111,6 +111,7 @@ struct VariantPart<true> {
     uint64_t bar_s[2];               // S of an even / odd tile is complete (the MMA warp's commit)
     uint64_t bar_p[2];               // P of an even / odd tile is written (one arrival per row warp with real rows)
     uint64_t bar_o[2];               // O includes an even / odd tile's product (commit)
+    uint64_t bar_q;                  // the queries of a piece's unit are in tensor memory (one arrival per row warp with real rows)
     uint64_t tmem_done;              // the row warps have made their last tensor-memory access
     uint64_t empty_k[kTcKStages];    // a K buffer's scores have been computed (commit)
     uint32_t tmem_base;
@@ -120,9 +121,8 @@ template <bool TC>
 struct __align__(1024) SmemT {
     static constexpr int kS = TC ? kTcStages : kStages;
     // The K/V ring.  The tensor-memory variant cuts the same memory differently: kTcStages V buffers, then
-    // kTcKStages K buffers (16 KiB each), then the unit's queries, [64-channel half][128 rows][128 B] with
-    // 16-byte pieces swizzled by row.
-    static constexpr int kBufs = TC ? (kTcStages + kTcKStages) / 2 + 1 : kStages;
+    // kTcKStages K buffers (16 KiB each).
+    static constexpr int kBufs = TC ? (kTcStages + kTcKStages) / 2 : kStages;
     unsigned char stage[kBufs][kStageBytes];
     uint64_t full[kS];
     uint64_t empty[kS];
@@ -139,7 +139,7 @@ struct __align__(1024) SmemT {
     int pieces_n;
     VariantPart<TC> v;
 };
-static_assert(2 * kTcRows * 128 == kStageBytes, "the query tile takes one stage buffer");
+static_assert((kTcStages + kTcKStages) % 2 == 0, "the K and V buffers fill whole stage buffers");
 using Smem = SmemT<false>;
 static_assert(sizeof(SmemT<true>) + 1024 <= 227 * 1024, "the tensor-memory variant's shared memory");
 
@@ -445,6 +445,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 mbar_init(&sm.v.bar_p[b], tc_row_warps);
                 mbar_init(&sm.v.bar_o[b], 1);
             }
+            mbar_init(&sm.v.bar_q, tc_row_warps);
             mbar_init(&sm.v.tmem_done, tc_row_warps);
             for (int b = 0; b < kTcKStages; ++b) mbar_init(&sm.v.empty_k[b], 1);
         }
@@ -927,20 +928,19 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     if constexpr (TC) {
     if (warp == kConsumerWarps + 1) {
         // =========================== MMA warp (tensor-memory variant) ====================
-        // Lane 0 issues, per tile, S = Q . K^T (8 MMAs of K = 16 over the 128 channels; Q and the K tile
-        // K-major in shared memory) and, once the row warps have written the tile's probabilities,
-        // O (+)= P . V (4 MMAs over the 64 tokens; P from tensor memory, the V tile MN-major).  The product
-        // of a tile is issued after the scores of the next one, so the tensor cores work on S(t + 1)
-        // while the row warps are busy with S(t).  The whole warp brings a unit's queries into shared
-        // memory (zero rows past the unit's) and clears the rows of a ragged last tile of V.
+        // Lane 0 issues, per tile, S = Q . K^T (8 MMAs of K = 16 over the 128 channels; Q from tensor memory,
+        // where the row warps put the unit's queries when a piece begins, the K tile K-major in shared
+        // memory) and, once the row warps have written the tile's probabilities, O (+)= P . V (4 MMAs over
+        // the 64 tokens; P from tensor memory, the V tile MN-major).  The tensor cores work on S(t + 1)
+        // while the row warps are busy with S(t).  The whole warp clears the rows of a ragged last tile of V.
         const uint32_t tbase = sm.v.tmem_base;
         const uint32_t t_o = tbase + 128;
         constexpr uint32_t idesc_qk = tc_idesc_bf16(kTcRows, kTileTokens, false);
         constexpr uint32_t idesc_pv = tc_idesc_bf16(kTcRows, kHeadDim, true);
-        const uint32_t q_addr = smem_u32(sm.stage[SmemK::kBufs - 1]);
+        const uint32_t t_q = tbase + 256;
+        int piece_no = 0;                          // pieces begun so far (phase of bar_q)
         bool dead = false;                         // a wait ran out: stop issuing, free the tensor memory, leave
         int ct = 0, piece_ct = 0;                  // computed tiles so far (of the CTA, of the piece)
-        int q_unit = -1;
 #ifdef SEER_DECODE_TRACE
         unsigned long long mm_tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         const long long mm_t0 = clock64();
@@ -955,12 +955,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         int it = 0;                                // next tile of the stream
         bool ended = false;
         uint32_t idle = 0;
-        // rows of the query tile past the unit's stay zero for the whole launch
-        for (int x = p.rows * 16 + lane; x < kTcRows * 16; x += 32) {
-            const int r = x >> 4, c16 = x & 15;
-            *reinterpret_cast<uint4*>(sm.stage[SmemK::kBufs - 1] + (c16 >> 3) * (kTcRows * 128) + r * 128 + ((c16 & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-        }
-        __syncwarp();
         while (!dead && (!ended || pend_n > 0)) {
             bool did = false;
             if (pend_n > 0) {
@@ -989,28 +983,17 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     mbar_try_wait(&sm.full[st], (it / kS) & 1);
                     __syncwarp();
                     const StageMeta mt = sm.meta[st];
+                    // the first tile of a piece has to find the piece's queries in tensor memory
+                    const bool q_ready = mt.nvalid < 0 || !(mt.flags & 1) ||
+                        __shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.v.bar_q, piece_no & 1) : 0, 0);
+                    if (q_ready) {
                     did = true;
                     if (mt.nvalid < 0) {
                         ended = true;
                     } else {
-                        if (mt.flags & 1) piece_ct = 0;
+                        if (mt.flags & 1) { piece_ct = 0; ++piece_no; }
                         const int nv = mt.nvalid;
                         if (nv > 0) {
-                            if (q_unit != mt.unit) {
-                                // every earlier S has been computed before the queries change
-                                if (ct > 0 && !mbar_wait(&sm.v.bar_s[(ct - 1) & 1], ((ct - 1) >> 1) & 1, p.status)) { dead = true; break; }
-                                // the unit's real rows, by asynchronous 16-byte copies all issued before any is waited for
-                                // (the rows past them were cleared once and stay zero)
-                                for (int x = lane; x < p.rows * 16; x += 32) {
-                                    const int r = x >> 4, c16 = x & 15;
-                                    cp_async16(sm.stage[SmemK::kBufs - 1] + (c16 >> 3) * (kTcRows * 128) + r * 128 + (((c16 & 7) ^ (r & 7)) << 4),
-                                               reinterpret_cast<const uint4*>(p.q + unit_row(p, mt.unit, r) * kHeadDim) + c16);
-                                }
-                                cp_async_wait_all();
-                                q_unit = mt.unit;
-                                fence_proxy_async_smem();
-                                __syncwarp();
-                            }
                             if (nv < kTileTokens) {
                                 // ragged tail: rows past the sequence end may hold anything; cleared in V so that a
                                 // zero probability times garbage cannot produce NaN
@@ -1029,7 +1012,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                                 const uint32_t k_addr = smem_u32(sm.stage[0]) + (kTcStages + it % kTcKStages) * kTileBytes;
 #pragma unroll
                                 for (int ks = 0; ks < kHeadDim / 16; ++ks)
-                                    tc_mma_ss(tbase + 64 * b, tc_smem_desc(q_addr + (ks >> 2) * (kTcRows * 128) + (ks & 3) * 32, 16, 1024),
+                                    tc_mma_ts(tbase + 64 * b, t_q + 8 * ks,
                                               tc_smem_desc(k_addr + (ks >> 2) * kHalfTileBytes + (ks & 3) * 32, 16, 1024), idesc_qk, ks > 0);
                                 tc_commit(&sm.v.bar_s[b]);
                                 tc_commit(&sm.v.empty_k[it % kTcKStages]);   // the K buffer has been read
@@ -1047,6 +1030,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                             }
                         }
                         ++it;
+                    }
                     }
                 }
             }
@@ -1108,6 +1092,31 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         const uint32_t t_o = tbase + 128;
         float m_ref = -INFINITY, l_run = 0.f;
         int ct = 0, piece_ct = 0;       // computed tiles so far (of the CTA, of the piece)
+        // A piece's queries go to tensor memory, this thread's row as 64 columns of bf16 pairs (zeros for a padding
+        // row): requested from global memory early, stored once every score of the piece before has been computed
+        // (this thread has then read the last of them); the MMA warp issues none of the new piece's before all
+        // row warps have arrived.
+        auto load_q = [&](int unit, uint4 (&qv)[16]) {
+            const uint4* qsrc = reinterpret_cast<const uint4*>(p.q + unit_row(p, unit, real ? row : 0) * kHeadDim);
+#pragma unroll
+            for (int x = 0; x < 16; ++x) qv[x] = real ? __ldg(qsrc + x) : make_uint4(0u, 0u, 0u, 0u);
+        };
+        auto store_q = [&](const uint4 (&qv)[16]) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t qr[32];
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    qr[4 * x] = qv[8 * h + x].x; qr[4 * x + 1] = qv[8 * h + x].y;
+                    qr[4 * x + 2] = qv[8 * h + x].z; qr[4 * x + 3] = qv[8 * h + x].w;
+                }
+                tmem_st32(tbase + 256 + 32 * h, qr);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.v.bar_q);
+        };
         if (!mbar_wait(&sm.full[0], 0, p.status)) return;
         if (tid == 0) SEER_STAMP(10);
         StageMeta mt = sm.meta[0];
@@ -1120,6 +1129,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 piece_tiles = 0;
                 piece_iv = mt.interval;
                 piece_ct = 0;
+                // (the first piece's queries; those of a later piece are put in place when the piece before it ends)
+                if (it == 0) {
+                    uint4 qv[16];
+                    load_q(mt.unit, qv);
+                    store_q(qv);
+                }
             }
             ++piece_tiles;
             const int nv = mt.nvalid;                          // cached tokens from the tile's first row on (capped at 64 + 7)
@@ -1221,12 +1236,18 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 // ---------------- the current piece ends here: every row thread stores its row -----------------
                 const int u = mt.unit;
                 const bool partial = piece_tiles < mt.unit_tiles;
+                // the next piece's queries travel while this piece's last product completes; once they are in
+                // tensor memory the MMA warp computes the next piece's first scores under the read-out below
+                const bool more = nx.nvalid >= 0;
+                uint4 qv[16];
+                if (more) load_q(nx.unit, qv);
                 if (piece_ct > 0) {
                     const int c = ct - 1;
                     if (!mbar_wait(&sm.v.bar_o[c & 1], (c >> 1) & 1, p.status)) return;
                     __syncwarp();
                     tc_fence_after_sync();
                 }
+                if (more) store_q(qv);
                 const size_t slot = (size_t)piece_iv + u;
                 float* po = p.part_o + slot * (8 * NT * kHeadDim) + row * kHeadDim;
                 float* pm = p.part_ml + slot * (kMlStride * NT);

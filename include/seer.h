@@ -114,11 +114,12 @@ typedef struct {
 /* Creates a context on CUDA device `device` and allocates its workspace
  * (workspace_bytes, 0 = a default of 64 MiB; partial results of split
  * sequences, gate scratch, status words).  *out is NULL on failure.
- * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT=16 makes
- * the multi-token decode calls with 17 to 64 rows per (sequence, KV head)
- * (q_len * group) run on the tcgen05 tensor cores with S, P and O in tensor
- * memory; the default, 8, is the mma.sync kernel, which is the faster one at
- * the sizes measured so far.  Results agree within the decode tolerance. */
+ * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT.  The
+ * multi-token decode calls with 17 to 64 rows per (sequence, KV head)
+ * (q_len * group) have two kernels: 16 = on the tcgen05 tensor cores with S, P,
+ * O and the queries in tensor memory, 8 = mma.sync.  Unset, up to 48 rows take
+ * the first and more rows the second (the faster one each, as measured).
+ * Results agree within the decode tolerance. */
 seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes);
 /* Frees the workspace.  The caller must have synchronised the streams used. */
 void seer_destroy(seer_ctx* ctx);

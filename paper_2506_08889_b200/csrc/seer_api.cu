@@ -49,7 +49,7 @@ struct seer_ctx {
     int pool_div;               // decode scheduling: share of tiles handed out dynamically
     int min_tiles;              // decode scheduling: fewest tiles of a CTA's range
     int sel_from_lens;          // set by seer_decode_step around its attention call (see DecodeParams)
-    int wide_variant;           // kernel variant code for more than 16 rows per unit: 16 (tcgen05) or 8 (mma.sync)
+    int wide_variant;           // kernel variant code for more than 16 rows per unit: 16 (tcgen05), 8 (mma.sync), 0 (by size)
     char err[512];
 };
 
@@ -211,7 +211,8 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     const int row_cap = wide ? 64 : 16;
     const int tok_per_launch = q_len < row_cap / group ? q_len : row_cap / group;
     const int n_tiles = wide ? 8 : tok_per_launch * group > 8 ? 2 : 1;    // (sizes the partial slots: 8 rows each)
-    const int variant = wide ? ctx->wide_variant : n_tiles;               // (the kernel: 16 = rows on M by tcgen05)
+    // (the kernel: 16 = rows on M by tcgen05, the faster one up to 48 rows; 8 = rows on M by mma.sync)
+    const int variant = !wide ? n_tiles : ctx->wide_variant ? ctx->wide_variant : tok_per_launch * group <= 48 ? 16 : 8;
     const int per_sm = decode_ctas_per_sm(sparse, paged, variant);
     if (per_sm <= 0) return fail(ctx, SEER_ERR_CUDA, "decode kernel cannot be resident (shared memory)");
     long long max_tiles = sparse ? (long long)U * ((max_sel + bpt - 1) / bpt) * tpb
@@ -331,8 +332,8 @@ seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes) {
     if (const char* e = getenv("SEER_DECODE_POOL_DIV")) ctx->pool_div = atoi(e);
     ctx->min_tiles = 4;
     if (const char* e = getenv("SEER_DECODE_MIN_TILES")) ctx->min_tiles = atoi(e);
-    ctx->wide_variant = 8;
-    if (const char* e = getenv("SEER_DECODE_WIDE_VARIANT")) ctx->wide_variant = atoi(e) == 16 ? 16 : 8;
+    ctx->wide_variant = 0;      // chosen by the number of rows
+    if (const char* e = getenv("SEER_DECODE_WIDE_VARIANT")) ctx->wide_variant = atoi(e) == 16 ? 16 : atoi(e) == 8 ? 8 : 0;
     ctx->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)64 << 20;
     if (ctx->ws_bytes < 4096) ctx->ws_bytes = 4096;     // (far too small for any call: every call checks)
     if (cudaMalloc(reinterpret_cast<void**>(&ctx->ws), ctx->ws_bytes) != cudaSuccess) {

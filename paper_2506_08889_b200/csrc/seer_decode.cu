@@ -57,11 +57,13 @@ constexpr int kWideTiles = 8;                              // N-tile count that 
 // The rows-on-M variant on the fifth-generation tensor cores (TC): one CTA per SM, a deeper ring, an extra
 // warp that issues the MMAs; S, P and O live in tensor memory.
 constexpr int kTcTilesCode = 16;                           // what the host passes as n_tiles to ask for it
-constexpr int kTcStages = 8;                               // V buffers (16 KiB each) = tiles between landing and product
-constexpr int kTcKStages = 4;                              // K buffers (16 KiB each): a K tile is free once its scores are computed
+constexpr int kTcStages = 7;                               // V buffers (16 KiB each) = tiles between landing and product
+constexpr int kTcKStages = 5;                              // K buffers (16 KiB each): a K tile is free once its scores are computed
 constexpr int kTcThreads = kThreads + 32;
 constexpr int kTcRows = 128;                               // M of the MMAs (rows past the unit's are zero)
-constexpr int kTcCols = 512;                               // tensor-memory columns: S/P twice 64, O 128, Q 64 (320, as a power of two)
+constexpr int kTcSBufs = 3;                                // S/P buffers: scores of up to three tiles ahead of their products
+constexpr int kTcOCol = 64 * kTcSBufs, kTcQCol = kTcOCol + 128;   // tensor-memory columns of O and of Q
+constexpr int kTcCols = 512;                               // S/P 3 x 64, O 128, Q 64 = 384 columns, as a power of two
 constexpr int kAheadMaxChunk = 8;                          // own chunks up to this size are claimed ahead
 constexpr int kAheadTiles = 3;                             // tiles left to issue when the next interval's claim is made
 constexpr int kSmemUnits = 128;                            // units whose tile-count prefix sums fit in shared memory
@@ -108,9 +110,9 @@ struct VariantPart {
 };
 template <>
 struct VariantPart<true> {
-    uint64_t bar_s[2];               // S of an even / odd tile is complete (the MMA warp's commit)
-    uint64_t bar_p[2];               // P of an even / odd tile is written (one arrival per row warp with real rows)
-    uint64_t bar_o[2];               // O includes an even / odd tile's product (commit)
+    uint64_t bar_s[kTcSBufs];        // S of a tile (buffer = tile number mod kTcSBufs) is complete (the MMA warp's commit)
+    uint64_t bar_p[kTcSBufs];        // P of such a tile is written (one arrival per row warp with real rows)
+    uint64_t bar_o[kTcSBufs];        // O includes such a tile's product (commit)
     uint64_t bar_q;                  // the queries of a piece's unit are in tensor memory (one arrival per row warp with real rows)
     uint64_t tmem_done;              // the row warps have made their last tensor-memory access
     uint64_t empty_k[kTcKStages];    // a K buffer's scores have been computed (commit)
@@ -440,7 +442,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             mbar_init(&sm.empty[s], TC ? 1 + tc_row_warps : kConsumerWarps);
         }
         if constexpr (TC) {
-            for (int b = 0; b < 2; ++b) {
+            for (int b = 0; b < kTcSBufs; ++b) {
                 mbar_init(&sm.v.bar_s[b], 1);
                 mbar_init(&sm.v.bar_p[b], tc_row_warps);
                 mbar_init(&sm.v.bar_o[b], 1);
@@ -934,10 +936,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         // the 64 tokens; P from tensor memory, the V tile MN-major).  The tensor cores work on S(t + 1)
         // while the row warps are busy with S(t).  The whole warp clears the rows of a ragged last tile of V.
         const uint32_t tbase = sm.v.tmem_base;
-        const uint32_t t_o = tbase + 128;
+        const uint32_t t_o = tbase + kTcOCol;
         constexpr uint32_t idesc_qk = tc_idesc_bf16(kTcRows, kTileTokens, false);
         constexpr uint32_t idesc_pv = tc_idesc_bf16(kTcRows, kHeadDim, true);
-        const uint32_t t_q = tbase + 256;
+        const uint32_t t_q = tbase + kTcQCol;
         int piece_no = 0;                          // pieces begun so far (phase of bar_q)
         bool dead = false;                         // a wait ran out: stop issuing, free the tensor memory, leave
         int ct = 0, piece_ct = 0;                  // computed tiles so far (of the CTA, of the piece)
@@ -946,20 +948,20 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         const long long mm_t0 = clock64();
 #endif
         // Two kinds of work, taken as they become possible: the scores of the next tile once it has landed
-        // (at most two tiles may be between their scores and their product: S is double-buffered), and the
+        // (at most three tiles may be between their scores and their product: S has three buffers), and the
         // product of the oldest such tile once its probabilities are written.  A stage is released by the
         // commit behind its product, so it is held no longer than the row warps need for its tile.
-        int pend_n = 0;                            // tiles whose product is still to be issued (0..2)
-        int pend_stage[2] = {0, 0};
-        bool pend_acc[2] = {false, false};         // indexed by the tile's parity (ct & 1)
+        int pend_n = 0;                            // tiles whose product is still to be issued (0..kTcSBufs)
+        int pend_stage[kTcSBufs] = {};
+        bool pend_acc[kTcSBufs] = {};              // indexed by the tile's S buffer (ct % kTcSBufs)
         int it = 0;                                // next tile of the stream
         bool ended = false;
         uint32_t idle = 0;
         while (!dead && (!ended || pend_n > 0)) {
             bool did = false;
             if (pend_n > 0) {
-                const int c = ct - pend_n, b = c & 1;
-                if (__shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.v.bar_p[b], (c >> 1) & 1) : 0, 0)) {
+                const int c = ct - pend_n, b = c % kTcSBufs;
+                if (__shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.v.bar_p[b], (c / kTcSBufs) & 1) : 0, 0)) {
                     __syncwarp();
                     if (lane == 0) {
                         tc_fence_after_sync();
@@ -976,7 +978,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     did = true;
                 }
             }
-            if (!ended && pend_n < 2) {
+            if (!ended && pend_n < kTcSBufs) {
                 const int st = it % kS;
                 if (__shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.full[st], (it / kS) & 1) : 0, 0)) {
                     // (every lane reads the metadata after lane 0 has seen the barrier's phase complete)
@@ -1006,7 +1008,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                                 fence_proxy_async_smem();
                                 __syncwarp();
                             }
-                            const int b = ct & 1;
+                            const int b = ct % kTcSBufs;
                             if (lane == 0) {
                                 tc_fence_after_sync();
                                 const uint32_t k_addr = smem_u32(sm.stage[0]) + (kTcStages + it % kTcKStages) * kTileBytes;
@@ -1089,7 +1091,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     int pubs = 0;                       // partials written so far (phase of merge_bar[0])
     if (32 * w < p.rows) {
         const uint32_t tbase = sm.v.tmem_base + ((uint32_t)(32 * w) << 16);
-        const uint32_t t_o = tbase + 128;
+        const uint32_t t_o = tbase + kTcOCol;
         float m_ref = -INFINITY, l_run = 0.f;
         int ct = 0, piece_ct = 0;       // computed tiles so far (of the CTA, of the piece)
         // A piece's queries go to tensor memory, this thread's row as 64 columns of bf16 pairs (zeros for a padding
@@ -1110,7 +1112,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     qr[4 * x] = qv[8 * h + x].x; qr[4 * x + 1] = qv[8 * h + x].y;
                     qr[4 * x + 2] = qv[8 * h + x].z; qr[4 * x + 3] = qv[8 * h + x].w;
                 }
-                tmem_st32(tbase + 256 + 32 * h, qr);
+                tmem_st32(tbase + kTcQCol + 32 * h, qr);
             }
             tmem_wait_st();
             tc_fence_before_sync();
@@ -1139,9 +1141,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             ++piece_tiles;
             const int nv = mt.nvalid;                          // cached tokens from the tile's first row on (capped at 64 + 7)
             if (nv > 0) {
-                const int b = ct & 1;
+                const int b = ct % kTcSBufs;
                 TC_T(t_a);
-                if (!mbar_wait(&sm.v.bar_s[b], (ct >> 1) & 1, p.status)) return;
+                if (!mbar_wait(&sm.v.bar_s[b], (ct / kTcSBufs) & 1, p.status)) return;
                 __syncwarp();
                 tc_fence_after_sync();
                 TC_T(t_b);
@@ -1184,7 +1186,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     if (piece_ct > 0) {
                         // O holds the earlier tiles' products: all of them are in once the last one is
                         const int c = ct - 1;
-                        if (!mbar_wait(&sm.v.bar_o[c & 1], (c >> 1) & 1, p.status)) return;
+                        if (!mbar_wait(&sm.v.bar_o[c % kTcSBufs], (c / kTcSBufs) & 1, p.status)) return;
                         __syncwarp();
                         tc_fence_after_sync();
 #pragma unroll 1
@@ -1243,7 +1245,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 if (more) load_q(nx.unit, qv);
                 if (piece_ct > 0) {
                     const int c = ct - 1;
-                    if (!mbar_wait(&sm.v.bar_o[c & 1], (c >> 1) & 1, p.status)) return;
+                    if (!mbar_wait(&sm.v.bar_o[c % kTcSBufs], (c / kTcSBufs) & 1, p.status)) return;
                     __syncwarp();
                     tc_fence_after_sync();
                 }

@@ -15,8 +15,9 @@ DEV = "cuda:0"
 @pytest.fixture(scope="module", params=["mma.sync", "tcgen05"])
 def ctx(request):
     """Every test of this file runs twice: units of 17 to 64 rows take the rows-on-M kernel, which exists as an
-    mma.sync variant (the default) and as a tcgen05 variant (S, P and O in tensor memory) that a context picks
-    up from SEER_DECODE_WIDE_VARIANT=16 when it is created.  Up to 16 rows both runs take the same kernels."""
+    mma.sync variant and as a tcgen05 variant (S, P, O and the queries in tensor memory); a context created with
+    SEER_DECODE_WIDE_VARIANT=8 or 16 takes that one at every size (unset: tcgen05 up to 48 rows).  Up to 16 rows
+    both runs take the same kernels."""
     import os
     old = os.environ.get("SEER_DECODE_WIDE_VARIANT")
     os.environ["SEER_DECODE_WIDE_VARIANT"] = "16" if request.param == "tcgen05" else "8"

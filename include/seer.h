@@ -306,9 +306,11 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
  * One decode step of one attention layer in a single call (paper Fig. 3): the compressed-K
  * update for the block that has just filled (Sec. 3.2, skipped when k_nope is NULL), gate scoring
  * and token-budget selection (Eq. 1a/1c, Sec. 3.1), block-sparse decode over the selected
- * blocks (Sec. 3.3).  Exactly the three calls
+ * blocks (Sec. 3.3).  The results are those of the three calls
  *     seer_kcomp_append(.., first_block = -1) ; seer_gate_select(.., scores_in = NULL) ; seer_sparse_decode
- * on `stream`, with one argument check and one host round trip instead of three.
+ * on `stream`, with one host round trip instead of three.  (The launches go out as gate, attention,
+ * append: the block that has just filled is the sequence's last block, which the gate takes without
+ * scoring it, so the entry the append writes is first read in the next step.)
  *  block_idx / block_cnt / max_sel: caller-owned scratch for the selected lists (they are
  *  outputs too: the lists the attention used).  Other arguments as in the three calls;
  *  kv->seq_lens is used as the sequence lengths of all three.

@@ -59,7 +59,7 @@ constexpr int kWideTiles = 8;                              // N-tile count that 
 constexpr int kTcTilesCode = 16;                           // what the host passes as n_tiles to ask for it
 constexpr int kTcStages = 7;                               // V buffers (16 KiB each) = tiles between landing and product
 constexpr int kTcKStages = 5;                              // K buffers (16 KiB each): a K tile is free once its scores are computed
-constexpr int kTcThreads = kThreads + 64;                   // + the two MMA-issuing warps
+constexpr int kTcThreads = kThreads + 32;
 constexpr int kTcRows = 128;                               // M of the MMAs (rows past the unit's are zero)
 constexpr int kTcSBufs = 3;                                // S/P buffers: scores of up to three tiles ahead of their products
 constexpr int kTcOCol = 64 * kTcSBufs, kTcQCol = kTcOCol + 128;   // tensor-memory columns of O and of Q
@@ -437,9 +437,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         const int tc_row_warps = min(kConsumerWarps, (p.rows + 31) / 32);
         for (int s = 0; s < kS; ++s) {
             mbar_init(&sm.full[s], 1);
-            // a stage is free once every consumer warp has arrived; tensor-memory variant: once the product that reads
-            // its V has completed (a commit) and the score warp and every row warp have taken the tile's metadata
-            mbar_init(&sm.empty[s], TC ? 2 + tc_row_warps : kConsumerWarps);
+            // a stage is free once every consumer warp has arrived; tensor-memory variant: once the MMAs that read
+            // it have completed (one commit) and every row warp has taken the tile's metadata
+            mbar_init(&sm.empty[s], TC ? 1 + tc_row_warps : kConsumerWarps);
         }
         if constexpr (TC) {
             for (int b = 0; b < kTcSBufs; ++b) {
@@ -929,106 +929,131 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 
     if constexpr (TC) {
     if (warp == kConsumerWarps + 1) {
-        // =========================== score warp (tensor-memory variant) ====================
-        // Lane 0 issues S = Q . K^T for every tile as soon as it has landed: 8 MMAs of K = 16 over the 128
-        // channels (M 128 x N 64; Q from tensor memory, where the row warps put the unit's queries when a piece
-        // begins; the K tile K-major in shared memory) into the tile's S buffer - one of three, so the scores run
-        // up to three tiles ahead of the products - and the commits behind them tell the row warps and free the
-        // K buffer.  An issuing thread gets one MMA out per 80 to 120 cycles, more than these small MMAs take to
-        // execute, which is why the products have an issuing warp of their own.  The whole warp clears the rows
-        // of a ragged last tile of V.  This warp also owns the tensor memory.
+        // =========================== MMA warp (tensor-memory variant) ====================
+        // Lane 0 issues, per tile, S = Q . K^T (8 MMAs of K = 16 over the 128 channels; Q from tensor memory,
+        // where the row warps put the unit's queries when a piece begins, the K tile K-major in shared
+        // memory) and, once the row warps have written the tile's probabilities, O (+)= P . V (4 MMAs over
+        // the 64 tokens; P from tensor memory, the V tile MN-major).  The tensor cores work on S(t + 1)
+        // while the row warps are busy with S(t).  The whole warp clears the rows of a ragged last tile of V.
         const uint32_t tbase = sm.v.tmem_base;
+        const uint32_t t_o = tbase + kTcOCol;
         constexpr uint32_t idesc_qk = tc_idesc_bf16(kTcRows, kTileTokens, false);
+        constexpr uint32_t idesc_pv = tc_idesc_bf16(kTcRows, kHeadDim, true);
         const uint32_t t_q = tbase + kTcQCol;
         int piece_no = 0;                          // pieces begun so far (phase of bar_q)
-        int ct = 0;                                // computed tiles so far
         bool dead = false;                         // a wait ran out: stop issuing, free the tensor memory, leave
-        for (int it = 0; !dead; ++it) {
-            const int st = it % kS, sk = it % kTcKStages;
-            if (!mbar_wait(&sm.full[st], (it / kS) & 1, p.status)) { dead = true; break; }
-            const StageMeta mt = sm.meta[st];
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.empty[st]);          // metadata taken
-            if (mt.nvalid < 0) break;
-            if (mt.flags & 1) {
-                // the first tile of a piece has to find the piece's queries in tensor memory
-                if (!mbar_wait(&sm.v.bar_q, piece_no & 1, p.status)) { dead = true; break; }
-                ++piece_no;
-            }
-            const int nv = mt.nvalid;
-            if (nv <= 0) {
-                if (lane == 0) mbar_arrive(&sm.v.empty_k[sk]);  // nothing was loaded: the K buffer goes straight back
-                continue;
-            }
-            const int b = ct % kTcSBufs;
-            // the S buffer is free once the product of the tile that had it before is complete
-            if (ct >= kTcSBufs && !mbar_wait(&sm.v.bar_o[b], ((ct - kTcSBufs) / kTcSBufs) & 1, p.status)) { dead = true; break; }
-            if (nv < kTileTokens) {
-                // ragged tail: rows past the sequence end may hold anything; cleared in V so that a zero
-                // probability times garbage cannot produce NaN
-                unsigned char* vt = sm.stage[0] + (size_t)st * kTileBytes;
-                for (int x = lane; x < (kTileTokens - nv) * 16; x += 32) {
-                    const int r = nv + (x >> 4), part = x & 15;
-                    *reinterpret_cast<uint4*>(vt + (part >> 3) * kHalfTileBytes + r * 128 + ((part & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-                }
-                fence_proxy_async_smem();
-            }
-            __syncwarp();
-            if (lane == 0) {
-                tc_fence_after_sync();
-                // (one descriptor per tile; a K step moves its start-address field, in units of 16 bytes)
-                const uint64_t kd = tc_smem_desc(smem_u32(sm.stage[0]) + (kTcStages + sk) * kTileBytes, 16, 1024);
+        int ct = 0, piece_ct = 0;                  // computed tiles so far (of the CTA, of the piece)
+#ifdef SEER_DECODE_TRACE
+        unsigned long long mm_tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const long long mm_t0 = clock64();
+#endif
+        // Two kinds of work, taken as they become possible: the scores of the next tile once it has landed
+        // (at most three tiles may be between their scores and their product: S has three buffers), and the
+        // product of the oldest such tile once its probabilities are written.  A stage is released by the
+        // commit behind its product, so it is held no longer than the row warps need for its tile.
+        int pend_n = 0;                            // tiles whose product is still to be issued (0..kTcSBufs)
+        int pend_stage[kTcSBufs] = {};
+        bool pend_acc[kTcSBufs] = {};              // indexed by the tile's S buffer (ct % kTcSBufs)
+        int it = 0;                                // next tile of the stream
+        bool ended = false;
+        uint32_t idle = 0;
+        while (!dead && (!ended || pend_n > 0)) {
+            bool did = false;
+            if (pend_n > 0) {
+                const int c = ct - pend_n, b = c % kTcSBufs;
+                if (__shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.v.bar_p[b], (c / kTcSBufs) & 1) : 0, 0)) {
+                    __syncwarp();
+                    if (lane == 0) {
+                        tc_fence_after_sync();
+                        const uint32_t v_addr = smem_u32(sm.stage[0]) + pend_stage[b] * kTileBytes;
 #pragma unroll
-                for (int ks = 0; ks < kHeadDim / 16; ++ks)
-                    tc_mma_ts(tbase + 64 * b, t_q + 8 * ks, kd + (uint64_t)(((ks >> 2) * kHalfTileBytes + (ks & 3) * 32) >> 4), idesc_qk, ks > 0);
-                tc_commit(&sm.v.bar_s[b]);
-                tc_commit(&sm.v.empty_k[sk]);                   // the K buffer has been read
+                        for (int ks = 0; ks < kTileTokens / 16; ++ks)
+                            tc_mma_ts(t_o, tbase + 64 * b + 8 * ks, tc_smem_desc(v_addr + ks * 2048, kHalfTileBytes, 1024), idesc_pv,
+                                      pend_acc[b] || ks > 0);
+                        tc_commit(&sm.empty[pend_stage[b]]);   // the stage's K and V have been read
+                        tc_commit(&sm.v.bar_o[b]);
+                    }
+                    __syncwarp();
+                    --pend_n;
+                    did = true;
+                }
             }
-            __syncwarp();
-            ++ct;
+            if (!ended && pend_n < kTcSBufs) {
+                const int st = it % kS;
+                if (__shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.full[st], (it / kS) & 1) : 0, 0)) {
+                    // (every lane reads the metadata after lane 0 has seen the barrier's phase complete)
+                    mbar_try_wait(&sm.full[st], (it / kS) & 1);
+                    __syncwarp();
+                    const StageMeta mt = sm.meta[st];
+                    // the first tile of a piece has to find the piece's queries in tensor memory
+                    const bool q_ready = mt.nvalid < 0 || !(mt.flags & 1) ||
+                        __shfl_sync(0xffffffffu, lane == 0 ? (int)mbar_test_wait(&sm.v.bar_q, piece_no & 1) : 0, 0);
+                    if (q_ready) {
+                    did = true;
+                    if (mt.nvalid < 0) {
+                        ended = true;
+                    } else {
+                        if (mt.flags & 1) { piece_ct = 0; ++piece_no; }
+                        const int nv = mt.nvalid;
+                        if (nv > 0) {
+                            if (nv < kTileTokens) {
+                                // ragged tail: rows past the sequence end may hold anything; cleared in V so that a
+                                // zero probability times garbage cannot produce NaN
+                                unsigned char* vt = sm.stage[0] + (size_t)st * kTileBytes;
+                                for (int x = lane; x < (kTileTokens - nv) * 16; x += 32) {
+                                    const int r = nv + (x >> 4), part = x & 15;
+                                    *reinterpret_cast<uint4*>(vt + (part >> 3) * kHalfTileBytes + r * 128 + ((part & 7) << 4)) =
+                                        make_uint4(0u, 0u, 0u, 0u);
+                                }
+                                fence_proxy_async_smem();
+                                __syncwarp();
+                            }
+                            const int b = ct % kTcSBufs;
+                            if (lane == 0) {
+                                tc_fence_after_sync();
+                                const uint32_t k_addr = smem_u32(sm.stage[0]) + (kTcStages + it % kTcKStages) * kTileBytes;
+#pragma unroll
+                                for (int ks = 0; ks < kHeadDim / 16; ++ks)
+                                    tc_mma_ts(tbase + 64 * b, t_q + 8 * ks,
+                                              tc_smem_desc(k_addr + (ks >> 2) * kHalfTileBytes + (ks & 3) * 32, 16, 1024), idesc_qk, ks > 0);
+                                tc_commit(&sm.v.bar_s[b]);
+                                tc_commit(&sm.v.empty_k[it % kTcKStages]);   // the K buffer has been read
+                            }
+                            __syncwarp();
+                            pend_stage[b] = st;
+                            pend_acc[b] = piece_ct > 0;
+                            ++pend_n;
+                            ++ct;
+                            ++piece_ct;
+                        } else {
+                            if (lane == 0) {                               // nothing was loaded: the buffers go straight back
+                                mbar_arrive(&sm.empty[st]);
+                                mbar_arrive(&sm.v.empty_k[it % kTcKStages]);
+                            }
+                        }
+                        ++it;
+                    }
+                    }
+                }
+            }
+            if (did) {
+                idle = 0;
+            } else if (++idle > 64) {
+                if (idle > (1u << 23)) {               // seconds: whatever this warp waits for will not come
+                    raise_status(p.status, DEV_TIMEOUT);
+                    dead = true;
+                }
+                __nanosleep(32);
+            }
         }
+#ifdef SEER_DECODE_TRACE
+        mm_tr[3] = (unsigned long long)(clock64() - mm_t0);
+        if (lane == 0) for (int k = 0; k < 8; ++k) p.trace[(size_t)blockIdx.x * kTraceSlots + 64 + k] = mm_tr[k];
+#endif
         // the tensor memory goes back once the row warps are done with it (or a wait has run out)
         mbar_wait(&sm.v.tmem_done, 0, p.status);
         __syncwarp();
         tmem_dealloc(tbase, kTcCols);
-        return;
-    }
-    if (warp == kConsumerWarps + 2) {
-        // =========================== product warp (tensor-memory variant) ====================
-        // Lane 0 issues O (+)= P . V for every tile once the row warps have written its probabilities: 4 MMAs
-        // over the 64 tokens (M 128 x N 128; P from tensor memory, the V tile MN-major in shared memory); the
-        // commits behind them free the V buffer and tell the row warps that O includes the tile.
-        const uint32_t tbase = sm.v.tmem_base;
-        const uint32_t t_o = tbase + kTcOCol;
-        constexpr uint32_t idesc_pv = tc_idesc_bf16(kTcRows, kHeadDim, true);
-        int ct = 0, piece_ct = 0;                  // computed tiles so far (of the CTA, of the piece)
-        for (int it = 0;; ++it) {
-            const int st = it % kS;
-            if (!mbar_wait(&sm.full[st], (it / kS) & 1, p.status)) break;
-            const StageMeta mt = sm.meta[st];
-            __syncwarp();
-            if (mt.nvalid < 0) break;
-            if (mt.flags & 1) piece_ct = 0;
-            if (mt.nvalid <= 0) {
-                if (lane == 0) mbar_arrive(&sm.empty[st]);      // nothing was loaded: the V buffer goes straight back
-                continue;
-            }
-            const int b = ct % kTcSBufs;
-            if (!mbar_wait(&sm.v.bar_p[b], (ct / kTcSBufs) & 1, p.status)) break;
-            __syncwarp();
-            if (lane == 0) {
-                tc_fence_after_sync();
-                const uint64_t vd = tc_smem_desc(smem_u32(sm.stage[0]) + st * kTileBytes, kHalfTileBytes, 1024);
-#pragma unroll
-                for (int ks = 0; ks < kTileTokens / 16; ++ks)
-                    tc_mma_ts(t_o, tbase + 64 * b + 8 * ks, vd + (uint64_t)((ks * 2048) >> 4), idesc_pv, piece_ct > 0 || ks > 0);
-                tc_commit(&sm.empty[st]);                       // the V buffer has been read
-                tc_commit(&sm.v.bar_o[b]);
-            }
-            __syncwarp();
-            ++ct;
-            ++piece_ct;
-        }
         return;
     }
     }

@@ -329,15 +329,16 @@ def run_ours(args):
 
     def e2e_step(lay):
         dbuf.copy_(hbuf, non_blocking=True)          # q, q_nope, the new token's K and V rows, lengths
-        lay["k"][:, :, L - 1, :] = dk_new            # the caller's append of the new token
-        lay["v"][:, :, L - 1, :] = dv_new
+        lay["k_last"].copy_(dk_new)                  # the caller's append of the new token
+        lay["v_last"].copy_(dv_new)
         ctx.seer_decode_step(shape, lay["kv_e2e"], lay["gate"], dq, dqn, lay["k"], budget, idx, cnt, k_sel, out,
                              stream=stream)
         hout.copy_(out, non_blocking=True)
-        torch.cuda.synchronize()
+        stream.synchronize()
 
     for lay in layers:
         lay["kv_e2e"] = binding.make_kv(lay["k"], lay["v"], dlens)
+        lay["k_last"], lay["v_last"] = lay["k"][:, :, L - 1, :], lay["v"][:, :, L - 1, :]   # (views: the rows the step appends)
     Ke = max(8, min(K, 300))
     for s in range(3):
         e2e_step(layers[s % n_layers])

@@ -55,12 +55,12 @@ constexpr int kMaxSteals = 14;                             // chunks a CTA may t
 constexpr int kFewTilesPerCta = 16;                        // up to this many tiles per CTA the number of ranges is chosen with care
 constexpr int kWideTiles = 8;                              // N-tile count that stands for the rows-on-M variant (up to 64 rows)
 // The rows-on-M variant on the fifth-generation tensor cores (TC): one CTA per SM, a deeper ring, an extra
-// warp that issues the MMAs; S, P and O live in tensor memory.
+// warp that issues the MMAs; S, P, O and the unit's queries live in tensor memory.
 constexpr int kTcTilesCode = 16;                           // what the host passes as n_tiles to ask for it
 constexpr int kTcStages = 7;                               // V buffers (16 KiB each) = tiles between landing and product
 constexpr int kTcKStages = 5;                              // K buffers (16 KiB each): a K tile is free once its scores are computed
 constexpr int kTcThreads = kThreads + 32;
-constexpr int kTcRows = 128;                               // M of the MMAs (rows past the unit's are zero)
+constexpr int kTcRows = 128;                               // M of the MMAs (rows past the unit's are padding: zero, or never read)
 constexpr int kTcSBufs = 3;                                // S/P buffers: scores of up to three tiles ahead of their products
 constexpr int kTcOCol = 64 * kTcSBufs, kTcQCol = kTcOCol + 128;   // tensor-memory columns of O and of Q
 constexpr int kTcCols = 512;                               // S/P 3 x 64, O 128, Q 64 = 384 columns, as a power of two
@@ -1073,7 +1073,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     // probabilities back over S as bf16 pairs (P) for the MMA warp's second product.  The reference maximum
     // only moves when the true one has grown by more than 2^8 since (probabilities stay below 2^8, exact in
     // bf16's range); O, which accumulates in tensor memory, is rescaled on those occasions only.
-    //     S (128 x 64 tok) = Q (128 x 128) . K^T      tcgen05.mma, Q and K K-major in shared memory
+    //     S (128 x 64 tok) = Q (128 x 128) . K^T      tcgen05.mma, Q from tensor memory, K K-major in shared memory
     //     O (128 x 128)   += P (128 x 64) . V          P from tensor memory, V MN-major in shared memory
     constexpr float kSlack = 8.f;
 #ifdef SEER_DECODE_TRACE

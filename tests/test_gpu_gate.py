@@ -9,7 +9,7 @@ import torch
 
 import oracle
 from paper_2506_08889_b200 import binding, synth
-from util import bits, check_attention, make_qkv, ref_sparse, kc_tolerance
+from util import bits, check_attention, make_qkv, ref_sparse, kc_tolerance, to_paged
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -487,4 +487,40 @@ def test_step_call_on_ragged_lengths_budget_above_and_below_the_block_counts(ctx
         assert np.array_equal(cnt.cpu().numpy(), want_cnt) and np.array_equal(idx.cpu().numpy(), want_idx)
         ref = ref_sparse(bits(q), bits(k), bits(v), lens, want_idx, want_cnt, b, 0.0884)
         check_attention(out, lse, *ref, what=f"step b={b} budget={budget}")
+    assert ctx.device_status() == binding.SEER_OK
+
+
+def test_step_call_on_a_paged_cache_with_ragged_lengths(ctx):
+    """seer_decode_step over a paged K/V pool (pages of 128 tokens under a random permutation) and ragged
+    lengths: inside the step the attention kernel counts its tiles from the sequence lengths before the gate
+    has finished, so the lists, the counts and the attention are checked against the oracle for budgets above
+    and below the sequences' block counts."""
+    B, Hq, Hkv, d, dg, S, b = 5, 10, 2, 128, 128, 4096, 64
+    nb = S // b
+    lens = np.array([S, 37 * b + 9, 3 * b, b + 1, 0], np.int32)
+    q, k, v = make_qkv(B, Hq, Hkv, S, d, 91, DEV)
+    kp, vp, table = to_paged(k, v, 128, 91)
+    qn = synth.normal_bf16((B, Hq, d), 91, "qn", DEV)
+    wq = synth.normal_bf16((Hkv, dg, 5 * d), 91, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nb, dg), 91, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    kv = binding.make_kv(kp, vp, lens_t, max_seq_len=S, page_table=table, page_size=128)
+    for budget, max_sel in [(20 * b, 20), (20 * b, 6), (2 * b, 8)]:
+        idx = torch.full((B, Hkv, max_sel), 55, dtype=torch.int32, device=DEV)
+        cnt = torch.full((B, Hkv), 55, dtype=torch.int32, device=DEV)
+        out = torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+        lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV)
+        for _ in range(2):                                  # (the second call's kernels overlap the first's)
+            ctx.seer_decode_step(shape, kv, gate, q, qn, None, budget, idx, cnt, max_sel, out, lse)
+        torch.cuda.synchronize()
+        sc = torch.zeros((B, Hkv, nb), dtype=torch.float32, device=DEV)
+        idx2, cnt2 = torch.zeros_like(idx), torch.zeros_like(cnt)
+        ctx.seer_gate_select(shape, gate, lens_t, qn, None, budget, idx2, cnt2, max_sel, scores_out=sc)
+        torch.cuda.synchronize()
+        want_idx, want_cnt = oracle.select(sc.cpu().numpy(), lens, b, budget, max_sel)
+        assert np.array_equal(cnt.cpu().numpy(), want_cnt) and np.array_equal(idx.cpu().numpy(), want_idx)
+        ref = ref_sparse(bits(q), bits(k), bits(v), lens, want_idx, want_cnt, b, 0.0884)
+        check_attention(out, lse, *ref, what=f"paged step budget={budget}")
     assert ctx.device_status() == binding.SEER_OK

@@ -349,11 +349,14 @@ __global__ void __launch_bounds__(kKcThreads, 4) kcomp_bulk_kernel(const KcompPa
 //   producer (1 warp)    keeps a ring of 64-row stages (one block, 16 KiB) full with tiled copies, so
 //                        the bytes in flight do not depend on what the other warps are doing;
 //   pooling (7 warps)    each takes one block at a time out of shared memory and leaves the block's
-//                        3*128 features (bf16; the mean as high part + correction) in one of two
-//                        feature buffers;
-//   projection (8 warps) warp w holds rows 16w .. 16w+15 of W_k as mma A fragments (96 registers) and,
-//                        once 16 blocks are pooled, multiplies them in (64 mma, nothing to fetch),
-//                        rotates and stores - while the pooling warps are already on the next item.
+//                        3*128 features (bf16; the mean as high part + correction: 512 numbers) in one of
+//                        two feature buffers, laid out as the tensor cores read a K-major operand;
+//   MMA (1 warp)         once 16 blocks are pooled, one thread multiplies them in: Y (128 rows of W_k x 16
+//                        blocks, fp32 in tensor memory) = W_k[h] (from tensor memory, where it stays while
+//                        the CTA's items have the same head) . features^T, 32 tcgen05.mma of K = 16;
+//   epilogue (4 warps)   thread r has row r of W_k and of Y: it puts its row of W_k[h] into tensor memory when
+//                        the head changes, reads its 16 products, and the four warps rotate and store -
+//                        while the pooling warps are already on the next item.
 // An item is 16 consecutive blocks of one (sequence, KV head); items are numbered head-major and dealt
 // round-robin, so a CTA changes head a handful of times per launch.
 //
@@ -373,7 +376,10 @@ constexpr int kStageBytes = kStageRows * kHeadDim * 2;
 constexpr int kStreamDGate = 128;
 constexpr int kLensCache = 2048;                       // sequences whose length is kept in shared memory
 constexpr int kPoolWarps = 7;                        // with 8 + 1 others: 16 warps, 128 registers each
-constexpr int kProjWarps = kStreamDGate / 16;
+constexpr int kProjWarps = 8;                        // warps 0..3 epilogue, 4 MMA, 5..7 unused
+constexpr int kEpiWarps = 4, kEpiThreads = 128;
+constexpr int kFeatBytes = 8 * kBulkBlocks * 128;      // one feature buffer
+constexpr int kKcTmemCols = 512;                       // W_k 256 columns (512 bf16 per row), Y twice 16
 constexpr int kProjThreads = 32 * kProjWarps;
 constexpr int kStreamThreads = 32 * (kProjWarps + kPoolWarps + 1);
 static_assert(kStreamStages <= 32, "one producer lane per ring slot");
@@ -384,16 +390,19 @@ struct __align__(1024) StreamSmem {
     // a stage: channels 0..63 of its 32 rows (128 B per row, 16-byte pieces swizzled by row as the copy engine
     // lays them out), then channels 64..127
     unsigned char ring[kStreamStages][kStageBytes];
-    // [max | min | avg]; once a buffer's features have been multiplied in, its start holds the 16 x 128
-    // fp32 products until they are rotated and stored
-    alignas(16) __nv_bfloat16 feat_hi[2][kBulkBlocks][kFeatStride];
-    alignas(16) __nv_bfloat16 feat_lo[2][kBulkBlocks][kLoStride];     // avg - bf16(avg)
+    // features of 16 blocks, twice: [8 slabs of 64 features][16 blocks][128 B], 16-byte pieces swizzled by
+    // block (what a K-major operand with the 128-byte swizzle looks like); slabs: max 0-1, min 2-3, the mean's
+    // high part 4-5, its correction 6-7
+    unsigned char feat[2][kFeatBytes];
+    float ybuf[kBulkBlocks][kStreamDGate];
     uint64_t full[kStreamStages], empty[kStreamStages];
     uint64_t feat_full[2], feat_empty[2];
+    uint64_t y_full[2], y_free[2];       // the products of an even / odd item are complete / have been read
+    uint64_t w_ready;                    // a head's W_k is in tensor memory
+    uint64_t tmem_done;                  // the epilogue warps have made their last tensor-memory access
+    uint32_t tmem_base;
     int lens[kLensCache];                                             // seq_lens, read once
 };
-static_assert(sizeof(float) * kBulkBlocks * kStreamDGate <= sizeof(__nv_bfloat16) * kBulkBlocks * kFeatStride,
-              "the products must fit in the feature buffer they replace");
 static_assert(sizeof(StreamSmem) + 1024 <= 227 * 1024, "one CTA's shared memory");
 static_assert(kStageBytes % 2048 == 0, "both halves of a stage start on a swizzle-pattern boundary");
 
@@ -405,7 +414,7 @@ static_assert(kStageBytes % 2048 == 0, "both halves of a stage start on a swizzl
 #define KC_ACC(slot, t0, t1)
 #endif
 
-__device__ __forceinline__ void proj_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kProjThreads) : "memory"); }
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
 __global__ void __launch_bounds__(kStreamThreads, 1)
 kcomp_stream_kernel(const __grid_constant__ CUtensorMap map_k, const KcompParams p) {
@@ -419,16 +428,23 @@ kcomp_stream_kernel(const __grid_constant__ CUtensorMap map_k, const KcompParams
         }
         for (int f = 0; f < 2; ++f) {
             mbar_init(&sm.feat_full[f], kPoolWarps);
-            mbar_init(&sm.feat_empty[f], kProjWarps);
+            mbar_init(&sm.feat_empty[f], 1);
+            mbar_init(&sm.y_full[f], 1);
+            mbar_init(&sm.y_free[f], kEpiWarps);
         }
+        mbar_init(&sm.w_ready, kEpiWarps);
+        mbar_init(&sm.tmem_done, kEpiWarps);
         mbar_fence_init();
     }
+    if (warp == kEpiWarps) tmem_alloc(&sm.tmem_base, kKcTmemCols);
+    tc_fence_before_sync();
     pdl_wait();
     pdl_launch_dependents();
     // A small load issued while the copies flood the memory system waits microseconds behind them: the
     // lengths are fetched once, before any copy is in flight.
     for (int x = tid; x < min(p.batch, kLensCache); x += kStreamThreads) sm.lens[x] = p.seq_lens[x];
     __syncthreads();
+    tc_fence_after_sync();
 
     const int b = p.block_size;                        // == kStreamRows
     const int groups = (p.num_blocks + kBulkBlocks - 1) / kBulkBlocks;
@@ -570,102 +586,131 @@ kcomp_stream_kernel(const __grid_constant__ CUtensorMap map_k, const KcompParams
                     for (int c = 0; c < 8; ++c) sum[c] += __shfl_xor_sync(0xffffffffu, sum[c], 16);
                 }
                 if (lane < 16) {
+                    // 8 features per kind and lane: one 16-byte piece each, at its swizzled place in row q of its slab
+                    uint4 pmax = make_uint4(0u, 0u, 0u, 0u), pmin = pmax, phi = pmax, plo = pmax;
+                    if (q < nb) {
+                        pmax = make_uint4(*reinterpret_cast<uint32_t*>(&mx[0]), *reinterpret_cast<uint32_t*>(&mx[1]),
+                                          *reinterpret_cast<uint32_t*>(&mx[2]), *reinterpret_cast<uint32_t*>(&mx[3]));
+                        pmin = make_uint4(*reinterpret_cast<uint32_t*>(&mn[0]), *reinterpret_cast<uint32_t*>(&mn[1]),
+                                          *reinterpret_cast<uint32_t*>(&mn[2]), *reinterpret_cast<uint32_t*>(&mn[3]));
+                        uint32_t hi[4], lo[4];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const __nv_bfloat162 zero = __float2bfloat162_rn(0.f);
-                        *reinterpret_cast<__nv_bfloat162*>(&sm.feat_hi[fb][q][8 * cchunk + 2 * c]) = q < nb ? mx[c] : zero;
-                        *reinterpret_cast<__nv_bfloat162*>(&sm.feat_hi[fb][q][kHeadDim + 8 * cchunk + 2 * c]) =
-                            q < nb ? mn[c] : zero;
+                        for (int c = 0; c < 8; c += 2) {
+                            const float a0 = sum[c] * (1.f / kStreamRows), a1 = sum[c + 1] * (1.f / kStreamRows);
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
+                            hi[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                            const float2 hf = bf16x2_to_float2(h2);
+                            lo[c >> 1] = pack_bf16x2(a0 - hf.x, a1 - hf.y);
+                        }
+                        phi = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                        plo = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                     }
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const float av = q < nb ? sum[c] * (1.f / kStreamRows) : 0.f;
-                        const __nv_bfloat16 av_hi = __float2bfloat16(av);
-                        sm.feat_hi[fb][q][2 * kHeadDim + 8 * cchunk + c] = av_hi;
-                        sm.feat_lo[fb][q][8 * cchunk + c] = __float2bfloat16(av - __bfloat162float(av_hi));
-                    }
+                    unsigned char* f0 = sm.feat[fb] + (cchunk >> 3) * (kBulkBlocks * 128) + q * 128 + (((cchunk & 7) ^ (q & 7)) << 4);
+                    *reinterpret_cast<uint4*>(f0) = pmax;
+                    *reinterpret_cast<uint4*>(f0 + 2 * kBulkBlocks * 128) = pmin;
+                    *reinterpret_cast<uint4*>(f0 + 4 * kBulkBlocks * 128) = phi;
+                    *reinterpret_cast<uint4*>(f0 + 6 * kBulkBlocks * 128) = plo;
                 }
             }
             block_no += nb;
             ++n_done;
+            fence_proxy_async_smem();              // the tensor cores read the features through the asynchronous proxy
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.feat_full[fb]);
 #ifdef SEER_DECODE_TRACE
             { const long long t_e = clock64(); tr[4] += (unsigned long long)(t_e - t_fe0); }
 #endif
         }
-    } else {
-        // ---- projection, rotation, store ----
-        const int g = lane >> 2, t4 = lane & 3;
-        const bool projects = warp < p.d_gate / 16;
-        uint32_t wa[3 * kHeadDim / 16][4];            // this warp's 16 rows of W_k as A fragments
+    } else if (warp == kEpiWarps) {
+        // ---- MMA warp: Y = W_k[h] . features^T per item, issued by lane 0 ----
+        const uint32_t tbase = sm.tmem_base;
+        constexpr uint32_t idesc = tc_idesc_bf16(128, kBulkBlocks, false);
+        int h_held = -1;
+        uint32_t n_done = 0, n_heads = 0;
+        for (int item = blockIdx.x; item < n_items && !dead; item += gridDim.x) {
+            int h, i, j_first;
+            const int nb = item_blocks(item, h, i, j_first);
+            if (nb == 0) continue;
+            if (h != h_held) {
+                // the epilogue warps put the new head's rows in place (after the last products of the old one)
+                if (!mbar_wait(&sm.w_ready, n_heads & 1u, p.status)) { dead = true; break; }
+                ++n_heads;
+                h_held = h;
+            }
+            const int fb = n_done & 1;
+            if (!mbar_wait(&sm.feat_full[fb], (n_done >> 1) & 1u, p.status)) { dead = true; break; }
+            // the Y buffer of two items ago has been read
+            if (n_done >= 2 && !mbar_wait(&sm.y_free[fb], ((n_done - 2) >> 1) & 1u, p.status)) { dead = true; break; }
+            __syncwarp();
+            if (lane == 0) {
+                tc_fence_after_sync();
+                const uint64_t fd = tc_smem_desc(smem_u32(sm.feat[fb]), 16, 1024);
+#pragma unroll 4
+                for (int ks = 0; ks < 32; ++ks)
+                    tc_mma_ts(tbase + 256 + 16 * fb, tbase + 8 * ks, fd + (uint64_t)(((ks >> 2) * (kBulkBlocks * 128) + (ks & 3) * 32) >> 4),
+                              idesc, ks > 0);
+                tc_commit(&sm.y_full[fb]);
+                tc_commit(&sm.feat_empty[fb]);         // the features have been read
+            }
+            __syncwarp();
+            ++n_done;
+        }
+        // the tensor memory goes back once the epilogue warps are done with it (or a wait has run out)
+        mbar_wait(&sm.tmem_done, 0, p.status);
+        __syncwarp();
+        tmem_dealloc(tbase, kKcTmemCols);
+    } else if (warp < kEpiWarps) {
+        // ---- epilogue: W_k into tensor memory, products out of it, rotation, store ----
+        const int r = tid;                            // row of W_k[h] and of Y, lane of tensor memory
+        const uint32_t tbase = sm.tmem_base + ((uint32_t)(32 * warp) << 16);
         int h_held = -1;
         uint32_t n_done = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
             int h, i, j_first;
             const int nb = item_blocks(item, h, i, j_first);
             if (nb == 0) continue;
-            if (h != h_held && projects) {
-                const uint32_t* w0 =
-                    reinterpret_cast<const uint32_t*>(p.w_k + ((size_t)h * p.d_gate + 16 * warp + g) * 3 * kHeadDim);
-                const uint32_t* w1 = w0 + 8 * (3 * kHeadDim / 2);
+            if (h != h_held) {
+                // (every product that used the old rows is complete: this thread has read the last of them)
+                const uint4* wrow = reinterpret_cast<const uint4*>(p.w_k + ((size_t)h * p.d_gate + min(r, p.d_gate - 1)) * 3 * kHeadDim);
+#pragma unroll 1
+                for (int c0 = 0; c0 < 8; ++c0) {          // 8 x 32 columns = 512 bf16: [max | min | avg | avg again]
+                    uint32_t wr[32];
+                    const int src = (c0 < 6 ? c0 : c0 - 2) * 8;   // (16-byte pieces of the row; the mean's weights serve its correction too)
 #pragma unroll
-                for (int ks = 0; ks < 3 * kHeadDim / 16; ++ks) {
-                    wa[ks][0] = __ldg(w0 + 8 * ks + t4);
-                    wa[ks][1] = __ldg(w1 + 8 * ks + t4);
-                    wa[ks][2] = __ldg(w0 + 8 * ks + 4 + t4);
-                    wa[ks][3] = __ldg(w1 + 8 * ks + 4 + t4);
+                    for (int x = 0; x < 8; ++x) {
+                        const uint4 v = r < p.d_gate ? __ldg(wrow + src + x) : make_uint4(0u, 0u, 0u, 0u);
+                        wr[4 * x] = v.x; wr[4 * x + 1] = v.y; wr[4 * x + 2] = v.z; wr[4 * x + 3] = v.w;
+                    }
+                    tmem_st32(tbase + 32 * c0, wr);
                 }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.w_ready);
+                h_held = h;
             }
-            h_held = h;
             const int fb = n_done & 1;
             KC_T(t_p0);
-            if (!dead && !mbar_wait(&sm.feat_full[fb], (n_done >> 1) & 1u, p.status)) dead = true;
+            if (!dead && !mbar_wait(&sm.y_full[fb], (n_done >> 1) & 1u, p.status)) dead = true;
             KC_T(t_p1);
             KC_ACC(0, t_p0, t_p1);
             ++n_done;
-            float acc[2][4];
+            __syncwarp();
+            tc_fence_after_sync();
+            uint32_t y[16];
+            tmem_ld16(tbase + 256 + 16 * fb, y);
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.y_free[fb]);
 #pragma unroll
-            for (int n = 0; n < 2; ++n)
-#pragma unroll
-                for (int x = 0; x < 4; ++x) acc[n][x] = 0.f;
-            if (projects) {
-#pragma unroll
-                for (int ks = 0; ks < 3 * kHeadDim / 16; ++ks) {
-#pragma unroll
-                    for (int n = 0; n < 2; ++n) {
-                        const __nv_bfloat16* fr = &sm.feat_hi[fb][8 * n + g][16 * ks + 2 * t4];
-                        mma_bf16_16816(acc[n], wa[ks], *reinterpret_cast<const uint32_t*>(fr),
-                                       *reinterpret_cast<const uint32_t*>(fr + 8));
-                        if (ks >= 2 * kHeadDim / 16) {        // the mean's correction term
-                            const __nv_bfloat16* fl = &sm.feat_lo[fb][8 * n + g][16 * ks - 2 * kHeadDim + 2 * t4];
-                            mma_bf16_16816(acc[n], wa[ks], *reinterpret_cast<const uint32_t*>(fl),
-                                           *reinterpret_cast<const uint32_t*>(fl + 8));
-                        }
-                    }
-                }
-            }
-            KC_T(t_pa);
-            KC_ACC(2, t_p1, t_pa);
-            proj_sync();                                    // every warp is done with the features
-            float (*ybuf)[kStreamDGate] = reinterpret_cast<float (*)[kStreamDGate]>(&sm.feat_hi[fb][0][0]);
-            if (projects) {
-#pragma unroll
-                for (int n = 0; n < 2; ++n) {
-                    ybuf[8 * n + 2 * t4][16 * warp + g] = acc[n][0];
-                    ybuf[8 * n + 2 * t4 + 1][16 * warp + g] = acc[n][1];
-                    ybuf[8 * n + 2 * t4][16 * warp + g + 8] = acc[n][2];
-                    ybuf[8 * n + 2 * t4 + 1][16 * warp + g + 8] = acc[n][3];
-                }
-            }
-            proj_sync();
-            KC_T(t_pb);
-            KC_ACC(3, t_pa, t_pb);
+            for (int q = 0; q < kBulkBlocks; ++q) sm.ybuf[q][r] = __uint_as_float(y[q]);
+            epi_sync();
             const int half = p.d_gate / 2;
             const int u = i * p.num_kv_heads + h;
             // eight rotary pairs per thread: two 16-byte stores instead of sixteen 2-byte ones (a store, too,
             // queues behind the copies)
-            for (int x = tid; x < nb * (half / 8); x += kProjThreads) {
+            for (int x = tid; x < nb * (half / 8); x += kEpiThreads) {
                 const int q = x / (half / 8), c0 = 8 * (x % (half / 8));
                 const int j = j_first + q;
                 uint32_t lo[4], hi[4];
@@ -676,7 +721,7 @@ kcomp_stream_kernel(const __grid_constant__ CUtensorMap map_k, const KcompParams
                     for (int k = 0; k < 2; ++k) {
                         float sn, cs;
                         rope_sincos((double)j * (double)b, p.inv_freq[c0 + e + k], &sn, &cs);
-                        const float a = ybuf[q][c0 + e + k], bb = ybuf[q][c0 + e + k + half];
+                        const float a = sm.ybuf[q][c0 + e + k], bb = sm.ybuf[q][c0 + e + k + half];
                         r0[k] = a * cs - bb * sn;
                         r1[k] = bb * cs + a * sn;
                     }
@@ -687,14 +732,13 @@ kcomp_stream_kernel(const __grid_constant__ CUtensorMap map_k, const KcompParams
                 *reinterpret_cast<uint4*>(dst) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 *reinterpret_cast<uint4*>(dst + half) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
             }
-            // the buffer may be refilled once all eight warps have read their products out of it; the next
-            // item's features and products are in the other buffer
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.feat_empty[fb]);
+            epi_sync();                                    // (the products' buffer is written again for the next item)
             KC_T(t_p2);
             KC_ACC(1, t_p1, t_p2);
-            KC_ACC(4, t_pb, t_p2);
         }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.tmem_done);
     }
 #ifdef SEER_DECODE_TRACE
     if (lane == 0) {

@@ -345,10 +345,10 @@ __global__ void __launch_bounds__(kKcThreads, 4) kcomp_bulk_kernel(const KcompPa
 
 
 // ---- bulk build, streaming variant (b = 64, d_gate <= 128) ----------------------------------------
-// One persistent CTA per SM, three kinds of warps that meet only through mbarriers:
+// One persistent CTA per SM, four kinds of warps that meet only through mbarriers:
 //   producer (1 warp)    keeps a ring of 64-row stages (one block, 16 KiB) full with tiled copies, so
 //                        the bytes in flight do not depend on what the other warps are doing;
-//   pooling (7 warps)    each takes one block at a time out of shared memory and leaves the block's
+//   pooling (10 warps)   each takes one block at a time out of shared memory and leaves the block's
 //                        3*128 features (bf16; the mean as high part + correction: 512 numbers) in one of
 //                        two feature buffers, laid out as the tensor cores read a K-major operand;
 //   MMA (1 warp)         once 16 blocks are pooled, one thread multiplies them in: Y (128 rows of W_k x 16
@@ -368,19 +368,18 @@ __global__ void __launch_bounds__(kKcThreads, 4) kcomp_bulk_kernel(const KcompPa
 // phase away from the barrier's own, which is what a parity wait needs to be unambiguous.  (With a
 // block-of-the-item -> warp rule a fast warp could ask for a slot's next use before the slot's current use
 // had landed for another warp, and the parity test would pass on stale data.)
-constexpr int kStreamStages = 7;                       // 112 KiB in flight per SM
+constexpr int kStreamStages = 10;                      // 160 KiB in flight per SM
 constexpr int kStreamRows = 64;                        // the block size this kernel is written for
 constexpr int kStageRows = kKcompStageRows;
 constexpr int kStagesPerBlock = kStreamRows / kStageRows;
 constexpr int kStageBytes = kStageRows * kHeadDim * 2;
 constexpr int kStreamDGate = 128;
 constexpr int kLensCache = 2048;                       // sequences whose length is kept in shared memory
-constexpr int kPoolWarps = 7;                        // with 8 + 1 others: 16 warps, 128 registers each
-constexpr int kProjWarps = 8;                        // warps 0..3 epilogue, 4 MMA, 5..7 unused
+constexpr int kPoolWarps = 10;                       // with 4 + 1 + 1 others: 16 warps
+constexpr int kProjWarps = 5;                        // warps 0..3 epilogue, 4 MMA
 constexpr int kEpiWarps = 4, kEpiThreads = 128;
 constexpr int kFeatBytes = 8 * kBulkBlocks * 128;      // one feature buffer
 constexpr int kKcTmemCols = 512;                       // W_k 256 columns (512 bf16 per row), Y twice 16
-constexpr int kProjThreads = 32 * kProjWarps;
 constexpr int kStreamThreads = 32 * (kProjWarps + kPoolWarps + 1);
 static_assert(kStreamStages <= 32, "one producer lane per ring slot");
 static_assert(kStreamStages % (kStagesPerBlock * kPoolWarps) == 0,

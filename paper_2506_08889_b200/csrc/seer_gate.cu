@@ -44,6 +44,28 @@ __device__ __forceinline__ float dot8(const uint4& a, const uint4& b) {
     return acc;
 }
 
+// v[k], k = 0..7, summed over a group of `group` = 8, 16 or 32 neighbouring lanes, eight sums for
+// 8 + (log2(group) - 3) shuffles: lanes exchange half of what they carry and go on with the other half,
+// so a lane ends with the group's sum of v[r], r = its low three lane bits in reverse order.
+__device__ __forceinline__ float reduce8(const float (&v)[8], int lane, int group) {
+    const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4;
+    float w4[4], w2[2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float keep = b0 ? v[i + 4] : v[i], send = b0 ? v[i] : v[i + 4];
+        w4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float keep = b1 ? w4[i + 2] : w4[i], send = b1 ? w4[i] : w4[i + 2];
+        w2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    }
+    const float keep = b2 ? w2[1] : w2[0], send = b2 ? w2[0] : w2[1];
+    float x = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    for (int off = 8; off < group; off <<= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    return x;
+}
+
 // Order-preserving key: larger score <-> larger key; -0 == +0; NaN below everything.
 __device__ __forceinline__ uint32_t score_key(float s) {
     if (s != s) return 0u;
@@ -451,7 +473,7 @@ __global__ void __launch_bounds__(kProjThreads) gate_qproj_kernel(const GatePara
 // last ticket runs the selection over all of the unit's scores.  No CTA waits for another.
 #ifdef SEER_GATE_TRACE
 #define GATE_STAMP(k) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
-    reinterpret_cast<unsigned long long*>(p.status)[((size_t)blockIdx.y * gridDim.x + blockIdx.x) * 8 + (k)] = t_; } } while (0)
+    reinterpret_cast<unsigned long long*>(p.status)[((size_t)blockIdx.y * gridDim.x + blockIdx.x) * 16 + (k)] = t_; } } while (0)
 #else
 #define GATE_STAMP(k) ((void)0)
 #endif
@@ -461,7 +483,7 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
     __shared__ int is_last;
     const int u = blockIdx.y, i = u / p.num_kv_heads;
     const int S = gridDim.x, slice = blockIdx.x;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int lpk = p.d_gate / 8;                      // lanes per key: 8, 16 or 32
     const int csub = tid & (lpk - 1);
     const int j0 = min(p.max_blocks, slice * per), j1 = min(p.max_blocks, j0 + per);
@@ -494,21 +516,19 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
     };
     load_q(0);
     const float inv = rsqrtf((float)p.d_gate);
+    const int lpk_shift = 31 - __clz(lpk);
+    const int krev = ((lane & 1) << 2) | (lane & 2) | ((lane >> 2) & 1);
     for (int cb = 0; cb < total; cb += kGateThreads * kBatch) {
-        // a key's score is the largest of its dot products with the query tokens' gate queries
-        float best[kBatch];
-#pragma unroll
-        for (int k = 0; k < kBatch; ++k) best[k] = -INFINITY;
+        // a key's score is the largest of its dot products with the query tokens' gate queries; after
+        // reduce8 a lane holds the sum of the key of its piece number krev
+        float best = -INFINITY;
         for (int t = 0; t < q_len; ++t) {
             if (q_len > 1) load_q(t);
             float acc[kBatch];
 #pragma unroll
             for (int k = 0; k < kBatch; ++k) acc[k] = dot8(kv[k], qsub);
-#pragma unroll
-            for (int k = 0; k < kBatch; ++k) {
-                for (int off = lpk >> 1; off > 0; off >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
-                best[k] = q_len > 1 ? fmaxf(best[k], acc[k]) : acc[k];
-            }
+            const float x = reduce8(acc, lane, lpk);
+            best = q_len > 1 ? fmaxf(best, x) : x;
         }
         const int cb_now = cb;
         if (cb + kGateThreads * kBatch < total) {      // next batch on its way while this one is stored
@@ -518,12 +538,9 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
                 kv[k] = c < total ? __ldg(kc + c) : make_uint4(0u, 0u, 0u, 0u);
             }
         }
-#pragma unroll
-        for (int k = 0; k < kBatch; ++k) {
-            const int c = cb_now + k * kGateThreads + tid;
-            const int j = j0 + c / lpk;
-            if (c < total && csub == 0 && j < n_cand) __stcg(sc_out + j, best[k] * inv);
-        }
+        const int c = cb_now + krev * kGateThreads + tid;
+        const int j = j0 + (c >> lpk_shift);
+        if (c < total && (csub & ~7) == 0 && j < n_cand) __stcg(sc_out + j, best * inv);
     }
     // ---- ticket: the last slice of the unit to finish does the selection --------------------
     GATE_STAMP(2);
@@ -681,12 +698,15 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     float* sc0 = cluster.map_shared_rank(sc_all, 0);
     float* sc_user = p.scores_user ? p.scores_user + (size_t)u * p.max_blocks : nullptr;
     const float inv = rsqrtf((float)p.d_gate);
-    // A key's score is the largest of its dot products with the query tokens' gate queries; the lanes
-    // that hold a key's pieces add up by shuffles.  best[k] belongs to piece cb + k * 512 + tid.
+    // A key's score is the largest of its dot products with the query tokens' gate queries.  A thread holds
+    // one piece of each of kBatch = 8 keys, the lpk lanes of a group the same 8 keys; reduce8 adds up over the
+    // group so that every lane ends with the sum of ONE of the keys (of piece number krev, the lane's low
+    // three bits reversed): each exchange halves the values a lane carries on.  Lanes 0..7 of a group store.
+    const int lpk_shift = 31 - __clz(lpk);
+    const int krev = ((lane & 1) << 2) | (lane & 2) | ((lane >> 2) & 1);
+    const bool storer = (csub & ~7) == 0;
     auto score_batch = [&](auto&& piece, int cb) {
-        float best[kBatch];
-#pragma unroll
-        for (int k = 0; k < kBatch; ++k) best[k] = -INFINITY;
+        float best = -INFINITY;
         for (int t = 0; t < q_len; ++t) {
             float qsub[8];
 #pragma unroll
@@ -694,22 +714,14 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
             float acc[kBatch];
 #pragma unroll
             for (int k = 0; k < kBatch; ++k) acc[k] = dot8(piece(k), qsub);
-            for (int off = lpk >> 1; off > 0; off >>= 1) {
-#pragma unroll
-                for (int k = 0; k < kBatch; ++k) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
-            }
-#pragma unroll
-            for (int k = 0; k < kBatch; ++k) best[k] = MULTI ? fmaxf(best[k], acc[k]) : acc[k];
+            const float x = reduce8(acc, lane, lpk);
+            best = MULTI ? fmaxf(best, x) : x;
         }
-#pragma unroll
-        for (int k = 0; k < kBatch; ++k) {
-            const int c = cb + k * kGateThreads + tid;
-            const int j = j0 + c / lpk;
-            if (c < total && csub == 0 && j < n_cand) {
-                const float v = best[k] * inv;
-                sc0[j] = v;
-                if (sc_user) sc_user[j] = v;
-            }
+        const int j = j0 + ((cb + krev * kGateThreads + tid) >> lpk_shift);
+        if (storer && j < j1 && j < n_cand) {
+            const float v = best * inv;
+            sc0[j] = v;
+            if (sc_user) sc_user[j] = v;
         }
     };
     // Batches alternate between the staged area (each thread reads back the pieces it copied itself)
@@ -718,7 +730,9 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     constexpr int kPieces = kGateThreads * kBatch;
     for (int cb = 0;;) {
         cp_async_wait_all();
+        if (cb == 0) GATE_STAMP(8);
         score_batch([&](int k) { const int pc = cb + k * kGateThreads + tid; return pc < total ? staged[pc - cb] : make_uint4(0u, 0u, 0u, 0u); }, cb);
+        if (cb == 0) GATE_STAMP(9);
         cb += kPieces;
         if (cb >= total) break;
         if (cb + kPieces < total) {

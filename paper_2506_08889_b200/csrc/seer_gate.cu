@@ -95,6 +95,7 @@ struct SelectSmem {
     uint32_t warp_min[kUnitThreads / 32], warp_max[kUnitThreads / 32];
     float red[kUnitThreads / 32];           // block reductions of the threshold method (its own array: the
                                             // selection that follows writes warp_min while slower warps still read)
+    uint32_t pre_min, pre_max;              // smallest and largest key, when the scoring warps have found them (cluster kernel)
     uint32_t prefix;
     int rem;
     int bin_cnt;                            // one-pass path: candidates in the boundary bin ...
@@ -108,13 +109,15 @@ struct SelectSmem {
 // candidate above it and the first few equal to it (the lower block number wins a tie), and
 // the forced last block closes the list.  Comparisons only: the result is exact.
 // NT = threads of the CTA; SMEM = the scores are in shared memory (else read from L2).
+// L_known >= 0: the sequence length, already loaded.  pre: sm.pre_min / sm.pre_max hold the candidates' smallest and
+// largest key and the histograms are clear (the cluster kernel sees to both before its last cluster barrier).
 template <int NT, bool CACHED, bool SMEM>
-__device__ void select_unit(const GateParams& p, int u, const float* sc, SelectSmem& sm) {
+__device__ void select_unit(const GateParams& p, int u, const float* sc, SelectSmem& sm, int L_known = -1, bool pre = false) {
     constexpr int kCachedT = CACHED ? (NT >= 1024 ? 4 : 8) : 1;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int i = u / p.num_kv_heads;
     int32_t* dst = p.block_idx + (size_t)u * p.max_sel;
-    const int L = p.seq_lens[i];
+    const int L = L_known >= 0 ? L_known : p.seq_lens[i];
     const int n_i = L > 0 ? (L + p.block_size - 1) / p.block_size : 0;
     if (n_i <= 0) {
         for (int e = tid; e < p.max_sel; e += NT) dst[e] = -1;
@@ -189,23 +192,28 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
         // for a handful of hot histogram bins.  The passes therefore work on key - min(key), whose
         // significant bits (those of max - min) are spread evenly: first the block-wide min and max.
         uint32_t kmin = 0xffffffffu, kmax = 0u;
-        if (CACHED) {
-#pragma unroll
-            for (int e = 0; e < kCachedT; ++e)
-                if (j_lo + e < j_hi) { kmin = min(kmin, keys[e]); kmax = max(kmax, keys[e]); }
+        if (pre) {
+            kmin = sm.pre_min;
+            kmax = sm.pre_max;
         } else {
-            for (int e = 0; j_lo + e < j_hi; ++e) { const uint32_t key = key_at(e); kmin = min(kmin, key); kmax = max(kmax, key); }
-        }
+            if (CACHED) {
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, off));
-            kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, off));
-        }
-        if (lane == 0) { sm.warp_min[warp] = kmin; sm.warp_max[warp] = kmax; }
-        for (int x = tid; x < 3 * kSelBins; x += NT) (&sm.hist[0][0])[x] = 0;
-        __syncthreads();
+                for (int e = 0; e < kCachedT; ++e)
+                    if (j_lo + e < j_hi) { kmin = min(kmin, keys[e]); kmax = max(kmax, keys[e]); }
+            } else {
+                for (int e = 0; j_lo + e < j_hi; ++e) { const uint32_t key = key_at(e); kmin = min(kmin, key); kmax = max(kmax, key); }
+            }
 #pragma unroll
-        for (int w2 = 0; w2 < NT / 32; ++w2) { kmin = min(kmin, sm.warp_min[w2]); kmax = max(kmax, sm.warp_max[w2]); }
+            for (int off = 16; off > 0; off >>= 1) {
+                kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, off));
+                kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, off));
+            }
+            if (lane == 0) { sm.warp_min[warp] = kmin; sm.warp_max[warp] = kmax; }
+            for (int x = tid; x < 3 * kSelBins; x += NT) (&sm.hist[0][0])[x] = 0;
+            __syncthreads();
+#pragma unroll
+            for (int w2 = 0; w2 < NT / 32; ++w2) { kmin = min(kmin, sm.warp_min[w2]); kmax = max(kmax, sm.warp_max[w2]); }
+        }
         int bits_left = 32 - __clz(max(kmax - kmin, 1u));     // significant bits of key - kmin
         uint32_t prefix = 0u;                                  // the digits found so far, of thr - kmin
         int rem = need;
@@ -396,9 +404,10 @@ __device__ void select_unit(const GateParams& p, int u, const float* sc, SelectS
 }
 
 template <int NT, bool SMEM>
-__device__ __forceinline__ void select_dispatch(const GateParams& p, int u, const float* sc, SelectSmem& sm) {
-    if (p.max_blocks <= (NT >= 1024 ? 4 : 8) * NT) select_unit<NT, true, SMEM>(p, u, sc, sm);
-    else select_unit<NT, false, SMEM>(p, u, sc, sm);
+__device__ __forceinline__ void select_dispatch(const GateParams& p, int u, const float* sc, SelectSmem& sm, int L_known = -1,
+                                                bool pre = false) {
+    if (p.max_blocks <= (NT >= 1024 ? 4 : 8) * NT) select_unit<NT, true, SMEM>(p, u, sc, sm, L_known, pre);
+    else select_unit<NT, false, SMEM>(p, u, sc, sm, L_known, pre);
 }
 
 // Selection on caller-provided scores: one CTA per unit.
@@ -642,6 +651,13 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
         const int pc = k * kGateThreads + tid;
         if (pc < total) cp_async16(staged + pc, kc + pc);
     }
+    // The first CTA, which will select, clears its histograms and the two words the scoring warps fold
+    // the smallest and largest key into (remote atomics, after the first cluster barrier) now, while
+    // the keys travel: the selection then starts with both in hand.
+    if (slice == 0) {
+        for (int x = tid; x < 3 * kSelBins; x += kGateThreads) (&sm.hist[0][0])[x] = 0;
+        if (tid == 0) { sm.pre_min = 0xffffffffu; sm.pre_max = 0u; }
+    }
     cluster_wait();                                    // every CTA of the cluster has started
     // ---- 1. gate queries --------------------------------------------------------------------------
     for (int item = gw; item < n_items; item += n_gw) {
@@ -705,6 +721,7 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     const int lpk_shift = 31 - __clz(lpk);
     const int krev = ((lane & 1) << 2) | (lane & 2) | ((lane >> 2) & 1);
     const bool storer = (csub & ~7) == 0;
+    uint32_t kmn = 0xffffffffu, kmx = 0u;              // smallest and largest key among the scores this thread stores
     auto score_batch = [&](auto&& piece, int cb) {
         float best = -INFINITY;
         for (int t = 0; t < q_len; ++t) {
@@ -722,6 +739,9 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
             const float v = best * inv;
             sc0[j] = v;
             if (sc_user) sc_user[j] = v;
+            const uint32_t key = score_key(v);
+            kmn = min(kmn, key);
+            kmx = max(kmx, key);
         }
     };
     // Batches alternate between the staged area (each thread reads back the pieces it copied itself)
@@ -753,12 +773,21 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
             }
         }
     }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        kmn = min(kmn, __shfl_xor_sync(0xffffffffu, kmn, off));
+        kmx = max(kmx, __shfl_xor_sync(0xffffffffu, kmx, off));
+    }
+    if (lane == 0 && kmn <= kmx) {
+        atomicMin(cluster.map_shared_rank(&sm.pre_min, 0), kmn);
+        atomicMax(cluster.map_shared_rank(&sm.pre_max, 0), kmx);
+    }
     GATE_STAMP(4);
     cluster.sync();
     GATE_STAMP(5);
     // ---- 3. selection by the first CTA ----------------------------------------------------------
     if (slice != 0) return;
-    select_dispatch<kGateThreads, true>(p, u, sc_all, sm);
+    select_dispatch<kGateThreads, true>(p, u, sc_all, sm, L, true);
     GATE_STAMP(6);
 }
 

@@ -49,6 +49,9 @@ struct seer_ctx {
     int pool_div;               // decode scheduling: share of tiles handed out dynamically
     int min_tiles;              // decode scheduling: fewest tiles of a CTA's range
     int sel_from_lens;          // set by seer_decode_step around its attention call (see DecodeParams)
+    int list_gen;               // != 0 inside seer_decode_step: the gate marks finished lists with it, the attention kernel waits per unit
+    int list_gen_last;          // the last such number handed out
+    int use_list_flags;         // 0: the attention kernel of a step waits for the whole gate kernel instead (SEER_STEP_LIST_FLAGS=0)
     int wide_variant;           // kernel variant code for more than 16 rows per unit: 16 (tcgen05), 8 (mma.sync), 0 (by size)
     char err[512];
 };
@@ -75,7 +78,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 constexpr int kMaxGridCtas = 148 * 2 * 4;   // generous bound on the decode grid, for workspace sizing
 
 struct WsLayout {
-    size_t sched, steal, tickets, gate_tickets, prefix, scratch;
+    size_t sched, steal, tickets, gate_tickets, list_flags, prefix, scratch;
     size_t part_o, part_ml, q_gate, scores, total;
 };
 
@@ -91,6 +94,7 @@ WsLayout ws_layout(int num_units, int slots, int d_gate, int max_blocks, int n_t
     w.steal = off; off = align_up(off + sizeof(int) * (size_t)kMaxGridCtas, 256);
     w.tickets = off; off = align_up(off + sizeof(unsigned long long) * (size_t)kMaxUnits, 256);
     w.gate_tickets = off; off = align_up(off + sizeof(int) * (size_t)kMaxUnits, 256);
+    w.list_flags = off; off = align_up(off + sizeof(int) * (size_t)kMaxUnits, 256);
     w.prefix = off; off = align_up(off + sizeof(int) * ((size_t)kMaxUnits + 1), 256);
     w.scratch = off;
     // decode view of the scratch
@@ -256,6 +260,10 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
     p.page_table_stride = kv->page_table_stride;
     p.max_sel = max_sel;
     p.sel_from_lens = sparse && q_len == 1 ? ctx->sel_from_lens : 0;
+    if (p.sel_from_lens > 0 && ctx->list_gen != 0) {
+        p.list_flags = reinterpret_cast<const int*>(ctx->ws + w.list_flags);
+        p.list_gen = ctx->list_gen;
+    }
     p.page_size = kv->page_size;
     p.num_pages = kv->num_pages;
     p.batch = shape->batch;
@@ -332,6 +340,8 @@ seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes) {
     if (const char* e = getenv("SEER_DECODE_POOL_DIV")) ctx->pool_div = atoi(e);
     ctx->min_tiles = 4;
     if (const char* e = getenv("SEER_DECODE_MIN_TILES")) ctx->min_tiles = atoi(e);
+    ctx->use_list_flags = 1;
+    if (const char* e = getenv("SEER_STEP_LIST_FLAGS")) ctx->use_list_flags = atoi(e) != 0;
     ctx->wide_variant = 0;      // chosen by the number of rows
     if (const char* e = getenv("SEER_DECODE_WIDE_VARIANT")) ctx->wide_variant = atoi(e) == 16 ? 16 : atoi(e) == 8 ? 8 : 0;
     ctx->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)64 << 20;
@@ -518,6 +528,10 @@ static seer_status gate_select_common(seer_ctx* ctx, const seer_shape* shape, co
     p.threshold = threshold;
     p.status = reinterpret_cast<unsigned int*>(ctx->ws);
     p.tickets = reinterpret_cast<int*>(ctx->ws + w.gate_tickets);
+    if (ctx->list_gen != 0) {
+        p.list_flags = reinterpret_cast<int*>(ctx->ws + w.list_flags);
+        p.list_gen = ctx->list_gen;
+    }
 #ifdef SEER_GATE_TRACE
     p.status = reinterpret_cast<unsigned int*>(ctx->ws + (ctx->ws_bytes - (size_t)(1 << 19)));
 #endif
@@ -645,17 +659,27 @@ seer_status seer_decode_step(seer_ctx* ctx, const seer_shape* shape, const seer_
     // The block that has just filled is the sequence's last block, which the gate always selects without
     // scoring it (Sec. 3.2): its compressed key is first needed in the next step.  The append is therefore
     // the step's last launch and does its work under the tail of the attention kernel.
-    seer_status st = seer_gate_select(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, token_budget, block_idx, block_cnt,
-                                      max_sel, nullptr, stream);
-    if (st != SEER_OK) return st;
     // With the token budget every list has min(budget in blocks, blocks of the sequence) entries (as long as the
     // compressed-key cache covers the longest sequence): the attention kernel then counts its tiles from the
-    // lengths, before the gate has finished, and waits for the gate only when it reads the lists.
+    // lengths, before the gate has finished, and waits, unit by unit, for the mark the gate kernel leaves when a
+    // unit's list is written.
+    if (!shape || !gate) return fail(ctx, SEER_ERR_INVALID_ARG, "shape or gate is NULL");
     const int k_blocks = token_budget / shape->block_size > 1 ? token_budget / shape->block_size : 1;
     const bool covered = (long long)gate->max_blocks * shape->block_size >= (long long)kv->max_seq_len;
+    if (covered && ctx->use_list_flags) {
+        ctx->list_gen_last = ctx->list_gen_last >= 0x7ffffff0 ? 1 : ctx->list_gen_last + 1;
+        ctx->list_gen = ctx->list_gen_last;
+    }
+    seer_status st = seer_gate_select(ctx, shape, gate, kv->seq_lens, q_nope, nullptr, token_budget, block_idx, block_cnt,
+                                      max_sel, nullptr, stream);
+    if (st != SEER_OK) {
+        ctx->list_gen = 0;
+        return st;
+    }
     ctx->sel_from_lens = covered ? (k_blocks < max_sel ? k_blocks : max_sel) : 0;
     st = seer_sparse_decode(ctx, shape, kv, q, block_idx, block_cnt, max_sel, out, lse, stream);
     ctx->sel_from_lens = 0;
+    ctx->list_gen = 0;
     if (st != SEER_OK || !k_nope) return st;
     return kcomp_append_common(ctx, shape, gate, kv->seq_lens, k_nope, k_nope_stride_batch, k_nope_stride_head,
                                k_nope_stride_token, k_nope_rows_block_local, -1, 1, 1, stream);

@@ -730,7 +730,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     ahead = 2;
                 }
             };
-            if (!producer_waited) {                  // the lists are read from here on
+            if (!producer_waited && !p.list_flags) {  // the lists are read from here on
                 pdl_wait();
                 producer_waited = true;
             }
@@ -767,6 +767,16 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                     const int i = unit_seq(p, my_u);
                     head = my_u - i * p.num_kv_heads;
                     const int L = p.seq_lens[i];
+                    if (SPARSE && p.list_flags) {
+                        // The gate kernel of the same step marks every unit whose list it has written: the tiles of
+                        // the early units are requested while it is still selecting for the late ones.  (That kernel
+                        // was launched before this one and all of its CTAs were resident before this one could start,
+                        // so it makes progress whatever this warp does; the wait is bounded all the same.)
+                        for (int spin = 0; ld_acquire_gpu(p.list_flags + my_u) != p.list_gen; ++spin) {
+                            if (spin > (1 << 20)) { raise_status(p.status, DEV_TIMEOUT); break; }
+                            __nanosleep(40);
+                        }
+                    }
                     if (SMALL) {
                         // a tile gathers the next bpt listed blocks of the unit
                         const int n_i = (L + p.block_size - 1) >> p.bs_shift;

@@ -252,6 +252,16 @@ __device__ __forceinline__ void prefetch_l2(const void* ptr, uint32_t bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr), "r"(bytes) : "memory");
 }
 
+// A flag another kernel's CTA writes once its data is in place: store with release, load with acquire (gpu scope).
+__device__ __forceinline__ void st_release_gpu(int* ptr, int v) {
+    asm volatile("st.release.gpu.global.b32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int* ptr) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+
 // sin and cos of pos * inv_freq for the rotary embedding.  The angle reaches 1e5..1e6 rad at
 // long context, so the product and the reduction to one turn are done in double (a handful
 // of operations); the reduced angle is then accurate to about 1e-10 turns and the fp32

@@ -410,6 +410,16 @@ __device__ __forceinline__ void select_dispatch(const GateParams& p, int u, cons
     else select_unit<NT, false, SMEM>(p, u, sc, sm, L_known, pre);
 }
 
+// The unit's list (entries, count, padding) is complete: tell a kernel that waits for it per unit.
+__device__ __forceinline__ void publish_list(const GateParams& p, int u) {
+    if (!p.list_flags) return;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        st_release_gpu(p.list_flags + u, p.list_gen);
+    }
+}
+
 // Selection on caller-provided scores: one CTA per unit.
 __global__ void __launch_bounds__(kGateThreads) gate_select_only_kernel(const GateParams p) {
     __shared__ SelectSmem sm;
@@ -417,6 +427,7 @@ __global__ void __launch_bounds__(kGateThreads) gate_select_only_kernel(const Ga
     pdl_wait();
     pdl_launch_dependents();
     select_dispatch<kGateThreads, false>(p, u, p.scores_in + (size_t)u * p.max_blocks, sm);
+    publish_list(p, u);
 }
 
 // ---- q_gate = RoPE_{L_i - 1}( W_q[h] . concat_g(Q_nope) )  (Eq. 1a) ---------------------------
@@ -565,6 +576,7 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_score_select_kernel(cons
     GATE_STAMP(4);
     if (!is_last) return;
     select_dispatch<kGateThreads, false>(p, u, sc_out, sm);   // reads the scores with ld.cg, after the ticket
+    publish_list(p, u);
     GATE_STAMP(5);
 }
 
@@ -788,6 +800,7 @@ __global__ void __launch_bounds__(kGateThreads, 2) gate_cluster_kernel(const Gat
     // ---- 3. selection by the first CTA ----------------------------------------------------------
     if (slice != 0) return;
     select_dispatch<kGateThreads, true>(p, u, sc_all, sm, L, true);
+    publish_list(p, u);
     GATE_STAMP(6);
 }
 

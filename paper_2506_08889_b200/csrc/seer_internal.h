@@ -68,6 +68,8 @@ struct DecodeParams {
     int min_tiles;                  // a CTA's range has at least this many tiles (fewer CTAs take part when work is short)
     int max_rounds;                 // most dynamic chunks per range (<= kMaxRounds; 0: none) -- bounds the partial slots
     float scale_log2;               // sm_scale * log2(e)
+    const int* list_flags;          // non-null: unit u's list is final once list_flags[u] == list_gen (written by the gate
+    int list_gen;                   // kernel of the same step); the producer warp then waits per unit, not for the gate's grid
     int sel_from_lens;              // > 0: every unit's list holds min(this, blocks of its sequence) entries, so the
                                     // counts follow from the lengths and the schedule can be made before the kernel
                                     // that writes the lists has finished (0: read block_cnt)
@@ -116,6 +118,8 @@ struct GateParams {
     float threshold;
     unsigned int* status;
     int* tickets;                   // [B*Hkv], zero between launches
+    int* list_flags;                // non-null: list_gen is stored (release) to list_flags[u] once unit u's list is written
+    int list_gen;
     double inv_freq[kMaxDGate / 2]; // rope_theta^(-2c/d_gate), computed on the host in double
 };
 // Launches the scoring kernels (unless scores_in is given) and the selection kernel.

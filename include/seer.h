@@ -114,7 +114,8 @@ typedef struct {
 /* Creates a context on CUDA device `device` and allocates its workspace
  * (workspace_bytes, 0 = a default of 64 MiB; partial results of split
  * sequences, gate scratch, status words).  *out is NULL on failure.
- * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT.  The
+ * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT and
+ * SEER_STEP_LIST_FLAGS (the latter under seer_decode_step).  The
  * multi-token decode calls with 17 to 64 rows per (sequence, KV head)
  * (q_len * group) have two kernels: 16 = on the tcgen05 tensor cores with S, P,
  * O and the queries in tensor memory, 8 = mma.sync.  Unset, up to 48 rows take
@@ -135,7 +136,8 @@ seer_status seer_get_device_status(seer_ctx* ctx, void* stream);
 
 /*
  * Diagnostic: exercises the path every bounded device-side wait of the library takes when it runs out
- * (Sec. 3.3's kernels never wait for one another; the waits are on the kernels' own copies in flight).
+ * (the waits are on a kernel's own copies in flight and, inside seer_decode_step, on the marks that the gate
+ * kernel launched just before it leaves for each finished list).
  * One CTA polls `polls` times (1 .. 2^20) on a barrier that nobody arrives at, gives up, sets the sticky
  * time-out bit and leaves a ticket and the scheduler counters non-zero, as a kernel that was cut short
  * would.  The next seer_get_device_status then returns SEER_ERR_TIMEOUT and clears those counters, after
@@ -310,7 +312,12 @@ seer_status seer_kcomp_append(seer_ctx* ctx, const seer_shape* shape, const seer
  *     seer_kcomp_append(.., first_block = -1) ; seer_gate_select(.., scores_in = NULL) ; seer_sparse_decode
  * on `stream`, with one host round trip instead of three.  (The launches go out as gate, attention,
  * append: the block that has just filled is the sequence's last block, which the gate takes without
- * scoring it, so the entry the append writes is first read in the next step.)
+ * scoring it, so the entry the append writes is first read in the next step.  When gate->max_blocks
+ * blocks cover kv->max_seq_len, the attention kernel knows every list's length from the sequence
+ * lengths and the budget; the gate kernel then marks each list as it finishes it and the attention
+ * kernel starts on a sequence's blocks as soon as that list is marked, with a bounded wait that ends
+ * in SEER_ERR_TIMEOUT.  SEER_STEP_LIST_FLAGS=0 in the environment at seer_create makes it wait for
+ * the whole gate kernel instead; the results are the same.)
  *  block_idx / block_cnt / max_sel: caller-owned scratch for the selected lists (they are
  *  outputs too: the lists the attention used).  Other arguments as in the three calls;
  *  kv->seq_lens is used as the sequence lengths of all three.

@@ -254,3 +254,54 @@ def test_result_does_not_depend_on_how_the_work_is_cut(ctx, monkeypatch):
         o2, l2 = _run_sparse(ctx, q, k, v, lens, idx, cnt, b, 0.0884)
         check_attention(o2, l2, *ref, what="repeat", strict=True)
     assert ctx.device_status() == binding.SEER_OK
+
+
+def test_counts_rewritten_by_the_kernel_just_before(ctx, monkeypatch):
+    # The sparse kernel makes its schedule from the lists' counts as they stand before its
+    # dependency wait and checks them against the final ones after it.  Here the kernel launched
+    # just before it (a selection on given scores) rewrites counts and lists every time, with a
+    # budget that alternates, and nothing synchronises in between: every result must be the
+    # oracle's for the lists of its own step, whether the early look saw the old or the new counts.
+    B, Hq, Hkv, d, b, nb = 2, 8, 4, 128, 64, 96
+    S = nb * b
+    lens = np.array([S, S - 3 * b - 11], np.int32)
+    q, k, v = make_qkv(B, Hq, Hkv, S, d, 77, DEV)
+    r = synth.np_rng(77, "scores")
+    sc = r.normal(size=(B, Hkv, nb)).astype(np.float32)
+    sc_t = torch.as_tensor(sc, device=DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    gate = binding.make_gate(128, 1.0e6, None, None, None, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    kv = binding.make_kv(k, v, lens_t)
+    max_sel = 40
+    budgets = [5 * b, 37 * b]
+    want = []
+    for bud in budgets:
+        i_w, c_w = oracle.select(sc, lens, b, bud, max_sel)
+        want.append((i_w, c_w, ref_sparse(bits(q), bits(k), bits(v), lens, i_w, c_w, b, 0.0884)))
+
+    def run(c):
+        idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+        cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+        steps = 24
+        outs = [torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=DEV) for _ in range(steps)]
+        lses = [torch.zeros((B, Hq), dtype=torch.float32, device=DEV) for _ in range(steps)]
+        torch.cuda.synchronize()
+        for s in range(steps):
+            c.seer_gate_select(shape, gate, lens_t, None, sc_t, budgets[s & 1], idx, cnt, max_sel)
+            c.seer_sparse_decode(shape, kv, q, idx, cnt, max_sel, outs[s], lses[s])
+        torch.cuda.synchronize()
+        for s in range(steps):
+            o_w, l_w, a_w = want[s & 1][2]
+            check_attention(outs[s], lses[s], o_w, l_w, a_w, what=f"step {s}")
+        assert np.array_equal(idx.cpu().numpy(), want[(steps - 1) & 1][0])
+        assert np.array_equal(cnt.cpu().numpy(), want[(steps - 1) & 1][1])
+        assert c.device_status() == binding.SEER_OK
+
+    run(ctx)
+    monkeypatch.setenv("SEER_DECODE_SPECULATE", "0")           # read when a context is created
+    plain = binding.Context(0)
+    try:
+        run(plain)
+    finally:
+        plain.close()

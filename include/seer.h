@@ -114,8 +114,9 @@ typedef struct {
 /* Creates a context on CUDA device `device` and allocates its workspace
  * (workspace_bytes, 0 = a default of 64 MiB; partial results of split
  * sequences, gate scratch, status words).  *out is NULL on failure.
- * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT and
- * SEER_STEP_LIST_FLAGS (the latter under seer_decode_step).  The
+ * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT,
+ * SEER_STEP_LIST_FLAGS (under seer_decode_step) and SEER_DECODE_SPECULATE
+ * (under seer_sparse_decode).  The
  * multi-token decode calls with 17 to 64 rows per (sequence, KV head)
  * (q_len * group) have two kernels: 16 = on the tcgen05 tensor cores with S, P,
  * O and the queries in tensor memory, 8 = mma.sync.  Unset, up to 48 rows take
@@ -177,6 +178,10 @@ seer_status seer_dense_decode(seer_ctx* ctx, const seer_shape* shape, const seer
  * tiles and dealt out evenly over the CTAs; pieces of one pair meet in a
  * log-sum-exp combine done by the last CTA to finish (no second launch).
  * A list with no valid entry gives out = 0, lse = -inf.
+ * block_cnt and seq_lens may be written by the kernel launched just before this
+ * call on the stream: the kernel looks at them early to prepare its schedule, but
+ * uses only what it reads once that kernel has completed (with up to 128
+ * (sequence, KV head) pairs; SEER_DECODE_SPECULATE=0 at seer_create: no early look).
  */
 seer_status seer_sparse_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv,
                                const void* q, const int32_t* block_idx,
@@ -194,10 +199,10 @@ seer_status seer_sparse_decode(seer_ctx* ctx, const seer_shape* shape, const see
  * as it serves all heads of the group.  q_len = 1 is seer_sparse_decode / seer_dense_decode.
  *  q   [B,q_len,Hq,d] bf16 contiguous;  out [B,q_len,Hq,d] bf16;  lse [B,q_len,Hq] fp32 or NULL.
  * A query that sees no listed token (also every query at a negative position, when
- * L_i < q_len) gets out = 0, lse = -inf.  Tokens share a launch -- and the selected K/V are read
- * once for all of them -- while q_len * (Hq/Hkv) <= 16; beyond that the call issues
- * ceil(q_len / floor(16 / (Hq/Hkv))) launches on the stream.  Other arguments, errors and the
- * treatment of the lists as in the single-token calls.
+ * L_i < q_len) gets out = 0, lse = -inf.  All tokens share one launch -- and the selected K/V
+ * are read once for all of them -- while q_len * (Hq/Hkv) <= 64 (with blocks of 16 or 32 tokens:
+ * <= 16); beyond that the call issues one launch per 64 (16) rows on the stream.  Other
+ * arguments, errors and the treatment of the lists as in the single-token calls.
  */
 seer_status seer_sparse_decode_multi(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv,
                                      const void* q, int q_len, const int32_t* block_idx,

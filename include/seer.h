@@ -114,9 +114,8 @@ typedef struct {
 /* Creates a context on CUDA device `device` and allocates its workspace
  * (workspace_bytes, 0 = a default of 64 MiB; partial results of split
  * sequences, gate scratch, status words).  *out is NULL on failure.
- * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT,
- * SEER_STEP_LIST_FLAGS (under seer_decode_step) and SEER_DECODE_SPECULATE
- * (under seer_sparse_decode).  The
+ * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT and
+ * SEER_STEP_LIST_FLAGS (the latter under seer_decode_step).  The
  * multi-token decode calls with 17 to 64 rows per (sequence, KV head)
  * (q_len * group) have two kernels: 16 = on the tcgen05 tensor cores with S, P,
  * O and the queries in tensor memory, 8 = mma.sync.  Unset, up to 48 rows take
@@ -178,10 +177,8 @@ seer_status seer_dense_decode(seer_ctx* ctx, const seer_shape* shape, const seer
  * tiles and dealt out evenly over the CTAs; pieces of one pair meet in a
  * log-sum-exp combine done by the last CTA to finish (no second launch).
  * A list with no valid entry gives out = 0, lse = -inf.
- * block_cnt and seq_lens may be written by the kernel launched just before this
- * call on the stream: the kernel looks at them early to prepare its schedule, but
- * uses only what it reads once that kernel has completed (with up to 128
- * (sequence, KV head) pairs; SEER_DECODE_SPECULATE=0 at seer_create: no early look).
+ * block_idx, block_cnt and seq_lens may be written by the kernel launched just
+ * before this call on the stream: they are read only once that kernel has completed.
  */
 seer_status seer_sparse_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv,
                                const void* q, const int32_t* block_idx,

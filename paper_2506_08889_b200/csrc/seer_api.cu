@@ -51,7 +51,6 @@ struct seer_ctx {
     int sel_from_lens;          // set by seer_decode_step around its attention call (see DecodeParams)
     int list_gen;               // != 0 inside seer_decode_step: the gate marks finished lists with it, the attention kernel waits per unit
     int list_gen_last;          // the last such number handed out
-    int speculate;              // 0: the sparse attention kernel reads the lists' counts only after its dependency wait (SEER_DECODE_SPECULATE=0)
     int use_list_flags;         // 0: the attention kernel of a step waits for the whole gate kernel instead (SEER_STEP_LIST_FLAGS=0)
     int wide_variant;           // kernel variant code for more than 16 rows per unit: 16 (tcgen05), 8 (mma.sync), 0 (by size)
     char err[512];
@@ -265,7 +264,6 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
         p.list_flags = reinterpret_cast<const int*>(ctx->ws + w.list_flags);
         p.list_gen = ctx->list_gen;
     }
-    p.speculate = sparse && block_cnt && p.sel_from_lens == 0 && ctx->speculate;
     p.page_size = kv->page_size;
     p.num_pages = kv->num_pages;
     p.batch = shape->batch;
@@ -344,8 +342,6 @@ seer_status seer_create(seer_ctx** out, int device, size_t workspace_bytes) {
     if (const char* e = getenv("SEER_DECODE_MIN_TILES")) ctx->min_tiles = atoi(e);
     ctx->use_list_flags = 1;
     if (const char* e = getenv("SEER_STEP_LIST_FLAGS")) ctx->use_list_flags = atoi(e) != 0;
-    ctx->speculate = 1;
-    if (const char* e = getenv("SEER_DECODE_SPECULATE")) ctx->speculate = atoi(e) != 0;
     ctx->wide_variant = 0;      // chosen by the number of rows
     if (const char* e = getenv("SEER_DECODE_WIDE_VARIANT")) ctx->wide_variant = atoi(e) == 16 ? 16 : atoi(e) == 8 ? 8 : 0;
     ctx->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)64 << 20;

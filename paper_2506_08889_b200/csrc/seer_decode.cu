@@ -169,17 +169,14 @@ __device__ __forceinline__ int unit_seq(const DecodeParams& p, int u) {
 }
 
 template <bool SPARSE, bool SMALL = false>
-__device__ __forceinline__ int tiles_of(const DecodeParams& p, int u, bool l2_only = false) {
-    // (l2_only: a read made before the kernel's dependency wait, of words that may still change; it must leave
-    // no line in the L1 cache, which is not coherent, for the reads after the wait to hit)
-    const int L = l2_only ? __ldcg(p.seq_lens + unit_seq(p, u)) : p.seq_lens[unit_seq(p, u)];
+__device__ __forceinline__ int tiles_of(const DecodeParams& p, int u) {
+    const int L = p.seq_lens[unit_seq(p, u)];
     if (SPARSE) {
         int c;
         if (p.sel_from_lens > 0) {
             c = min(p.sel_from_lens, (L + p.block_size - 1) >> p.bs_shift);     // (the lists are not final yet)
         } else {
-            // not behind the test on L: both loads in flight
-            c = p.block_cnt ? (l2_only ? __ldcg(p.block_cnt + u) : p.block_cnt[u]) : p.max_sel;
+            c = p.block_cnt ? p.block_cnt[u] : p.max_sel;     // not behind the test on L: both loads in flight
         }
         c = max(0, min(c, p.max_sel));
         return L <= 0 ? 0 : (SMALL ? (c + p.blocks_per_tile - 1) >> p.bpt_shift : c << p.tpb_shift);
@@ -486,17 +483,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     // The producer warp puts its wait off when the lists' lengths follow from the sequence lengths: it then
     // makes the schedule and finds its first unit while the kernel that writes the lists is still running, and
     // waits just before it reads a list.  (Everything it touches before that was final before that kernel began.)
-    // With lists of the caller's (p.speculate) it does the same on a guess: the counts it reads before the wait may
-    // still be changed by the kernel before this one, so they only serve to have the schedule ready; after the wait
-    // the warp reads the counts again, and if any differs it starts over with the final ones.  (Most launches follow
-    // a kernel that leaves the counts alone, or writes the values they had one step earlier.)
-    bool spec = SPARSE && p.speculate && p.sel_from_lens == 0 && U <= kSmemUnits && warp == kConsumerWarps;
-    bool producer_waited = !((SPARSE && p.sel_from_lens > 0 && warp == kConsumerWarps) || spec);
+    bool producer_waited = !(SPARSE && p.sel_from_lens > 0 && warp == kConsumerWarps);
     if (producer_waited) pdl_wait();
     if (tid == 0) SEER_STAMP(9);
 
     if (warp == kConsumerWarps) {
-    redo:
         // =========================== producer warp ====================================
         // The warp first sums the units' tile counts by itself (the consumer warps do not need the
         // result to start waiting) and derives the schedule.  The prefix sums of the counts, by which
@@ -508,8 +499,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         int mine = 0, t_min = 0x7fffffff, t_max = 0;
 #pragma unroll 1
         for (int u = u_lo; u < u_hi; ++u) {
-            const int t = tiles_of<SPARSE, SMALL>(p, u, spec);
-            if (t == 0 && cta == 0 && !spec) write_zero_unit(p, u);       // units without work: zeros, -inf
+            const int t = tiles_of<SPARSE, SMALL>(p, u);
+            if (t == 0 && cta == 0) write_zero_unit(p, u);       // units without work: zeros, -inf
             if (smem_pfx) sm.upfx[u + 1] = t;                      // (the count for now)
             mine += t;
             t_min = min(t_min, t);
@@ -645,30 +636,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             }
             return best;
         };
-        // Guessed counts: the final ones of this lane's units are asked for right after the wait (kSpecPer loads in
-        // flight beside the first list entries) and compared before the first tile is requested.
-        constexpr int kSpecPer = (kSmemUnits + 31) / 32;
-        int chk[kSpecPer];
-        bool chk_pending = false;
-        auto chk_load = [&]() {
-#pragma unroll
-            for (int k = 0; k < kSpecPer; ++k) chk[k] = u_lo + k < u_hi ? tiles_of<SPARSE, SMALL>(p, u_lo + k) : -1;
-            chk_pending = true;
-        };
-        auto chk_same = [&]() -> bool {
-            bool same = true;
-#pragma unroll
-            for (int k = 0; k < kSpecPer; ++k)
-                if (u_lo + k < u_hi) same = same && chk[k] == sm.upfx[u_lo + k + 1] - sm.upfx[u_lo + k];
-            chk_pending = false;
-            same = __all_sync(0xffffffffu, same);
-            if (same && cta == 0) {
-#pragma unroll
-                for (int k = 0; k < kSpecPer; ++k)
-                    if (u_lo + k < u_hi && chk[k] == 0) write_zero_unit(p, u_lo + k);
-            }
-            return same;
-        };
         for (;;) {
             {
                 int c = 0, j = 0;
@@ -766,7 +733,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
             if (!producer_waited && !p.list_flags) {  // the lists are read from here on
                 pdl_wait();
                 producer_waited = true;
-                if (spec) chk_load();
             }
             const bool fresh = !contiguous;          // this interval starts a new piece
             int ce = iv_begin - cpu;                  // offset of the next tile inside unit cu
@@ -797,7 +763,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 const int bpt = SMALL ? p.blocks_per_tile : 1;           // (a compile-time 1 for blocks of 64 or 128 tokens)
                 int nvalid = 0, head = 0, flags = 0;
                 int row[4] = {0, 0, 0, 0}, outer[4] = {0, 0, 0, 0};
-                bool bad = false;                  // (reported below, once the counts behind these tiles are known to be final)
                 if (my_u >= 0) {
                     const int i = unit_seq(p, my_u);
                     head = my_u - i * p.num_kv_heads;
@@ -822,14 +787,14 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                             const int e = my_e * bpt + sb;
                             if (sb < bpt && e < cnt_u) {
                                 const int blk = p.block_idx[(size_t)my_u * p.max_sel + e];
-                                if (blk >= n_i) bad = true;
+                                if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
                                 if (blk >= 0 && blk < n_i) {
                                     const int tok0 = blk * p.block_size;
                                     int nv = max(0, min(p.block_size + 7, L - tok0));
                                     if (PAGED && nv > 0) {
                                         const int pg = p.page_table[(size_t)i * p.page_table_stride + tok0 / p.page_size];
                                         if (pg < 0 || pg >= p.num_pages) {
-                                            bad = true;
+                                            raise_status(p.status, DEV_BAD_INDEX);
                                             nv = 0;
                                         }
                                         outer[sb] = pg;
@@ -847,7 +812,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                         if (SPARSE) {
                             const int blk = p.block_idx[(size_t)my_u * p.max_sel + (my_e >> p.tpb_shift)];
                             const int n_i = (L + p.block_size - 1) >> p.bs_shift;
-                            if (blk >= n_i) bad = true;
+                            if (blk >= n_i) raise_status(p.status, DEV_BAD_INDEX);
                             if (blk >= 0 && blk < n_i) {
                                 tok0 = (blk << p.bs_shift) + (my_e & (p.tiles_per_block - 1)) * kTileTokens;
                                 nvalid = max(0, min(kTileTokens + 7, L - tok0));
@@ -860,7 +825,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                             if (nvalid > 0) {
                                 const int pg = p.page_table[(size_t)i * p.page_table_stride + tok0 / p.page_size];
                                 if (pg < 0 || pg >= p.num_pages) {
-                                    bad = true;
+                                    raise_status(p.status, DEV_BAD_INDEX);
                                     nvalid = 0;
                                 }
                                 outer[0] = pg;
@@ -876,14 +841,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 } else if (lane < n_chunk) {
                     // the counts changed under us: keep the pipeline protocol, load nothing
                     my_u = 0; my_ut = 1; flags = 1;
-                    bad = true;
+                    raise_status(p.status, DEV_BAD_INDEX);
                 }
-                if (chk_pending && !chk_same()) {
-                    // the counts were not final when the schedule was made: once more, with those read after the wait
-                    spec = false;
-                    goto redo;
-                }
-                if (bad) raise_status(p.status, DEV_BAD_INDEX);
                 for (int s = 0; s < n_chunk; ++s, ++it) {
                     if (n_tiles - (t + s) == min(n_tiles, kAheadTiles)) ask_ahead();
                     const int s_nvalid = __shfl_sync(0xffffffffu, nvalid, s);
@@ -958,15 +917,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                 }
             }
         }
-        if (!producer_waited) {                      // (a CTA without tiles: the counters below belong to this launch only after the wait)
-            pdl_wait();
-            producer_waited = true;
-            if (spec) chk_load();
-        }
-        if (chk_pending && !chk_same()) {
-            spec = false;
-            goto redo;
-        }
+        if (!producer_waited) pdl_wait();            // (a CTA without tiles: the counters below belong to this launch only after the wait)
         if (lane == 0) {
             // end-of-stream marker for the consumers
             const int st = it % kS;

@@ -73,8 +73,6 @@ struct DecodeParams {
     int sel_from_lens;              // > 0: every unit's list holds min(this, blocks of its sequence) entries, so the
                                     // counts follow from the lengths and the schedule can be made before the kernel
                                     // that writes the lists has finished (0: read block_cnt)
-    int speculate;                  // 1: the schedule is made from the counts as they stand before the dependency wait
-                                    // and checked against the final ones after it (sparse, block_cnt given, few units)
     unsigned int* status;
     unsigned long long* tickets;    // [num_units]: tiles done << 32 | valid-slot bits; zero between launches
     int* sched;                     // [2]: theft cursor, exit counter; zero between launches

@@ -256,12 +256,11 @@ def test_result_does_not_depend_on_how_the_work_is_cut(ctx, monkeypatch):
     assert ctx.device_status() == binding.SEER_OK
 
 
-def test_counts_rewritten_by_the_kernel_just_before(ctx, monkeypatch):
-    # The sparse kernel makes its schedule from the lists' counts as they stand before its
-    # dependency wait and checks them against the final ones after it.  Here the kernel launched
-    # just before it (a selection on given scores) rewrites counts and lists every time, with a
-    # budget that alternates, and nothing synchronises in between: every result must be the
-    # oracle's for the lists of its own step, whether the early look saw the old or the new counts.
+def test_counts_rewritten_by_the_kernel_just_before(ctx):
+    # The kernel launched just before the sparse decode (a selection on given scores) rewrites counts
+    # and lists every time, with a budget that alternates, and nothing synchronises in between: the
+    # decode kernel may begin its set-up under that kernel's tail, but every result must be the
+    # oracle's for the lists of its own step.
     B, Hq, Hkv, d, b, nb = 2, 8, 4, 128, 64, 96
     S = nb * b
     lens = np.array([S, S - 3 * b - 11], np.int32)
@@ -279,29 +278,19 @@ def test_counts_rewritten_by_the_kernel_just_before(ctx, monkeypatch):
     for bud in budgets:
         i_w, c_w = oracle.select(sc, lens, b, bud, max_sel)
         want.append((i_w, c_w, ref_sparse(bits(q), bits(k), bits(v), lens, i_w, c_w, b, 0.0884)))
-
-    def run(c):
-        idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
-        cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
-        steps = 24
-        outs = [torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=DEV) for _ in range(steps)]
-        lses = [torch.zeros((B, Hq), dtype=torch.float32, device=DEV) for _ in range(steps)]
-        torch.cuda.synchronize()
-        for s in range(steps):
-            c.seer_gate_select(shape, gate, lens_t, None, sc_t, budgets[s & 1], idx, cnt, max_sel)
-            c.seer_sparse_decode(shape, kv, q, idx, cnt, max_sel, outs[s], lses[s])
-        torch.cuda.synchronize()
-        for s in range(steps):
-            o_w, l_w, a_w = want[s & 1][2]
-            check_attention(outs[s], lses[s], o_w, l_w, a_w, what=f"step {s}")
-        assert np.array_equal(idx.cpu().numpy(), want[(steps - 1) & 1][0])
-        assert np.array_equal(cnt.cpu().numpy(), want[(steps - 1) & 1][1])
-        assert c.device_status() == binding.SEER_OK
-
-    run(ctx)
-    monkeypatch.setenv("SEER_DECODE_SPECULATE", "0")           # read when a context is created
-    plain = binding.Context(0)
-    try:
-        run(plain)
-    finally:
-        plain.close()
+    idx = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+    cnt = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+    steps = 24
+    outs = [torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=DEV) for _ in range(steps)]
+    lses = [torch.zeros((B, Hq), dtype=torch.float32, device=DEV) for _ in range(steps)]
+    torch.cuda.synchronize()
+    for s in range(steps):
+        ctx.seer_gate_select(shape, gate, lens_t, None, sc_t, budgets[s & 1], idx, cnt, max_sel)
+        ctx.seer_sparse_decode(shape, kv, q, idx, cnt, max_sel, outs[s], lses[s])
+    torch.cuda.synchronize()
+    for s in range(steps):
+        o_w, l_w, a_w = want[s & 1][2]
+        check_attention(outs[s], lses[s], o_w, l_w, a_w, what=f"step {s}")
+    assert np.array_equal(idx.cpu().numpy(), want[(steps - 1) & 1][0])
+    assert np.array_equal(cnt.cpu().numpy(), want[(steps - 1) & 1][1])
+    assert ctx.device_status() == binding.SEER_OK

@@ -298,6 +298,18 @@ def run_ours(args):
     bulk_ms, _ = repeated(lambda s: ctx.seer_kcomp_append(shape, layers[s % n_layers]["gate"], lens_t, layers[s % n_layers]["k"],
                                                           first_block=0, num_blocks=n_blocks - 1, stream=stream),
                           max(4, min(K, 8 * n_layers)))
+    # what a kernel that only reads gets out of this GPU's memory: the library's read probe over one layer's K and V
+    # caches per launch (4.3 GB, rotating over the layers), the ceiling the decode kernels' figures are set against
+    probe_chk = torch.zeros(1, dtype=torch.int64, device=dev)
+    probe_bytes = layers[0]["k"].numel() * 2
+
+    def probe(s):
+        lay = layers[s % n_layers]
+        ctx.seer_debug_read_bandwidth(lay["k"], probe_bytes, probe_chk, stream=stream)
+        ctx.seer_debug_read_bandwidth(lay["v"], probe_bytes, probe_chk, stream=stream)
+
+    probe_ms, _ = repeated(probe, max(4, min(K, 4 * n_layers)))
+    probe_gbs = 2 * probe_bytes / (probe_ms * 1e-3) / 1e9
     clocks = sampler.stop()
 
     # ---- end to end through the same API with host buffers ----------------------------------
@@ -389,7 +401,11 @@ def run_ours(args):
                          # the same kernel launched back to back (no event between launches, so that each
                          # launch's set-up overlaps its predecessor's tail as it does inside the step)
                          "us_per_launch_back_to_back": round(sparse_b2b_ms * 1e3, 2),
-                         "frac_back_to_back": round(decode_bytes / (sparse_b2b_ms * 1e-3) / 1e9 / peak, 4)},
+                         "frac_back_to_back": round(decode_bytes / (sparse_b2b_ms * 1e-3) / 1e9 / peak, 4),
+                         # against what a read-only kernel reaches on this GPU (the library's probe, same run)
+                         "read_probe_GBps": round(probe_gbs, 1),
+                         "frac_of_read_probe": round(kern_gbs / probe_gbs, 4),
+                         "frac_back_to_back_of_read_probe": round(decode_bytes / (sparse_b2b_ms * 1e-3) / 1e9 / probe_gbs, 4)},
             "extra": {
                 "tokens_per_s_per_layer": round(world * B / (step_ms * 1e-3), 1),
                 "selected_kv_bytes_per_step": sel_kv_bytes,

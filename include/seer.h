@@ -144,6 +144,16 @@ seer_status seer_get_device_status(seer_ctx* ctx, void* stream);
  * which the context works as before.  Asynchronous on `stream`; faults nothing.
  */
 seer_status seer_debug_wait_timeout(seer_ctx* ctx, int polls, void* stream);
+/*
+ * Diagnostic for the roofline (the paper's kernel is "primarily I/O-bound", Sec. 4.4: its ceiling is what a
+ * kernel that only reads gets out of the memory): reads `bytes` bytes at `src` once -- device memory,
+ * 16-byte aligned, `bytes` a multiple of 16 -- with plain 16-byte loads, eight in flight per thread, and
+ * leaves the exclusive-or of all their 32-bit words in the low half of *checksum (device memory, 8 bytes,
+ * cleared by the call).  Timed by the caller over a buffer larger than the L2 cache it gives the read
+ * bandwidth that the decode kernels' achieved figures can be set against.  Asynchronous on `stream`.
+ */
+seer_status seer_debug_read_bandwidth(seer_ctx* ctx, const void* src, size_t bytes, unsigned long long* checksum,
+                                      void* stream);
 /* Workspace bytes a context needs for calls of this shape (upper bound);
  * max_blocks = largest number of blocks per sequence. */
 size_t seer_workspace_bytes(const seer_shape* shape, int max_blocks, int d_gate);

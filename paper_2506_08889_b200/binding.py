@@ -32,7 +32,7 @@ EXPORTS = [
     "seer_dense_decode", "seer_sparse_decode", "seer_gate_select", "seer_kcomp_append",
     "seer_gate_select_static", "seer_decode_step", "seer_gate_select_threshold",
     "seer_sparse_decode_multi", "seer_dense_decode_multi", "seer_gate_select_multi", "seer_decode_step_multi",
-    "seer_debug_wait_timeout", "seer_gate_select_threshold_multi",
+    "seer_debug_wait_timeout", "seer_gate_select_threshold_multi", "seer_debug_read_bandwidth",
 ]
 
 
@@ -123,6 +123,8 @@ def lib() -> ctypes.CDLL:
                                    vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, i32, vp, vp, vp]
     L.seer_debug_wait_timeout.restype = i32
     L.seer_debug_wait_timeout.argtypes = [vp, i32, vp]
+    L.seer_debug_read_bandwidth.restype = i32
+    L.seer_debug_read_bandwidth.argtypes = [vp, vp, ctypes.c_size_t, vp, vp]
     L.seer_gate_select_static.restype = i32
     L.seer_gate_select_static.argtypes = [i32, ctypes.POINTER(SeerShape), ctypes.POINTER(SeerGate), vp, vp, i32,
                                           vp, vp, i32, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
@@ -210,6 +212,10 @@ class Context:
 
     def seer_debug_wait_timeout(self, polls: int, stream=None):
         self._check(lib().seer_debug_wait_timeout(self._h, int(polls), _stream(stream)))
+
+    def seer_debug_read_bandwidth(self, src, nbytes: int, checksum, stream=None):
+        self._check(lib().seer_debug_read_bandwidth(self._h, _ptr(src), ctypes.c_size_t(int(nbytes)), _ptr(checksum),
+                                                    _stream(stream)))
 
     # ---- the four operations (names follow the C ABI) ------------------------------------
     def seer_dense_decode(self, shape: SeerShape, kv: SeerKV, q, out, lse=None, stream=None):

@@ -408,7 +408,63 @@ __global__ void debug_wait_timeout_kernel(unsigned int* status, unsigned long lo
         steal[1] = 1 | (1 << 16);
     }
 }
+
+// Reads n16 16-byte words once, eight loads in flight per thread, and folds their 32-bit words into one
+// checksum (so that no load can be dropped): what a kernel that only reads can get out of the memory.
+constexpr int kProbeThreads = 512;
+__global__ void __launch_bounds__(kProbeThreads, 2) read_probe_kernel(const uint4* __restrict__ src, size_t n16,
+                                                                    unsigned long long* checksum) {
+    const size_t stride = (size_t)gridDim.x * kProbeThreads;
+    size_t i = (size_t)blockIdx.x * kProbeThreads + threadIdx.x;
+    uint4 acc = make_uint4(0u, 0u, 0u, 0u);
+    for (; i + 7 * stride < n16; i += 8 * stride) {
+        uint4 v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = __ldcs(src + i + k * stride);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            acc.x ^= v[k].x;
+            acc.y ^= v[k].y;
+            acc.z ^= v[k].z;
+            acc.w ^= v[k].w;
+        }
+    }
+    for (; i < n16; i += stride) {
+        const uint4 v = __ldcs(src + i);
+        acc.x ^= v.x;
+        acc.y ^= v.y;
+        acc.z ^= v.z;
+        acc.w ^= v.w;
+    }
+    unsigned int x = acc.x ^ acc.y ^ acc.z ^ acc.w;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x ^= __shfl_xor_sync(0xffffffffu, x, o);
+    if ((threadIdx.x & 31) == 0 && x != 0u) atomicXor(checksum, (unsigned long long)x);
+}
 }  // namespace
+
+seer_status seer_debug_read_bandwidth(seer_ctx* ctx, const void* src, size_t bytes, unsigned long long* checksum,
+                                      void* stream) {
+    if (!ctx) return SEER_ERR_INVALID_ARG;
+    if (!src || !checksum) return fail(ctx, SEER_ERR_INVALID_ARG, "src or checksum is NULL");
+    if ((reinterpret_cast<uintptr_t>(src) & 15) || (bytes & 15) || (reinterpret_cast<uintptr_t>(checksum) & 7))
+        return fail(ctx, SEER_ERR_INVALID_ARG, "src and bytes must be multiples of 16, checksum 8-byte aligned");
+    cudaError_t ce = cudaSetDevice(ctx->device);
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ce = cudaMemsetAsync(checksum, 0, sizeof(unsigned long long), s);
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "memset: %s", cudaGetErrorString(ce));
+    if (bytes == 0) return SEER_OK;
+    const size_t n16 = bytes / 16;
+    size_t grid = (n16 + kProbeThreads - 1) / kProbeThreads;
+    const size_t full = (size_t)ctx->num_sms * 2;
+    if (grid > full) grid = full;
+    read_probe_kernel<<<(unsigned int)grid, kProbeThreads, 0, s>>>(static_cast<const uint4*>(src), n16, checksum);
+    ce = cudaGetLastError();
+    if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "launch: %s", cudaGetErrorString(ce));
+    ctx->launches += 1;
+    return SEER_OK;
+}
 
 seer_status seer_debug_wait_timeout(seer_ctx* ctx, int polls, void* stream) {
     if (!ctx) return SEER_ERR_INVALID_ARG;

@@ -282,6 +282,17 @@ def run_ours(args):
         step(layers[s % n_layers], evs[s])
     barrier()
     sparse_ms = float(np.median([a.elapsed_time(bq) for a, bq in evs]))
+    # what two event records cost around a launch that does next to nothing (a one-element fill), taken the same way:
+    # the part of the bracketed figure above that belongs to the bracketing, reported beside it, never subtracted
+    tiny = torch.zeros(1, dtype=torch.int32, device=dev)
+    barrier()
+    for s in range(n_ev):
+        step(layers[s % n_layers])
+        evs[s][0].record()
+        tiny.fill_(1)
+        evs[s][1].record()
+    barrier()
+    empty_ms = float(np.median([a.elapsed_time(bq) for a, bq in evs]))
 
     # dense decode on the same tensors (speed-up denominator), same protocol
     Kd = max(8, min(K, 200))
@@ -394,7 +405,7 @@ def run_ours(args):
                          "peak": peak, "unit": "GB/s", "frac": round(kern_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
                          "frac_of_nominal_8000": round(kern_gbs / NOMINAL_HBM_GBS, 4),
                          "algorithmic_bytes_per_launch": decode_bytes, "us_per_launch": round(sparse_ms * 1e3, 2),
-                         "event_samples": n_ev,
+                         "event_samples": n_ev, "empty_launch_between_events_us": round(empty_ms * 1e3, 2),
                          "traffic": (int(NCU_READ_BYTES_PER_2_SEQUENCES * B / 2 * (1.0 - args.sparsity) / 0.1
                                          + NCU_WRITE_BYTES_PER_LAUNCH) if abs(args.sparsity - 0.9) < 1e-9 else None),
                          "traffic_note": "ncu capture at batch 2, scaled by the units processed",

@@ -524,3 +524,68 @@ def test_step_call_on_a_paged_cache_with_ragged_lengths(ctx):
         ref = ref_sparse(bits(q), bits(k), bits(v), lens, want_idx, want_cnt, b, 0.0884)
         check_attention(out, lse, *ref, what=f"paged step budget={budget}")
     assert ctx.device_status() == binding.SEER_OK
+
+
+def test_steps_back_to_back_with_and_without_the_list_marks(monkeypatch):
+    """Many seer_decode_step calls in a row without a synchronisation, the queries alternating between two
+    draws (so that consecutive steps select different blocks and a mark or a list left by an earlier step
+    would give a wrong result), on ragged lengths: every step's lists are the oracle's selection on the
+    scores the gate computes, every output the oracle's attention over those lists -- with the per-unit
+    marks between the gate and the attention kernel (default) and with SEER_STEP_LIST_FLAGS=0."""
+    B, Hq, Hkv, d, dg, b, S = 4, 8, 2, 128, 128, 64, 8192
+    nb = S // b
+    lens = np.array([S, S - 5 * b - 9, 40 * b + 1, 3 * b], np.int32)
+    _, k, v = make_qkv(B, Hq, Hkv, S, d, 91, DEV)
+    qs = [synth.normal_bf16((B, Hq, d), 91, f"q{j}", DEV) for j in range(2)]
+    qns = [synth.normal_bf16((B, Hq, d), 91, f"qn{j}", DEV) for j in range(2)]
+    wq = synth.normal_bf16((Hkv, dg, 4 * d), 91, "wq", DEV, std=0.02)
+    kc = synth.normal_bf16((B, Hkv, nb, dg), 91, "kc", DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    gate = binding.make_gate(dg, THETA, wq, None, kc, nb)
+    lens_t = torch.as_tensor(lens, device=DEV)
+    kv = binding.make_kv(k, v, lens_t)
+    budget, max_sel, steps = 24 * b, 24, 16
+
+    def run(c):
+        # what each of the two query draws must give: scores from the gate alone, the rest from the oracle
+        want = []
+        for j in range(2):
+            sc = torch.zeros((B, Hkv, nb), dtype=torch.float32, device=DEV)
+            i0 = torch.zeros((B, Hkv, max_sel), dtype=torch.int32, device=DEV)
+            c0 = torch.zeros((B, Hkv), dtype=torch.int32, device=DEV)
+            c.seer_gate_select(shape, gate, lens_t, qns[j], None, budget, i0, c0, max_sel, scores_out=sc)
+            torch.cuda.synchronize()
+            w_idx, w_cnt = oracle.select(sc.cpu().numpy(), lens, b, budget, max_sel)
+            want.append((w_idx, w_cnt, ref_sparse(bits(qs[j]), bits(k), bits(v), lens, w_idx, w_cnt, b, 0.0884)))
+        assert not np.array_equal(want[0][0], want[1][0])          # the two draws do select differently
+        idx = [torch.full((B, Hkv, max_sel), 55, dtype=torch.int32, device=DEV) for _ in range(steps)]
+        cnt = [torch.full((B, Hkv), 55, dtype=torch.int32, device=DEV) for _ in range(steps)]
+        outs = [torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV) for _ in range(steps)]
+        lses = [torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV) for _ in range(steps)]
+        shared_idx = torch.full((B, Hkv, max_sel), 55, dtype=torch.int32, device=DEV)
+        shared_cnt = torch.full((B, Hkv), 55, dtype=torch.int32, device=DEV)
+        torch.cuda.synchronize()
+        for s in range(steps):
+            # even steps reuse one list buffer (each gate overwrites the lists the previous attention read),
+            # odd steps have their own, kept for the comparison
+            li, lc = (shared_idx, shared_cnt) if s % 4 == 0 else (idx[s], cnt[s])
+            c.seer_decode_step(shape, kv, gate, qs[s & 1], qns[s & 1], None, budget, li, lc, max_sel, outs[s], lses[s])
+        torch.cuda.synchronize()
+        for s in range(steps):
+            w_idx, w_cnt, (o_w, l_w, a_w) = want[s & 1]
+            if s % 4 != 0:
+                assert np.array_equal(idx[s].cpu().numpy(), w_idx) and np.array_equal(cnt[s].cpu().numpy(), w_cnt), s
+            check_attention(outs[s], lses[s], o_w, l_w, a_w, what=f"step {s}")
+        assert c.device_status() == binding.SEER_OK
+
+    with_marks = binding.Context(0)
+    try:
+        run(with_marks)
+    finally:
+        with_marks.close()
+    monkeypatch.setenv("SEER_STEP_LIST_FLAGS", "0")             # read when a context is created
+    without = binding.Context(0)
+    try:
+        run(without)
+    finally:
+        without.close()

@@ -5,6 +5,7 @@
 // distributed shared memory carrying the gate query and the scores between the steps.  Beyond that
 // size the same steps run as a projection kernel and a score + selection kernel (the second a
 // programmatic dependent of the first) that go through global memory and per-unit tickets.
+#include <cstdlib>
 #include <cooperative_groups.h>
 
 #include "seer_device.cuh"
@@ -851,6 +852,27 @@ cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* la
         // one cluster per unit: slices of about 512 compressed keys, at most 8 CTAs
         int S = (p.max_blocks + 511) / 512;
         S = S < 1 ? 1 : (S > 8 ? 8 : S);
+        // With few units (small batches) the clusters are widened while they all still fit the SMs at one CTA
+        // each and a slice keeps 128 keys or more: the projection's rows and the keys of a unit are then spread
+        // over more SMs, and the chain of phases gets shorter.
+        {
+            static int sm_count[kMaxDevices] = {};
+            const int slot = current_device_slot();
+            if (sm_count[slot] == 0) {
+                int dev = 0, n = 0;
+                if (cudaGetDevice(&dev) == cudaSuccess &&
+                    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+                    sm_count[slot] = n;
+                else
+                    sm_count[slot] = 1;
+            }
+            static int widen = -1;
+            if (widen < 0) {
+                const char* e = getenv("SEER_GATE_WIDEN");
+                widen = e ? atoi(e) : 1;
+            }
+            while (widen && 2 * S <= 8 && U * 2 * S <= widen * sm_count[slot] && (p.max_blocks + 2 * S - 1) / (2 * S) >= 128) S *= 2;
+        }
         const int per = (p.max_blocks + S - 1) / S;
         const bool multi = p.q_len > 1;
         switch (nit) {

@@ -174,6 +174,9 @@ uint64_t seer_launch_count(const seer_ctx* ctx);
  */
 seer_status seer_dense_decode(seer_ctx* ctx, const seer_shape* shape, const seer_kv* kv,
                               const void* q, void* out, float* lse, void* stream);
+/* Stream capture: the decode calls (dense, sparse, their _multi forms and the step calls) give every launch
+ * counters that the host advances per call, so a CUDA graph captured from them could not be replayed
+ * correctly; on a stream that is being captured they return SEER_ERR_UNSUPPORTED and enqueue nothing. */
 
 /*
  * Block-sparse split-KV flash decoding (Sec. 3.3): the same sum restricted to

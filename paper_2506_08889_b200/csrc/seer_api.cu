@@ -206,6 +206,15 @@ seer_status decode_common(seer_ctx* ctx, const seer_shape* shape, const seer_kv*
 
     cudaError_t ce = cudaSetDevice(ctx->device);
     if (ce != cudaSuccess) return fail(ctx, SEER_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce));
+    // A decode launch carries counters that the host advances per call (the stamp of its partial results, the
+    // number its step's list marks must show): replayed from a captured graph they would repeat, and partials or
+    // marks left by the previous replay would pass for this one's.  Refuse rather than compute wrong results.
+    {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(static_cast<cudaStream_t>(stream), &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone)
+            return fail(ctx, SEER_ERR_UNSUPPORTED,
+                        "the stream is being captured: decode launches carry per-call counters and cannot be replayed from a graph");
+    }
     // Query tokens share a launch while (tokens x group) fits the kernel's 16 rows; more tokens
     // take further launches over the same lists (each reads the selected K/V once).
     // Up to 16 rows ride on the MMA's N side (tokens on M); more than 16 rows (with blocks of 64 or 128 tokens)

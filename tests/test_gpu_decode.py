@@ -294,3 +294,34 @@ def test_counts_rewritten_by_the_kernel_just_before(ctx):
     assert np.array_equal(idx.cpu().numpy(), want[(steps - 1) & 1][0])
     assert np.array_equal(cnt.cpu().numpy(), want[(steps - 1) & 1][1])
     assert ctx.device_status() == binding.SEER_OK
+
+
+def test_decode_refuses_a_stream_that_is_being_captured(ctx):
+    # a decode launch carries per-call counters, so a graph captured from it could not be replayed:
+    # the call must say so instead of enqueueing anything, and work again once the capture is over
+    B, Hq, Hkv, d, b, S = 1, 4, 1, 128, 64, 1024
+    lens = np.array([S], np.int32)
+    q, k, v = make_qkv(B, Hq, Hkv, S, d, 5, DEV)
+    shape = binding.make_shape(B, Hq, Hkv, d, b, 0.0884)
+    lens_t = torch.as_tensor(lens, device=DEV)      # (kept alive: the kv struct holds its address only)
+    kv = binding.make_kv(k, v, lens_t)
+    out = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=DEV)
+    fill = torch.zeros(8, device=DEV)
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        try:
+            fill.add_(1.0)                         # (something to capture, so that the graph is not empty)
+            with pytest.raises(binding.SeerError) as e:
+                ctx.seer_dense_decode(shape, kv, q, out, stream=side)
+            assert e.value.status == binding.SEER_ERR_UNSUPPORTED
+        finally:
+            graph.capture_end()
+    torch.cuda.synchronize()
+    ctx.seer_dense_decode(shape, kv, q, out)
+    torch.cuda.synchronize()
+    ref = ref_dense(bits(q), bits(k), bits(v), lens, 0.0884)
+    check_attention(out, None, ref[0], None, ref[2], what="after the capture")
+    assert ctx.device_status() == binding.SEER_OK

@@ -142,6 +142,20 @@ def max_over_ranks(values, device="cpu"):
     return [float(x) for x in t.cpu()]
 
 
+def repeat_blocks(timed_block, n, min_s, max_repeats=200, device="cpu"):
+    """Repeats `timed_block(n)` (ms per call of a block of n calls) until `min_s` seconds have been timed;
+    returns (median block, number of blocks).  Every block's time is first replaced by its maximum over the
+    ranks, so that all ranks see the same numbers and stop after the same block -- the blocks contain
+    barriers, and ranks that went on for different numbers of blocks would wait for one another forever."""
+    import numpy as np
+    blocks, total = [], 0.0
+    while not blocks or (total < min_s and len(blocks) < max_repeats):
+        ms = max_over_ranks([timed_block(n)], device)[0]
+        blocks.append(ms)
+        total += ms * n * 1e-3
+    return float(np.median(blocks)), len(blocks)
+
+
 def job_throughput_gbs(world: int, bytes_per_rank: int, ms: float) -> float:
     """Whole-job GB/s: all ranks' bytes over the slowest rank's time."""
     return world * bytes_per_rank / (ms * 1e-3) / 1e9
@@ -262,12 +276,7 @@ def run_ours(args):
     def repeated(fn, n, min_s=None, max_repeats=200):
         """Median over repeated blocks of n calls (ms per call), and the number of blocks."""
         min_s = args.min_timed_s if min_s is None else min_s
-        blocks, total = [], 0.0
-        while not blocks or (total < min_s and len(blocks) < max_repeats):
-            ms = timed_block(fn, n)
-            blocks.append(ms)
-            total += ms * n * 1e-3
-        return float(np.median(blocks)), len(blocks)
+        return repeat_blocks(lambda m: timed_block(fn, m), n, min_s, max_repeats, dev)
 
     launches0 = ctx.launch_count()
     step_ms, repeats = repeated(lambda s: step(layers[s % n_layers]), K)
@@ -365,16 +374,15 @@ def run_ours(args):
     Ke = max(8, min(K, 300))
     for s in range(3):
         e2e_step(layers[s % n_layers])
-    e2e_blocks, e2e_total = [], 0.0
-    while not e2e_blocks or (e2e_total < args.min_timed_s and len(e2e_blocks) < 200):
+    def e2e_block(n):
         barrier()
         w0 = time.perf_counter()
-        for s in range(Ke):
+        for s in range(n):
             e2e_step(layers[s % n_layers])
         barrier()
-        e2e_blocks.append((time.perf_counter() - w0) * 1e3 / Ke)
-        e2e_total += e2e_blocks[-1] * Ke * 1e-3
-    e2e_ms = float(np.median(e2e_blocks))
+        return (time.perf_counter() - w0) * 1e3 / n
+
+    e2e_ms, _ = repeat_blocks(e2e_block, Ke, args.min_timed_s, 200, dev)
     assert ctx.device_status() == binding.SEER_OK
 
     # ---- reduce over ranks -------------------------------------------------------------------

@@ -117,7 +117,8 @@ typedef struct {
  * Read from the environment at creation: SEER_DECODE_WIDE_VARIANT and
  * SEER_STEP_LIST_FLAGS (the latter under seer_decode_step); read at the
  * process's first gate call: SEER_GATE_WIDEN (0: the gate's clusters keep one
- * CTA per 512 compressed keys also when there are few sequences).  The
+ * CTA per 512 compressed keys also when there are few sequences; n: they may be
+ * widened while all of them fit the SMs at n CTAs each, default 2).  The
  * multi-token decode calls with 17 to 64 rows per (sequence, KV head)
  * (q_len * group) have two kernels: 16 = on the tcgen05 tensor cores with S, P,
  * O and the queries in tensor memory, 8 = mma.sync.  Unset, up to 48 rows take

@@ -852,8 +852,8 @@ cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* la
         // one cluster per unit: slices of about 512 compressed keys, at most 8 CTAs
         int S = (p.max_blocks + 511) / 512;
         S = S < 1 ? 1 : (S > 8 ? 8 : S);
-        // With few units (small batches) the clusters are widened while they all still fit the SMs at one CTA
-        // each and a slice keeps 128 keys or more: the projection's rows and the keys of a unit are then spread
+        // With few units (small batches) the clusters are widened while they all still fit the SMs at two CTAs
+        // each (what the kernel's shared memory allows) and a slice keeps 128 keys or more: the projection's rows and the keys of a unit are then spread
         // over more SMs, and the chain of phases gets shorter.
         {
             static int sm_count[kMaxDevices] = {};
@@ -869,7 +869,7 @@ cudaError_t launch_gate_select(const GateParams& p, cudaStream_t stream, int* la
             static int widen = -1;
             if (widen < 0) {
                 const char* e = getenv("SEER_GATE_WIDEN");
-                widen = e ? atoi(e) : 1;
+                widen = e ? atoi(e) : 2;         // (CTAs per SM that the clusters may fill; 0: no widening)
             }
             while (widen && 2 * S <= 8 && U * 2 * S <= widen * sm_count[slot] && (p.max_blocks + 2 * S - 1) / (2 * S) >= 128) S *= 2;
         }

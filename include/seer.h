@@ -118,7 +118,11 @@ typedef struct {
  * SEER_STEP_LIST_FLAGS (the latter under seer_decode_step); read at the
  * process's first gate call: SEER_GATE_WIDEN (0: the gate's clusters keep one
  * CTA per 512 compressed keys also when there are few sequences; n: they may be
- * widened while all of them fit the SMs at n CTAs each, default 2).  The
+ * widened while all of them fit the SMs at n CTAs each, default 2).  Also at
+ * creation, for experiments with the decode kernel's work split:
+ * SEER_DECODE_POOL_DIV (1/n of a CTA's tiles are handed out dynamically;
+ * default 4, 0 = a static split) and SEER_DECODE_MIN_TILES (fewest tiles a CTA
+ * takes when work is short; default 4).  The
  * multi-token decode calls with 17 to 64 rows per (sequence, KV head)
  * (q_len * group) have two kernels: 16 = on the tcgen05 tensor cores with S, P,
  * O and the queries in tensor memory, 8 = mma.sync.  Unset, up to 48 rows take
